@@ -1,0 +1,141 @@
+/* libef: one two-way compressed step of dist-EF-blockSGDM on a single B200.
+ *
+ * The library implements the data-parallel hot path of Algorithm 4 (distributed blockwise
+ * momentum SGD with error feedback) of arXiv 1905.10936 for M simulated workers that all
+ * live on one GPU.  One iteration t is
+ *
+ *     for each worker i in [0, M):  ef_worker_step(ctx, i, g_{t,i})
+ *     ef_server_step(ctx)
+ *
+ * All entry points are plain C.  "device" pointers are CUDA device pointers of the current
+ * device, "host" pointers are ordinary host pointers.  The library never allocates device
+ * memory: the caller hands over one workspace (size from ef_workspace_bytes) and keeps
+ * owning it.  Every call only enqueues work on the CUDA stream given to ef_init and returns
+ * without synchronising; results are ordered on that stream.
+ *
+ * There is no CPU fallback: on a device that is not compute capability 10.x ef_init fails
+ * with EF_ERR_UNSUPPORTED_DEVICE.
+ *
+ * Packed sign layout (a convention of this library; the paper only fixes "one bit per sign
+ * in {-1,+1}", Appendix A): block b owns ceil(d_b/32) consecutive 32-bit words, blocks in
+ * order, every block starting on a word boundary.  Element k of the block is bit (k mod 32),
+ * least significant bit first, of the block's word floor(k/32).  Bit 1 means the element is
+ * negative (decodes to -1), bit 0 means it is >= 0 (decodes to +1; sign(+-0) = +1).  Unused
+ * high bits of a block's last word are 0.  Scales are B consecutive floats, scale_b =
+ * ||v_{G_b}||_1 / d_b (Section 3.2).  The decoded message is Delta_j = (bit ? -1 : +1) * scale_b.
+ */
+#ifndef EF_H_
+#define EF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ef_ctx ef_ctx;   /* opaque host object; owns no device memory */
+
+enum ef_status {
+    EF_OK = 0,
+    EF_ERR_INVALID_ARG = 1,        /* a size, index, pointer or hyper-parameter is out of range */
+    EF_ERR_BAD_STATE = 2,          /* call order violated (see ef_worker_step / ef_server_step) */
+    EF_ERR_WORKSPACE = 3,          /* workspace null or smaller than ef_workspace_bytes */
+    EF_ERR_ALIGNMENT = 4,          /* a device pointer is not 16-byte aligned */
+    EF_ERR_CUDA = 5,               /* a CUDA runtime call failed; see ef_last_cuda_error */
+    EF_ERR_UNSUPPORTED_DEVICE = 6, /* current device is not compute capability 10.x */
+    EF_ERR_TIMEOUT = 7             /* reserved: a bounded device-side wait gave up */
+};
+
+/* Flags for ef_workspace_bytes / ef_init. */
+#define EF_FLAG_HOST_STAGING 1u    /* reserve two d-float staging buffers for ef_worker_step_host */
+
+/* Maximum number of simulated workers. */
+#define EF_MAX_WORKERS 4096
+
+/* Workspace size in bytes for a problem (Algorithm 4, "Input" and "Initialize" lines):
+ * d parameters, B blocks given by B+1 non-decreasing host offsets with offsets[0] = 0,
+ * offsets[B] = d and every block non-empty (1/d_b appears in Prop. 1), M workers.
+ * Pure host computation; needs no GPU.  Errors: EF_ERR_INVALID_ARG. */
+int ef_workspace_bytes(int64_t d, int32_t B, const int64_t* offsets /* host, B+1 */,
+                       int32_t M, uint32_t flags, size_t* bytes /* out */);
+
+/* Creates a context and initialises the state of Algorithm 4 in the workspace:
+ * x_0 = 0, m_{-1,i} = 0, e_{0,i} = 0, etilde_0 = 0, t = 0 (Algorithm 4, "Initialize").
+ * mu in [0, 1) is the momentum parameter, eta > 0 the (constant) stepsize, so the factor
+ * eta_{t-1}/eta_t of Algorithm 4 is 1 (at t = 0 it multiplies a zero residual).
+ * workspace: device, 256-byte aligned, at least ef_workspace_bytes; borrowed until ef_destroy.
+ * cuda_stream: a cudaStream_t (0 = default stream) on which all work of this context runs.
+ * Errors: INVALID_ARG, WORKSPACE, ALIGNMENT, UNSUPPORTED_DEVICE, CUDA.  On error *out = NULL
+ * and nothing was launched. */
+int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets /* host, B+1 */,
+            int32_t M, float mu, float eta, uint32_t flags,
+            void* workspace /* device */, size_t workspace_bytes, void* cuda_stream);
+
+/* Worker side of one iteration for worker i (Algorithm 4, the "on each worker i" lines):
+ *   m_{t,i} = mu m_{t-1,i} + g_{t,i};  p_{t,i} = mu m_{t,i} + g_{t,i} + e_{t,i};
+ *   Delta_{t,i} = C_B(p_{t,i}) (packed signs + one scale per block, Section 3.2);
+ *   e_{t+1,i} = p_{t,i} - Delta_{t,i}.
+ * grad: device, d floats, 16-byte aligned, borrowed until the enqueued kernel has run.
+ * Writes the packed words and scales readable through ef_worker_words / ef_worker_scales.
+ * Workers may be stepped in any order, each exactly once per iteration.
+ * Non-finite gradients are not checked; they propagate into the block's scale.
+ * Errors: INVALID_ARG (i, null), ALIGNMENT, BAD_STATE (worker i already stepped in this
+ * iteration), CUDA. */
+int ef_worker_step(ef_ctx* ctx, int32_t i, const float* grad /* device */);
+
+/* Same as ef_worker_step with the gradient in HOST memory (pinned memory recommended): the
+ * gradient is copied to a staging buffer on an internal copy stream, double-buffered so that
+ * the copy of worker i+1 overlaps the kernel of worker i.  grad is borrowed until the copy
+ * has completed (ordered before everything later enqueued on the context's stream).
+ * Requires EF_FLAG_HOST_STAGING at ef_init, else EF_ERR_BAD_STATE. */
+int ef_worker_step_host(ef_ctx* ctx, int32_t i, const float* grad /* host */);
+
+/* Server side of one iteration (Algorithm 4, the "on server" lines) plus the parameter
+ * update every worker performs after the pull (Algorithm 4, x_{t+1} = x_t - eta Deltatilde_t;
+ * all replicas of x are identical, so it is done once):
+ *   ptilde_t = (1/M) sum_i Delta_{t,i} + etilde_t;  Deltatilde_t = C_B(ptilde_t);
+ *   etilde_{t+1} = ptilde_t - Deltatilde_t;  x_{t+1} = x_t - eta Deltatilde_t.
+ * The average is evaluated as sum over ascending i of (+-)(scale_{i,b} / M) in fp32.
+ * Errors: BAD_STATE unless every worker has been stepped exactly once since the last
+ * server step; CUDA. */
+int ef_server_step(ef_ctx* ctx);
+
+/* Copies the server's message of the last ef_server_step (packed words, then scales) to host
+ * memory, asynchronously on the context's stream.  words: ef_num_words words; scales: B floats.
+ * Errors: INVALID_ARG (null), CUDA. */
+int ef_read_update_host(ef_ctx* ctx, uint32_t* words /* host */, float* scales /* host */);
+
+/* Zero-copy device views, valid until ef_destroy; contents are ordered on the context's stream.
+ * i in [0, M); NULL on a bad index. */
+const uint32_t* ef_worker_words(ef_ctx* ctx, int32_t i);   /* ef_num_words words */
+const float*    ef_worker_scales(ef_ctx* ctx, int32_t i);  /* B floats */
+const uint32_t* ef_server_words(ef_ctx* ctx);
+const float*    ef_server_scales(ef_ctx* ctx);
+float*          ef_params(ef_ctx* ctx);   /* x, d floats; the caller may write x_0 or edit x between iterations */
+int64_t         ef_num_words(ef_ctx* ctx);/* W = sum_b ceil(d_b / 32) */
+
+/* State access for tests and checkpoints.  All pointers are device pointers to d floats,
+ * 16-byte aligned.  i in [0, M) names a worker; i = -1 names the server (residual only).
+ * The residual is stored internally in a deferred form (the corrected vector p_t plus the
+ * block scale); ef_get_residual writes the residual e_{t+1} = p_t - Delta_t itself.
+ * ef_set_state overwrites momentum (ignored for the server, may be NULL there) and residual.
+ * Errors: INVALID_ARG, ALIGNMENT, BAD_STATE (called in the middle of an iteration), CUDA. */
+int ef_get_momentum(ef_ctx* ctx, int32_t i, float* dst);
+int ef_get_residual(ef_ctx* ctx, int32_t i, float* dst);
+int ef_set_state(ef_ctx* ctx, int32_t i, const float* momentum, const float* residual);
+int ef_step_count(ef_ctx* ctx, int64_t* t /* out: completed iterations */);
+
+/* Number of kernels this context has launched so far (for launch accounting). */
+int64_t ef_launch_count(ef_ctx* ctx);
+
+const char* ef_strerror(int status);
+int ef_last_cuda_error(ef_ctx* ctx);      /* the cudaError_t of the last EF_ERR_CUDA, else 0 */
+
+/* Frees the host object.  Does not touch the workspace.  NULL is allowed. */
+int ef_destroy(ef_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* EF_H_ */

@@ -1,0 +1,182 @@
+"""Thin ctypes binding of libef (see include/ef.h): argument marshalling only.
+
+Every function has the name and the argument order of its C counterpart.  Device pointers
+are passed as integers (``tensor.data_ptr()``); torch is used only to own device memory and
+to name the CUDA stream.  There is no fallback: if the shared library is missing the import
+of a symbol raises, and on a device that is not compute capability 10.x ``ef_init`` fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libef.so")
+
+EF_OK = 0
+EF_ERR_INVALID_ARG = 1
+EF_ERR_BAD_STATE = 2
+EF_ERR_WORKSPACE = 3
+EF_ERR_ALIGNMENT = 4
+EF_ERR_CUDA = 5
+EF_ERR_UNSUPPORTED_DEVICE = 6
+EF_ERR_TIMEOUT = 7
+EF_FLAG_HOST_STAGING = 1
+EF_MAX_WORKERS = 4096
+
+_vp, _i64, _i32, _u32, _f32 = (ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_uint32,
+                               ctypes.c_float)
+
+# name -> (restype, argtypes); mirrors include/ef.h
+SIGNATURES = {
+    "ef_workspace_bytes": (ctypes.c_int, [_i64, _i32, _vp, _i32, _u32, ctypes.POINTER(ctypes.c_size_t)]),
+    "ef_init": (ctypes.c_int, [ctypes.POINTER(_vp), _i64, _i32, _vp, _i32, _f32, _f32, _u32, _vp,
+                               ctypes.c_size_t, _vp]),
+    "ef_worker_step": (ctypes.c_int, [_vp, _i32, _vp]),
+    "ef_worker_step_host": (ctypes.c_int, [_vp, _i32, _vp]),
+    "ef_server_step": (ctypes.c_int, [_vp]),
+    "ef_read_update_host": (ctypes.c_int, [_vp, _vp, _vp]),
+    "ef_worker_words": (_vp, [_vp, _i32]),
+    "ef_worker_scales": (_vp, [_vp, _i32]),
+    "ef_server_words": (_vp, [_vp]),
+    "ef_server_scales": (_vp, [_vp]),
+    "ef_params": (_vp, [_vp]),
+    "ef_num_words": (_i64, [_vp]),
+    "ef_get_momentum": (ctypes.c_int, [_vp, _i32, _vp]),
+    "ef_get_residual": (ctypes.c_int, [_vp, _i32, _vp]),
+    "ef_set_state": (ctypes.c_int, [_vp, _i32, _vp, _vp]),
+    "ef_step_count": (ctypes.c_int, [_vp, ctypes.POINTER(_i64)]),
+    "ef_launch_count": (_i64, [_vp]),
+    "ef_strerror": (ctypes.c_char_p, [ctypes.c_int]),
+    "ef_last_cuda_error": (ctypes.c_int, [_vp]),
+    "ef_destroy": (ctypes.c_int, [_vp]),
+}
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads libef.so from the package directory; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise OSError(f"{LIB_PATH} is missing: build it with "
+                          "`python -m paper_1905_10936_b200.build` (there is no fallback path)")
+        lib = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+class EFError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = load_library().ef_strerror(status).decode()
+        super().__init__(f"{where}: {msg} (status {status})")
+
+
+def _check(status: int, where: str) -> None:
+    if status != EF_OK:
+        raise EFError(status, where)
+
+
+def _offsets_array(offsets: Sequence[int]) -> np.ndarray:
+    return np.ascontiguousarray(offsets, dtype=np.int64)
+
+
+# ---- functions with the C names ------------------------------------------------------------
+def ef_workspace_bytes(d: int, B: int, offsets, M: int, flags: int = 0) -> int:
+    off = _offsets_array(offsets)
+    out = ctypes.c_size_t(0)
+    _check(load_library().ef_workspace_bytes(d, B, off.ctypes.data, M, flags, ctypes.byref(out)),
+           "ef_workspace_bytes")
+    return out.value
+
+
+def ef_init(d: int, B: int, offsets, M: int, mu: float, eta: float, flags: int,
+            workspace_ptr: int, workspace_bytes: int, cuda_stream: int) -> int:
+    off = _offsets_array(offsets)
+    ctx = _vp(None)
+    _check(load_library().ef_init(ctypes.byref(ctx), d, B, off.ctypes.data, M, mu, eta, flags,
+                                  workspace_ptr, workspace_bytes, cuda_stream), "ef_init")
+    return ctx.value
+
+
+def ef_worker_step(ctx: int, i: int, grad_ptr: int) -> None:
+    _check(load_library().ef_worker_step(ctx, i, grad_ptr), "ef_worker_step")
+
+
+def ef_worker_step_host(ctx: int, i: int, grad_host_ptr: int) -> None:
+    _check(load_library().ef_worker_step_host(ctx, i, grad_host_ptr), "ef_worker_step_host")
+
+
+def ef_server_step(ctx: int) -> None:
+    _check(load_library().ef_server_step(ctx), "ef_server_step")
+
+
+def ef_read_update_host(ctx: int, words_host_ptr: int, scales_host_ptr: int) -> None:
+    _check(load_library().ef_read_update_host(ctx, words_host_ptr, scales_host_ptr),
+           "ef_read_update_host")
+
+
+def ef_worker_words(ctx: int, i: int) -> Optional[int]:
+    return load_library().ef_worker_words(ctx, i)
+
+
+def ef_worker_scales(ctx: int, i: int) -> Optional[int]:
+    return load_library().ef_worker_scales(ctx, i)
+
+
+def ef_server_words(ctx: int) -> Optional[int]:
+    return load_library().ef_server_words(ctx)
+
+
+def ef_server_scales(ctx: int) -> Optional[int]:
+    return load_library().ef_server_scales(ctx)
+
+
+def ef_params(ctx: int) -> Optional[int]:
+    return load_library().ef_params(ctx)
+
+
+def ef_num_words(ctx: int) -> int:
+    return load_library().ef_num_words(ctx)
+
+
+def ef_get_momentum(ctx: int, i: int, dst_ptr: int) -> None:
+    _check(load_library().ef_get_momentum(ctx, i, dst_ptr), "ef_get_momentum")
+
+
+def ef_get_residual(ctx: int, i: int, dst_ptr: int) -> None:
+    _check(load_library().ef_get_residual(ctx, i, dst_ptr), "ef_get_residual")
+
+
+def ef_set_state(ctx: int, i: int, momentum_ptr: Optional[int], residual_ptr: int) -> None:
+    _check(load_library().ef_set_state(ctx, i, momentum_ptr, residual_ptr), "ef_set_state")
+
+
+def ef_step_count(ctx: int) -> int:
+    t = _i64(0)
+    _check(load_library().ef_step_count(ctx, ctypes.byref(t)), "ef_step_count")
+    return t.value
+
+
+def ef_launch_count(ctx: int) -> int:
+    return load_library().ef_launch_count(ctx)
+
+
+def ef_last_cuda_error(ctx: int) -> int:
+    return load_library().ef_last_cuda_error(ctx)
+
+
+def ef_strerror(status: int) -> str:
+    return load_library().ef_strerror(status).decode()
+
+
+def ef_destroy(ctx: int) -> None:
+    _check(load_library().ef_destroy(ctx), "ef_destroy")

@@ -1,0 +1,397 @@
+// Host side of libef: argument checking, workspace layout, tile table, kernel launches.
+// The interface is documented in include/ef.h.
+#include "../../include/ef.h"
+#include "ef_kernels.cuh"
+
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+namespace {
+
+using efk::Block;
+using efk::Tile;
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
+
+// Rows of four elements per thread and tile; a tile is 1024*U elements.
+constexpr int kU = 4;
+constexpr int kTileLen = 1024 * kU;
+
+struct Layout {
+    int64_t d = 0, W = 0;
+    int32_t B = 0, M = 0;
+    int64_t num_tiles = 0;
+    size_t dpad = 0, wpad = 0, bpad = 0, tpad = 0;    // padded element counts per sub-buffer
+    size_t off_x = 0, off_m = 0, off_pb = 0, off_spb = 0, off_words = 0, off_scales = 0,
+           off_rscale = 0, off_partials = 0, off_tickets = 0, off_tiles = 0, off_blocks = 0,
+           off_stage = 0, total = 0;
+};
+
+int check_problem(int64_t d, int32_t B, const int64_t* offsets, int32_t M) {
+    if (!offsets || d < 1 || B < 1 || M < 1 || M > EF_MAX_WORKERS) return EF_ERR_INVALID_ARG;
+    if (offsets[0] != 0 || offsets[B] != d) return EF_ERR_INVALID_ARG;
+    for (int32_t b = 0; b < B; ++b)
+        if (offsets[b + 1] <= offsets[b]) return EF_ERR_INVALID_ARG;
+    return EF_OK;
+}
+
+int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_t flags,
+                Layout* L) {
+    int rc = check_problem(d, B, offsets, M);
+    if (rc != EF_OK) return rc;
+    if (flags & ~EF_FLAG_HOST_STAGING) return EF_ERR_INVALID_ARG;
+    L->d = d; L->B = B; L->M = M;
+    int64_t W = 0, T = 0;
+    for (int32_t b = 0; b < B; ++b) {
+        const int64_t db = offsets[b + 1] - offsets[b];
+        W += (db + 31) / 32;
+        T += (db + kTileLen - 1) / kTileLen;
+    }
+    if (T > 0x7fffffffLL) return EF_ERR_INVALID_ARG;
+    L->W = W; L->num_tiles = T;
+    L->dpad = align_up((size_t)d * 4) / 4;
+    L->wpad = align_up((size_t)W * 4) / 4;
+    L->bpad = align_up((size_t)B * 4) / 4;
+    L->tpad = align_up((size_t)T * 8) / 8;
+    const size_t M1 = (size_t)M + 1;
+    size_t o = 0;
+    L->off_x = o;        o += L->dpad * 4;
+    L->off_m = o;        o += (size_t)M * L->dpad * 4;
+    L->off_pb = o;       o += (size_t)M * L->dpad * 4;
+    L->off_spb = o;      o += L->dpad * 4;
+    L->off_words = o;    o += M1 * L->wpad * 4;
+    L->off_scales = o;   o += M1 * L->bpad * 4;
+    L->off_rscale = o;   o += M1 * L->bpad * 4;
+    L->off_partials = o; o += M1 * L->tpad * 8;
+    L->off_tickets = o;  o += M1 * L->bpad * 4;
+    L->off_tiles = o;    o += align_up((size_t)T * sizeof(Tile));
+    L->off_blocks = o;   o += align_up((size_t)B * sizeof(Block));
+    L->off_stage = o;
+    if (flags & EF_FLAG_HOST_STAGING) o += 2 * L->dpad * 4;
+    L->total = o;
+    return EF_OK;
+}
+
+}  // namespace
+
+struct ef_ctx {
+    Layout L;
+    float mu = 0.f, eta = 0.f;
+    uint32_t flags = 0;
+    char* ws = nullptr;
+    cudaStream_t stream = nullptr;
+    int64_t t = 0;
+    int64_t launches = 0;
+    int last_cuda = 0;
+    int pending = 0;                       // workers stepped in the current iteration
+    std::vector<uint8_t> stepped;
+    std::vector<Tile> h_tiles;             // kept alive: source of an asynchronous upload
+    std::vector<Block> h_blocks;
+    // host-staging path
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_copied[2] = {nullptr, nullptr};
+    cudaEvent_t ev_free[2] = {nullptr, nullptr};
+    int64_t host_calls = 0;
+
+    float* x() const { return (float*)(ws + L.off_x); }
+    float* m(int i) const { return (float*)(ws + L.off_m) + (size_t)i * L.dpad; }
+    float* pb(int i) const {   // i == M: server
+        return i < L.M ? (float*)(ws + L.off_pb) + (size_t)i * L.dpad : (float*)(ws + L.off_spb);
+    }
+    uint32_t* words(int i) const { return (uint32_t*)(ws + L.off_words) + (size_t)i * L.wpad; }
+    float* scales(int i) const { return (float*)(ws + L.off_scales) + (size_t)i * L.bpad; }
+    float* rscale(int i) const { return (float*)(ws + L.off_rscale) + (size_t)i * L.bpad; }
+    double* partials(int i) const { return (double*)(ws + L.off_partials) + (size_t)i * L.tpad; }
+    unsigned* tickets(int i) const { return (unsigned*)(ws + L.off_tickets) + (size_t)i * L.bpad; }
+    const Tile* tiles() const { return (const Tile*)(ws + L.off_tiles); }
+    const Block* blocks() const { return (const Block*)(ws + L.off_blocks); }
+    float* stage(int s) const { return (float*)(ws + L.off_stage) + (size_t)s * L.dpad; }
+};
+
+namespace {
+
+int cuda_fail(ef_ctx* c, cudaError_t e) {
+    if (c) c->last_cuda = (int)e;
+    return EF_ERR_CUDA;
+}
+#define EF_CUDA(c, call)                                         \
+    do {                                                         \
+        cudaError_t e_ = (call);                                 \
+        if (e_ != cudaSuccess) return cuda_fail((c), e_);        \
+    } while (0)
+
+inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+int launch_worker(ef_ctx* c, int i, const float* grad) {
+    efk::WorkerArgs a;
+    a.g = grad; a.m = c->m(i); a.pb = c->pb(i); a.words = c->words(i);
+    a.scale_out = c->scales(i); a.rscale = c->rscale(i);
+    a.partials = c->partials(i); a.tickets = c->tickets(i);
+    a.tiles = c->tiles(); a.blocks = c->blocks(); a.mu = c->mu;
+    efk::ef_worker_kernel<kU><<<(unsigned)c->L.num_tiles, efk::kThreads, 0, c->stream>>>(a);
+    EF_CUDA(c, cudaGetLastError());
+    c->launches += 1;
+    return EF_OK;
+}
+
+template <int MT>
+void launch_server_t(ef_ctx* c, const efk::ServerArgs& a) {
+    efk::ef_server_kernel<kU, MT>
+        <<<(unsigned)c->L.num_tiles, efk::kThreads, (size_t)c->L.M * sizeof(float), c->stream>>>(a);
+}
+
+int launch_server(ef_ctx* c) {
+    const int M = c->L.M;
+    efk::ServerArgs a;
+    a.wwords = c->words(0); a.wstride = (long long)c->L.wpad;
+    a.wscales = c->scales(0); a.sstride = (int)c->L.bpad; a.M = M;
+    a.pb = c->pb(M); a.words = c->words(M); a.scale_out = c->scales(M); a.rscale = c->rscale(M);
+    a.partials = c->partials(M); a.tickets = c->tickets(M);
+    a.tiles = c->tiles(); a.blocks = c->blocks();
+    switch (M) {
+        case 1: launch_server_t<1>(c, a); break;
+        case 2: launch_server_t<2>(c, a); break;
+        case 4: launch_server_t<4>(c, a); break;
+        case 7: launch_server_t<7>(c, a); break;
+        case 8: launch_server_t<8>(c, a); break;
+        default: launch_server_t<0>(c, a); break;
+    }
+    EF_CUDA(c, cudaGetLastError());
+    efk::ApplyArgs p;
+    p.x = c->x(); p.words = c->words(M); p.scales = c->scales(M); p.tiles = c->tiles();
+    p.eta = c->eta;
+    efk::ef_apply_kernel<kU><<<(unsigned)c->L.num_tiles, efk::kThreads, 0, c->stream>>>(p);
+    EF_CUDA(c, cudaGetLastError());
+    c->launches += 2;
+    return EF_OK;
+}
+
+int check_worker_call(ef_ctx* c, int32_t i, const float* grad) {
+    if (!c || !grad || i < 0 || i >= c->L.M) return EF_ERR_INVALID_ARG;
+    if (c->stepped[i]) return EF_ERR_BAD_STATE;
+    return EF_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int ef_workspace_bytes(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_t flags,
+                       size_t* bytes) {
+    if (!bytes) return EF_ERR_INVALID_ARG;
+    Layout L;
+    const int rc = make_layout(d, B, offsets, M, flags, &L);
+    if (rc != EF_OK) return rc;
+    *bytes = L.total;
+    return EF_OK;
+}
+
+int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t M, float mu,
+            float eta, uint32_t flags, void* workspace, size_t workspace_bytes,
+            void* cuda_stream) {
+    if (!out) return EF_ERR_INVALID_ARG;
+    *out = nullptr;
+    Layout L;
+    int rc = make_layout(d, B, offsets, M, flags, &L);
+    if (rc != EF_OK) return rc;
+    if (!(mu >= 0.f && mu < 1.f)) return EF_ERR_INVALID_ARG;
+    if (!(eta > 0.f) || !std::isfinite(eta)) return EF_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < L.total) return EF_ERR_WORKSPACE;
+    if (((uintptr_t)workspace & (kAlign - 1)) != 0) return EF_ERR_ALIGNMENT;
+
+    int dev = -1;
+    cudaError_t ce = cudaGetDevice(&dev);
+    if (ce != cudaSuccess) return EF_ERR_CUDA;
+    int major = 0;
+    ce = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (ce != cudaSuccess) return EF_ERR_CUDA;
+    if (major != 10) return EF_ERR_UNSUPPORTED_DEVICE;
+
+    ef_ctx* c = new (std::nothrow) ef_ctx();
+    if (!c) return EF_ERR_INVALID_ARG;
+    c->L = L; c->mu = mu; c->eta = eta; c->flags = flags;
+    c->ws = (char*)workspace;
+    c->stream = (cudaStream_t)cuda_stream;
+    c->stepped.assign(M, 0);
+
+    // tile and block tables
+    c->h_tiles.reserve((size_t)L.num_tiles);
+    c->h_blocks.resize((size_t)B);
+    int64_t word = 0;
+    for (int32_t b = 0; b < B; ++b) {
+        const int64_t start = offsets[b], len = offsets[b + 1] - offsets[b];
+        Block& blk = c->h_blocks[b];
+        blk.start = start; blk.len = len; blk.word = word;
+        blk.tile_begin = (int)c->h_tiles.size();
+        for (int64_t o = 0; o < len; o += kTileLen) {
+            Tile t;
+            t.start = start + o; t.word = word + o / 32;
+            t.len = (int)((len - o < kTileLen) ? (len - o) : kTileLen);
+            t.block = b; t.pad0 = 0; t.pad1 = 0;
+            c->h_tiles.push_back(t);
+        }
+        blk.tile_count = (int)c->h_tiles.size() - blk.tile_begin;
+        word += (len + 31) / 32;
+    }
+
+    auto fail = [&](cudaError_t e) { delete c; (void)e; return EF_ERR_CUDA; };
+    // Algorithm 4 "Initialize": x_0, m, e, etilde = 0; also words, scales, tickets, partials.
+    if ((ce = cudaMemsetAsync(c->ws, 0, L.off_tiles, c->stream)) != cudaSuccess) return fail(ce);
+    if ((ce = cudaMemcpyAsync(c->ws + L.off_tiles, c->h_tiles.data(),
+                              c->h_tiles.size() * sizeof(Tile), cudaMemcpyHostToDevice,
+                              c->stream)) != cudaSuccess) return fail(ce);
+    if ((ce = cudaMemcpyAsync(c->ws + L.off_blocks, c->h_blocks.data(),
+                              c->h_blocks.size() * sizeof(Block), cudaMemcpyHostToDevice,
+                              c->stream)) != cudaSuccess) return fail(ce);
+    if (flags & EF_FLAG_HOST_STAGING) {
+        if ((ce = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking)) != cudaSuccess)
+            return fail(ce);
+        for (int s = 0; s < 2; ++s) {
+            if ((ce = cudaEventCreateWithFlags(&c->ev_copied[s], cudaEventDisableTiming)) != cudaSuccess ||
+                (ce = cudaEventCreateWithFlags(&c->ev_free[s], cudaEventDisableTiming)) != cudaSuccess) {
+                ef_destroy(c);
+                return EF_ERR_CUDA;
+            }
+        }
+    }
+    *out = c;
+    return EF_OK;
+}
+
+int ef_worker_step(ef_ctx* c, int32_t i, const float* grad) {
+    int rc = check_worker_call(c, i, grad);
+    if (rc != EF_OK) return rc;
+    if (!aligned16(grad)) return EF_ERR_ALIGNMENT;
+    rc = launch_worker(c, i, grad);
+    if (rc != EF_OK) return rc;
+    c->stepped[i] = 1; c->pending += 1;
+    return EF_OK;
+}
+
+int ef_worker_step_host(ef_ctx* c, int32_t i, const float* grad) {
+    int rc = check_worker_call(c, i, grad);
+    if (rc != EF_OK) return rc;
+    if (!(c->flags & EF_FLAG_HOST_STAGING)) return EF_ERR_BAD_STATE;
+    const int s = (int)(c->host_calls & 1);
+    // the staging slot is free once the kernel that last read it has finished
+    if (c->host_calls >= 2) EF_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->ev_free[s], 0));
+    EF_CUDA(c, cudaMemcpyAsync(c->stage(s), grad, (size_t)c->L.d * 4, cudaMemcpyHostToDevice,
+                               c->copy_stream));
+    EF_CUDA(c, cudaEventRecord(c->ev_copied[s], c->copy_stream));
+    EF_CUDA(c, cudaStreamWaitEvent(c->stream, c->ev_copied[s], 0));
+    rc = launch_worker(c, i, c->stage(s));
+    if (rc != EF_OK) return rc;
+    EF_CUDA(c, cudaEventRecord(c->ev_free[s], c->stream));
+    c->host_calls += 1;
+    c->stepped[i] = 1; c->pending += 1;
+    return EF_OK;
+}
+
+int ef_server_step(ef_ctx* c) {
+    if (!c) return EF_ERR_INVALID_ARG;
+    if (c->pending != c->L.M) return EF_ERR_BAD_STATE;
+    const int rc = launch_server(c);
+    if (rc != EF_OK) return rc;
+    std::fill(c->stepped.begin(), c->stepped.end(), (uint8_t)0);
+    c->pending = 0;
+    c->t += 1;
+    return EF_OK;
+}
+
+int ef_read_update_host(ef_ctx* c, uint32_t* words, float* scales) {
+    if (!c || !words || !scales) return EF_ERR_INVALID_ARG;
+    const int M = c->L.M;
+    EF_CUDA(c, cudaMemcpyAsync(words, c->words(M), (size_t)c->L.W * 4, cudaMemcpyDeviceToHost,
+                               c->stream));
+    EF_CUDA(c, cudaMemcpyAsync(scales, c->scales(M), (size_t)c->L.B * 4, cudaMemcpyDeviceToHost,
+                               c->stream));
+    return EF_OK;
+}
+
+const uint32_t* ef_worker_words(ef_ctx* c, int32_t i) {
+    return (c && i >= 0 && i < c->L.M) ? c->words(i) : nullptr;
+}
+const float* ef_worker_scales(ef_ctx* c, int32_t i) {
+    return (c && i >= 0 && i < c->L.M) ? c->scales(i) : nullptr;
+}
+const uint32_t* ef_server_words(ef_ctx* c) { return c ? c->words(c->L.M) : nullptr; }
+const float* ef_server_scales(ef_ctx* c) { return c ? c->scales(c->L.M) : nullptr; }
+float* ef_params(ef_ctx* c) { return c ? c->x() : nullptr; }
+int64_t ef_num_words(ef_ctx* c) { return c ? c->L.W : -1; }
+
+int ef_get_momentum(ef_ctx* c, int32_t i, float* dst) {
+    if (!c || !dst || i < 0 || i >= c->L.M) return EF_ERR_INVALID_ARG;
+    if (!aligned16(dst)) return EF_ERR_ALIGNMENT;
+    EF_CUDA(c, cudaMemcpyAsync(dst, c->m(i), (size_t)c->L.d * 4, cudaMemcpyDeviceToDevice,
+                               c->stream));
+    return EF_OK;
+}
+
+int ef_get_residual(ef_ctx* c, int32_t i, float* dst) {
+    if (!c || !dst || i < -1 || i >= c->L.M) return EF_ERR_INVALID_ARG;
+    if (!aligned16(dst)) return EF_ERR_ALIGNMENT;
+    const int k = (i < 0) ? c->L.M : i;
+    efk::ResidualArgs a;
+    a.pb = c->pb(k); a.rscale = c->rscale(k); a.dst = dst; a.tiles = c->tiles();
+    efk::ef_residual_kernel<kU><<<(unsigned)c->L.num_tiles, efk::kThreads, 0, c->stream>>>(a);
+    EF_CUDA(c, cudaGetLastError());
+    c->launches += 1;
+    return EF_OK;
+}
+
+int ef_set_state(ef_ctx* c, int32_t i, const float* momentum, const float* residual) {
+    if (!c || !residual || i < -1 || i >= c->L.M) return EF_ERR_INVALID_ARG;
+    if (i >= 0 && !momentum) return EF_ERR_INVALID_ARG;
+    if (!aligned16(residual) || (momentum && !aligned16(momentum))) return EF_ERR_ALIGNMENT;
+    if (c->pending != 0) return EF_ERR_BAD_STATE;
+    const int k = (i < 0) ? c->L.M : i;
+    const size_t nbytes = (size_t)c->L.d * 4;
+    if (i >= 0)
+        EF_CUDA(c, cudaMemcpyAsync(c->m(i), momentum, nbytes, cudaMemcpyDeviceToDevice, c->stream));
+    // deferred form with scale 0: p -+ 0 gives back the residual exactly
+    EF_CUDA(c, cudaMemcpyAsync(c->pb(k), residual, nbytes, cudaMemcpyDeviceToDevice, c->stream));
+    EF_CUDA(c, cudaMemsetAsync(c->rscale(k), 0, (size_t)c->L.B * 4, c->stream));
+    return EF_OK;
+}
+
+int ef_step_count(ef_ctx* c, int64_t* t) {
+    if (!c || !t) return EF_ERR_INVALID_ARG;
+    *t = c->t;
+    return EF_OK;
+}
+
+int64_t ef_launch_count(ef_ctx* c) { return c ? c->launches : -1; }
+
+const char* ef_strerror(int status) {
+    switch (status) {
+        case EF_OK: return "ok";
+        case EF_ERR_INVALID_ARG: return "invalid argument";
+        case EF_ERR_BAD_STATE: return "call order violated";
+        case EF_ERR_WORKSPACE: return "workspace missing or too small";
+        case EF_ERR_ALIGNMENT: return "pointer not sufficiently aligned";
+        case EF_ERR_CUDA: return "CUDA runtime error";
+        case EF_ERR_UNSUPPORTED_DEVICE: return "device is not compute capability 10.x";
+        case EF_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+int ef_last_cuda_error(ef_ctx* c) { return c ? c->last_cuda : 0; }
+
+int ef_destroy(ef_ctx* c) {
+    if (!c) return EF_OK;
+    for (int s = 0; s < 2; ++s) {
+        if (c->ev_copied[s]) cudaEventDestroy(c->ev_copied[s]);
+        if (c->ev_free[s]) cudaEventDestroy(c->ev_free[s]);
+    }
+    if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+    delete c;
+    return EF_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,113 @@
+"""Convenience holder around the C-ABI context: owns the torch workspace tensor and exposes
+the device views as torch tensors.  No arithmetic of the method happens here."""
+from __future__ import annotations
+
+import ctypes
+from typing import Optional
+
+import numpy as np
+import torch
+
+from . import binding as ef
+
+
+def _as_tensor(ptr: int, n: int, dtype: torch.dtype, device: torch.device) -> torch.Tensor:
+    """Zero-copy torch view of `n` elements of device memory at `ptr`."""
+    itemsize = torch.empty((), dtype=dtype).element_size()
+
+    class _Holder:
+        __cuda_array_interface__ = {
+            "shape": (n,), "typestr": {torch.float32: "<f4", torch.int32: "<i4"}[dtype],
+            "data": (ptr, False), "version": 3, "strides": (itemsize,),
+        }
+    return torch.as_tensor(_Holder(), device=device)
+
+
+class EFEngine:
+    """One dist-EF-blockSGDM problem on the current CUDA device."""
+
+    def __init__(self, offsets, M: int, mu: float, eta: float, host_staging: bool = False,
+                 stream: Optional[torch.cuda.Stream] = None, device: Optional[torch.device] = None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("EFEngine needs a CUDA device (there is no CPU path)")
+        self.device = torch.device(device if device is not None else f"cuda:{torch.cuda.current_device()}")
+        self.offsets = np.ascontiguousarray(offsets, dtype=np.int64)
+        self.B = len(self.offsets) - 1
+        self.d = int(self.offsets[-1])
+        self.M = int(M)
+        flags = ef.EF_FLAG_HOST_STAGING if host_staging else 0
+        nbytes = ef.ef_workspace_bytes(self.d, self.B, self.offsets, self.M, flags)
+        self.workspace_bytes = nbytes
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            self.stream = stream if stream is not None else torch.cuda.current_stream()
+            self.ctx = ef.ef_init(self.d, self.B, self.offsets, self.M, float(mu), float(eta), flags,
+                                  self.workspace.data_ptr(), nbytes, self.stream.cuda_stream)
+        self.W = ef.ef_num_words(self.ctx)
+
+    def close(self):
+        if getattr(self, "ctx", None):
+            ef.ef_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- steps ------------------------------------------------------------------------------
+    def worker_step(self, i: int, grad: torch.Tensor) -> None:
+        assert grad.is_cuda and grad.dtype == torch.float32 and grad.numel() == self.d
+        assert grad.is_contiguous()
+        ef.ef_worker_step(self.ctx, i, grad.data_ptr())
+
+    def worker_step_host(self, i: int, grad: torch.Tensor) -> None:
+        assert (not grad.is_cuda) and grad.dtype == torch.float32 and grad.numel() == self.d
+        assert grad.is_contiguous()
+        ef.ef_worker_step_host(self.ctx, i, grad.data_ptr())
+
+    def server_step(self) -> None:
+        ef.ef_server_step(self.ctx)
+
+    def read_update_host(self, words: torch.Tensor, scales: torch.Tensor) -> None:
+        assert words.numel() == self.W and scales.numel() == self.B
+        ef.ef_read_update_host(self.ctx, words.data_ptr(), scales.data_ptr())
+
+    # ---- views ------------------------------------------------------------------------------
+    def worker_words(self, i: int) -> torch.Tensor:
+        return _as_tensor(ef.ef_worker_words(self.ctx, i), self.W, torch.int32, self.device)
+
+    def worker_scales(self, i: int) -> torch.Tensor:
+        return _as_tensor(ef.ef_worker_scales(self.ctx, i), self.B, torch.float32, self.device)
+
+    def server_words(self) -> torch.Tensor:
+        return _as_tensor(ef.ef_server_words(self.ctx), self.W, torch.int32, self.device)
+
+    def server_scales(self) -> torch.Tensor:
+        return _as_tensor(ef.ef_server_scales(self.ctx), self.B, torch.float32, self.device)
+
+    def params(self) -> torch.Tensor:
+        return _as_tensor(ef.ef_params(self.ctx), self.d, torch.float32, self.device)
+
+    def momentum(self, i: int) -> torch.Tensor:
+        out = torch.empty(self.d, dtype=torch.float32, device=self.device)
+        ef.ef_get_momentum(self.ctx, i, out.data_ptr())
+        return out
+
+    def residual(self, i: int = -1) -> torch.Tensor:
+        out = torch.empty(self.d, dtype=torch.float32, device=self.device)
+        ef.ef_get_residual(self.ctx, i, out.data_ptr())
+        return out
+
+    def set_state(self, i: int, momentum: Optional[torch.Tensor], residual: torch.Tensor) -> None:
+        ef.ef_set_state(self.ctx, i, momentum.data_ptr() if momentum is not None else None,
+                        residual.data_ptr())
+
+    @property
+    def step_count(self) -> int:
+        return ef.ef_step_count(self.ctx)
+
+    @property
+    def launch_count(self) -> int:
+        return ef.ef_launch_count(self.ctx)

@@ -1,0 +1,213 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_1905_10936_b200 import binding as ef
+from paper_1905_10936_b200 import workloads as wl
+from paper_1905_10936_b200.engine import EFEngine
+from parity import run_parity, BlockSample, compare_state, words_np
+
+pytestmark = pytest.mark.gpu
+
+TILE = 4096   # elements per tile of the library build (1024 * rows per thread)
+
+
+def _wl(name, sizes, M, mu=0.9, eta=0.1, steps=5, law="normal", scale_range=None, cid=50):
+    return wl.custom_workload(name, sizes, M, mu, eta, steps, law, scale_range, config_id=cid)
+
+
+# ------------------------------------------------------------------ small and ragged layouts
+@pytest.mark.parametrize("sizes,M", [
+    ([4], 1), ([1], 2), ([2, 2], 2), ([64], 3),
+    ([1] * 50, 4),                                   # identity compressor: d_b = 1
+    ([10, 32, 458, 500], 1),                         # M = 1: server repeats the worker message
+    ([3, 5, 31, 33, 63, 65, 127, 129], 3),           # unaligned block starts: scalar path
+    ([40, 64, 5, 300, 7, 1000, 13], 5),              # mixed aligned / unaligned
+    ([TILE], 2), ([TILE - 1], 2), ([TILE + 1], 2), ([TILE - 4, 8, TILE + 4], 7),
+    ([2 * TILE, TILE // 2, 3 * TILE + 36, 100], 8),  # several tiles per block + ragged tails
+    ([5 * TILE + 2, 3, 2 * TILE + 1, 4 * TILE], 2),  # multi-tile blocks on the scalar path
+    ([1000] * 40, 16), ([12345, 54321, 99999], 9),   # generic-M server path
+])
+def test_small_layouts(sizes, M):
+    w = _wl("small", sizes, M, steps=6)
+    eng, orc, stats = run_parity(w)
+    assert stats["adopted"] <= 2
+
+
+@pytest.mark.parametrize("mu,eta", [(0.0, 0.1), (0.5, 1.0), (0.99, 1e-3)])
+def test_hyper_parameters(mu, eta):
+    w = _wl("hp", [TILE + 100, 777, 2 * TILE], 3, mu=mu, eta=eta, steps=6, scale_range=(1e-3, 1.0))
+    run_parity(w)
+
+
+def test_zero_gradients_and_zero_blocks():
+    """All-zero blocks: scale 0, every bit 0, state stays 0 (sign(0) = +1)."""
+    w = _wl("zeros", [100, TILE, 64], 2, steps=3)
+    z = torch.zeros(w.d)
+    g = torch.randn(w.d); g[100:100 + TILE] = 0
+    grads = [[z, z], [g, g.flip(0) * 0 + g], [z, z]]
+    eng, orc, _ = run_parity(w, grads=grads)
+    assert eng.worker_scales(0)[1].item() == 0.0
+
+
+def test_worker_order_does_not_matter():
+    w = _wl("order", [TILE + 5, 333], 4, steps=3)
+    es = None
+    a = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    b = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    for t in range(3):
+        gs = [w.draw_grad(t, i, "cuda") for i in range(w.M)]
+        for i in range(w.M):
+            a.worker_step(i, gs[i])
+        for i in reversed(range(w.M)):
+            b.worker_step(i, gs[i])
+        a.server_step(); b.server_step()
+    assert torch.equal(a.params(), b.params())
+    assert torch.equal(a.server_words(), b.server_words())
+    assert torch.equal(a.residual(-1), b.residual(-1))
+
+
+def test_runs_are_deterministic():
+    w = wl.make_workload(2)
+    outs = []
+    for rep in range(2):
+        e = EFEngine(w.offsets, w.M, w.mu, w.eta)
+        es = w.element_scales("cuda")
+        for t in range(3):
+            for i in range(w.M):
+                e.worker_step(i, w.draw_grad(t, i, "cuda", es))
+            e.server_step()
+        outs.append((e.params().clone(), e.server_words().clone(), e.server_scales().clone(),
+                     e.residual(0)))
+    for x, y in zip(*outs):
+        assert torch.equal(x, y)
+
+
+# ------------------------------------------------------------------ benchmark configurations
+def test_config1_flat_2_20():
+    w = wl.make_workload(1)
+    eng, orc, stats = run_parity(w)
+    assert stats["scale_bit_mismatch"] <= 1
+
+
+def test_config2_resnet20_layout():
+    w = wl.make_workload(2)
+    eng, orc, stats = run_parity(w)
+    assert stats["scale_bit_mismatch"] <= 2
+
+
+def test_config3_resnet50_layout():
+    w = wl.make_workload(3)
+    run_parity(w, check_every_step=False)
+
+
+def test_config4_flat_2_28_sampled_blocks():
+    """Full-size launch (d = 2^28, M = 7, 20 steps); the oracle follows 6 of the 256 blocks."""
+    w = wl.make_workload(4)
+    run_parity(w, blocks=[0, 1, 100, 127, 128, 255], check_every_step=False)
+
+
+def test_config5_gpt2_layout_sampled_blocks():
+    """Full-size launch; the oracle follows the embedding block (51M elements, 12.5k tiles),
+    the position table and one whole transformer layer, plus the last block."""
+    w = wl.make_workload(5)
+    layer7 = list(range(2 + 12 * 7, 2 + 12 * 8))
+    run_parity(w, blocks=[0, 1] + layer7 + [w.B - 1], check_every_step=False)
+
+
+# ------------------------------------------------------------------ state access / checkpoint
+def test_checkpoint_roundtrip_is_bit_exact():
+    """5 steps, export (x, m_i, e_i, etilde), import into a fresh context, 5 more steps:
+    identical to 10 straight steps."""
+    w = _wl("ckpt", [TILE + 37, 640, 3 * TILE], 3, steps=10, scale_range=(1e-2, 1.0))
+    es = w.element_scales("cuda")
+    a = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    b = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    for t in range(5):
+        for i in range(w.M):
+            a.worker_step(i, w.draw_grad(t, i, "cuda", es))
+        a.server_step()
+    b.params().copy_(a.params())
+    for i in range(w.M):
+        b.set_state(i, a.momentum(i), a.residual(i))
+    b.set_state(-1, None, a.residual(-1))
+    for t in range(5, 10):
+        for i in range(w.M):
+            g = w.draw_grad(t, i, "cuda", es)
+            a.worker_step(i, g); b.worker_step(i, g)
+        a.server_step(); b.server_step()
+    assert torch.equal(a.params(), b.params())
+    assert torch.equal(a.server_words(), b.server_words())
+    assert torch.equal(a.server_scales(), b.server_scales())
+    for i in range(-1, w.M):
+        assert torch.equal(a.residual(i), b.residual(i))
+
+
+def test_caller_may_set_initial_parameters():
+    w = _wl("x0", [500, TILE], 2, steps=2)
+    x0 = torch.randn(w.d, device="cuda")
+    a = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    b = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    b.params().copy_(x0)
+    for t in range(2):
+        for i in range(w.M):
+            g = w.draw_grad(t, i, "cuda")
+            a.worker_step(i, g); b.worker_step(i, g)
+        a.server_step(); b.server_step()
+    # the update is independent of x: x_T - x_0 is the same up to rounding of the adds
+    assert torch.allclose(b.params() - x0, a.params(), rtol=0, atol=1e-6)
+
+
+# ------------------------------------------------------------------ host-buffer entry points
+def test_host_staging_path_matches_device_path():
+    w = _wl("host", [TILE * 3 + 11, 100, TILE], 3, steps=4)
+    a = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    b = EFEngine(w.offsets, w.M, w.mu, w.eta, host_staging=True)
+    words = torch.empty(b.W, dtype=torch.int32).pin_memory()
+    scales = torch.empty(b.B, dtype=torch.float32).pin_memory()
+    for t in range(4):
+        hs = [w.draw_grad(t, i, "cpu").pin_memory() for i in range(w.M)]
+        for i in range(w.M):
+            a.worker_step(i, hs[i].cuda())
+            b.worker_step_host(i, hs[i])
+        a.server_step(); b.server_step()
+        b.read_update_host(words, scales)
+        torch.cuda.synchronize()
+        assert torch.equal(words, a.server_words().cpu())
+        assert torch.equal(scales, a.server_scales().cpu())
+    assert torch.equal(a.params(), b.params())
+
+
+# ------------------------------------------------------------------ error paths on a device
+def test_error_paths_on_device():
+    w = _wl("err", [64, 64], 2)
+    e = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    g = torch.zeros(w.d + 4, device="cuda")
+    with pytest.raises(ef.EFError) as ei:
+        ef.ef_worker_step(e.ctx, 0, g.data_ptr() + 4)
+    assert ei.value.status == ef.EF_ERR_ALIGNMENT
+    with pytest.raises(ef.EFError) as ei:
+        ef.ef_server_step(e.ctx)
+    assert ei.value.status == ef.EF_ERR_BAD_STATE
+    ef.ef_worker_step(e.ctx, 1, g.data_ptr())
+    with pytest.raises(ef.EFError) as ei:
+        ef.ef_worker_step(e.ctx, 1, g.data_ptr())
+    assert ei.value.status == ef.EF_ERR_BAD_STATE
+    with pytest.raises(ef.EFError) as ei:
+        ef.ef_worker_step(e.ctx, 2, g.data_ptr())
+    assert ei.value.status == ef.EF_ERR_INVALID_ARG
+    with pytest.raises(ef.EFError) as ei:
+        ef.ef_worker_step_host(e.ctx, 0, g.data_ptr())
+    assert ei.value.status == ef.EF_ERR_BAD_STATE          # no staging buffers requested
+    with pytest.raises(ef.EFError) as ei:
+        e.set_state(0, g[:w.d], g[:w.d])
+    assert ei.value.status == ef.EF_ERR_BAD_STATE          # in the middle of an iteration
+    ef.ef_worker_step(e.ctx, 0, g.data_ptr())
+    ef.ef_server_step(e.ctx)
+    assert e.step_count == 1 and e.launch_count == 4
+    ws = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(ef.EFError) as ei:
+        ef.ef_init(w.d, w.B, w.offsets, w.M, 0.9, 0.1, 0, ws.data_ptr(), 1024, 0)
+    assert ei.value.status == ef.EF_ERR_WORKSPACE
+    torch.cuda.synchronize()
