@@ -49,6 +49,12 @@ enum ef_status {
 
 /* Flags for ef_workspace_bytes / ef_init. */
 #define EF_FLAG_HOST_STAGING 1u    /* reserve two d-float staging buffers for ef_worker_step_host */
+/* How the per-block L1 sums of blocks larger than one tile are completed.  By default the
+ * library chooses: inside the main kernels for small (launch-bound) problems, in a tiny
+ * follow-up kernel for large (bandwidth-bound) ones.  Both give bit-identical scales.  At
+ * most one of the two flags may be set. */
+#define EF_FLAG_FUSED_SCALE 2u     /* always complete the sums inside the main kernels */
+#define EF_FLAG_SPLIT_SCALE 4u     /* always use the follow-up kernel */
 
 /* Maximum number of simulated workers. */
 #define EF_MAX_WORKERS 4096

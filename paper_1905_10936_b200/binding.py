@@ -25,6 +25,8 @@ EF_ERR_CUDA = 5
 EF_ERR_UNSUPPORTED_DEVICE = 6
 EF_ERR_TIMEOUT = 7
 EF_FLAG_HOST_STAGING = 1
+EF_FLAG_FUSED_SCALE = 2
+EF_FLAG_SPLIT_SCALE = 4
 EF_MAX_WORKERS = 4096
 
 _vp, _i64, _i32, _u32, _f32 = (ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_uint32,

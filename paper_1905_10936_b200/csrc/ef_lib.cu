@@ -21,6 +21,8 @@ inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a
 // Rows of four elements per thread and tile; a tile is 1024*U elements.
 constexpr int kU = 4;
 constexpr int kTileLen = 1024 * kU;
+// Grids up to this many tiles (about two waves of CTAs) finalise block scales in-kernel.
+constexpr int64_t kFusedMaxTiles = 1024;
 
 struct Layout {
     int64_t d = 0, W = 0;
@@ -29,7 +31,8 @@ struct Layout {
     size_t dpad = 0, wpad = 0, bpad = 0, tpad = 0;    // padded element counts per sub-buffer
     size_t off_x = 0, off_m = 0, off_pb = 0, off_spb = 0, off_words = 0, off_scales = 0,
            off_rscale = 0, off_partials = 0, off_tickets = 0, off_tiles = 0, off_blocks = 0,
-           off_stage = 0, total = 0;
+           off_multi = 0, off_stage = 0, total = 0;
+    int32_t num_multi = 0;                            // blocks that span more than one tile
 };
 
 int check_problem(int64_t d, int32_t B, const int64_t* offsets, int32_t M) {
@@ -44,13 +47,16 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
                 Layout* L) {
     int rc = check_problem(d, B, offsets, M);
     if (rc != EF_OK) return rc;
-    if (flags & ~EF_FLAG_HOST_STAGING) return EF_ERR_INVALID_ARG;
+    if (flags & ~(EF_FLAG_HOST_STAGING | EF_FLAG_FUSED_SCALE | EF_FLAG_SPLIT_SCALE))
+        return EF_ERR_INVALID_ARG;
+    if ((flags & EF_FLAG_FUSED_SCALE) && (flags & EF_FLAG_SPLIT_SCALE)) return EF_ERR_INVALID_ARG;
     L->d = d; L->B = B; L->M = M;
     int64_t W = 0, T = 0;
     for (int32_t b = 0; b < B; ++b) {
         const int64_t db = offsets[b + 1] - offsets[b];
         W += (db + 31) / 32;
         T += (db + kTileLen - 1) / kTileLen;
+        if (db > kTileLen) L->num_multi += 1;
     }
     if (T > 0x7fffffffLL) return EF_ERR_INVALID_ARG;
     L->W = W; L->num_tiles = T;
@@ -71,6 +77,7 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
     L->off_tickets = o;  o += M1 * L->bpad * 4;
     L->off_tiles = o;    o += align_up((size_t)T * sizeof(Tile));
     L->off_blocks = o;   o += align_up((size_t)B * sizeof(Block));
+    L->off_multi = o;    o += align_up((size_t)L->num_multi * sizeof(int32_t) + 4);
     L->off_stage = o;
     if (flags & EF_FLAG_HOST_STAGING) o += 2 * L->dpad * 4;
     L->total = o;
@@ -92,6 +99,8 @@ struct ef_ctx {
     std::vector<uint8_t> stepped;
     std::vector<Tile> h_tiles;             // kept alive: source of an asynchronous upload
     std::vector<Block> h_blocks;
+    std::vector<int32_t> h_multi;
+    int fused = 0;                         // block scales finalised inside the main kernels
     // host-staging path
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t ev_copied[2] = {nullptr, nullptr};
@@ -110,6 +119,7 @@ struct ef_ctx {
     unsigned* tickets(int i) const { return (unsigned*)(ws + L.off_tickets) + (size_t)i * L.bpad; }
     const Tile* tiles() const { return (const Tile*)(ws + L.off_tiles); }
     const Block* blocks() const { return (const Block*)(ws + L.off_blocks); }
+    const int* multi() const { return (const int*)(ws + L.off_multi); }
     float* stage(int s) const { return (float*)(ws + L.off_stage) + (size_t)s * L.dpad; }
 };
 
@@ -127,16 +137,29 @@ int cuda_fail(ef_ctx* c, cudaError_t e) {
 
 inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
+// Non-fused mode: adds the per-tile partial sums of every multi-tile block of buffer set k
+// (worker k, or the server for k == M) after the kernel that produced them.
+int launch_scale(ef_ctx* c, int k) {
+    if (c->fused || c->L.num_multi == 0) return EF_OK;
+    efk::ScaleArgs a;
+    a.partials = c->partials(k); a.blocks = c->blocks(); a.multi = c->multi();
+    a.scale_out = c->scales(k); a.rscale = c->rscale(k);
+    efk::ef_scale_kernel<<<(unsigned)c->L.num_multi, efk::kThreads, 0, c->stream>>>(a);
+    EF_CUDA(c, cudaGetLastError());
+    c->launches += 1;
+    return EF_OK;
+}
+
 int launch_worker(ef_ctx* c, int i, const float* grad) {
     efk::WorkerArgs a;
     a.g = grad; a.m = c->m(i); a.pb = c->pb(i); a.words = c->words(i);
     a.scale_out = c->scales(i); a.rscale = c->rscale(i);
     a.partials = c->partials(i); a.tickets = c->tickets(i);
-    a.tiles = c->tiles(); a.blocks = c->blocks(); a.mu = c->mu;
+    a.tiles = c->tiles(); a.blocks = c->blocks(); a.mu = c->mu; a.fused = c->fused;
     efk::ef_worker_kernel<kU><<<(unsigned)c->L.num_tiles, efk::kThreads, 0, c->stream>>>(a);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
-    return EF_OK;
+    return launch_scale(c, i);
 }
 
 template <int MT>
@@ -152,22 +175,30 @@ int launch_server(ef_ctx* c) {
     a.wscales = c->scales(0); a.sstride = (int)c->L.bpad; a.M = M;
     a.pb = c->pb(M); a.words = c->words(M); a.scale_out = c->scales(M); a.rscale = c->rscale(M);
     a.partials = c->partials(M); a.tickets = c->tickets(M);
-    a.tiles = c->tiles(); a.blocks = c->blocks();
+    a.tiles = c->tiles(); a.blocks = c->blocks(); a.fused = c->fused;
     switch (M) {
         case 1: launch_server_t<1>(c, a); break;
         case 2: launch_server_t<2>(c, a); break;
+        case 3: launch_server_t<3>(c, a); break;
         case 4: launch_server_t<4>(c, a); break;
+        case 5: launch_server_t<5>(c, a); break;
+        case 6: launch_server_t<6>(c, a); break;
         case 7: launch_server_t<7>(c, a); break;
         case 8: launch_server_t<8>(c, a); break;
         default: launch_server_t<0>(c, a); break;
     }
     EF_CUDA(c, cudaGetLastError());
+    c->launches += 1;
+    {
+        const int rc = launch_scale(c, M);
+        if (rc != EF_OK) return rc;
+    }
     efk::ApplyArgs p;
     p.x = c->x(); p.words = c->words(M); p.scales = c->scales(M); p.tiles = c->tiles();
     p.eta = c->eta;
     efk::ef_apply_kernel<kU><<<(unsigned)c->L.num_tiles, efk::kThreads, 0, c->stream>>>(p);
     EF_CUDA(c, cudaGetLastError());
-    c->launches += 2;
+    c->launches += 1;
     return EF_OK;
 }
 
@@ -236,8 +267,14 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
             c->h_tiles.push_back(t);
         }
         blk.tile_count = (int)c->h_tiles.size() - blk.tile_begin;
+        if (blk.tile_count > 1) c->h_multi.push_back(b);
         word += (len + 31) / 32;
     }
+    // Small grids are launch-bound: finish block scales inside the main kernels.  Large grids
+    // are bandwidth-bound: the per-CTA fence of the fused form costs more than a tiny launch.
+    if (flags & EF_FLAG_FUSED_SCALE) c->fused = 1;
+    else if (flags & EF_FLAG_SPLIT_SCALE) c->fused = 0;
+    else c->fused = (L.num_tiles <= kFusedMaxTiles) ? 1 : 0;
 
     auto fail = [&](cudaError_t e) { delete c; (void)e; return EF_ERR_CUDA; };
     // Algorithm 4 "Initialize": x_0, m, e, etilde = 0; also words, scales, tickets, partials.
@@ -247,6 +284,10 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
                               c->stream)) != cudaSuccess) return fail(ce);
     if ((ce = cudaMemcpyAsync(c->ws + L.off_blocks, c->h_blocks.data(),
                               c->h_blocks.size() * sizeof(Block), cudaMemcpyHostToDevice,
+                              c->stream)) != cudaSuccess) return fail(ce);
+    if (!c->h_multi.empty() &&
+        (ce = cudaMemcpyAsync(c->ws + L.off_multi, c->h_multi.data(),
+                              c->h_multi.size() * sizeof(int32_t), cudaMemcpyHostToDevice,
                               c->stream)) != cudaSuccess) return fail(ce);
     if (flags & EF_FLAG_HOST_STAGING) {
         if ((ce = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking)) != cudaSuccess)

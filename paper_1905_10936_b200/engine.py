@@ -27,7 +27,7 @@ class EFEngine:
     """One dist-EF-blockSGDM problem on the current CUDA device."""
 
     def __init__(self, offsets, M: int, mu: float, eta: float, host_staging: bool = False,
-                 stream: Optional[torch.cuda.Stream] = None, device: Optional[torch.device] = None):
+                 scale_mode: str = "auto", stream: Optional[torch.cuda.Stream] = None, device: Optional[torch.device] = None):
         if not torch.cuda.is_available():
             raise RuntimeError("EFEngine needs a CUDA device (there is no CPU path)")
         self.device = torch.device(device if device is not None else f"cuda:{torch.cuda.current_device()}")
@@ -36,6 +36,7 @@ class EFEngine:
         self.d = int(self.offsets[-1])
         self.M = int(M)
         flags = ef.EF_FLAG_HOST_STAGING if host_staging else 0
+        flags |= {"auto": 0, "fused": ef.EF_FLAG_FUSED_SCALE, "split": ef.EF_FLAG_SPLIT_SCALE}[scale_mode]
         nbytes = ef.ef_workspace_bytes(self.d, self.B, self.offsets, self.M, flags)
         self.workspace_bytes = nbytes
         with torch.cuda.device(self.device):

@@ -81,10 +81,10 @@ def assert_scales_close(got: np.ndarray, ref: np.ndarray, what: str):
 
 def run_parity(w: Workload, steps: Optional[int] = None, blocks: Optional[Sequence[int]] = None,
                grads: Optional[List[List[torch.Tensor]]] = None, check_every_step: bool = True,
-               device: str = "cuda"):
+               device: str = "cuda", scale_mode: str = "auto"):
     """Runs `steps` iterations on both sides; returns (engine, oracle, stats)."""
     steps = w.steps if steps is None else steps
-    eng = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    eng = EFEngine(w.offsets, w.M, w.mu, w.eta, scale_mode=scale_mode)
     smp = BlockSample(w.offsets, blocks)
     orc = Oracle(smp.sub_offsets, w.M, w.mu, w.eta)
     es = w.element_scales(device)

@@ -29,9 +29,10 @@ def _wl(name, sizes, M, mu=0.9, eta=0.1, steps=5, law="normal", scale_range=None
     ([5 * TILE + 2, 3, 2 * TILE + 1, 4 * TILE], 2),  # multi-tile blocks on the scalar path
     ([1000] * 40, 16), ([12345, 54321, 99999], 9),   # generic-M server path
 ])
-def test_small_layouts(sizes, M):
+@pytest.mark.parametrize("scale_mode", ["fused", "split"])
+def test_small_layouts(sizes, M, scale_mode):
     w = _wl("small", sizes, M, steps=6)
-    eng, orc, stats = run_parity(w)
+    eng, orc, stats = run_parity(w, scale_mode=scale_mode)
     assert stats["adopted"] <= 2
 
 
@@ -68,11 +69,11 @@ def test_worker_order_does_not_matter():
     assert torch.equal(a.residual(-1), b.residual(-1))
 
 
-def test_runs_are_deterministic():
+def test_runs_are_deterministic_and_scale_modes_agree():
     w = wl.make_workload(2)
     outs = []
-    for rep in range(2):
-        e = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    for mode in ("fused", "fused", "split"):
+        e = EFEngine(w.offsets, w.M, w.mu, w.eta, scale_mode=mode)
         es = w.element_scales("cuda")
         for t in range(3):
             for i in range(w.M):
@@ -80,8 +81,9 @@ def test_runs_are_deterministic():
             e.server_step()
         outs.append((e.params().clone(), e.server_words().clone(), e.server_scales().clone(),
                      e.residual(0)))
-    for x, y in zip(*outs):
-        assert torch.equal(x, y)
+    for other in outs[1:]:
+        for x, y in zip(outs[0], other):
+            assert torch.equal(x, y)
 
 
 # ------------------------------------------------------------------ benchmark configurations
@@ -100,6 +102,11 @@ def test_config2_resnet20_layout():
 def test_config3_resnet50_layout():
     w = wl.make_workload(3)
     run_parity(w, check_every_step=False)
+
+
+def test_config3_fused_scale_mode():
+    w = wl.make_workload(3)
+    run_parity(w, steps=3, check_every_step=False, scale_mode="fused")
 
 
 def test_config4_flat_2_28_sampled_blocks():
@@ -205,7 +212,7 @@ def test_error_paths_on_device():
     assert ei.value.status == ef.EF_ERR_BAD_STATE          # in the middle of an iteration
     ef.ef_worker_step(e.ctx, 0, g.data_ptr())
     ef.ef_server_step(e.ctx)
-    assert e.step_count == 1 and e.launch_count == 4
+    assert e.step_count == 1 and e.launch_count == 4      # 2 worker + server + apply kernels
     ws = torch.empty(1024, dtype=torch.uint8, device="cuda")
     with pytest.raises(ef.EFError) as ei:
         ef.ef_init(w.d, w.B, w.offsets, w.M, 0.9, 0.1, 0, ws.data_ptr(), 1024, 0)
