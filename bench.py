@@ -153,7 +153,7 @@ def run_reference(args) -> None:
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    w = wl.make_workload(args.config)
+    w = load_workload(args)
     budget_s = 90.0
     per_block = np.mean(w.sizes) * oracle_ns_per_param(w.M) * 1e-9
     n_blocks = int(max(1, min(w.B, budget_s / ((args.steps + args.warmup) * per_block))))
@@ -195,7 +195,7 @@ def run_ours(args) -> None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    w = wl.make_workload(args.config)
+    w = load_workload(args)
     K, W = args.steps, args.warmup
     eng = EFEngine(w.offsets, w.M, w.mu, w.eta)
     es = w.element_scales(dev)
@@ -338,12 +338,22 @@ def eng_state_gib(w: wl.Workload) -> float:
     return (w.d * 4.0 * (2 * w.M + 2) + w.d * 4.0 * w.M) / 2 ** 30
 
 
+def load_workload(args) -> wl.Workload:
+    w = wl.make_workload(args.config)
+    if args.blocks and args.blocks < w.B:
+        w = wl.custom_workload(f"{w.name}-first{args.blocks}blocks", w.sizes[:args.blocks], w.M,
+                               w.mu, w.eta, w.steps, w.law, w.scale_range, config_id=w.config_id)
+    return w
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=4, help="workload 1..5 (default: flat 2^28)")
+    ap.add_argument("--blocks", type=int, default=0,
+                    help="use only the first N blocks of the workload (small cases for profiling)")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")

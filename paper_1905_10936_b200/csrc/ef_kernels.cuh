@@ -8,12 +8,18 @@
 // second pass over p, the residual is kept in a *deferred* form: the buffer stores p_t and the
 // block's scale s_t, and the next iteration rebuilds e_{t+1,j} = p_{t,j} -+ s_t in registers
 // while loading (one fp32 add, the same single rounding as the eager form).  The sign used is
-// (p_{t,j} < 0), which is exactly the bit that was sent.  Each launch is therefore one
+// that of p_{t,j}, which is exactly the bit that was sent.  Each launch is therefore one
 // streaming pass: read g, m, p_prev; write m, p; write 1 bit per element; plus one fp64
-// partial sum per tile.  The partial sums of a block are added in a fixed order, either by a
+// partial sum per CTA.  The partial sums of a block are added in a fixed order, either by a
 // tiny follow-up kernel (large grids: the kernel boundary orders the partial sums for free,
 // whereas a device-wide fence in every CTA costs about 8% of the streaming rate) or, for small
 // launch-bound grids, by the last CTA to finish the block (one atomic ticket, no waiting).
+//
+// Work decomposition.  The flat vector is cut into tiles of at most kTileChunks chunks of
+// 1024*U elements; a tile never crosses a block boundary.  The worker and apply kernels run
+// one CTA per chunk (three read and two write streams of 16 KB each per CTA keep enough bytes
+// in flight).  The server kernel has one read and one write stream only, so one CTA walks all
+// chunks of a tile and stages them two chunks ahead through shared memory with cp.async.
 //
 // Arithmetic is IEEE binary32 with explicit round-to-nearest intrinsics in a fixed order so
 // that results do not depend on compiler contraction; block sums are binary64.
@@ -27,14 +33,15 @@ namespace efk {
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr unsigned kFull = 0xffffffffu;
+constexpr int kTileChunks = 4;        // chunks per tile; also partial-sum slots per tile
 
-// A tile is a run of at most 1024*U consecutive elements inside one block.  Tiles of a block
-// start at multiples of the tile length from the block's first element, so a tile always
-// starts on a packed-word boundary.
+// A tile is a run of at most kTileChunks*1024*U consecutive elements inside one block.  Tiles
+// of a block start at multiples of the tile length from the block's first element, so tiles
+// and chunks always start on a packed-word boundary.
 struct __align__(16) Tile {
     long long start;   // flat index of the first element
     long long word;    // index of the first packed word
-    int len;           // elements in this tile (1 .. 1024*U)
+    int len;           // elements in this tile
     int block;         // block id
     int pad0, pad1;
 };
@@ -56,7 +63,7 @@ struct WorkerArgs {
     uint32_t* words;       // packed signs of p_{t,i}
     float* scale_out;      // per-block scales of the message
     float* rscale;         // per-block scale that belongs to pb (in: t-1, out: t)
-    double* partials;      // one fp64 partial L1 sum per tile
+    double* partials;      // kTileChunks fp64 partial L1 sums per tile
     unsigned* tickets;     // one arrival counter per block (0 between launches)
     const Tile* tiles;
     const Block* blocks;
@@ -84,7 +91,7 @@ struct ServerArgs {
 struct ScaleArgs {
     const double* partials;
     const Block* blocks;
-    const int* multi;        // ids of the blocks that span more than one tile
+    const int* multi;        // ids of the blocks that span more than one chunk
     float* scale_out;
     float* rscale;
 };
@@ -114,9 +121,29 @@ __device__ __forceinline__ void st_stream(float* p, float4 v) {
     __stcg(reinterpret_cast<float4*>(p), v);
 }
 
-// e_{t+1,j} = p_{t,j} - s * sign(p_{t,j}) with sign(+-0) = +1 (Algorithm 4; Appendix A).
+// Sign convention: sign(+-0) = +1 (Appendix A maps signs to {-1,+1}), i.e. "negative" means
+// p < 0.  The kernels test the IEEE sign bit instead, which is the same predicate for every
+// value except -0.0, and -0.0 never occurs in a residual buffer: the scale s is >= +0, so
+// e = p - s*sign(p) is never -0 (x - x = +0 in round-to-nearest), hence p = u + e is never -0,
+// the buffers start at +0 and ef_set_state adds +0 to what it imports.  (NaN is unspecified.)
+//
+// e_{t+1,j} = p_{t,j} - s * sign(p_{t,j})   (Algorithm 4): one rounding, as p + s or p - s.
 __device__ __forceinline__ float residual_of(float pb, float s) {
-    return (pb < 0.f) ? __fadd_rn(pb, s) : __fsub_rn(pb, s);
+    const float signed_s = __uint_as_float((__float_as_uint(pb) & 0x80000000u) | __float_as_uint(s));
+    return __fsub_rn(pb, signed_s);
+}
+
+// Sign bits of four values as a nibble, element k in bit k.
+__device__ __forceinline__ unsigned sign_nibble(const float (&v)[4]) {
+    unsigned n = __float_as_uint(v[3]) >> 31;
+    n = __funnelshift_l(__float_as_uint(v[2]), n, 1);
+    n = __funnelshift_l(__float_as_uint(v[1]), n, 1);
+    n = __funnelshift_l(__float_as_uint(v[0]), n, 1);
+    return n;
+}
+
+__device__ __forceinline__ double abs_sum4(const float (&v)[4]) {
+    return ((double)fabsf(v[0]) + (double)fabsf(v[1])) + ((double)fabsf(v[2]) + (double)fabsf(v[3]));
 }
 
 __device__ __forceinline__ double warp_sum(double v) {
@@ -139,16 +166,17 @@ __device__ __forceinline__ double cta_sum(double v, double* s_sum) {
     return S;
 }
 
-// Adds the partial sums of block b in a fixed order (thread k takes tiles k, k+256, ...; then
+// Adds the partial sums of block b in a fixed order (thread k takes slots k, k+256, ...; then
 // the CTA tree) and writes the scale s_b = ||p_b||_1 / d_b (Section 3.2).  Called by a whole CTA.
 __device__ __forceinline__ void sum_partials_and_write(const Block& b, int block_id,
                                                        const double* __restrict__ partials,
                                                        float* __restrict__ scale_out,
                                                        float* __restrict__ rscale,
                                                        double* s_sum) {
+    const double* src = partials + (long long)b.tile_begin * kTileChunks;
+    const int n = b.tile_count * kTileChunks;
     double v = 0.0;
-    for (int k = threadIdx.x; k < b.tile_count; k += kThreads)
-        v += __ldcg(&partials[b.tile_begin + k]);
+    for (int k = threadIdx.x; k < n; k += kThreads) v += __ldcg(&src[k]);
     const double S = cta_sum(v, s_sum);
     if (threadIdx.x == 0) {
         const float s = (float)(S / (double)b.len);
@@ -157,12 +185,15 @@ __device__ __forceinline__ void sum_partials_and_write(const Block& b, int block
     }
 }
 
-// End of a tile: turns the tile's |p| sum into the block scale or a published partial sum.
-// Single-tile blocks are finished directly.  For larger blocks the tile's partial sum is
-// stored; if `fused`, the CTA that arrives last at the block's ticket also adds all partial
-// sums (no CTA ever waits for another one), otherwise ef_scale_kernel does that after this
-// launch.
-__device__ __forceinline__ void finish_block(double acc, int tile_index, const Tile& t,
+// End of a CTA's work: turns its |p| sum into the block scale or a published partial sum.
+//   slot      partial-sum slot of this CTA; `zero_slots` further slots are set to 0
+//   alone     this CTA covered the whole block: write the scale directly
+//   expected  number of CTAs that arrive at the block's ticket in fused mode
+// For blocks covered by several CTAs the partial sum is stored; if `fused`, the CTA that
+// arrives last at the block's ticket also adds all partial sums (no CTA ever waits for another
+// one), otherwise ef_scale_kernel does that after this launch.
+__device__ __forceinline__ void finish_block(double acc, long long slot, int zero_slots, bool alone,
+                                             unsigned expected, int block_id,
                                              const Block* __restrict__ blocks,
                                              double* __restrict__ partials,
                                              unsigned* __restrict__ tickets,
@@ -172,18 +203,18 @@ __device__ __forceinline__ void finish_block(double acc, int tile_index, const T
     __shared__ int s_last;
     const double S = cta_sum(acc, s_sum);
     if (threadIdx.x == 0) {
-        const Block b = blocks[t.block];
         int last = 0;
-        if (b.tile_count == 1) {
-            const float s = (float)(S / (double)b.len);
-            scale_out[t.block] = s;
-            rscale[t.block] = s;
+        if (alone) {
+            const float s = (float)(S / (double)blocks[block_id].len);
+            scale_out[block_id] = s;
+            rscale[block_id] = s;
         } else {
-            partials[tile_index] = S;
+            partials[slot] = S;
+            for (int z = 1; z <= zero_slots; ++z) partials[slot + z] = 0.0;
             if (fused) {
                 __threadfence();
-                const unsigned old = atomicAdd(&tickets[t.block], 1u);
-                last = (old + 1u == (unsigned)b.tile_count);
+                const unsigned old = atomicAdd(&tickets[block_id], 1u);
+                last = (old + 1u == expected);
             }
         }
         s_last = last;
@@ -192,12 +223,12 @@ __device__ __forceinline__ void finish_block(double acc, int tile_index, const T
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    const Block b = blocks[t.block];
-    sum_partials_and_write(b, t.block, partials, scale_out, rscale, s_sum);
-    if (threadIdx.x == 0) tickets[t.block] = 0u;      // ready for the next launch
+    const Block b = blocks[block_id];
+    sum_partials_and_write(b, block_id, partials, scale_out, rscale, s_sum);
+    if (threadIdx.x == 0) tickets[block_id] = 0u;      // ready for the next launch
 }
 
-// Follow-up kernel of the non-fused mode: one CTA per multi-tile block.
+// Follow-up kernel of the non-fused mode: one CTA per block that spans more than one chunk.
 __global__ void __launch_bounds__(kThreads) ef_scale_kernel(const ScaleArgs a) {
     __shared__ double s_sum[kWarps];
     const int block_id = a.multi[blockIdx.x];
@@ -234,8 +265,19 @@ __device__ __forceinline__ void store4(float* p, int o, int len, bool full, cons
     }
 }
 
+// Chunk `sub` of tile t as a tile of its own (len <= 0 if the tile has no such chunk).
+template <int U>
+__device__ __forceinline__ Tile chunk_of(const Tile& t, int sub) {
+    Tile c = t;
+    c.start += (long long)sub * (1024 * U);
+    c.word += sub * (1024 * U / 32);
+    const int rest = t.len - sub * (1024 * U);
+    c.len = rest < 1024 * U ? rest : 1024 * U;
+    return c;
+}
+
 // ------------------------------------------------------------------ worker kernel
-// One tile per CTA.  Warp w owns the 128*U consecutive elements starting at w*128*U; in row u
+// One chunk per CTA.  Warp w owns the 128*U consecutive elements starting at w*128*U; in row u
 // lane l holds elements u*128 + 4l .. +3 (a 128-bit access, 512 contiguous bytes per warp).
 template <int U, bool FULL>
 __device__ __forceinline__ double worker_rows(const WorkerArgs& a, const Tile& t, float sp) {
@@ -255,7 +297,6 @@ __device__ __forceinline__ double worker_rows(const WorkerArgs& a, const Tile& t
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const int o = o0 + u * 128;
-        unsigned nib = 0;
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             const float e = residual_of(p[u][k], sp);                // e_{t,i}
@@ -264,10 +305,9 @@ __device__ __forceinline__ double worker_rows(const WorkerArgs& a, const Tile& t
             float pv = __fadd_rn(v, e);                              // p_t
             if (!FULL && o + k >= t.len) pv = 0.f;
             p[u][k] = pv;
-            nib |= (pv < 0.f ? 1u : 0u) << k;
         }
-        acc += ((double)fabsf(p[u][0]) + (double)fabsf(p[u][1])) +
-               ((double)fabsf(p[u][2]) + (double)fabsf(p[u][3]));
+        const unsigned nib = sign_nibble(p[u]);
+        acc += abs_sum4(p[u]);
         const unsigned w = pack_nibbles(nib, lane);
         store4(mp + u * 128, o, t.len, FULL, m[u]);
         store4(pp + u * 128, o, t.len, FULL, p[u]);
@@ -276,7 +316,7 @@ __device__ __forceinline__ double worker_rows(const WorkerArgs& a, const Tile& t
     return acc;
 }
 
-// Fallback for tiles that do not start on a 16-byte boundary: 32-bit accesses, one ballot per
+// Fallback for chunks that do not start on a 16-byte boundary: 32-bit accesses, one ballot per
 // 32 elements.
 __device__ __forceinline__ double worker_rows_scalar(const WorkerArgs& a, const Tile& t, float sp) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -304,30 +344,49 @@ __device__ __forceinline__ double worker_rows_scalar(const WorkerArgs& a, const 
 
 template <int U>
 __global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a) {
-    const Tile t = a.tiles[blockIdx.x];
-    const float sp = a.rscale[t.block];
-    double acc;
-    if ((t.start & 3) != 0)
-        acc = worker_rows_scalar(a, t, sp);
-    else if (t.len == 1024 * U)
-        acc = worker_rows<U, true>(a, t, sp);
-    else
-        acc = worker_rows<U, false>(a, t, sp);
-    finish_block(acc, blockIdx.x, t, a.blocks, a.partials, a.tickets, a.scale_out, a.rscale, a.fused);
+    const Tile t = chunk_of<U>(a.tiles[blockIdx.x / kTileChunks], blockIdx.x % kTileChunks);
+    const Block b = a.blocks[t.block];
+    const bool alone = b.len <= 1024 * U;              // the block is this single chunk
+    if (t.len <= 0 && alone) return;
+    double acc = 0.0;
+    if (t.len > 0) {
+        const float sp = a.rscale[t.block];
+        if ((t.start & 3) != 0)
+            acc = worker_rows_scalar(a, t, sp);
+        else if (t.len == 1024 * U)
+            acc = worker_rows<U, true>(a, t, sp);
+        else
+            acc = worker_rows<U, false>(a, t, sp);
+    }
+    finish_block(acc, blockIdx.x, 0, alone, (unsigned)(b.tile_count * kTileChunks), t.block,
+                 a.blocks, a.partials, a.tickets, a.scale_out, a.rscale, a.fused);
 }
 
 // ------------------------------------------------------------------ server kernel
 // a_j = sum over ascending i of (bit_i ? -c_i : +c_i), c_i = fl(scale_{i,b} / M), the first
 // term taken as is (Algorithm 4, server line: (1/M) sum_i Delta_{t,i}).
 //
-// For M <= 8 the 2^M possible values of a_j inside one block are tabulated once per CTA in
-// shared memory (each entry is the same chain of fp32 additions, so the table is exact) and an
-// element costs one lookup instead of M dependent additions with 2 bit operations each.  The
-// index of element k of a lane is the byte k of R, where bit (8k + i) of R is worker i's sign
-// bit: each worker's nibble n (its 4 sign bits for the lane's 4 elements) is spread with
-// (n * 0x00204081) & 0x01010101, which moves bit k to bit 8k without carries, and shifted
-// left by i.
+// For M <= 8 the possible values of a_j inside one block are tabulated once per CTA in shared
+// memory (each entry is the same chain of fp32 additions, so the table is exact) and an
+// element costs one lookup instead of M dependent additions with 2 bit operations each.
+//
+// Building the table index without per-worker work in every lane: the 8 lanes that share a
+// packed word each load the word of ONE worker (lane q -> worker q).  Seen as an 8x8 matrix of
+// nibbles (row = worker, column = lane whose 4 elements the nibble belongs to), a three-stage
+// butterfly over the lanes (xor 4: half-words, xor 2: bytes, xor 1: nibbles) transposes it, so
+// lane r ends with N = the 8 workers' nibbles for its own 4 elements.  Two delta swaps of the
+// bit-index (4 <-> 1, 3 <-> 0) then turn N into R, whose byte k holds the 8 sign bits of
+// element k, worker i at bit kLutPos(i).  Byte k of R indexes the table.
 constexpr int kMaxLutWorkers = 8;
+
+__host__ __device__ constexpr int kLutPos(int i) {
+    return 4 * (i & 1) + 2 * ((i >> 2) & 1) + ((i >> 1) & 1);
+}
+__host__ __device__ constexpr int kLutSize(int M) {   // 1 << (highest used bit position + 1)
+    int hi = 0;
+    for (int i = 0; i < M; ++i) hi = kLutPos(i) > hi ? kLutPos(i) : hi;
+    return 1 << (hi + 1);
+}
 
 __device__ __forceinline__ void build_scaled(const ServerArgs& a, int block, int M, float* s_c) {
     for (int i = threadIdx.x; i < M; i += kThreads)
@@ -336,65 +395,162 @@ __device__ __forceinline__ void build_scaled(const ServerArgs& a, int block, int
 
 template <int MT>
 __device__ __forceinline__ void build_lut(const float* s_c, float* s_lut) {
-    for (int pat = threadIdx.x; pat < (1 << MT); pat += kThreads) {
-        float v = (pat & 1) ? -s_c[0] : s_c[0];
+    for (int idx = threadIdx.x; idx < kLutSize(MT); idx += kThreads) {
+        float v = ((idx >> kLutPos(0)) & 1) ? -s_c[0] : s_c[0];
 #pragma unroll
-        for (int i = 1; i < MT; ++i) v = __fadd_rn(v, ((pat >> i) & 1) ? -s_c[i] : s_c[i]);
-        s_lut[pat] = v;
+        for (int i = 1; i < MT; ++i)
+            v = __fadd_rn(v, ((idx >> kLutPos(i)) & 1) ? -s_c[i] : s_c[i]);
+        s_lut[idx] = v;
     }
 }
 
-template <int U, int MT, bool FULL>
-__device__ __forceinline__ double server_rows_lut(const ServerArgs& a, const Tile& t, float sp,
-                                                  float* s_c, float* s_lut) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int o0 = warp * (128 * U) + lane * 4;
-    const int sh = (lane & 7) * 4;
-    float* pp = a.pb + t.start + o0;
-    const uint32_t* wp = a.wwords + t.word + (o0 >> 5);
-    float p[U][4];
-    unsigned w[U][MT];
-    // all global loads first; the table is built while they are in flight
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-        load4(pp + u * 128, o0 + u * 128, t.len, FULL, p[u]);
-#pragma unroll
-        for (int i = 0; i < MT; ++i)
-            w[u][i] = (FULL || o0 + u * 128 < t.len) ? __ldg(wp + (long long)i * a.wstride + u * 4) : 0u;
+__device__ __forceinline__ unsigned delta_swap(unsigned x, int d, unsigned mask) {
+    const unsigned t = ((x >> d) ^ x) & mask;
+    return x ^ t ^ (t << d);
+}
+
+// Lane-dependent constants of the butterfly (q = lane & 7).
+struct Butterfly {
+    unsigned sel1, sel2, keep3;
+    int rot3;
+    __device__ __forceinline__ explicit Butterfly(int q)
+        : sel1((q & 4) ? 0x3276u : 0x5410u), sel2((q & 2) ? 0x3715u : 0x6240u),
+          keep3((q & 1) ? 0xF0F0F0F0u : 0x0F0F0F0Fu), rot3((q & 1) ? 28 : 4) {}
+    // w: this lane's worker word (lane q of the 8-lane group holds worker q, 0 if q >= M).
+    // Returns R: byte k = table index of the lane's element k.
+    __device__ __forceinline__ unsigned indices(unsigned w) const {
+        unsigned x = w;
+        x = __byte_perm(x, __shfl_xor_sync(kFull, x, 4), sel1);
+        x = __byte_perm(x, __shfl_xor_sync(kFull, x, 2), sel2);
+        const unsigned y = __shfl_xor_sync(kFull, x, 1);
+        x = (x & keep3) | (__funnelshift_l(y, y, rot3) & ~keep3);
+        x = delta_swap(x, 14, 0x0000CCCCu);
+        return delta_swap(x, 7, 0x00AA00AAu);
     }
+};
+
+// Asynchronous global->shared copies (LDGSTS).  Every thread copies exactly the bytes it will
+// read back itself, so completion is tracked per thread with wait_group and no barrier or
+// flag wait is involved.
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(
+                     (unsigned)__cvta_generic_to_shared(smem)), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async4(void* smem, const void* gmem) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(
+                     (unsigned)__cvta_generic_to_shared(smem)), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+constexpr int kServerStages = 3;
+// Dynamic shared memory of the server kernel: staging ring, then M scaled scales.
+template <int U>
+__host__ __device__ constexpr size_t server_ring_bytes() {
+    return (size_t)kServerStages * U * kThreads * (sizeof(float4) + sizeof(unsigned));
+}
+
+// Table path: one CTA walks the chunks of its tile.  Full chunks are staged through a ring of
+// kServerStages shared-memory slots filled two chunks ahead with cp.async, so loads stay in
+// flight during the lookups without costing registers; a ragged last chunk is loaded directly.
+template <int U, int MT>
+__device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Tile& t, float sp,
+                                                  unsigned char* ring, float* s_c, float* s_lut) {
+    constexpr int kChunk = 1024 * U;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int q = lane & 7;
+    const int o0 = warp * (128 * U) + lane * 4;
+    const Butterfly bf(q);
+    float* const pbase = a.pb + t.start + o0;
+    const uint32_t* const wbase =
+        a.wwords + (long long)(q < MT ? q : 0) * a.wstride + t.word + (o0 >> 5);
+    const int nfull = t.len / kChunk;              // chunks staged through shared memory
+    const int tail = t.len - nfull * kChunk;       // ragged rest (only at the end of a block)
+    const char* lut = reinterpret_cast<const char*>(s_lut);
+    // slot (stage s, row u) of this thread: consecutive threads are 16 (4) bytes apart
+    float4* const ring_p = reinterpret_cast<float4*>(ring) + threadIdx.x;
+    unsigned* const ring_w =
+        reinterpret_cast<unsigned*>(ring + (size_t)kServerStages * U * kThreads * sizeof(float4)) +
+        threadIdx.x;
+    double acc = 0.0;
+
+    auto issue_chunk = [&](int c) {
+        if (c < nfull) {
+            const int s = c % kServerStages;
+            const float* pp = pbase + (long long)c * kChunk;
+            const uint32_t* wp = wbase + c * (kChunk / 32);
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                cp_async16(ring_p + (s * U + u) * kThreads, pp + u * 128);
+                if (q < MT) cp_async4(ring_w + (s * U + u) * kThreads, wp + u * 4);
+            }
+        }
+        cp_async_commit();                 // one (possibly empty) group per chunk index
+    };
+    auto compute_chunk = [&](int c, int clen, float (&p)[U][4], unsigned (&w)[U]) {
+        const bool full = clen == kChunk;
+        float* pp = pbase + (long long)c * kChunk;
+        uint32_t* words = a.words + t.word + c * (kChunk / 32);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int o = o0 + u * 128;
+            const unsigned R = bf.indices(w[u]);
+            float avg[4];
+            avg[0] = *reinterpret_cast<const float*>(lut + ((R << 2) & 0x3FCu));
+            avg[1] = *reinterpret_cast<const float*>(lut + ((R >> 6) & 0x3FCu));
+            avg[2] = *reinterpret_cast<const float*>(lut + ((R >> 14) & 0x3FCu));
+            avg[3] = *reinterpret_cast<const float*>(lut + ((R >> 22) & 0x3FCu));
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                float pv = __fadd_rn(avg[k], residual_of(p[u][k], sp));      // ptilde_t
+                if (!full && o + k >= clen) pv = 0.f;
+                p[u][k] = pv;
+            }
+            const unsigned nib = sign_nibble(p[u]);
+            acc += abs_sum4(p[u]);
+            const unsigned word = pack_nibbles(nib, lane);
+            store4(pp + u * 128, o, clen, full, p[u]);
+            if (q == 0 && (full || o < clen)) words[o >> 5] = word;
+        }
+    };
+
+    float p[U][4];
+    unsigned w[U];
+    issue_chunk(0);                        // in flight while the table is built
+    issue_chunk(1);
     build_scaled(a, t.block, MT, s_c);
     __syncthreads();
     build_lut<MT>(s_c, s_lut);
     __syncthreads();
-    double acc = 0.0;
+    for (int c = 0; c < nfull; ++c) {
+        issue_chunk(c + 2);                // reuses the slot this thread consumed at c - 1
+        cp_async_wait<2>();                // groups c+1 and c+2 may still be in flight
+        const int s = c % kServerStages;
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-        const int o = o0 + u * 128;
-        unsigned R = 0;
-#pragma unroll
-        for (int i = 0; i < MT; ++i) {
-            const unsigned n = (w[u][i] >> sh) & 0xFu;
-            R |= (n * (0x00204081u << i)) & (0x01010101u << i);
+        for (int u = 0; u < U; ++u) {
+            const float4 v = ring_p[(s * U + u) * kThreads];
+            p[u][0] = v.x; p[u][1] = v.y; p[u][2] = v.z; p[u][3] = v.w;
+            w[u] = (q < MT) ? ring_w[(s * U + u) * kThreads] : 0u;
         }
-        unsigned nib = 0;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const float avg = s_lut[(R >> (8 * k)) & 0xFFu];
-            float pv = __fadd_rn(avg, residual_of(p[u][k], sp));      // ptilde_t
-            if (!FULL && o + k >= t.len) pv = 0.f;
-            p[u][k] = pv;
-            nib |= (pv < 0.f ? 1u : 0u) << k;
-        }
-        acc += ((double)fabsf(p[u][0]) + (double)fabsf(p[u][1])) +
-               ((double)fabsf(p[u][2]) + (double)fabsf(p[u][3]));
-        const unsigned word = pack_nibbles(nib, lane);
-        store4(pp + u * 128, o, t.len, FULL, p[u]);
-        if ((lane & 7) == 0 && (FULL || o < t.len)) a.words[t.word + (o >> 5)] = word;
+        compute_chunk(c, kChunk, p, w);
     }
+    if (tail > 0) {
+        const float* pp = pbase + (long long)nfull * kChunk;
+        const uint32_t* wp = wbase + nfull * (kChunk / 32);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int o = o0 + u * 128;
+            load4(pp + u * 128, o, tail, false, p[u]);
+            w[u] = (q < MT && (o & ~31) < tail) ? __ldg(wp + u * 4) : 0u;
+        }
+        compute_chunk(nfull, tail, p, w);
+    }
+    cp_async_wait<0>();
     return acc;
 }
 
-// Direct evaluation for any M (and for tiles that are not 16-byte aligned).
+// Direct evaluation for any M.
 __device__ __forceinline__ void average4(const ServerArgs& a, const float* s_c, long long wi,
                                          int sh, float (&avg)[4]) {
     const uint32_t* wp = a.wwords + wi;
@@ -410,39 +566,39 @@ __device__ __forceinline__ void average4(const ServerArgs& a, const float* s_c, 
     }
 }
 
-template <int U, bool FULL>
+template <int U>
 __device__ __forceinline__ double server_rows(const ServerArgs& a, const Tile& t, float sp,
                                               const float* s_c) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int o0 = warp * (128 * U) + lane * 4;
     const int sh = (lane & 7) * 4;
+    const bool full = t.len == 1024 * U;
     float* pp = a.pb + t.start + o0;
     float p[U][4];
 #pragma unroll
-    for (int u = 0; u < U; ++u) load4(pp + u * 128, o0 + u * 128, t.len, FULL, p[u]);
+    for (int u = 0; u < U; ++u) load4(pp + u * 128, o0 + u * 128, t.len, full, p[u]);
     double acc = 0.0;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const int o = o0 + u * 128;
         float avg[4] = {0.f, 0.f, 0.f, 0.f};
-        if (FULL || o < t.len) average4(a, s_c, t.word + (o >> 5), sh, avg);
-        unsigned nib = 0;
+        if (full || o < t.len) average4(a, s_c, t.word + (o >> 5), sh, avg);
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             float pv = __fadd_rn(avg[k], residual_of(p[u][k], sp));   // ptilde_t
-            if (!FULL && o + k >= t.len) pv = 0.f;
+            if (!full && o + k >= t.len) pv = 0.f;
             p[u][k] = pv;
-            nib |= (pv < 0.f ? 1u : 0u) << k;
         }
-        acc += ((double)fabsf(p[u][0]) + (double)fabsf(p[u][1])) +
-               ((double)fabsf(p[u][2]) + (double)fabsf(p[u][3]));
+        const unsigned nib = sign_nibble(p[u]);
+        acc += abs_sum4(p[u]);
         const unsigned w = pack_nibbles(nib, lane);
-        store4(pp + u * 128, o, t.len, FULL, p[u]);
-        if ((lane & 7) == 0 && (FULL || o < t.len)) a.words[t.word + (o >> 5)] = w;
+        store4(pp + u * 128, o, t.len, full, p[u]);
+        if ((lane & 7) == 0 && (full || o < t.len)) a.words[t.word + (o >> 5)] = w;
     }
     return acc;
 }
 
+// Any alignment, any M, any tile length.
 __device__ __forceinline__ double server_rows_scalar(const ServerArgs& a, const Tile& t, float sp,
                                                      const float* s_c) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -470,37 +626,41 @@ __device__ __forceinline__ double server_rows_scalar(const ServerArgs& a, const 
     return acc;
 }
 
-// MT = number of workers when 1 <= M <= 8 (table path), MT = 0 for any other M.
+// One tile per CTA.  MT = number of workers when 1 <= M <= 8 (table path), 0 for any other M.
 template <int U, int MT>
 __global__ void __launch_bounds__(kThreads) ef_server_kernel(const ServerArgs a) {
-    extern __shared__ float s_c[];                     // M scaled worker scales
-    __shared__ float s_lut[MT > 0 ? (1 << MT) : 1];
+    // dynamic shared memory: [staging ring (table path only)] [M scaled worker scales]
+    extern __shared__ __align__(16) unsigned char s_dyn[];
+    float* s_c = reinterpret_cast<float*>(s_dyn + (MT > 0 ? server_ring_bytes<U>() : 0));
+    __shared__ float s_lut[MT > 0 ? kLutSize(MT) : 1];
     const Tile t = a.tiles[blockIdx.x];
     const float sp = a.rscale[t.block];
-    double acc;
+    double acc = 0.0;
     if (MT > 0 && (t.start & 3) == 0) {
-        if (t.len == 1024 * U)
-            acc = server_rows_lut<U, (MT > 0 ? MT : 1), true>(a, t, sp, s_c, s_lut);
-        else
-            acc = server_rows_lut<U, (MT > 0 ? MT : 1), false>(a, t, sp, s_c, s_lut);
+        acc = server_tile_lut<U, (MT > 0 ? MT : 1)>(a, t, sp, s_dyn, s_c, s_lut);
     } else {
         build_scaled(a, t.block, a.M, s_c);
         __syncthreads();
-        if ((t.start & 3) != 0)
+        if ((t.start & 3) != 0) {
             acc = server_rows_scalar(a, t, sp, s_c);
-        else if (t.len == 1024 * U)
-            acc = server_rows<U, true>(a, t, sp, s_c);
-        else
-            acc = server_rows<U, false>(a, t, sp, s_c);
+        } else {
+            for (int c = 0; c * (1024 * U) < t.len; ++c)
+                acc += server_rows<U>(a, chunk_of<U>(t, c), sp, s_c);
+        }
     }
-    finish_block(acc, blockIdx.x, t, a.blocks, a.partials, a.tickets, a.scale_out, a.rscale, a.fused);
+    const Block b = a.blocks[t.block];
+    finish_block(acc, (long long)blockIdx.x * kTileChunks, kTileChunks - 1, b.len <= 1024 * U,
+                 (unsigned)b.tile_count, t.block, a.blocks, a.partials, a.tickets, a.scale_out,
+                 a.rscale, a.fused);
 }
 
 // ------------------------------------------------------------------ parameter update
 // x_{t+1,j} = x_{t,j} - eta * stilde_b * sign(ptilde_j)  (Algorithm 4, worker line after the pull)
+// One chunk per CTA.
 template <int U>
 __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
-    const Tile t = a.tiles[blockIdx.x];
+    const Tile t = chunk_of<U>(a.tiles[blockIdx.x / kTileChunks], blockIdx.x % kTileChunks);
+    if (t.len <= 0) return;
     const float step = __fmul_rn(a.eta, a.scales[t.block]);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if ((t.start & 3) != 0) {
@@ -530,20 +690,32 @@ __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
 #pragma unroll
     for (int u = 0; u < U; ++u) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-            x[u][k] = ((nib[u] >> k) & 1u) ? __fadd_rn(x[u][k], step) : __fsub_rn(x[u][k], step);
+        for (int k = 0; k < 4; ++k) {   // x - step*sign: subtract step with the sign bit flipped in
+            const float signed_step =
+                __uint_as_float(__float_as_uint(step) ^ ((nib[u] << (31 - k)) & 0x80000000u));
+            x[u][k] = __fsub_rn(x[u][k], signed_step);
+        }
         store4(xp + u * 128, o0 + u * 128, t.len, full, x[u]);
     }
 }
 
 // ------------------------------------------------------------------ residual materialisation
 // dst_j = p_j - s_b * sign(p_j): the residual e_{t+1} in its plain form (tests, checkpoints).
-template <int U>
+// One tile per CTA.
 __global__ void __launch_bounds__(kThreads) ef_residual_kernel(const ResidualArgs a) {
     const Tile t = a.tiles[blockIdx.x];
     const float s = a.rscale[t.block];
     for (int o = threadIdx.x; o < t.len; o += kThreads)
         a.dst[t.start + o] = residual_of(a.pb[t.start + o], s);
+}
+
+// Import of a residual (ef_set_state): adding +0 maps -0 to +0 and changes nothing else, which
+// keeps the "no -0 in a residual buffer" invariant of the sign-bit tests above.
+__global__ void __launch_bounds__(kThreads) ef_import_kernel(const float* __restrict__ src,
+                                                             float* __restrict__ dst, long long n) {
+    for (long long j = blockIdx.x * (long long)kThreads + threadIdx.x; j < n;
+         j += (long long)gridDim.x * kThreads)
+        dst[j] = __fadd_rn(src[j], 0.0f);
 }
 
 }  // namespace efk

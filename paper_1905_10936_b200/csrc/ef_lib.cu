@@ -3,6 +3,7 @@
 #include "../../include/ef.h"
 #include "ef_kernels.cuh"
 
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -18,11 +19,13 @@ using efk::Tile;
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
 
-// Rows of four elements per thread and tile; a tile is 1024*U elements.
+// Rows of four elements per thread and chunk: a chunk is 1024*U elements (one CTA of the worker
+// and apply kernels), a tile is kTileChunks chunks (one CTA of the server kernel).
 constexpr int kU = 4;
-constexpr int kTileLen = 1024 * kU;
-// Grids up to this many tiles (about two waves of CTAs) finalise block scales in-kernel.
-constexpr int64_t kFusedMaxTiles = 1024;
+constexpr int kChunkLen = 1024 * kU;
+constexpr int kTileLen = kChunkLen * efk::kTileChunks;
+// Grids up to this many chunks (about two waves of CTAs) finalise block scales in-kernel.
+constexpr int64_t kFusedMaxChunks = 1024;
 
 struct Layout {
     int64_t d = 0, W = 0;
@@ -32,7 +35,7 @@ struct Layout {
     size_t off_x = 0, off_m = 0, off_pb = 0, off_spb = 0, off_words = 0, off_scales = 0,
            off_rscale = 0, off_partials = 0, off_tickets = 0, off_tiles = 0, off_blocks = 0,
            off_multi = 0, off_stage = 0, total = 0;
-    int32_t num_multi = 0;                            // blocks that span more than one tile
+    int32_t num_multi = 0;                            // blocks that span more than one chunk
 };
 
 int check_problem(int64_t d, int32_t B, const int64_t* offsets, int32_t M) {
@@ -56,14 +59,14 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
         const int64_t db = offsets[b + 1] - offsets[b];
         W += (db + 31) / 32;
         T += (db + kTileLen - 1) / kTileLen;
-        if (db > kTileLen) L->num_multi += 1;
+        if (db > kChunkLen) L->num_multi += 1;
     }
-    if (T > 0x7fffffffLL) return EF_ERR_INVALID_ARG;
+    if (T * efk::kTileChunks > 0x7fffffffLL) return EF_ERR_INVALID_ARG;
     L->W = W; L->num_tiles = T;
     L->dpad = align_up((size_t)d * 4) / 4;
     L->wpad = align_up((size_t)W * 4) / 4;
     L->bpad = align_up((size_t)B * 4) / 4;
-    L->tpad = align_up((size_t)T * 8) / 8;
+    L->tpad = align_up((size_t)T * efk::kTileChunks * 8) / 8;   // partial-sum slots
     const size_t M1 = (size_t)M + 1;
     size_t o = 0;
     L->off_x = o;        o += L->dpad * 4;
@@ -137,7 +140,7 @@ int cuda_fail(ef_ctx* c, cudaError_t e) {
 
 inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
-// Non-fused mode: adds the per-tile partial sums of every multi-tile block of buffer set k
+// Non-fused mode: adds the partial sums of every block larger than one chunk of buffer set k
 // (worker k, or the server for k == M) after the kernel that produced them.
 int launch_scale(ef_ctx* c, int k) {
     if (c->fused || c->L.num_multi == 0) return EF_OK;
@@ -156,16 +159,23 @@ int launch_worker(ef_ctx* c, int i, const float* grad) {
     a.scale_out = c->scales(i); a.rscale = c->rscale(i);
     a.partials = c->partials(i); a.tickets = c->tickets(i);
     a.tiles = c->tiles(); a.blocks = c->blocks(); a.mu = c->mu; a.fused = c->fused;
-    efk::ef_worker_kernel<kU><<<(unsigned)c->L.num_tiles, efk::kThreads, 0, c->stream>>>(a);
+    efk::ef_worker_kernel<kU><<<(unsigned)(c->L.num_tiles * efk::kTileChunks), efk::kThreads, 0, c->stream>>>(a);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
     return launch_scale(c, i);
 }
 
 template <int MT>
-void launch_server_t(ef_ctx* c, const efk::ServerArgs& a) {
-    efk::ef_server_kernel<kU, MT>
-        <<<(unsigned)c->L.num_tiles, efk::kThreads, (size_t)c->L.M * sizeof(float), c->stream>>>(a);
+cudaError_t launch_server_t(ef_ctx* c, const efk::ServerArgs& a) {
+    const size_t smem = (MT > 0 ? efk::server_ring_bytes<kU>() : 0) + (size_t)c->L.M * sizeof(float);
+    if (smem > 48 * 1024) {
+        const cudaError_t e = cudaFuncSetAttribute(efk::ef_server_kernel<kU, MT>,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    efk::ef_server_kernel<kU, MT><<<(unsigned)c->L.num_tiles, efk::kThreads, smem, c->stream>>>(a);
+    return cudaGetLastError();
 }
 
 int launch_server(ef_ctx* c) {
@@ -176,18 +186,19 @@ int launch_server(ef_ctx* c) {
     a.pb = c->pb(M); a.words = c->words(M); a.scale_out = c->scales(M); a.rscale = c->rscale(M);
     a.partials = c->partials(M); a.tickets = c->tickets(M);
     a.tiles = c->tiles(); a.blocks = c->blocks(); a.fused = c->fused;
+    cudaError_t le;
     switch (M) {
-        case 1: launch_server_t<1>(c, a); break;
-        case 2: launch_server_t<2>(c, a); break;
-        case 3: launch_server_t<3>(c, a); break;
-        case 4: launch_server_t<4>(c, a); break;
-        case 5: launch_server_t<5>(c, a); break;
-        case 6: launch_server_t<6>(c, a); break;
-        case 7: launch_server_t<7>(c, a); break;
-        case 8: launch_server_t<8>(c, a); break;
-        default: launch_server_t<0>(c, a); break;
+        case 1: le = launch_server_t<1>(c, a); break;
+        case 2: le = launch_server_t<2>(c, a); break;
+        case 3: le = launch_server_t<3>(c, a); break;
+        case 4: le = launch_server_t<4>(c, a); break;
+        case 5: le = launch_server_t<5>(c, a); break;
+        case 6: le = launch_server_t<6>(c, a); break;
+        case 7: le = launch_server_t<7>(c, a); break;
+        case 8: le = launch_server_t<8>(c, a); break;
+        default: le = launch_server_t<0>(c, a); break;
     }
-    EF_CUDA(c, cudaGetLastError());
+    EF_CUDA(c, le);
     c->launches += 1;
     {
         const int rc = launch_scale(c, M);
@@ -196,7 +207,7 @@ int launch_server(ef_ctx* c) {
     efk::ApplyArgs p;
     p.x = c->x(); p.words = c->words(M); p.scales = c->scales(M); p.tiles = c->tiles();
     p.eta = c->eta;
-    efk::ef_apply_kernel<kU><<<(unsigned)c->L.num_tiles, efk::kThreads, 0, c->stream>>>(p);
+    efk::ef_apply_kernel<kU><<<(unsigned)(c->L.num_tiles * efk::kTileChunks), efk::kThreads, 0, c->stream>>>(p);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
     return EF_OK;
@@ -267,14 +278,14 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
             c->h_tiles.push_back(t);
         }
         blk.tile_count = (int)c->h_tiles.size() - blk.tile_begin;
-        if (blk.tile_count > 1) c->h_multi.push_back(b);
+        if (len > kChunkLen) c->h_multi.push_back(b);
         word += (len + 31) / 32;
     }
     // Small grids are launch-bound: finish block scales inside the main kernels.  Large grids
     // are bandwidth-bound: the per-CTA fence of the fused form costs more than a tiny launch.
     if (flags & EF_FLAG_FUSED_SCALE) c->fused = 1;
     else if (flags & EF_FLAG_SPLIT_SCALE) c->fused = 0;
-    else c->fused = (L.num_tiles <= kFusedMaxTiles) ? 1 : 0;
+    else c->fused = (L.num_tiles * efk::kTileChunks <= kFusedMaxChunks) ? 1 : 0;
 
     auto fail = [&](cudaError_t e) { delete c; (void)e; return EF_ERR_CUDA; };
     // Algorithm 4 "Initialize": x_0, m, e, etilde = 0; also words, scales, tickets, partials.
@@ -379,7 +390,7 @@ int ef_get_residual(ef_ctx* c, int32_t i, float* dst) {
     const int k = (i < 0) ? c->L.M : i;
     efk::ResidualArgs a;
     a.pb = c->pb(k); a.rscale = c->rscale(k); a.dst = dst; a.tiles = c->tiles();
-    efk::ef_residual_kernel<kU><<<(unsigned)c->L.num_tiles, efk::kThreads, 0, c->stream>>>(a);
+    efk::ef_residual_kernel<<<(unsigned)c->L.num_tiles, efk::kThreads, 0, c->stream>>>(a);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
     return EF_OK;
@@ -394,8 +405,14 @@ int ef_set_state(ef_ctx* c, int32_t i, const float* momentum, const float* resid
     const size_t nbytes = (size_t)c->L.d * 4;
     if (i >= 0)
         EF_CUDA(c, cudaMemcpyAsync(c->m(i), momentum, nbytes, cudaMemcpyDeviceToDevice, c->stream));
-    // deferred form with scale 0: p -+ 0 gives back the residual exactly
-    EF_CUDA(c, cudaMemcpyAsync(c->pb(k), residual, nbytes, cudaMemcpyDeviceToDevice, c->stream));
+    // deferred form with scale 0: p -+ 0 gives back the residual exactly (-0 is stored as +0)
+    {
+        const long long n = c->L.d;
+        const unsigned grid = (unsigned)std::min<long long>((n + efk::kThreads - 1) / efk::kThreads, 148 * 16);
+        efk::ef_import_kernel<<<grid, efk::kThreads, 0, c->stream>>>(residual, c->pb(k), n);
+        EF_CUDA(c, cudaGetLastError());
+        c->launches += 1;
+    }
     EF_CUDA(c, cudaMemsetAsync(c->rscale(k), 0, (size_t)c->L.B * 4, c->stream));
     return EF_OK;
 }

@@ -10,7 +10,8 @@ from parity import run_parity, BlockSample, compare_state, words_np
 
 pytestmark = pytest.mark.gpu
 
-TILE = 4096   # elements per tile of the library build (1024 * rows per thread)
+TILE = 4096   # elements per chunk of the library build (1024 * rows per thread)
+BIG = 4 * TILE  # elements per tile (one server CTA walks up to four chunks)
 
 
 def _wl(name, sizes, M, mu=0.9, eta=0.1, steps=5, law="normal", scale_range=None, cid=50):
@@ -28,6 +29,8 @@ def _wl(name, sizes, M, mu=0.9, eta=0.1, steps=5, law="normal", scale_range=None
     ([2 * TILE, TILE // 2, 3 * TILE + 36, 100], 8),  # several tiles per block + ragged tails
     ([5 * TILE + 2, 3, 2 * TILE + 1, 4 * TILE], 2),  # multi-tile blocks on the scalar path
     ([1000] * 40, 16), ([12345, 54321, 99999], 9),   # generic-M server path
+    ([BIG], 7), ([BIG + 1, BIG - 1], 4), ([BIG - 4, 3 * BIG + TILE + 4, 2 * BIG + 2 * TILE], 7),
+    ([2 * TILE + 8, BIG + 3 * TILE, 5 * BIG + 100], 3),
 ])
 @pytest.mark.parametrize("scale_mode", ["fused", "split"])
 def test_small_layouts(sizes, M, scale_mode):
@@ -50,6 +53,38 @@ def test_zero_gradients_and_zero_blocks():
     grads = [[z, z], [g, g.flip(0) * 0 + g], [z, z]]
     eng, orc, _ = run_parity(w, grads=grads)
     assert eng.worker_scales(0)[1].item() == 0.0
+
+
+def test_negative_zero_inputs_follow_the_oracle():
+    """sign(-0) = +1: gradients made of -0.0 and exact cancellations must give the oracle's bits."""
+    w = _wl("negzero", [64, TILE, 96], 2, steps=4)
+    nz = torch.full((w.d,), -0.0)
+    g = torch.randn(w.d)
+    g[:64] = -0.0                       # a block that stays exactly zero
+    g[64:64 + 200:2] = -0.0
+    grads = [[nz, nz], [g, -g], [nz, g], [-g, nz]]
+    eng, orc, stats = run_parity(w, grads=grads)
+    assert stats["adopted"] == 0
+
+
+def test_imported_negative_zero_residual_is_canonicalised():
+    w = _wl("negzero-import", [TILE + 8, 40], 2, steps=2)
+    a = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    b = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    m0 = torch.randn(w.d, device="cuda")
+    e_pos = torch.zeros(w.d, device="cuda")
+    e_neg = torch.full((w.d,), -0.0, device="cuda")
+    for i in range(w.M):
+        a.set_state(i, m0, e_pos); b.set_state(i, m0, e_neg)
+    a.set_state(-1, None, e_pos); b.set_state(-1, None, e_neg)
+    for t in range(2):
+        for i in range(w.M):
+            g = w.draw_grad(t, i, "cuda")
+            a.worker_step(i, g); b.worker_step(i, g)
+        a.server_step(); b.server_step()
+    assert torch.equal(a.params(), b.params())
+    assert torch.equal(a.worker_words(0), b.worker_words(0))
+    assert torch.equal(a.residual(-1), b.residual(-1))
 
 
 def test_worker_order_does_not_matter():
