@@ -366,42 +366,51 @@ __global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a)
 // a_j = sum over ascending i of (bit_i ? -c_i : +c_i), c_i = fl(scale_{i,b} / M), the first
 // term taken as is (Algorithm 4, server line: (1/M) sum_i Delta_{t,i}).
 //
-// For M <= 8 the possible values of a_j inside one block are tabulated once per CTA in shared
-// memory (each entry is the same chain of fp32 additions, so the table is exact) and an
-// element costs one lookup instead of M dependent additions with 2 bit operations each.
+// For M <= 8 the sum over the first min(M, 6) workers is tabulated once per CTA in shared
+// memory (each entry is the same chain of fp32 additions, so the table is exact) and workers
+// 6 and 7 are added to the looked-up value directly, in order.  An element then costs one
+// lookup plus at most two additions instead of M dependent additions with 2 bit operations
+// each.  The table has at most 64 entries and is stored 32 times, entry e of copy l at word
+// 32*e + l, so that lane l always reads bank l: the lookups are free of bank conflicts.
 //
 // Building the table index without per-worker work in every lane: the 8 lanes that share a
-// packed word each load the word of ONE worker (lane q -> worker q).  Seen as an 8x8 matrix of
-// nibbles (row = worker, column = lane whose 4 elements the nibble belongs to), a three-stage
-// butterfly over the lanes (xor 4: half-words, xor 2: bytes, xor 1: nibbles) transposes it, so
-// lane r ends with N = the 8 workers' nibbles for its own 4 elements.  Two delta swaps of the
-// bit-index (4 <-> 1, 3 <-> 0) then turn N into R, whose byte k holds the 8 sign bits of
-// element k, worker i at bit kLutPos(i).  Byte k of R indexes the table.
+// packed word each load the word of ONE worker (lane q -> worker kLaneWorker(q)).  Seen as an
+// 8x8 matrix of nibbles (row = lane that loaded it, column = lane whose 4 elements the nibble
+// belongs to), a three-stage butterfly over the lanes (xor 4: half-words, xor 2: bytes, xor 1:
+// nibbles) transposes it, so lane r ends with N = the 8 nibbles for its own 4 elements.  Two
+// delta swaps of the bit-index (4 <-> 1, 3 <-> 0) then turn N into R, whose byte k holds the 8
+// sign bits of element k; the data loaded by lane q lands at bit kLaneWorker(q), i.e. worker w
+// sits at bit w.
 constexpr int kMaxLutWorkers = 8;
+constexpr int kLutWorkers = 6;        // workers covered by the table
+constexpr int kLutCopies = 32;        // one copy per lane
 
-__host__ __device__ constexpr int kLutPos(int i) {
-    return 4 * (i & 1) + 2 * ((i >> 2) & 1) + ((i >> 1) & 1);
+__host__ __device__ constexpr int kLaneWorker(int q) {
+    return 4 * (q & 1) + 2 * ((q >> 2) & 1) + ((q >> 1) & 1);
 }
-__host__ __device__ constexpr int kLutSize(int M) {   // 1 << (highest used bit position + 1)
-    int hi = 0;
-    for (int i = 0; i < M; ++i) hi = kLutPos(i) > hi ? kLutPos(i) : hi;
-    return 1 << (hi + 1);
-}
+__host__ __device__ constexpr int kLutEntries(int M) { return 1 << (M < kLutWorkers ? M : kLutWorkers); }
 
 __device__ __forceinline__ void build_scaled(const ServerArgs& a, int block, int M, float* s_c) {
     for (int i = threadIdx.x; i < M; i += kThreads)
         s_c[i] = __fdiv_rn(a.wscales[(long long)i * a.sstride + block], (float)M);
 }
 
+// s_base[idx] = (+-c_0) +- c_1 ... +- c_{T-1}, bit i of idx set = worker i negative, T = min(M, 6);
+// then every entry is written once per copy.  Ends with a barrier.
 template <int MT>
-__device__ __forceinline__ void build_lut(const float* s_c, float* s_lut) {
-    for (int idx = threadIdx.x; idx < kLutSize(MT); idx += kThreads) {
-        float v = ((idx >> kLutPos(0)) & 1) ? -s_c[0] : s_c[0];
+__device__ __forceinline__ void build_lut(const float* s_c, float* s_base, float* s_lut) {
+    constexpr int T = MT < kLutWorkers ? MT : kLutWorkers;
+    if (threadIdx.x < (1 << T)) {
+        const int idx = threadIdx.x;
+        float v = (idx & 1) ? -s_c[0] : s_c[0];
 #pragma unroll
-        for (int i = 1; i < MT; ++i)
-            v = __fadd_rn(v, ((idx >> kLutPos(i)) & 1) ? -s_c[i] : s_c[i]);
-        s_lut[idx] = v;
+        for (int i = 1; i < T; ++i) v = __fadd_rn(v, ((idx >> i) & 1) ? -s_c[i] : s_c[i]);
+        s_base[idx] = v;
     }
+    __syncthreads();
+    for (int e = threadIdx.x; e < (1 << T) * kLutCopies; e += kThreads)
+        s_lut[e] = s_base[e / kLutCopies];
+    __syncthreads();
 }
 
 __device__ __forceinline__ unsigned delta_swap(unsigned x, int d, unsigned mask) {
@@ -416,8 +425,8 @@ struct Butterfly {
     __device__ __forceinline__ explicit Butterfly(int q)
         : sel1((q & 4) ? 0x3276u : 0x5410u), sel2((q & 2) ? 0x3715u : 0x6240u),
           keep3((q & 1) ? 0xF0F0F0F0u : 0x0F0F0F0Fu), rot3((q & 1) ? 28 : 4) {}
-    // w: this lane's worker word (lane q of the 8-lane group holds worker q, 0 if q >= M).
-    // Returns R: byte k = table index of the lane's element k.
+    // w: the packed word this lane loaded (worker kLaneWorker(q), or 0 if there is no such worker).
+    // Returns R: bit 8k + i = sign bit of worker i for the lane's element k.
     __device__ __forceinline__ unsigned indices(unsigned w) const {
         unsigned x = w;
         x = __byte_perm(x, __shfl_xor_sync(kFull, x, 4), sel1);
@@ -456,24 +465,28 @@ __host__ __device__ constexpr size_t server_ring_bytes() {
 // flight during the lookups without costing registers; a ragged last chunk is loaded directly.
 template <int U, int MT>
 __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Tile& t, float sp,
-                                                  unsigned char* ring, float* s_c, float* s_lut) {
+                                                  unsigned char* ring, float* s_c, float* s_base,
+                                                  float* s_lut) {
     constexpr int kChunk = 1024 * U;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q = lane & 7;
     const int o0 = warp * (128 * U) + lane * 4;
+    const int wq = kLaneWorker(q);                 // the worker whose words this lane loads
+    const bool has_w = wq < MT;
     const Butterfly bf(q);
     float* const pbase = a.pb + t.start + o0;
     const uint32_t* const wbase =
-        a.wwords + (long long)(q < MT ? q : 0) * a.wstride + t.word + (o0 >> 5);
+        a.wwords + (long long)(has_w ? wq : 0) * a.wstride + t.word + (o0 >> 5);
     const int nfull = t.len / kChunk;              // chunks staged through shared memory
     const int tail = t.len - nfull * kChunk;       // ragged rest (only at the end of a block)
-    const char* lut = reinterpret_cast<const char*>(s_lut);
+    const char* lut = reinterpret_cast<const char*>(s_lut + lane);   // this lane's copy
     // slot (stage s, row u) of this thread: consecutive threads are 16 (4) bytes apart
     float4* const ring_p = reinterpret_cast<float4*>(ring) + threadIdx.x;
     unsigned* const ring_w =
         reinterpret_cast<unsigned*>(ring + (size_t)kServerStages * U * kThreads * sizeof(float4)) +
         threadIdx.x;
     double acc = 0.0;
+    unsigned c6 = 0, c7 = 0;               // bit patterns of the scaled scales of workers 6, 7
 
     auto issue_chunk = [&](int c) {
         if (c < nfull) {
@@ -483,7 +496,7 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 cp_async16(ring_p + (s * U + u) * kThreads, pp + u * 128);
-                if (q < MT) cp_async4(ring_w + (s * U + u) * kThreads, wp + u * 4);
+                if (has_w) cp_async4(ring_w + (s * U + u) * kThreads, wp + u * 4);
             }
         }
         cp_async_commit();                 // one (possibly empty) group per chunk index
@@ -496,11 +509,22 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
         for (int u = 0; u < U; ++u) {
             const int o = o0 + u * 128;
             const unsigned R = bf.indices(w[u]);
+            // byte offset of entry (R_k & 63) in this lane's copy: 128 * index
             float avg[4];
-            avg[0] = *reinterpret_cast<const float*>(lut + ((R << 2) & 0x3FCu));
-            avg[1] = *reinterpret_cast<const float*>(lut + ((R >> 6) & 0x3FCu));
-            avg[2] = *reinterpret_cast<const float*>(lut + ((R >> 14) & 0x3FCu));
-            avg[3] = *reinterpret_cast<const float*>(lut + ((R >> 22) & 0x3FCu));
+            avg[0] = *reinterpret_cast<const float*>(lut + ((R << 7) & 0x1F80u));
+            avg[1] = *reinterpret_cast<const float*>(lut + ((R >> 1) & 0x1F80u));
+            avg[2] = *reinterpret_cast<const float*>(lut + ((R >> 9) & 0x1F80u));
+            avg[3] = *reinterpret_cast<const float*>(lut + ((R >> 17) & 0x1F80u));
+            if (MT > 6) {                  // workers 6 and 7 follow in order
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    avg[k] = __fadd_rn(avg[k], __uint_as_float(c6 ^ ((R << (25 - 8 * k)) & 0x80000000u)));
+            }
+            if (MT > 7) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    avg[k] = __fadd_rn(avg[k], __uint_as_float(c7 ^ ((R << (24 - 8 * k)) & 0x80000000u)));
+            }
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 float pv = __fadd_rn(avg[k], residual_of(p[u][k], sp));      // ptilde_t
@@ -521,8 +545,9 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
     issue_chunk(1);
     build_scaled(a, t.block, MT, s_c);
     __syncthreads();
-    build_lut<MT>(s_c, s_lut);
-    __syncthreads();
+    build_lut<MT>(s_c, s_base, s_lut);
+    c6 = __float_as_uint(s_c[MT > 6 ? 6 : 0]);
+    c7 = __float_as_uint(s_c[MT > 7 ? 7 : 0]);
     for (int c = 0; c < nfull; ++c) {
         issue_chunk(c + 2);                // reuses the slot this thread consumed at c - 1
         cp_async_wait<2>();                // groups c+1 and c+2 may still be in flight
@@ -531,7 +556,7 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
         for (int u = 0; u < U; ++u) {
             const float4 v = ring_p[(s * U + u) * kThreads];
             p[u][0] = v.x; p[u][1] = v.y; p[u][2] = v.z; p[u][3] = v.w;
-            w[u] = (q < MT) ? ring_w[(s * U + u) * kThreads] : 0u;
+            w[u] = has_w ? ring_w[(s * U + u) * kThreads] : 0u;
         }
         compute_chunk(c, kChunk, p, w);
     }
@@ -542,7 +567,7 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
         for (int u = 0; u < U; ++u) {
             const int o = o0 + u * 128;
             load4(pp + u * 128, o, tail, false, p[u]);
-            w[u] = (q < MT && (o & ~31) < tail) ? __ldg(wp + u * 4) : 0u;
+            w[u] = (has_w && (o & ~31) < tail) ? __ldg(wp + u * 4) : 0u;
         }
         compute_chunk(nfull, tail, p, w);
     }
@@ -632,12 +657,13 @@ __global__ void __launch_bounds__(kThreads) ef_server_kernel(const ServerArgs a)
     // dynamic shared memory: [staging ring (table path only)] [M scaled worker scales]
     extern __shared__ __align__(16) unsigned char s_dyn[];
     float* s_c = reinterpret_cast<float*>(s_dyn + (MT > 0 ? server_ring_bytes<U>() : 0));
-    __shared__ float s_lut[MT > 0 ? kLutSize(MT) : 1];
+    __shared__ float s_base[MT > 0 ? kLutEntries(MT) : 1];
+    __shared__ float s_lut[MT > 0 ? kLutEntries(MT) * kLutCopies : 1];
     const Tile t = a.tiles[blockIdx.x];
     const float sp = a.rscale[t.block];
     double acc = 0.0;
     if (MT > 0 && (t.start & 3) == 0) {
-        acc = server_tile_lut<U, (MT > 0 ? MT : 1)>(a, t, sp, s_dyn, s_c, s_lut);
+        acc = server_tile_lut<U, (MT > 0 ? MT : 1)>(a, t, sp, s_dyn, s_c, s_base, s_lut);
     } else {
         build_scaled(a, t.block, a.M, s_c);
         __syncthreads();
