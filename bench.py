@@ -37,7 +37,7 @@ UNIT = "params/s"
 
 # DRAM traffic per launch of the worker kernel measured by ncu (dram__bytes_read.sum +
 # dram__bytes_write.sum), in bytes per parameter; see profiles/ for the capture it comes from.
-NCU_WORKER_TRAFFIC_BYTES_PER_PARAM = None
+NCU_WORKER_TRAFFIC_BYTES_PER_PARAM = 19.91   # 5.3445e9 bytes per launch at d = 2^28
 
 
 # --------------------------------------------------------------------------- byte counts

@@ -26,6 +26,7 @@
 #pragma once
 
 #include <cstdint>
+#include <type_traits>
 #include <cuda_runtime.h>
 
 namespace efk {
@@ -501,8 +502,9 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
         }
         cp_async_commit();                 // one (possibly empty) group per chunk index
     };
-    auto compute_chunk = [&](int c, int clen, float (&p)[U][4], unsigned (&w)[U]) {
-        const bool full = clen == kChunk;
+    // full_c: std::true_type for a whole chunk (no bounds checks), std::false_type for the tail
+    auto compute_chunk = [&](auto full_c, int c, int clen, float (&p)[U][4], unsigned (&w)[U]) {
+        constexpr bool full = decltype(full_c)::value;
         float* pp = pbase + (long long)c * kChunk;
         uint32_t* words = a.words + t.word + c * (kChunk / 32);
 #pragma unroll
@@ -558,7 +560,7 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
             p[u][0] = v.x; p[u][1] = v.y; p[u][2] = v.z; p[u][3] = v.w;
             w[u] = has_w ? ring_w[(s * U + u) * kThreads] : 0u;
         }
-        compute_chunk(c, kChunk, p, w);
+        compute_chunk(std::true_type{}, c, kChunk, p, w);
     }
     if (tail > 0) {
         const float* pp = pbase + (long long)nfull * kChunk;
@@ -569,7 +571,7 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
             load4(pp + u * 128, o, tail, false, p[u]);
             w[u] = (has_w && (o & ~31) < tail) ? __ldg(wp + u * 4) : 0u;
         }
-        compute_chunk(nfull, tail, p, w);
+        compute_chunk(std::false_type{}, nfull, tail, p, w);
     }
     cp_async_wait<0>();
     return acc;
