@@ -44,7 +44,8 @@ enum ef_status {
     EF_ERR_ALIGNMENT = 4,          /* a device pointer is not 16-byte aligned */
     EF_ERR_CUDA = 5,               /* a CUDA runtime call failed; see ef_last_cuda_error */
     EF_ERR_UNSUPPORTED_DEVICE = 6, /* current device is not compute capability 10.x */
-    EF_ERR_TIMEOUT = 7             /* reserved: a bounded device-side wait gave up */
+    EF_ERR_TIMEOUT = 7,            /* reserved: a bounded device-side wait gave up */
+    EF_ERR_TOO_LARGE = 8           /* ef_worker_step_noalloc: n exceeds EF_NOALLOC_MAX_ELEMS */
 };
 
 /* Flags for ef_workspace_bytes / ef_init. */
@@ -134,6 +135,42 @@ int ef_step_count(ef_ctx* ctx, int64_t* t /* out: completed iterations */);
 
 /* Number of kernels this context has launched so far (for launch accounting). */
 int64_t ef_launch_count(ef_ctx* ctx);
+
+/* (The paper has no counterpart for this entry point; it exists for deployment reasons.)
+ * The worker step of one block for callers that must not allocate device memory where they
+ * step the optimizer: code that runs while another framework owns the allocator or the stream
+ * (callbacks, plugins with a fixed arena), and latency-critical loops that cannot afford the
+ * device-wide synchronisation an allocation may imply.  Unlike the context API it takes no
+ * workspace: its scratch (one fp64 partial sum per 4096 elements and an arrival counter, 33 KB)
+ * is a fixed array inside the library image, which every GPU that loads the library keeps until
+ * the process exits.  The call itself performs no cudaMalloc/cudaFree and uses no allocating
+ * library routine.
+ *
+ * Computes, for ONE block of n elements and state kept by the caller (all device pointers):
+ *   momentum[n]        in/out  m <- mu*m + grad
+ *   residual[n]        in/out  deferred residual buffer: holds p of the previous call on entry
+ *                              and p = mu*m + grad + e on exit, where e_j = p_prev_j - s_prev *
+ *                              sign(p_prev_j); start from zeros
+ *   residual_scale[1]  in/out  s_prev on entry, the new scale on exit; start from zero
+ *   words[ceil(n/32)]  out     packed signs of p (layout as described at the top of this file)
+ *   scale[1]           out     ||p||_1 / n
+ * i.e. exactly what ef_worker_step computes for a layout with a single block, bit for bit.
+ * grad, momentum and residual must be 16-byte aligned.  Work is enqueued on cuda_stream; no
+ * host synchronisation.
+ *
+ * Limits and sharing: n <= EF_NOALLOC_MAX_ELEMS, else EF_ERR_TOO_LARGE and nothing is launched.
+ * All calls on a device share the one scratch array: calls that may overlap on the GPU (different
+ * streams, or several host threads) race on it and must be serialised by the caller; calls
+ * queued on one stream are safe.  The array keeps the previous call's contents; the call clears
+ * the one cell that has to start at zero itself.
+ *
+ * The first call on each device looks up the array's device address (a short, one-time set-up
+ * under a lock); make that first call outside any stream capture.
+ * Errors: INVALID_ARG, TOO_LARGE, ALIGNMENT, UNSUPPORTED_DEVICE, CUDA. */
+#define EF_NOALLOC_MAX_ELEMS (1 << 24)
+int ef_worker_step_noalloc(const float* grad, float* momentum, float* residual,
+                           float* residual_scale, int64_t n, float mu,
+                           uint32_t* words, float* scale, void* cuda_stream);
 
 const char* ef_strerror(int status);
 int ef_last_cuda_error(ef_ctx* ctx);      /* the cudaError_t of the last EF_ERR_CUDA, else 0 */

@@ -24,6 +24,8 @@ EF_ERR_ALIGNMENT = 4
 EF_ERR_CUDA = 5
 EF_ERR_UNSUPPORTED_DEVICE = 6
 EF_ERR_TIMEOUT = 7
+EF_ERR_TOO_LARGE = 8
+EF_NOALLOC_MAX_ELEMS = 1 << 24
 EF_FLAG_HOST_STAGING = 1
 EF_FLAG_FUSED_SCALE = 2
 EF_FLAG_SPLIT_SCALE = 4
@@ -52,6 +54,7 @@ SIGNATURES = {
     "ef_set_state": (ctypes.c_int, [_vp, _i32, _vp, _vp]),
     "ef_step_count": (ctypes.c_int, [_vp, ctypes.POINTER(_i64)]),
     "ef_launch_count": (_i64, [_vp]),
+    "ef_worker_step_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _f32, _vp, _vp, _vp]),
     "ef_strerror": (ctypes.c_char_p, [ctypes.c_int]),
     "ef_last_cuda_error": (ctypes.c_int, [_vp]),
     "ef_destroy": (ctypes.c_int, [_vp]),
@@ -170,6 +173,16 @@ def ef_step_count(ctx: int) -> int:
 
 def ef_launch_count(ctx: int) -> int:
     return load_library().ef_launch_count(ctx)
+
+
+def ef_worker_step_noalloc(grad_ptr: int, momentum_ptr: int, residual_ptr: int,
+                           residual_scale_ptr: int, n: int, mu: float, words_ptr: int,
+                           scale_ptr: int, cuda_stream: int) -> None:
+    """Worker step of one block without any workspace (scratch is a fixed array in the library);
+    for callers that must not allocate device memory.  See include/ef.h for the contract."""
+    _check(load_library().ef_worker_step_noalloc(grad_ptr, momentum_ptr, residual_ptr,
+                                                 residual_scale_ptr, n, mu, words_ptr, scale_ptr,
+                                                 cuda_stream), "ef_worker_step_noalloc")
 
 
 def ef_last_cuda_error(ctx: int) -> int:

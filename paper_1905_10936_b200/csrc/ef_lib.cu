@@ -8,6 +8,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -435,6 +436,7 @@ const char* ef_strerror(int status) {
         case EF_ERR_CUDA: return "CUDA runtime error";
         case EF_ERR_UNSUPPORTED_DEVICE: return "device is not compute capability 10.x";
         case EF_ERR_TIMEOUT: return "device-side wait timed out";
+        case EF_ERR_TOO_LARGE: return "size exceeds the fixed scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }
@@ -453,3 +455,130 @@ int ef_destroy(ef_ctx* c) {
 }
 
 }  // extern "C"
+
+// =============================================================================================
+// ef_worker_step_noalloc: the worker step for callers that cannot allocate device memory.
+//
+// Some hosts of this library are not allowed to call cudaMalloc at the point where they step
+// the optimizer: code running inside a CUDA-graph capture or another framework's stream
+// callback, plugins that were handed a fixed arena and must not grow it, and real-time loops
+// where an allocation (which may synchronise the whole device) is not tolerable.  The regular
+// entry points avoid allocation by taking a caller-sized workspace; this variant needs not even
+// that: its scratch memory (one fp64 partial sum per 4096-element chunk plus one arrival
+// counter) lives in a fixed array inside the library image, so the caller passes only the
+// inputs and outputs of the step.  The price is a size limit (EF_NOALLOC_MAX_ELEMS) and that all
+// calls on a device share the one array.
+// =============================================================================================
+namespace {
+
+constexpr int kNoAllocMaxChunks = EF_NOALLOC_MAX_ELEMS / kChunkLen;
+// Scratch of the no-allocation entry point: [0, kNoAllocMaxChunks) partial sums, then one
+// 8-byte cell whose low word is the arrival counter.  Every GPU that loads the library holds
+// this array (33 KB) until the process exits.
+static __device__ __align__(256) double ef_noalloc_scratch[kNoAllocMaxChunks + 1];
+
+struct NoAllocArgs {
+    efk::WorkerArgs w;        // g, m, pb, words, mu (tables unused)
+    float* rscale_io;         // scale that belongs to pb: read at entry, replaced at exit
+    float* scale_out;         // the message's scale
+    double* partials;         // device address of ef_noalloc_scratch
+    unsigned* ticket;         // arrival counter inside the scratch array (0 at launch)
+    long long n;
+    int chunks;
+};
+
+// Same element arithmetic, chunking and summation order as ef_worker_kernel on a layout with
+// a single block of n elements; chunk geometry is computed instead of read from a table.
+template <int U>
+__global__ void __launch_bounds__(efk::kThreads) ef_worker_noalloc_kernel(const NoAllocArgs a) {
+    __shared__ double s_sum[efk::kWarps];
+    __shared__ int s_last;
+    Tile t;
+    t.start = (long long)blockIdx.x * (1024 * U);
+    t.word = (long long)blockIdx.x * (1024 * U / 32);
+    const long long rest = a.n - t.start;
+    t.len = (int)(rest < 1024 * U ? rest : 1024 * U);
+    t.block = 0; t.pad0 = 0; t.pad1 = 0;
+    const float sp = *a.rscale_io;
+    const double acc = (t.len == 1024 * U) ? efk::worker_rows<U, true>(a.w, t, sp)
+                                           : efk::worker_rows<U, false>(a.w, t, sp);
+    double S = efk::cta_sum(acc, s_sum);
+    if (threadIdx.x == 0) {
+        int last = 0;
+        if (a.chunks == 1) {
+            const float s = (float)(S / (double)a.n);
+            *a.scale_out = s;
+            *a.rscale_io = s;
+        } else {
+            a.partials[blockIdx.x] = S;
+            __threadfence();
+            last = (atomicAdd(a.ticket, 1u) + 1u == (unsigned)a.chunks);
+        }
+        s_last = last;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    double v = 0.0;
+    for (int k = threadIdx.x; k < a.chunks; k += efk::kThreads) v += __ldcg(&a.partials[k]);
+    S = efk::cta_sum(v, s_sum);
+    if (threadIdx.x == 0) {
+        const float s = (float)(S / (double)a.n);
+        *a.scale_out = s;
+        *a.rscale_io = s;       // every CTA has read the old value before it took its ticket
+    }
+}
+
+constexpr int kNoAllocMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+double* g_noalloc_ptr[kNoAllocMaxDevices] = {};   // device address of the scratch, per device
+
+}  // namespace
+
+extern "C" int ef_worker_step_noalloc(const float* grad, float* momentum, float* residual,
+                                      float* residual_scale, int64_t n, float mu,
+                                      uint32_t* words, float* scale, void* cuda_stream) {
+    if (!grad || !momentum || !residual || !residual_scale || !words || !scale || n < 1)
+        return EF_ERR_INVALID_ARG;
+    if (!(mu >= 0.f && mu < 1.f)) return EF_ERR_INVALID_ARG;
+    if (n > (int64_t)EF_NOALLOC_MAX_ELEMS) return EF_ERR_TOO_LARGE;
+    if (!aligned16(grad) || !aligned16(momentum) || !aligned16(residual)) return EF_ERR_ALIGNMENT;
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return EF_ERR_CUDA;
+    if (dev < 0 || dev >= kNoAllocMaxDevices) return EF_ERR_UNSUPPORTED_DEVICE;
+    double* scratch = nullptr;
+    {
+        // One-time set-up per device, done by the first call on that device (with the device
+        // current).  In host code the array's name is only a stand-in for the symbol, not a
+        // device address, so the address is looked up once and kept.
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (!g_noalloc_ptr[dev]) {
+            int major = 0;
+            if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+                return EF_ERR_CUDA;
+            if (major != 10) return EF_ERR_UNSUPPORTED_DEVICE;
+            double* p = nullptr;
+            if (cudaGetSymbolAddress((void**)&p, ef_noalloc_scratch) != cudaSuccess || !p)
+                return EF_ERR_CUDA;
+            g_noalloc_ptr[dev] = p;
+        }
+        scratch = g_noalloc_ptr[dev];
+    }
+
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    NoAllocArgs a;
+    a.w.g = grad; a.w.m = momentum; a.w.pb = residual; a.w.words = words;
+    a.w.scale_out = nullptr; a.w.rscale = nullptr; a.w.partials = nullptr; a.w.tickets = nullptr;
+    a.w.tiles = nullptr; a.w.blocks = nullptr; a.w.mu = mu; a.w.fused = 1;
+    a.rscale_io = residual_scale; a.scale_out = scale;
+    a.partials = scratch;
+    a.ticket = reinterpret_cast<unsigned*>(scratch + kNoAllocMaxChunks);
+    a.n = n;
+    a.chunks = (int)((n + kChunkLen - 1) / kChunkLen);
+    // The array keeps whatever the previous call left; only the counter must start at zero.
+    if (cudaMemsetAsync(a.ticket, 0, sizeof(double), stream) != cudaSuccess) return EF_ERR_CUDA;
+    ef_worker_noalloc_kernel<kU><<<(unsigned)a.chunks, efk::kThreads, 0, stream>>>(a);
+    if (cudaGetLastError() != cudaSuccess) return EF_ERR_CUDA;
+    return EF_OK;
+}
