@@ -197,14 +197,26 @@ def run_ours(args) -> None:
 
     w = load_workload(args)
     K, W = args.steps, args.warmup
-    eng = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    # all work of the context runs on this (non-default) stream, which is also made current
+    stream = torch.cuda.Stream(device=dev)
+    torch.cuda.set_stream(stream)
+    eng = EFEngine(w.offsets, w.M, w.mu, w.eta, stream=stream)
     es = w.element_scales(dev)
-    grads = [w.draw_grad(0, i, dev, es) for i in range(w.M)]      # pre-staged in HBM
+    stride = (w.d + 3) // 4 * 4
+    gall = torch.zeros(w.M, stride, dtype=torch.float32, device=dev)   # pre-staged in HBM
+    grads = [w.draw_grad(0, i, dev, es, out=gall[i, :w.d]) for i in range(w.M)]
     del es
+    batched = not args.per_worker_calls
+
+    def worker_calls():
+        if batched:
+            eng.worker_step_all(gall)          # all M workers in one launch
+        else:
+            for i in range(w.M):
+                eng.worker_step(i, grads[i])
 
     def one_step():
-        for i in range(w.M):
-            eng.worker_step(i, grads[i])
+        worker_calls()
         eng.server_step()
 
     for _ in range(W):
@@ -217,8 +229,7 @@ def run_ours(args) -> None:
     barrier()
     for k in range(K):
         ev[k][0].record()
-        for i in range(w.M):
-            eng.worker_step(i, grads[i])
+        worker_calls()
         ev[k][1].record()
         eng.server_step()
         ev[k][2].record()
@@ -226,19 +237,44 @@ def run_ours(args) -> None:
     clocks = sampler.stop()
     launches = eng.launch_count - launches0
     total_ms = ev[0][0].elapsed_time(ev[K - 1][2])
-    worker_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / (K * w.M)
+    launches_per_step_worker = 1 if batched else w.M
+    worker_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / (K * launches_per_step_worker)
     server_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / K
     if world > 1:
         tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         total_ms = float(tt.item())
 
+    # ---- the same step replayed from a CUDA graph (launch gaps shrink; matters for small layouts)
+    graph_info = None
+    if args.graph:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            one_step()
+        for _ in range(3):
+            g.replay()
+        barrier()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for _ in range(K):
+            g.replay()
+        g1.record()
+        barrier()
+        g_ms = g0.elapsed_time(g1)
+        if world > 1:
+            tt = torch.tensor([g_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            g_ms = float(tt.item())
+        graph_info = {"ms_per_step": g_ms / K, "value": world * w.d * K / (g_ms * 1e-3),
+                      "unit": UNIT, "note": "one whole step captured once, replayed K times"}
+        del g
+
     # ---- end to end: host gradients in, packed update out, copies inside the timed region
     e2e = None
     if not args.no_e2e:
         del eng
         torch.cuda.empty_cache()
-        eng2 = EFEngine(w.offsets, w.M, w.mu, w.eta, host_staging=True)
+        eng2 = EFEngine(w.offsets, w.M, w.mu, w.eta, host_staging=True, stream=stream)
         hgrads = []
         for i in range(w.M):
             h = torch.empty(w.d, dtype=torch.float32).pin_memory()
@@ -284,7 +320,7 @@ def run_ours(args) -> None:
         return
 
     peak, peak_kind = measured_hbm_peak()
-    wbytes = worker_call_bytes(w.d, w.B)
+    wbytes = worker_call_bytes(w.d, w.B) * (w.M if batched else 1)
     sbytes = server_call_bytes(w.d, w.B, w.M)
     w_gbs = wbytes / (worker_ms * 1e-3) / 1e9
     s_gbs = sbytes / (server_ms * 1e-3) / 1e9
@@ -296,6 +332,7 @@ def run_ours(args) -> None:
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
         "config": {"workload": w.name, "d": w.d, "B": w.B, "M": w.M, "mu": w.mu, "eta": w.eta,
+                   "worker_calls": "ef_worker_step_all" if batched else "ef_worker_step x M",
                    "per_gpu": "each rank owns one such layout (block-range shard of an "
                               "N-times larger problem)",
                    "l2": f"no flush: state+gradients {state_gib:.1f} GiB per GPU, far larger "
@@ -304,11 +341,13 @@ def run_ours(args) -> None:
         "e2e": e2e,
         "gpu_launches": int(launches * world),
         "roofline": {
-            "kernel": "ef_worker_kernel", "bound": "hbm", "achieved": w_gbs, "peak": peak,
+            "kernel": "ef_worker_kernel", "call": ("ef_worker_step_all: M workers per launch" if batched
+                                                   else "ef_worker_step: one worker per launch"),
+            "bound": "hbm", "achieved": w_gbs, "peak": peak,
             "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": w_gbs / peak,
             "frac_of_8000_nominal": w_gbs / 8000.0,
             "bytes_per_launch": wbytes, "ms_per_launch": worker_ms,
-            "traffic": (NCU_WORKER_TRAFFIC_BYTES_PER_PARAM * w.d
+            "traffic": (NCU_WORKER_TRAFFIC_BYTES_PER_PARAM * w.d * (w.M if batched else 1)
                         if NCU_WORKER_TRAFFIC_BYTES_PER_PARAM else None),
         },
         "roofline_server": {
@@ -319,6 +358,8 @@ def run_ours(args) -> None:
         },
         "step_gbs": step_bytes(w.d, w.B, w.M) / (total_ms / K * 1e-3) / 1e9,
     }
+    if graph_info is not None:
+        line["cuda_graph"] = graph_info
     if world == 1 and not args.no_cpu_baseline:
         per_block = np.mean(w.sizes) * oracle_ns_per_param(w.M) * 1e-9
         steps_c = 2
@@ -356,7 +397,11 @@ def main():
                     help="use only the first N blocks of the workload (small cases for profiling)")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--per-worker-calls", action="store_true",
+                    help="step the workers with M ef_worker_step calls instead of one ef_worker_step_all")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--graph", action="store_true",
+                    help="also time the step replayed from a CUDA graph (extra key cuda_graph)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3:

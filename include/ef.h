@@ -13,6 +13,10 @@
  * owning it.  Every call only enqueues work on the CUDA stream given to ef_init and returns
  * without synchronising; results are ordered on that stream.
  *
+ * Because the step calls (ef_worker_step, ef_server_step) only enqueue kernels on that stream,
+ * a caller may record them into a CUDA graph by capturing the stream; the host-side counters
+ * and call-order checks then see the captured calls only, not the replays.
+ *
  * There is no CPU fallback: on a device that is not compute capability 10.x ef_init fails
  * with EF_ERR_UNSUPPORTED_DEVICE.
  *
@@ -90,6 +94,14 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets /* host, 
  * Errors: INVALID_ARG (i, null), ALIGNMENT, BAD_STATE (worker i already stepped in this
  * iteration), CUDA. */
 int ef_worker_step(ef_ctx* ctx, int32_t i, const float* grad /* device */);
+
+/* All M workers in one launch: the same computation as ef_worker_step(ctx, i, grads + i*stride)
+ * for i = 0 .. M-1 (the workers are independent of each other, Algorithm 4), with one kernel
+ * launch instead of M.  grads: device, 16-byte aligned; stride: elements between the gradients
+ * of consecutive workers, >= d and a multiple of 4.  No worker may have been stepped yet in
+ * this iteration.  Results are bit-identical to the per-worker calls.
+ * Errors: INVALID_ARG, ALIGNMENT, BAD_STATE, CUDA. */
+int ef_worker_step_all(ef_ctx* ctx, const float* grads /* device, M gradients */, int64_t stride);
 
 /* Same as ef_worker_step with the gradient in HOST memory (pinned memory recommended): the
  * gradient is copied to a staging buffer on an internal copy stream, double-buffered so that

@@ -40,6 +40,7 @@ SIGNATURES = {
     "ef_init": (ctypes.c_int, [ctypes.POINTER(_vp), _i64, _i32, _vp, _i32, _f32, _f32, _u32, _vp,
                                ctypes.c_size_t, _vp]),
     "ef_worker_step": (ctypes.c_int, [_vp, _i32, _vp]),
+    "ef_worker_step_all": (ctypes.c_int, [_vp, _vp, _i64]),
     "ef_worker_step_host": (ctypes.c_int, [_vp, _i32, _vp]),
     "ef_server_step": (ctypes.c_int, [_vp]),
     "ef_read_update_host": (ctypes.c_int, [_vp, _vp, _vp]),
@@ -114,6 +115,10 @@ def ef_init(d: int, B: int, offsets, M: int, mu: float, eta: float, flags: int,
 
 def ef_worker_step(ctx: int, i: int, grad_ptr: int) -> None:
     _check(load_library().ef_worker_step(ctx, i, grad_ptr), "ef_worker_step")
+
+
+def ef_worker_step_all(ctx: int, grads_ptr: int, stride: int) -> None:
+    _check(load_library().ef_worker_step_all(ctx, grads_ptr, stride), "ef_worker_step_all")
 
 
 def ef_worker_step_host(ctx: int, i: int, grad_host_ptr: int) -> None:

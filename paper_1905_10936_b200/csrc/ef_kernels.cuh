@@ -70,6 +70,9 @@ struct WorkerArgs {
     const Block* blocks;
     float mu;
     int fused;             // 1: last CTA of a block finalises its scale; 0: ef_scale_kernel does
+    // batched launches: blockIdx.y selects the worker; its buffers lie at these strides
+    long long g_stride, state_stride, word_stride, partial_stride;
+    int scale_stride;      // also the stride of the ticket arrays
 };
 
 struct ServerArgs {
@@ -95,6 +98,8 @@ struct ScaleArgs {
     const int* multi;        // ids of the blocks that span more than one chunk
     float* scale_out;
     float* rscale;
+    long long partial_stride;   // blockIdx.y selects the buffer set (worker)
+    int scale_stride;
 };
 
 struct ApplyArgs {
@@ -234,7 +239,9 @@ __global__ void __launch_bounds__(kThreads) ef_scale_kernel(const ScaleArgs a) {
     __shared__ double s_sum[kWarps];
     const int block_id = a.multi[blockIdx.x];
     const Block b = a.blocks[block_id];
-    sum_partials_and_write(b, block_id, a.partials, a.scale_out, a.rscale, s_sum);
+    const long long so = (long long)blockIdx.y * a.scale_stride;
+    sum_partials_and_write(b, block_id, a.partials + blockIdx.y * a.partial_stride,
+                           a.scale_out + so, a.rscale + so, s_sum);
 }
 
 // Packs the four sign bits each lane holds (nibble, element k in bit k) into 32-bit words:
@@ -343,8 +350,21 @@ __device__ __forceinline__ double worker_rows_scalar(const WorkerArgs& a, const 
     return acc;
 }
 
+// grid.x = chunks, grid.y = workers stepped by this launch (1 for ef_worker_step).
 template <int U>
-__global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a) {
+__global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a0) {
+    WorkerArgs a = a0;
+    {
+        const long long wi = blockIdx.y;
+        a.g += wi * a.g_stride;
+        a.m += wi * a.state_stride;
+        a.pb += wi * a.state_stride;
+        a.words += wi * a.word_stride;
+        a.partials += wi * a.partial_stride;
+        a.scale_out += wi * a.scale_stride;
+        a.rscale += wi * a.scale_stride;
+        a.tickets += wi * a.scale_stride;
+    }
     const Tile t = chunk_of<U>(a.tiles[blockIdx.x / kTileChunks], blockIdx.x % kTileChunks);
     const Block b = a.blocks[t.block];
     const bool alone = b.len <= 1024 * U;              // the block is this single chunk

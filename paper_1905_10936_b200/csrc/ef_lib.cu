@@ -143,39 +143,69 @@ inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
 // Non-fused mode: adds the partial sums of every block larger than one chunk of buffer set k
 // (worker k, or the server for k == M) after the kernel that produced them.
-int launch_scale(ef_ctx* c, int k) {
+int launch_scale(ef_ctx* c, int k, int count = 1) {
     if (c->fused || c->L.num_multi == 0) return EF_OK;
     efk::ScaleArgs a;
     a.partials = c->partials(k); a.blocks = c->blocks(); a.multi = c->multi();
     a.scale_out = c->scales(k); a.rscale = c->rscale(k);
-    efk::ef_scale_kernel<<<(unsigned)c->L.num_multi, efk::kThreads, 0, c->stream>>>(a);
+    a.partial_stride = (long long)c->L.tpad; a.scale_stride = (int)c->L.bpad;
+    efk::ef_scale_kernel<<<dim3((unsigned)c->L.num_multi, (unsigned)count), efk::kThreads, 0,
+                           c->stream>>>(a);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
     return EF_OK;
 }
 
-int launch_worker(ef_ctx* c, int i, const float* grad) {
+// Steps workers i .. i+count-1; worker i+k reads its gradient at grad + k*g_stride.
+int launch_worker(ef_ctx* c, int i, const float* grad, int count = 1, long long g_stride = 0) {
     efk::WorkerArgs a;
     a.g = grad; a.m = c->m(i); a.pb = c->pb(i); a.words = c->words(i);
     a.scale_out = c->scales(i); a.rscale = c->rscale(i);
     a.partials = c->partials(i); a.tickets = c->tickets(i);
     a.tiles = c->tiles(); a.blocks = c->blocks(); a.mu = c->mu; a.fused = c->fused;
-    efk::ef_worker_kernel<kU><<<(unsigned)(c->L.num_tiles * efk::kTileChunks), efk::kThreads, 0, c->stream>>>(a);
+    a.g_stride = g_stride; a.state_stride = (long long)c->L.dpad;
+    a.word_stride = (long long)c->L.wpad; a.partial_stride = (long long)c->L.tpad;
+    a.scale_stride = (int)c->L.bpad;
+    efk::ef_worker_kernel<kU><<<dim3((unsigned)(c->L.num_tiles * efk::kTileChunks), (unsigned)count),
+                                efk::kThreads, 0, c->stream>>>(a);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
-    return launch_scale(c, i);
+    return launch_scale(c, i, count);
+}
+
+template <int MT>
+size_t server_smem_bytes(int M) {
+    return (MT > 0 ? efk::server_ring_bytes<kU>() : 0) + (size_t)M * sizeof(float);
+}
+
+// Raises the dynamic shared-memory limit of the server kernel this context will use.  Done once
+// in ef_init so that the step calls themselves only enqueue work.
+template <int MT>
+cudaError_t prepare_server_t(int M) {
+    const size_t smem = server_smem_bytes<MT>(M);
+    if (smem <= 48 * 1024) return cudaSuccess;
+    return cudaFuncSetAttribute(efk::ef_server_kernel<kU, MT>,
+                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+}
+
+cudaError_t prepare_server(int M) {
+    switch (M) {
+        case 1: return prepare_server_t<1>(M);
+        case 2: return prepare_server_t<2>(M);
+        case 3: return prepare_server_t<3>(M);
+        case 4: return prepare_server_t<4>(M);
+        case 5: return prepare_server_t<5>(M);
+        case 6: return prepare_server_t<6>(M);
+        case 7: return prepare_server_t<7>(M);
+        case 8: return prepare_server_t<8>(M);
+        default: return prepare_server_t<0>(M);
+    }
 }
 
 template <int MT>
 cudaError_t launch_server_t(ef_ctx* c, const efk::ServerArgs& a) {
-    const size_t smem = (MT > 0 ? efk::server_ring_bytes<kU>() : 0) + (size_t)c->L.M * sizeof(float);
-    if (smem > 48 * 1024) {
-        const cudaError_t e = cudaFuncSetAttribute(efk::ef_server_kernel<kU, MT>,
-                                                   cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)smem);
-        if (e != cudaSuccess) return e;
-    }
-    efk::ef_server_kernel<kU, MT><<<(unsigned)c->L.num_tiles, efk::kThreads, smem, c->stream>>>(a);
+    efk::ef_server_kernel<kU, MT><<<(unsigned)c->L.num_tiles, efk::kThreads,
+                                    server_smem_bytes<MT>(c->L.M), c->stream>>>(a);
     return cudaGetLastError();
 }
 
@@ -301,6 +331,7 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
         (ce = cudaMemcpyAsync(c->ws + L.off_multi, c->h_multi.data(),
                               c->h_multi.size() * sizeof(int32_t), cudaMemcpyHostToDevice,
                               c->stream)) != cudaSuccess) return fail(ce);
+    if ((ce = prepare_server(M)) != cudaSuccess) return fail(ce);
     if (flags & EF_FLAG_HOST_STAGING) {
         if ((ce = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking)) != cudaSuccess)
             return fail(ce);
@@ -323,6 +354,17 @@ int ef_worker_step(ef_ctx* c, int32_t i, const float* grad) {
     rc = launch_worker(c, i, grad);
     if (rc != EF_OK) return rc;
     c->stepped[i] = 1; c->pending += 1;
+    return EF_OK;
+}
+
+int ef_worker_step_all(ef_ctx* c, const float* grads, int64_t stride) {
+    if (!c || !grads || stride < c->L.d) return EF_ERR_INVALID_ARG;
+    if (!aligned16(grads) || (stride & 3) != 0) return EF_ERR_ALIGNMENT;
+    if (c->pending != 0) return EF_ERR_BAD_STATE;
+    const int rc = launch_worker(c, 0, grads, c->L.M, (long long)stride);
+    if (rc != EF_OK) return rc;
+    std::fill(c->stepped.begin(), c->stepped.end(), (uint8_t)1);
+    c->pending = c->L.M;
     return EF_OK;
 }
 
@@ -571,6 +613,8 @@ extern "C" int ef_worker_step_noalloc(const float* grad, float* momentum, float*
     a.w.g = grad; a.w.m = momentum; a.w.pb = residual; a.w.words = words;
     a.w.scale_out = nullptr; a.w.rscale = nullptr; a.w.partials = nullptr; a.w.tickets = nullptr;
     a.w.tiles = nullptr; a.w.blocks = nullptr; a.w.mu = mu; a.w.fused = 1;
+    a.w.g_stride = 0; a.w.state_stride = 0; a.w.word_stride = 0; a.w.partial_stride = 0;
+    a.w.scale_stride = 0;
     a.rscale_io = residual_scale; a.scale_out = scale;
     a.partials = scratch;
     a.ticket = reinterpret_cast<unsigned*>(scratch + kNoAllocMaxChunks);

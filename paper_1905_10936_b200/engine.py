@@ -63,6 +63,12 @@ class EFEngine:
         assert grad.is_contiguous()
         ef.ef_worker_step(self.ctx, i, grad.data_ptr())
 
+    def worker_step_all(self, grads: torch.Tensor) -> None:
+        """grads: [M, stride] fp32 on the device, row i = gradient of worker i (stride >= d)."""
+        assert grads.is_cuda and grads.dtype == torch.float32 and grads.dim() == 2
+        assert grads.shape[0] == self.M and grads.shape[1] >= self.d and grads.stride(1) == 1
+        ef.ef_worker_step_all(self.ctx, grads.data_ptr(), grads.stride(0))
+
     def worker_step_host(self, i: int, grad: torch.Tensor) -> None:
         assert (not grad.is_cuda) and grad.dtype == torch.float32 and grad.numel() == self.d
         assert grad.is_contiguous()

@@ -81,7 +81,7 @@ def assert_scales_close(got: np.ndarray, ref: np.ndarray, what: str):
 
 def run_parity(w: Workload, steps: Optional[int] = None, blocks: Optional[Sequence[int]] = None,
                grads: Optional[List[List[torch.Tensor]]] = None, check_every_step: bool = True,
-               device: str = "cuda", scale_mode: str = "auto"):
+               device: str = "cuda", scale_mode: str = "auto", batched: bool = False):
     """Runs `steps` iterations on both sides; returns (engine, oracle, stats)."""
     steps = w.steps if steps is None else steps
     eng = EFEngine(w.offsets, w.M, w.mu, w.eta, scale_mode=scale_mode)
@@ -89,11 +89,24 @@ def run_parity(w: Workload, steps: Optional[int] = None, blocks: Optional[Sequen
     orc = Oracle(smp.sub_offsets, w.M, w.mu, w.eta)
     es = w.element_scales(device)
     gbuf = torch.empty(w.d, dtype=torch.float32, device=device)
+    # batched mode: all M gradients in one [M, stride] tensor, one ef_worker_step_all per step
+    stride = (w.d + 3) // 4 * 4
+    gall = torch.zeros(w.M, stride, dtype=torch.float32, device=device) if batched else None
     stats = {"adopted": 0, "scale_bit_mismatch": 0, "scales_compared": 0, "adopted_list": []}
     for t in range(steps):
+        if batched:
+            for i in range(w.M):
+                if grads is not None:
+                    gall[i, :w.d].copy_(grads[t][i])
+                else:
+                    w.draw_grad(t, i, device, es, out=gall[i, :w.d])
+            eng.worker_step_all(gall)
         for i in range(w.M):
-            g = grads[t][i].to(device) if grads is not None else w.draw_grad(t, i, device, es, out=gbuf)
-            eng.worker_step(i, g)
+            if batched:
+                g = gall[i, :w.d]
+            else:
+                g = grads[t][i].to(device) if grads is not None else w.draw_grad(t, i, device, es, out=gbuf)
+                eng.worker_step(i, g)
             gw = smp.words(eng.worker_words(i))
             ad = orc.worker_step(i, smp.elems(g), hint=gw)
             stats["adopted"] += len(ad)

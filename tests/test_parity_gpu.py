@@ -39,6 +39,42 @@ def test_small_layouts(sizes, M, scale_mode):
     assert stats["adopted"] <= 2
 
 
+@pytest.mark.parametrize("sizes,M", [
+    ([3, 5, 31, 33, 63, 65, 127, 129], 3), ([40, 64, 5, 300, 7, 1000, 13], 5),
+    ([2 * TILE, TILE // 2, 3 * TILE + 36, 100], 8), ([BIG - 4, 3 * BIG + TILE + 4, 2 * BIG + 2 * TILE], 7),
+    ([12345, 54321, 99999], 9),
+])
+@pytest.mark.parametrize("scale_mode", ["fused", "split"])
+def test_batched_worker_call(sizes, M, scale_mode):
+    """ef_worker_step_all: all workers in one launch, checked against the oracle."""
+    w = _wl("batched", sizes, M, steps=5)
+    run_parity(w, scale_mode=scale_mode, batched=True)
+
+
+def test_batched_and_per_worker_calls_are_bit_identical():
+    w = wl.make_workload(2)
+    es = w.element_scales("cuda")
+    a = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    b = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    stride = (w.d + 3) // 4 * 4
+    gall = torch.zeros(w.M, stride, device="cuda")
+    for t in range(3):
+        for i in range(w.M):
+            w.draw_grad(t, i, "cuda", es, out=gall[i, :w.d])
+            a.worker_step(i, gall[i, :w.d])
+        b.worker_step_all(gall)
+        for i in range(w.M):
+            assert torch.equal(a.worker_words(i), b.worker_words(i))
+            assert torch.equal(a.worker_scales(i), b.worker_scales(i))
+        a.server_step(); b.server_step()
+    assert torch.equal(a.params(), b.params())
+    for i in range(-1, w.M):
+        assert torch.equal(a.residual(i), b.residual(i))
+    with pytest.raises(ef.EFError) as ei:                      # mixing is refused mid-iteration
+        a.worker_step(0, gall[0, :w.d]); a.worker_step_all(gall)
+    assert ei.value.status == ef.EF_ERR_BAD_STATE
+
+
 @pytest.mark.parametrize("mu,eta", [(0.0, 0.1), (0.5, 1.0), (0.99, 1e-3)])
 def test_hyper_parameters(mu, eta):
     w = _wl("hp", [TILE + 100, 777, 2 * TILE], 3, mu=mu, eta=eta, steps=6, scale_range=(1e-3, 1.0))
@@ -139,15 +175,21 @@ def test_config3_resnet50_layout():
     run_parity(w, check_every_step=False)
 
 
+def test_config3_batched_worker_call():
+    w = wl.make_workload(3)
+    run_parity(w, steps=4, check_every_step=False, batched=True)
+
+
 def test_config3_fused_scale_mode():
     w = wl.make_workload(3)
     run_parity(w, steps=3, check_every_step=False, scale_mode="fused")
 
 
 def test_config4_flat_2_28_sampled_blocks():
-    """Full-size launch (d = 2^28, M = 7, 20 steps); the oracle follows 6 of the 256 blocks."""
+    """Full-size launch (d = 2^28, M = 7, 20 steps) in the configuration bench.py times (all
+    workers in one ef_worker_step_all launch); the oracle follows 6 of the 256 blocks."""
     w = wl.make_workload(4)
-    run_parity(w, blocks=[0, 1, 100, 127, 128, 255], check_every_step=False)
+    run_parity(w, blocks=[0, 1, 100, 127, 128, 255], check_every_step=False, batched=True)
 
 
 def test_config5_gpt2_layout_sampled_blocks():
