@@ -16,10 +16,11 @@
 // launch-bound grids, by the last CTA to finish the block (one atomic ticket, no waiting).
 //
 // Work decomposition.  The flat vector is cut into tiles of at most kTileChunks chunks of
-// 1024*U elements; a tile never crosses a block boundary.  The worker and apply kernels run
-// one CTA per chunk (three read and two write streams of 16 KB each per CTA keep enough bytes
-// in flight).  The server kernel has one read and one write stream only, so one CTA walks all
-// chunks of a tile and stages them two chunks ahead through shared memory with cp.async.
+// 1024*U elements; a tile never crosses a block boundary.  The worker kernel runs one CTA per
+// chunk (three read and two write streams of 16 KB each per CTA keep enough bytes in flight).
+// The server and apply kernels have one read and one write stream only, so one CTA walks all
+// chunks of a tile: the server kernel stages them two chunks ahead through shared memory with
+// cp.async, the apply kernel loads chunk c+1 into a second register set while it updates c.
 //
 // Arithmetic is IEEE binary32 with explicit round-to-nearest intrinsics in a fixed order so
 // that results do not depend on compiler contraction; block sums are binary64.
@@ -474,7 +475,7 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-constexpr int kServerStages = 3;
+constexpr int kServerStages = 2;
 // Dynamic shared memory of the server kernel: staging ring, then M scaled scales.
 template <int U>
 __host__ __device__ constexpr size_t server_ring_bytes() {
@@ -563,16 +564,16 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
 
     float p[U][4];
     unsigned w[U];
-    issue_chunk(0);                        // in flight while the table is built
-    issue_chunk(1);
+#pragma unroll
+    for (int c = 0; c < kServerStages - 1; ++c) issue_chunk(c);   // in flight while the table is built
     build_scaled(a, t.block, MT, s_c);
     __syncthreads();
     build_lut<MT>(s_c, s_base, s_lut);
     c6 = __float_as_uint(s_c[MT > 6 ? 6 : 0]);
     c7 = __float_as_uint(s_c[MT > 7 ? 7 : 0]);
     for (int c = 0; c < nfull; ++c) {
-        issue_chunk(c + 2);                // reuses the slot this thread consumed at c - 1
-        cp_async_wait<2>();                // groups c+1 and c+2 may still be in flight
+        issue_chunk(c + kServerStages - 1);      // reuses the slot this thread consumed at c - 1
+        cp_async_wait<kServerStages - 1>();      // only the groups after chunk c may be in flight
         const int s = c % kServerStages;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -704,14 +705,15 @@ __global__ void __launch_bounds__(kThreads) ef_server_kernel(const ServerArgs a)
 
 // ------------------------------------------------------------------ parameter update
 // x_{t+1,j} = x_{t,j} - eta * stilde_b * sign(ptilde_j)  (Algorithm 4, worker line after the pull)
-// One chunk per CTA.
+// One tile per CTA; chunk c+1 is loaded into a second register set while chunk c is updated, so
+// the tile descriptor's latency is paid once per tile and loads stay in flight.
 template <int U>
 __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
-    const Tile t = chunk_of<U>(a.tiles[blockIdx.x / kTileChunks], blockIdx.x % kTileChunks);
-    if (t.len <= 0) return;
-    const float step = __fmul_rn(a.eta, a.scales[t.block]);
+    constexpr int kChunk = 1024 * U;
+    const Tile t = a.tiles[blockIdx.x];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if ((t.start & 3) != 0) {
+        const float step = __fmul_rn(a.eta, a.scales[t.block]);
         const int rows = (t.len + 31) >> 5;
         for (int r = warp; r < rows; r += kWarps) {
             const int o = r * 32 + lane;
@@ -723,27 +725,50 @@ __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
         }
         return;
     }
-    const bool full = (t.len == 1024 * U);
     const int o0 = warp * (128 * U) + lane * 4;
     const int sh = (lane & 7) * 4;
-    float* xp = a.x + t.start + o0;
-    float x[U][4];
-    unsigned nib[U];
+    float* const xbase = a.x + t.start + o0;
+    const uint32_t* const wbase = a.words + t.word + (o0 >> 5);
+    const int nchunks = (t.len + kChunk - 1) / kChunk;
+
+    auto load_chunk = [&](int c, float (&x)[U][4], unsigned (&nib)[U]) {
+        const int clen = min(kChunk, t.len - c * kChunk);
+        const bool full = clen == kChunk;
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-        const int o = o0 + u * 128;
-        load4(xp + u * 128, o, t.len, full, x[u]);
-        nib[u] = (full || o < t.len) ? (__ldg(a.words + t.word + (o >> 5)) >> sh) : 0u;
-    }
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {   // x - step*sign: subtract step with the sign bit flipped in
-            const float signed_step =
-                __uint_as_float(__float_as_uint(step) ^ ((nib[u] << (31 - k)) & 0x80000000u));
-            x[u][k] = __fsub_rn(x[u][k], signed_step);
+        for (int u = 0; u < U; ++u) {
+            const int o = o0 + u * 128;
+            load4(xbase + (long long)c * kChunk + u * 128, o, clen, full, x[u]);
+            nib[u] = (full || o < clen) ? __ldg(wbase + c * (kChunk / 32) + u * 4) : 0u;
         }
-        store4(xp + u * 128, o0 + u * 128, t.len, full, x[u]);
+    };
+    float step = 0.f;
+    auto update_chunk = [&](int c, float (&x)[U][4], unsigned (&nib)[U]) {
+        const int clen = min(kChunk, t.len - c * kChunk);
+        const bool full = clen == kChunk;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const unsigned n = nib[u] >> sh;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {   // x - step*sign: subtract step with the sign bit flipped in
+                const float signed_step =
+                    __uint_as_float(__float_as_uint(step) ^ ((n << (31 - k)) & 0x80000000u));
+                x[u][k] = __fsub_rn(x[u][k], signed_step);
+            }
+            store4(xbase + (long long)c * kChunk + u * 128, o0 + u * 128, clen, full, x[u]);
+        }
+    };
+
+    float xA[U][4], xB[U][4];
+    unsigned nA[U], nB[U];
+    load_chunk(0, xA, nA);
+    step = __fmul_rn(a.eta, a.scales[t.block]);        // its latency overlaps the first loads
+    for (int c = 0; c < nchunks; c += 2) {
+        if (c + 1 < nchunks) load_chunk(c + 1, xB, nB);
+        update_chunk(c, xA, nA);
+        if (c + 1 < nchunks) {
+            if (c + 2 < nchunks) load_chunk(c + 2, xA, nA);
+            update_chunk(c + 1, xB, nB);
+        }
     }
 }
 
