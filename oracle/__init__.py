@@ -50,7 +50,11 @@ def _load():
     lib.efo_worker_step.argtypes = [vp, i32, vp, vp, vp, i64]
     lib.efo_server_step.restype = i64
     lib.efo_server_step.argtypes = [vp, vp, vp, i64]
-    for name in ("efo_params", "efo_last_p"):
+    lib.efo_set_eta.restype = i32
+    lib.efo_set_eta.argtypes = [vp, f32]
+    lib.efo_set_weight_decay.restype = i32
+    lib.efo_set_weight_decay.argtypes = [vp, f32]
+    for name in ("efo_params", "efo_last_p", "efo_decay_momentum"):
         getattr(lib, name).restype = vp
         getattr(lib, name).argtypes = [vp]
     for name in ("efo_momentum", "efo_residual", "efo_words", "efo_scales"):
@@ -119,6 +123,18 @@ class Oracle:
         if n < 0:
             raise RuntimeError("efo_server_step: not every worker has stepped")
         return self._adopt[:min(n, self.ADOPT_CAP)].copy()
+
+    def set_eta(self, eta: float) -> None:
+        if self._lib.efo_set_eta(self._h, float(eta)) != 0:
+            raise RuntimeError("efo_set_eta: bad value or called in the middle of an iteration")
+
+    def set_weight_decay(self, lam: float) -> None:
+        if self._lib.efo_set_weight_decay(self._h, float(lam)) != 0:
+            raise RuntimeError("efo_set_weight_decay: bad value or called in the middle of an iteration")
+
+    @property
+    def decay_momentum(self) -> np.ndarray:
+        return _view(self._lib.efo_decay_momentum(self._h), self.d, np.float32)
 
     # ---- views (live; copy if you need a snapshot) ---------------------------
     @property

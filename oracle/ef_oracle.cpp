@@ -17,9 +17,21 @@
 // with the blockwise compressor of Section 3.2:
 //   C_B(v) = [ ||v_{G_b}||_1 / d_b * sign(v_{G_b}) ]_{b=1..B}.
 //
+// Stepsize sequence (Algorithms 2-4, "stepsize sequence {eta_t}"): efo_set_eta changes the
+// stepsize of the coming iteration; both residuals are then rescaled by
+// r = fl(eta_{t-1} / eta_t) (one fp32 multiplication, e <- fl(r e)) before they are added.
+// Weight decay (Appendix A): kept out of the compressor; every worker keeps an extra momentum
+//   mtilde_t = mu mtilde_{t-1} + lambda x_t,   x_{t+1} = x_t - eta_t (Deltatilde_t + mu mtilde_t + lambda x_t),
+// done once here because all replicas of x are identical.
+//
 // Readings where the paper is silent (each is a convention of this repository):
-//   * constant stepsize eta, so eta_{t-1}/eta_t = 1 for t >= 1; at t = 0 the ratio multiplies
-//     e_0 = etilde_0 = 0 (the paper's eta_{-1} = 0), so no multiplication is performed;
+//   * until efo_set_eta is called the stepsize is constant, so eta_{t-1}/eta_t = 1; at t = 0 the
+//     paper's ratio (eta_{-1} = 0) multiplies e_0 = etilde_0 = 0, which the ratio 1 reproduces;
+//   * the rescale is e <- fl(r e) with r = fl(eta_{t-1}/eta_t) computed once in fp32 (for r = 1
+//     this is the identity, bit for bit);
+//   * with weight decay the update is evaluated as
+//       wd = fl(lambda x); mtilde = fma(mu, mtilde, wd); v = fma(mu, mtilde, wd);
+//       x <- fl( fl(x -+ fl(eta s_b)) - fl(eta v) );
 //   * state and element arithmetic are IEEE binary32 in the fixed order written below, block
 //     L1 sums are accumulated sequentially in binary64 and rounded once to binary32 (the scale
 //     is a float32 on the wire, Section 3.2);
@@ -56,7 +68,10 @@ struct Oracle {
     int32_t B = 0;
     int32_t M = 0;
     float mu = 0.f;
-    float eta = 0.f;
+    float eta = 0.f;                     // eta_t of the coming iteration
+    float eta_prev = 0.f;                // eta_{t-1}: stepsize of the last completed iteration
+    float lambda = 0.f;                  // weight decay (0 = off)
+    std::vector<float> mt;               // weight-decay momentum mtilde (allocated when lambda > 0)
     int64_t W = 0;                       // total packed words
     int64_t t = 0;                       // completed iterations
     std::vector<int64_t> off;            // B+1 element offsets
@@ -78,7 +93,7 @@ struct Oracle {
 // Returns the number of adopted elements appended to `adopted`.
 int64_t compress_block(const float* p, int64_t lo, int64_t hi,
                        float* scale_out, uint32_t* words_out /* block's first word */,
-                       float* resid, float* x, float eta,
+                       float* resid, float* x, float eta, float mu, float lambda, float* mt,
                        const uint32_t* hint /* block's first word or null */,
                        int64_t* adopted, int64_t adopted_cap, int64_t adopted_n)
 {
@@ -106,7 +121,18 @@ int64_t compress_block(const float* p, int64_t lo, int64_t hi,
         }
         if (neg) words_out[k >> 5] |= (1u << (k & 31));
         resid[j] = neg ? (p[j] + s) : (p[j] - s);
-        if (x) x[j] = neg ? (x[j] + step) : (x[j] - step);
+        if (x) {
+            if (lambda > 0.0f) {                       // Appendix A: decay outside the compressor
+                const float wd = lambda * x[j];
+                mt[j] = std::fmaf(mu, mt[j], wd);      // mtilde_t = mu mtilde_{t-1} + lambda x_t
+                const float v = std::fmaf(mu, mt[j], wd);
+                const float xs = neg ? (x[j] + step) : (x[j] - step);
+                const float ev = eta * v;
+                x[j] = xs - ev;
+            } else {
+                x[j] = neg ? (x[j] + step) : (x[j] - step);
+            }
+        }
     }
     return adopted_n;
 }
@@ -123,7 +149,7 @@ void* efo_init(int64_t d, int32_t B, const int64_t* offsets, int32_t M, float mu
     if (!(mu >= 0.f && mu < 1.f) || !(eta > 0.f) || !std::isfinite(eta)) return nullptr;
     Oracle* o = new (std::nothrow) Oracle();
     if (!o) return nullptr;
-    o->d = d; o->B = B; o->M = M; o->mu = mu; o->eta = eta;
+    o->d = d; o->B = B; o->M = M; o->mu = mu; o->eta = eta; o->eta_prev = eta;
     o->off.assign(offsets, offsets + B + 1);
     o->woff.assign(B + 1, 0);
     for (int32_t b = 0; b < B; ++b)
@@ -158,16 +184,19 @@ int64_t efo_worker_step(void* h, int32_t i, const float* grad, const uint32_t* h
     float* e = o->e[i].data();
     float* p = o->p.data();
     const float mu = o->mu;
+    const float r = o->eta_prev / o->eta;                    // eta_{t-1} / eta_t
     int64_t n_adopted = 0;
     for (int32_t b = 0; b < o->B; ++b) {
         const int64_t lo = o->off[b], hi = o->off[b + 1];
         for (int64_t j = lo; j < hi; ++j) {
             m[j] = std::fmaf(mu, m[j], grad[j]);             // m_t = mu m_{t-1} + g_t
             const float u = std::fmaf(mu, m[j], grad[j]);    // mu m_t + g_t
-            p[j] = u + e[j];                                 // + e_t   (stepsize ratio 1)
+            const float es = r * e[j];                       // (eta_{t-1}/eta_t) e_t
+            p[j] = u + es;
         }
         n_adopted = compress_block(p, lo, hi, &o->scales[i][b],
-                                   o->words[i].data() + o->woff[b], e, nullptr, 0.f,
+                                   o->words[i].data() + o->woff[b], e, nullptr, 0.f, 0.f, 0.f,
+                                   nullptr,
                                    hint ? hint + o->woff[b] : nullptr,
                                    adopted, adopted_cap, n_adopted);
     }
@@ -185,6 +214,7 @@ int64_t efo_server_step(void* h, const uint32_t* hint, int64_t* adopted, int64_t
     float* p = o->p.data();
     float* et = o->et.data();
     const int32_t M = o->M;
+    const float r = o->eta_prev / o->eta;                    // eta_{t-1} / eta_t
     std::vector<float> c(M);
     int64_t n_adopted = 0;
     for (int32_t b = 0; b < o->B; ++b) {
@@ -198,17 +228,44 @@ int64_t efo_server_step(void* h, const uint32_t* hint, int64_t* adopted, int64_t
                 const float v = ((w >> (k & 31)) & 1u) ? -c[i] : c[i];   // decoded Delta_{t,i} / M
                 a = (i == 0) ? v : (a + v);
             }
-            p[j] = a + et[j];                                 // ptilde_t
+            const float es = r * et[j];                       // (eta_{t-1}/eta_t) etilde_t
+            p[j] = a + es;                                    // ptilde_t
         }
         n_adopted = compress_block(p, lo, hi, &o->sscales[b],
                                    o->swords.data() + o->woff[b], et, o->x.data(), o->eta,
+                                   o->mu, o->lambda, o->lambda > 0.f ? o->mt.data() : nullptr,
                                    hint ? hint + o->woff[b] : nullptr,
                                    adopted, adopted_cap, n_adopted);
     }
     for (int32_t i = 0; i < M; ++i) o->stepped[i] = 0;
+    o->eta_prev = o->eta;
     o->t += 1;
     return n_adopted;
 }
+
+// Stepsize of the coming iteration (between iterations only).  Returns 0, or -1 on misuse.
+int32_t efo_set_eta(void* h, float eta)
+{
+    Oracle* o = static_cast<Oracle*>(h);
+    if (!o || !(eta > 0.f) || !std::isfinite(eta)) return -1;
+    for (int32_t i = 0; i < o->M; ++i) if (o->stepped[i]) return -1;
+    o->eta = eta;
+    return 0;
+}
+
+// Weight decay lambda >= 0 (Appendix A); allocates mtilde = 0 on first use.
+int32_t efo_set_weight_decay(void* h, float lambda)
+{
+    Oracle* o = static_cast<Oracle*>(h);
+    if (!o || !(lambda >= 0.f) || !std::isfinite(lambda)) return -1;
+    for (int32_t i = 0; i < o->M; ++i) if (o->stepped[i]) return -1;
+    o->lambda = lambda;
+    if (lambda > 0.f && o->mt.empty()) o->mt.assign(o->d, 0.f);
+    return 0;
+}
+
+float* efo_decay_momentum(void* h) { Oracle* o = static_cast<Oracle*>(h);
+                                     return o->mt.empty() ? nullptr : o->mt.data(); }
 
 // Raw views into the oracle's state (valid until efo_destroy).
 float*    efo_params(void* h)               { return static_cast<Oracle*>(h)->x.data(); }
