@@ -19,7 +19,7 @@
 //
 // Stepsize sequence (Algorithms 2-4, "stepsize sequence {eta_t}"): efo_set_eta changes the
 // stepsize of the coming iteration; both residuals are then rescaled by
-// r = fl(eta_{t-1} / eta_t) (one fp32 multiplication, e <- fl(r e)) before they are added.
+// r = fl(eta_{t-1} / eta_t) as they are added: p = fma(r, e, mu m + g), ptilde = fma(r, etilde, a).
 // Weight decay (Appendix A): kept out of the compressor; every worker keeps an extra momentum
 //   mtilde_t = mu mtilde_{t-1} + lambda x_t,   x_{t+1} = x_t - eta_t (Deltatilde_t + mu mtilde_t + lambda x_t),
 // done once here because all replicas of x are identical.
@@ -27,8 +27,8 @@
 // Readings where the paper is silent (each is a convention of this repository):
 //   * until efo_set_eta is called the stepsize is constant, so eta_{t-1}/eta_t = 1; at t = 0 the
 //     paper's ratio (eta_{-1} = 0) multiplies e_0 = etilde_0 = 0, which the ratio 1 reproduces;
-//   * the rescale is e <- fl(r e) with r = fl(eta_{t-1}/eta_t) computed once in fp32 (for r = 1
-//     this is the identity, bit for bit);
+//   * the rescaled residual enters through one fused multiply-add, p = fma(r, e, u), with
+//     r = fl(eta_{t-1}/eta_t) computed once in fp32 (for r = 1 this is fl(u + e), bit for bit);
 //   * with weight decay the update is evaluated as
 //       wd = fl(lambda x); mtilde = fma(mu, mtilde, wd); v = fma(mu, mtilde, wd);
 //       x <- fl( fl(x -+ fl(eta s_b)) - fl(eta v) );
@@ -191,8 +191,7 @@ int64_t efo_worker_step(void* h, int32_t i, const float* grad, const uint32_t* h
         for (int64_t j = lo; j < hi; ++j) {
             m[j] = std::fmaf(mu, m[j], grad[j]);             // m_t = mu m_{t-1} + g_t
             const float u = std::fmaf(mu, m[j], grad[j]);    // mu m_t + g_t
-            const float es = r * e[j];                       // (eta_{t-1}/eta_t) e_t
-            p[j] = u + es;
+            p[j] = std::fmaf(r, e[j], u);                    // + (eta_{t-1}/eta_t) e_t
         }
         n_adopted = compress_block(p, lo, hi, &o->scales[i][b],
                                    o->words[i].data() + o->woff[b], e, nullptr, 0.f, 0.f, 0.f,
@@ -228,8 +227,7 @@ int64_t efo_server_step(void* h, const uint32_t* hint, int64_t* adopted, int64_t
                 const float v = ((w >> (k & 31)) & 1u) ? -c[i] : c[i];   // decoded Delta_{t,i} / M
                 a = (i == 0) ? v : (a + v);
             }
-            const float es = r * et[j];                       // (eta_{t-1}/eta_t) etilde_t
-            p[j] = a + es;                                    // ptilde_t
+            p[j] = std::fmaf(r, et[j], a);                    // ptilde_t = a + (eta_{t-1}/eta_t) etilde_t
         }
         n_adopted = compress_block(p, lo, hi, &o->sscales[b],
                                    o->swords.data() + o->woff[b], et, o->x.data(), o->eta,
