@@ -60,6 +60,7 @@ enum ef_status {
  * most one of the two flags may be set. */
 #define EF_FLAG_FUSED_SCALE 2u     /* always complete the sums inside the main kernels */
 #define EF_FLAG_SPLIT_SCALE 4u     /* always use the follow-up kernel */
+#define EF_FLAG_WEIGHT_DECAY 8u    /* reserve the d-float decay momentum for ef_set_weight_decay */
 
 /* Maximum number of simulated workers. */
 #define EF_MAX_WORKERS 4096
@@ -119,6 +120,22 @@ int ef_worker_step_host(ef_ctx* ctx, int32_t i, const float* grad /* host */);
  * Errors: BAD_STATE unless every worker has been stepped exactly once since the last
  * server step; CUDA. */
 int ef_server_step(ef_ctx* ctx);
+
+/* Stepsize of the coming iteration (Algorithms 2-4 take a stepsize sequence {eta_t}).  In that
+ * iteration both the workers' and the server's residual enter rescaled by eta_{t-1}/eta_t
+ * (computed in fp32; p = fma(ratio, e, mu m + g)), where eta_{t-1} is the stepsize of the last
+ * completed iteration (the value given to ef_init before any iteration has run).  Without this
+ * call the stepsize stays constant and the ratio is exactly 1.  Only between iterations.
+ * Errors: INVALID_ARG (eta <= 0 or not finite), BAD_STATE (in the middle of an iteration). */
+int ef_set_eta(ef_ctx* ctx, float eta);
+
+/* Weight decay lambda >= 0, kept out of the compressor as in Appendix A: every worker (here:
+ * once) keeps a decay momentum mtilde_t = mu mtilde_{t-1} + lambda x_t and the update becomes
+ * x_{t+1} = x_t - eta_t (Deltatilde_t + mu mtilde_t + lambda x_t).  Needs EF_FLAG_WEIGHT_DECAY at
+ * ef_init (the momentum starts at 0).  lambda = 0 switches it off.  Only between iterations.
+ * Errors: INVALID_ARG, BAD_STATE (flag missing, or in the middle of an iteration). */
+int ef_set_weight_decay(ef_ctx* ctx, float lambda);
+float* ef_decay_momentum(ef_ctx* ctx);    /* mtilde, d floats (NULL without the flag); may be edited between iterations */
 
 /* Copies the server's message of the last ef_server_step (packed words, then scales) to host
  * memory, asynchronously on the context's stream.  words: ef_num_words words; scales: B floats.

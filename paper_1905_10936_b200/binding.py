@@ -29,6 +29,7 @@ EF_NOALLOC_MAX_ELEMS = 1 << 24
 EF_FLAG_HOST_STAGING = 1
 EF_FLAG_FUSED_SCALE = 2
 EF_FLAG_SPLIT_SCALE = 4
+EF_FLAG_WEIGHT_DECAY = 8
 EF_MAX_WORKERS = 4096
 
 _vp, _i64, _i32, _u32, _f32 = (ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_uint32,
@@ -43,6 +44,9 @@ SIGNATURES = {
     "ef_worker_step_all": (ctypes.c_int, [_vp, _vp, _i64]),
     "ef_worker_step_host": (ctypes.c_int, [_vp, _i32, _vp]),
     "ef_server_step": (ctypes.c_int, [_vp]),
+    "ef_set_eta": (ctypes.c_int, [_vp, _f32]),
+    "ef_set_weight_decay": (ctypes.c_int, [_vp, _f32]),
+    "ef_decay_momentum": (_vp, [_vp]),
     "ef_read_update_host": (ctypes.c_int, [_vp, _vp, _vp]),
     "ef_worker_words": (_vp, [_vp, _i32]),
     "ef_worker_scales": (_vp, [_vp, _i32]),
@@ -127,6 +131,18 @@ def ef_worker_step_host(ctx: int, i: int, grad_host_ptr: int) -> None:
 
 def ef_server_step(ctx: int) -> None:
     _check(load_library().ef_server_step(ctx), "ef_server_step")
+
+
+def ef_set_eta(ctx: int, eta: float) -> None:
+    _check(load_library().ef_set_eta(ctx, eta), "ef_set_eta")
+
+
+def ef_set_weight_decay(ctx: int, lam: float) -> None:
+    _check(load_library().ef_set_weight_decay(ctx, lam), "ef_set_weight_decay")
+
+
+def ef_decay_momentum(ctx: int) -> Optional[int]:
+    return load_library().ef_decay_momentum(ctx)
 
 
 def ef_read_update_host(ctx: int, words_host_ptr: int, scales_host_ptr: int) -> None:

@@ -70,6 +70,7 @@ struct WorkerArgs {
     const Tile* tiles;
     const Block* blocks;
     float mu;
+    float ratio;           // eta_{t-1} / eta_t: rescale of the residual (1 for a constant stepsize)
     int fused;             // 1: last CTA of a block finalises its scale; 0: ef_scale_kernel does
     // batched launches: blockIdx.y selects the worker; its buffers lie at these strides
     long long g_stride, state_stride, word_stride, partial_stride;
@@ -91,6 +92,7 @@ struct ServerArgs {
     const Tile* tiles;
     const Block* blocks;
     int fused;
+    float ratio;             // eta_{t-1} / eta_t
 };
 
 struct ScaleArgs {
@@ -109,6 +111,9 @@ struct ApplyArgs {
     const float* scales;     // server scales
     const Tile* tiles;
     float eta;
+    // weight decay kept out of the compressor (Appendix A); used by the DECAY instantiation only
+    float* mt;               // decay momentum mtilde
+    float mu, lambda;
 };
 
 struct ResidualArgs {
@@ -135,6 +140,8 @@ __device__ __forceinline__ void st_stream(float* p, float4 v) {
 // the buffers start at +0 and ef_set_state adds +0 to what it imports.  (NaN is unspecified.)
 //
 // e_{t+1,j} = p_{t,j} - s * sign(p_{t,j})   (Algorithm 4): one rounding, as p + s or p - s.
+// It enters the next corrected vector as fma(eta_{t-1}/eta_t, e, .), which is fl(. + e) for a
+// constant stepsize.
 __device__ __forceinline__ float residual_of(float pb, float s) {
     const float signed_s = __uint_as_float((__float_as_uint(pb) & 0x80000000u) | __float_as_uint(s));
     return __fsub_rn(pb, signed_s);
@@ -311,7 +318,7 @@ __device__ __forceinline__ double worker_rows(const WorkerArgs& a, const Tile& t
             const float e = residual_of(p[u][k], sp);                // e_{t,i}
             m[u][k] = __fmaf_rn(a.mu, m[u][k], g[u][k]);             // m_t = mu m_{t-1} + g
             const float v = __fmaf_rn(a.mu, m[u][k], g[u][k]);       // mu m_t + g
-            float pv = __fadd_rn(v, e);                              // p_t
+            float pv = __fmaf_rn(a.ratio, e, v);                     // p_t = v + (eta_{t-1}/eta_t) e
             if (!FULL && o + k >= t.len) pv = 0.f;
             p[u][k] = pv;
         }
@@ -340,7 +347,7 @@ __device__ __forceinline__ double worker_rows_scalar(const WorkerArgs& a, const 
             const float g = a.g[j];
             const float e = residual_of(a.pb[j], sp);
             const float m = __fmaf_rn(a.mu, a.m[j], g);
-            pv = __fadd_rn(__fmaf_rn(a.mu, m, g), e);
+            pv = __fmaf_rn(a.ratio, e, __fmaf_rn(a.mu, m, g));
             a.m[j] = m;
             a.pb[j] = pv;
         }
@@ -550,7 +557,7 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
             }
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                float pv = __fadd_rn(avg[k], residual_of(p[u][k], sp));      // ptilde_t
+                float pv = __fmaf_rn(a.ratio, residual_of(p[u][k], sp), avg[k]);   // ptilde_t
                 if (!full && o + k >= clen) pv = 0.f;
                 p[u][k] = pv;
             }
@@ -633,7 +640,7 @@ __device__ __forceinline__ double server_rows(const ServerArgs& a, const Tile& t
         if (full || o < t.len) average4(a, s_c, t.word + (o >> 5), sh, avg);
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            float pv = __fadd_rn(avg[k], residual_of(p[u][k], sp));   // ptilde_t
+            float pv = __fmaf_rn(a.ratio, residual_of(p[u][k], sp), avg[k]);   // ptilde_t
             if (!full && o + k >= t.len) pv = 0.f;
             p[u][k] = pv;
         }
@@ -664,7 +671,7 @@ __device__ __forceinline__ double server_rows_scalar(const ServerArgs& a, const 
                 avg = (i == 0) ? v : __fadd_rn(avg, v);
             }
             const long long j = t.start + o;
-            pv = __fadd_rn(avg, residual_of(a.pb[j], sp));
+            pv = __fmaf_rn(a.ratio, residual_of(a.pb[j], sp), avg);
             a.pb[j] = pv;
         }
         acc += (double)fabsf(pv);
@@ -707,7 +714,22 @@ __global__ void __launch_bounds__(kThreads) ef_server_kernel(const ServerArgs a)
 // x_{t+1,j} = x_{t,j} - eta * stilde_b * sign(ptilde_j)  (Algorithm 4, worker line after the pull)
 // One tile per CTA; chunk c+1 is loaded into a second register set while chunk c is updated, so
 // the tile descriptor's latency is paid once per tile and loads stay in flight.
-template <int U>
+//
+// DECAY adds the weight-decay side path of Appendix A, which is not compressed:
+//   mtilde_t = mu mtilde_{t-1} + lambda x_t;  x_{t+1} = x_t - eta (Deltatilde_t + mu mtilde_t + lambda x_t),
+// evaluated as wd = fl(lambda x); mtilde = fma(mu, mtilde, wd); v = fma(mu, mtilde, wd);
+// x = fl(fl(x -+ eta s_b) - fl(eta v)).
+template <bool DECAY>
+__device__ __forceinline__ float apply_one(const ApplyArgs& a, float x, float signed_step, float* mt) {
+    const float xs = __fsub_rn(x, signed_step);
+    if (!DECAY) return xs;
+    const float wd = __fmul_rn(a.lambda, x);
+    *mt = __fmaf_rn(a.mu, *mt, wd);
+    const float v = __fmaf_rn(a.mu, *mt, wd);
+    return __fsub_rn(xs, __fmul_rn(a.eta, v));
+}
+
+template <int U, bool DECAY>
 __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
     constexpr int kChunk = 1024 * U;
     const Tile t = a.tiles[blockIdx.x];
@@ -720,7 +742,9 @@ __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
             if (o < t.len) {
                 const unsigned w = __ldg(a.words + t.word + r);
                 const long long j = t.start + o;
-                a.x[j] = ((w >> lane) & 1u) ? __fadd_rn(a.x[j], step) : __fsub_rn(a.x[j], step);
+                float mt = DECAY ? a.mt[j] : 0.f;
+                a.x[j] = apply_one<DECAY>(a, a.x[j], ((w >> lane) & 1u) ? -step : step, &mt);
+                if (DECAY) a.mt[j] = mt;
             }
         }
         return;
@@ -728,21 +752,24 @@ __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
     const int o0 = warp * (128 * U) + lane * 4;
     const int sh = (lane & 7) * 4;
     float* const xbase = a.x + t.start + o0;
+    float* const mbase = DECAY ? a.mt + t.start + o0 : nullptr;
     const uint32_t* const wbase = a.words + t.word + (o0 >> 5);
     const int nchunks = (t.len + kChunk - 1) / kChunk;
+    constexpr int UM = DECAY ? U : 1;      // the decay momentum is only held when it is used
 
-    auto load_chunk = [&](int c, float (&x)[U][4], unsigned (&nib)[U]) {
+    auto load_chunk = [&](int c, float (&x)[U][4], float (&mt)[UM][4], unsigned (&nib)[U]) {
         const int clen = min(kChunk, t.len - c * kChunk);
         const bool full = clen == kChunk;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int o = o0 + u * 128;
             load4(xbase + (long long)c * kChunk + u * 128, o, clen, full, x[u]);
+            if (DECAY) load4(mbase + (long long)c * kChunk + u * 128, o, clen, full, mt[DECAY ? u : 0]);
             nib[u] = (full || o < clen) ? __ldg(wbase + c * (kChunk / 32) + u * 4) : 0u;
         }
     };
     float step = 0.f;
-    auto update_chunk = [&](int c, float (&x)[U][4], unsigned (&nib)[U]) {
+    auto update_chunk = [&](int c, float (&x)[U][4], float (&mt)[UM][4], unsigned (&nib)[U]) {
         const int clen = min(kChunk, t.len - c * kChunk);
         const bool full = clen == kChunk;
 #pragma unroll
@@ -752,22 +779,24 @@ __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
             for (int k = 0; k < 4; ++k) {   // x - step*sign: subtract step with the sign bit flipped in
                 const float signed_step =
                     __uint_as_float(__float_as_uint(step) ^ ((n << (31 - k)) & 0x80000000u));
-                x[u][k] = __fsub_rn(x[u][k], signed_step);
+                x[u][k] = apply_one<DECAY>(a, x[u][k], signed_step, &mt[DECAY ? u : 0][k]);
             }
             store4(xbase + (long long)c * kChunk + u * 128, o0 + u * 128, clen, full, x[u]);
+            if (DECAY)
+                store4(mbase + (long long)c * kChunk + u * 128, o0 + u * 128, clen, full, mt[DECAY ? u : 0]);
         }
     };
 
-    float xA[U][4], xB[U][4];
+    float xA[U][4], xB[U][4], mA[UM][4], mB[UM][4];
     unsigned nA[U], nB[U];
-    load_chunk(0, xA, nA);
+    load_chunk(0, xA, mA, nA);
     step = __fmul_rn(a.eta, a.scales[t.block]);        // its latency overlaps the first loads
     for (int c = 0; c < nchunks; c += 2) {
-        if (c + 1 < nchunks) load_chunk(c + 1, xB, nB);
-        update_chunk(c, xA, nA);
+        if (c + 1 < nchunks) load_chunk(c + 1, xB, mB, nB);
+        update_chunk(c, xA, mA, nA);
         if (c + 1 < nchunks) {
-            if (c + 2 < nchunks) load_chunk(c + 2, xA, nA);
-            update_chunk(c + 1, xB, nB);
+            if (c + 2 < nchunks) load_chunk(c + 2, xA, mA, nA);
+            update_chunk(c + 1, xB, mB, nB);
         }
     }
 }

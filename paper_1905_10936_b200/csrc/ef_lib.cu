@@ -35,7 +35,7 @@ struct Layout {
     size_t dpad = 0, wpad = 0, bpad = 0, tpad = 0;    // padded element counts per sub-buffer
     size_t off_x = 0, off_m = 0, off_pb = 0, off_spb = 0, off_words = 0, off_scales = 0,
            off_rscale = 0, off_partials = 0, off_tickets = 0, off_tiles = 0, off_blocks = 0,
-           off_multi = 0, off_stage = 0, total = 0;
+           off_multi = 0, off_stage = 0, off_mt = 0, total = 0;
     int32_t num_multi = 0;                            // blocks that span more than one chunk
 };
 
@@ -51,7 +51,8 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
                 Layout* L) {
     int rc = check_problem(d, B, offsets, M);
     if (rc != EF_OK) return rc;
-    if (flags & ~(EF_FLAG_HOST_STAGING | EF_FLAG_FUSED_SCALE | EF_FLAG_SPLIT_SCALE))
+    if (flags & ~(EF_FLAG_HOST_STAGING | EF_FLAG_FUSED_SCALE | EF_FLAG_SPLIT_SCALE |
+                  EF_FLAG_WEIGHT_DECAY))
         return EF_ERR_INVALID_ARG;
     if ((flags & EF_FLAG_FUSED_SCALE) && (flags & EF_FLAG_SPLIT_SCALE)) return EF_ERR_INVALID_ARG;
     L->d = d; L->B = B; L->M = M;
@@ -74,6 +75,7 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
     L->off_m = o;        o += (size_t)M * L->dpad * 4;
     L->off_pb = o;       o += (size_t)M * L->dpad * 4;
     L->off_spb = o;      o += L->dpad * 4;
+    L->off_mt = o;       if (flags & EF_FLAG_WEIGHT_DECAY) o += L->dpad * 4;
     L->off_words = o;    o += M1 * L->wpad * 4;
     L->off_scales = o;   o += M1 * L->bpad * 4;
     L->off_rscale = o;   o += M1 * L->bpad * 4;
@@ -93,6 +95,8 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
 struct ef_ctx {
     Layout L;
     float mu = 0.f, eta = 0.f;
+    float eta_prev = 0.f;                  // stepsize of the last completed iteration
+    float lambda = 0.f;                    // weight decay (needs EF_FLAG_WEIGHT_DECAY)
     uint32_t flags = 0;
     char* ws = nullptr;
     cudaStream_t stream = nullptr;
@@ -124,6 +128,7 @@ struct ef_ctx {
     const Tile* tiles() const { return (const Tile*)(ws + L.off_tiles); }
     const Block* blocks() const { return (const Block*)(ws + L.off_blocks); }
     const int* multi() const { return (const int*)(ws + L.off_multi); }
+    float* mt() const { return (float*)(ws + L.off_mt); }
     float* stage(int s) const { return (float*)(ws + L.off_stage) + (size_t)s * L.dpad; }
 };
 
@@ -163,6 +168,7 @@ int launch_worker(ef_ctx* c, int i, const float* grad, int count = 1, long long 
     a.scale_out = c->scales(i); a.rscale = c->rscale(i);
     a.partials = c->partials(i); a.tickets = c->tickets(i);
     a.tiles = c->tiles(); a.blocks = c->blocks(); a.mu = c->mu; a.fused = c->fused;
+    a.ratio = c->eta_prev / c->eta;
     a.g_stride = g_stride; a.state_stride = (long long)c->L.dpad;
     a.word_stride = (long long)c->L.wpad; a.partial_stride = (long long)c->L.tpad;
     a.scale_stride = (int)c->L.bpad;
@@ -217,6 +223,7 @@ int launch_server(ef_ctx* c) {
     a.pb = c->pb(M); a.words = c->words(M); a.scale_out = c->scales(M); a.rscale = c->rscale(M);
     a.partials = c->partials(M); a.tickets = c->tickets(M);
     a.tiles = c->tiles(); a.blocks = c->blocks(); a.fused = c->fused;
+    a.ratio = c->eta_prev / c->eta;
     cudaError_t le;
     switch (M) {
         case 1: le = launch_server_t<1>(c, a); break;
@@ -237,8 +244,11 @@ int launch_server(ef_ctx* c) {
     }
     efk::ApplyArgs p;
     p.x = c->x(); p.words = c->words(M); p.scales = c->scales(M); p.tiles = c->tiles();
-    p.eta = c->eta;
-    efk::ef_apply_kernel<kU><<<(unsigned)c->L.num_tiles, efk::kThreads, 0, c->stream>>>(p);
+    p.eta = c->eta; p.mu = c->mu; p.lambda = c->lambda; p.mt = c->mt();
+    if (c->lambda > 0.f)
+        efk::ef_apply_kernel<kU, true><<<(unsigned)c->L.num_tiles, efk::kThreads, 0, c->stream>>>(p);
+    else
+        efk::ef_apply_kernel<kU, false><<<(unsigned)c->L.num_tiles, efk::kThreads, 0, c->stream>>>(p);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
     return EF_OK;
@@ -287,7 +297,7 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
 
     ef_ctx* c = new (std::nothrow) ef_ctx();
     if (!c) return EF_ERR_INVALID_ARG;
-    c->L = L; c->mu = mu; c->eta = eta; c->flags = flags;
+    c->L = L; c->mu = mu; c->eta = eta; c->eta_prev = eta; c->flags = flags;
     c->ws = (char*)workspace;
     c->stream = (cudaStream_t)cuda_stream;
     c->stepped.assign(M, 0);
@@ -394,8 +404,27 @@ int ef_server_step(ef_ctx* c) {
     if (rc != EF_OK) return rc;
     std::fill(c->stepped.begin(), c->stepped.end(), (uint8_t)0);
     c->pending = 0;
+    c->eta_prev = c->eta;
     c->t += 1;
     return EF_OK;
+}
+
+int ef_set_eta(ef_ctx* c, float eta) {
+    if (!c || !(eta > 0.f) || !std::isfinite(eta)) return EF_ERR_INVALID_ARG;
+    if (c->pending != 0) return EF_ERR_BAD_STATE;
+    c->eta = eta;
+    return EF_OK;
+}
+
+int ef_set_weight_decay(ef_ctx* c, float lambda) {
+    if (!c || !(lambda >= 0.f) || !std::isfinite(lambda)) return EF_ERR_INVALID_ARG;
+    if (c->pending != 0 || !(c->flags & EF_FLAG_WEIGHT_DECAY)) return EF_ERR_BAD_STATE;
+    c->lambda = lambda;
+    return EF_OK;
+}
+
+float* ef_decay_momentum(ef_ctx* c) {
+    return (c && (c->flags & EF_FLAG_WEIGHT_DECAY)) ? c->mt() : nullptr;
 }
 
 int ef_read_update_host(ef_ctx* c, uint32_t* words, float* scales) {
@@ -612,7 +641,7 @@ extern "C" int ef_worker_step_noalloc(const float* grad, float* momentum, float*
     NoAllocArgs a;
     a.w.g = grad; a.w.m = momentum; a.w.pb = residual; a.w.words = words;
     a.w.scale_out = nullptr; a.w.rscale = nullptr; a.w.partials = nullptr; a.w.tickets = nullptr;
-    a.w.tiles = nullptr; a.w.blocks = nullptr; a.w.mu = mu; a.w.fused = 1;
+    a.w.tiles = nullptr; a.w.blocks = nullptr; a.w.mu = mu; a.w.ratio = 1.f; a.w.fused = 1;
     a.w.g_stride = 0; a.w.state_stride = 0; a.w.word_stride = 0; a.w.partial_stride = 0;
     a.w.scale_stride = 0;
     a.rscale_io = residual_scale; a.scale_out = scale;

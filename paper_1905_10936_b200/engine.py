@@ -27,7 +27,7 @@ class EFEngine:
     """One dist-EF-blockSGDM problem on the current CUDA device."""
 
     def __init__(self, offsets, M: int, mu: float, eta: float, host_staging: bool = False,
-                 scale_mode: str = "auto", stream: Optional[torch.cuda.Stream] = None, device: Optional[torch.device] = None):
+                 scale_mode: str = "auto", weight_decay: bool = False, stream: Optional[torch.cuda.Stream] = None, device: Optional[torch.device] = None):
         if not torch.cuda.is_available():
             raise RuntimeError("EFEngine needs a CUDA device (there is no CPU path)")
         self.device = torch.device(device if device is not None else f"cuda:{torch.cuda.current_device()}")
@@ -36,6 +36,7 @@ class EFEngine:
         self.d = int(self.offsets[-1])
         self.M = int(M)
         flags = ef.EF_FLAG_HOST_STAGING if host_staging else 0
+        flags |= ef.EF_FLAG_WEIGHT_DECAY if weight_decay else 0
         flags |= {"auto": 0, "fused": ef.EF_FLAG_FUSED_SCALE, "split": ef.EF_FLAG_SPLIT_SCALE}[scale_mode]
         nbytes = ef.ef_workspace_bytes(self.d, self.B, self.offsets, self.M, flags)
         self.workspace_bytes = nbytes
@@ -76,6 +77,15 @@ class EFEngine:
 
     def server_step(self) -> None:
         ef.ef_server_step(self.ctx)
+
+    def set_eta(self, eta: float) -> None:
+        ef.ef_set_eta(self.ctx, float(eta))
+
+    def set_weight_decay(self, lam: float) -> None:
+        ef.ef_set_weight_decay(self.ctx, float(lam))
+
+    def decay_momentum(self) -> torch.Tensor:
+        return _as_tensor(ef.ef_decay_momentum(self.ctx), self.d, torch.float32, self.device)
 
     def read_update_host(self, words: torch.Tensor, scales: torch.Tensor) -> None:
         assert words.numel() == self.W and scales.numel() == self.B

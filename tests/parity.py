@@ -81,12 +81,21 @@ def assert_scales_close(got: np.ndarray, ref: np.ndarray, what: str):
 
 def run_parity(w: Workload, steps: Optional[int] = None, blocks: Optional[Sequence[int]] = None,
                grads: Optional[List[List[torch.Tensor]]] = None, check_every_step: bool = True,
-               device: str = "cuda", scale_mode: str = "auto", batched: bool = False):
+               device: str = "cuda", scale_mode: str = "auto", batched: bool = False,
+               etas: Optional[Sequence[float]] = None, weight_decay: float = 0.0,
+               x0: Optional[torch.Tensor] = None):
     """Runs `steps` iterations on both sides; returns (engine, oracle, stats)."""
     steps = w.steps if steps is None else steps
-    eng = EFEngine(w.offsets, w.M, w.mu, w.eta, scale_mode=scale_mode)
+    eta0 = w.eta if etas is None else etas[0]
+    eng = EFEngine(w.offsets, w.M, w.mu, eta0, scale_mode=scale_mode, weight_decay=weight_decay > 0)
     smp = BlockSample(w.offsets, blocks)
-    orc = Oracle(smp.sub_offsets, w.M, w.mu, w.eta)
+    orc = Oracle(smp.sub_offsets, w.M, w.mu, eta0)
+    if weight_decay > 0:
+        eng.set_weight_decay(weight_decay)
+        orc.set_weight_decay(weight_decay)
+    if x0 is not None:
+        eng.params().copy_(x0.to(device))
+        orc.x[:] = smp.elems(x0.to(device))
     es = w.element_scales(device)
     gbuf = torch.empty(w.d, dtype=torch.float32, device=device)
     # batched mode: all M gradients in one [M, stride] tensor, one ef_worker_step_all per step
@@ -94,6 +103,9 @@ def run_parity(w: Workload, steps: Optional[int] = None, blocks: Optional[Sequen
     gall = torch.zeros(w.M, stride, dtype=torch.float32, device=device) if batched else None
     stats = {"adopted": 0, "scale_bit_mismatch": 0, "scales_compared": 0, "adopted_list": []}
     for t in range(steps):
+        if etas is not None and t > 0:
+            eng.set_eta(etas[t])
+            orc.set_eta(etas[t])
         if batched:
             for i in range(w.M):
                 if grads is not None:
@@ -131,6 +143,9 @@ def run_parity(w: Workload, steps: Optional[int] = None, blocks: Optional[Sequen
         if check_every_step or t == steps - 1:
             compare_state(eng, orc, smp, f"after step {t}")
     assert eng.step_count == steps == orc.t
+    if weight_decay > 0:
+        assert_blockwise_close(smp.elems(eng.decay_momentum()), orc.decay_momentum, smp.sub_offsets,
+                               "decay momentum")
     return eng, orc, stats
 
 

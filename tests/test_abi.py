@@ -42,6 +42,8 @@ def test_workspace_bytes_accounts_for_all_state():
     assert state + words <= n <= state + words + (1 << 20)
     n2 = ef.ef_workspace_bytes(d, B, off, M, ef.EF_FLAG_HOST_STAGING)
     assert n2 - n == 2 * 4 * d
+    n3 = ef.ef_workspace_bytes(d, B, off, M, ef.EF_FLAG_WEIGHT_DECAY)
+    assert n3 - n == 4 * d
 
 
 @pytest.mark.parametrize("d,offsets,M", [
@@ -70,7 +72,7 @@ def test_init_validates_before_using_the_device():
         ef.ef_init(128, 2, off, 2, 0.9, 0.1, 0, 264, 1 << 30, 0)
     assert ei.value.status == ef.EF_ERR_ALIGNMENT
     with pytest.raises(ef.EFError) as ei:
-        ef.ef_init(128, 2, off, 2, 0.9, 0.1, 8, 256, 1 << 30, 0)     # unknown flag
+        ef.ef_init(128, 2, off, 2, 0.9, 0.1, 16, 256, 1 << 30, 0)    # unknown flag
     assert ei.value.status == ef.EF_ERR_INVALID_ARG
     with pytest.raises(ef.EFError) as ei:                            # contradictory flags
         ef.ef_init(128, 2, off, 2, 0.9, 0.1, ef.EF_FLAG_FUSED_SCALE | ef.EF_FLAG_SPLIT_SCALE,

@@ -81,6 +81,41 @@ def test_hyper_parameters(mu, eta):
     run_parity(w)
 
 
+# ------------------------------------------------------------------ stepsize sequence, weight decay
+@pytest.mark.parametrize("batched", [False, True])
+def test_stepsize_schedule(batched):
+    """eta_t changes between iterations; residuals are rescaled by eta_{t-1}/eta_t."""
+    w = _wl("sched", [TILE + 100, 777, 2 * BIG + 36, 3], 3, steps=8, scale_range=(1e-3, 1.0))
+    etas = [0.1, 0.1, 0.05, 0.2, 0.01, 0.01, 0.3, 0.1]
+    run_parity(w, etas=etas, batched=batched)
+
+
+@pytest.mark.parametrize("sizes,M", [([TILE + 100, 777, 2 * BIG + 36, 3], 3),
+                                      ([3, 5, 31, 33, 63, 65, 127, 129], 2)])
+def test_weight_decay_side_path(sizes, M):
+    w = _wl("decay", sizes, M, steps=6, scale_range=(1e-2, 1.0))
+    x0 = torch.randn(w.d)
+    run_parity(w, weight_decay=0.05, x0=x0)
+
+
+def test_schedule_and_weight_decay_on_resnet20_layout():
+    w = wl.make_workload(2)
+    etas = [0.1] * 3 + [0.01] * 3 + [0.001] * 4
+    run_parity(w, etas=etas, weight_decay=5e-4, x0=torch.randn(w.d) * 0.1, batched=True)
+
+
+def test_weight_decay_needs_the_flag():
+    w = _wl("nodecay", [64], 1)
+    e = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    with pytest.raises(ef.EFError) as ei:
+        e.set_weight_decay(0.1)
+    assert ei.value.status == ef.EF_ERR_BAD_STATE
+    with pytest.raises(ef.EFError) as ei:
+        e.set_eta(0.0)
+    assert ei.value.status == ef.EF_ERR_INVALID_ARG
+    assert ef.ef_decay_momentum(e.ctx) is None
+
+
 def test_zero_gradients_and_zero_blocks():
     """All-zero blocks: scale 0, every bit 0, state stays 0 (sign(0) = +1)."""
     w = _wl("zeros", [100, TILE, 64], 2, steps=3)
