@@ -37,7 +37,7 @@ UNIT = "params/s"
 
 # DRAM traffic per launch of the worker kernel measured by ncu (dram__bytes_read.sum +
 # dram__bytes_write.sum), in bytes per parameter; see profiles/ for the capture it comes from.
-NCU_WORKER_TRAFFIC_BYTES_PER_PARAM = 19.91   # 5.3445e9 bytes per launch at d = 2^28
+NCU_WORKER_TRAFFIC_BYTES_PER_PARAM = 20.10   # 37.766e9 bytes per 7-worker launch at d = 2^28
 
 
 # --------------------------------------------------------------------------- byte counts
@@ -200,7 +200,9 @@ def run_ours(args) -> None:
     # all work of the context runs on this (non-default) stream, which is also made current
     stream = torch.cuda.Stream(device=dev)
     torch.cuda.set_stream(stream)
-    eng = EFEngine(w.offsets, w.M, w.mu, w.eta, stream=stream)
+    eng = EFEngine(w.offsets, w.M, w.mu, w.eta, stream=stream, weight_decay=args.weight_decay > 0)
+    if args.weight_decay > 0:
+        eng.set_weight_decay(args.weight_decay)
     es = w.element_scales(dev)
     stride = (w.d + 3) // 4 * 4
     gall = torch.zeros(w.M, stride, dtype=torch.float32, device=dev)   # pre-staged in HBM
@@ -321,7 +323,7 @@ def run_ours(args) -> None:
 
     peak, peak_kind = measured_hbm_peak()
     wbytes = worker_call_bytes(w.d, w.B) * (w.M if batched else 1)
-    sbytes = server_call_bytes(w.d, w.B, w.M)
+    sbytes = server_call_bytes(w.d, w.B, w.M) + (8.0 * w.d if args.weight_decay > 0 else 0.0)
     w_gbs = wbytes / (worker_ms * 1e-3) / 1e9
     s_gbs = sbytes / (server_ms * 1e-3) / 1e9
     state_gib = eng_state_gib(w)
@@ -332,6 +334,7 @@ def run_ours(args) -> None:
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
         "config": {"workload": w.name, "d": w.d, "B": w.B, "M": w.M, "mu": w.mu, "eta": w.eta,
+                   "weight_decay": args.weight_decay,
                    "worker_calls": "ef_worker_step_all" if batched else "ef_worker_step x M",
                    "per_gpu": "each rank owns one such layout (block-range shard of an "
                               "N-times larger problem)",
@@ -399,6 +402,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--per-worker-calls", action="store_true",
                     help="step the workers with M ef_worker_step calls instead of one ef_worker_step_all")
+    ap.add_argument("--weight-decay", type=float, default=0.0,
+                    help="enable the weight-decay side path (adds a d-float momentum to the server call)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--graph", action="store_true",
                     help="also time the step replayed from a CUDA graph (extra key cuda_graph)")
