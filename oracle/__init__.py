@@ -60,6 +60,8 @@ def _load():
     for name in ("efo_momentum", "efo_residual", "efo_words", "efo_scales"):
         getattr(lib, name).restype = vp
         getattr(lib, name).argtypes = [vp, i32]
+    lib.efo_diagnostics.restype = vp
+    lib.efo_diagnostics.argtypes = [vp, i32]
     _lib = lib
     return lib
 
@@ -160,3 +162,7 @@ class Oracle:
 
     def scales(self, i: int = -1) -> np.ndarray:
         return _view(self._lib.efo_scales(self._h, i), self.B, np.float32)
+
+    def diagnostics(self, i: int) -> np.ndarray:
+        """[B, 4] float64: ||p_b||_1, ||p_b||_2^2, ||g_b||_1, ||g_b||_2^2 of worker i's last call."""
+        return _view(self._lib.efo_diagnostics(self._h, i), 4 * self.B, np.float64).reshape(self.B, 4)

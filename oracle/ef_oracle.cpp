@@ -24,6 +24,12 @@
 //   mtilde_t = mu mtilde_{t-1} + lambda x_t,   x_{t+1} = x_t - eta_t (Deltatilde_t + mu mtilde_t + lambda x_t),
 // done once here because all replicas of x are identical.
 //
+// Diagnostics (Section 3.2, Fig. 1): every worker call also records, per block, ||p_b||_1,
+// ||p_b||_2^2, ||g_b||_1 and ||g_b||_2^2 (binary64 sums), from which follow
+//   phi(p) = min_b ||p_b||_1^2 / (d_b ||p_b||_2^2)            (Prop. 1),
+//   delta of the non-block compressor = ||p||_1^2 / (d ||p||_2^2)   (Section 3.2),
+//   coefficient of variation of |g| in block b = sqrt(d_b ||g_b||_2^2 / ||g_b||_1^2 - 1).
+//
 // Readings where the paper is silent (each is a convention of this repository):
 //   * until efo_set_eta is called the stepsize is constant, so eta_{t-1}/eta_t = 1; at t = 0 the
 //     paper's ratio (eta_{-1} = 0) multiplies e_0 = etilde_0 = 0, which the ratio 1 reproduces;
@@ -86,6 +92,9 @@ struct Oracle {
     std::vector<uint32_t> swords;        // server packed signs
     std::vector<float> sscales;          // server block scales
     std::vector<uint8_t> stepped;        // worker i has pushed in this iteration
+    // Diagnostics of the last worker call of each worker (the quantities behind Fig. 1):
+    // per block ||p_b||_1, ||p_b||_2^2, ||g_b||_1, ||g_b||_2^2, accumulated in binary64.
+    std::vector<std::vector<double>> diag;   // [M][4*B]
 };
 
 // Compress p[lo,hi) of block b (Section 3.2), write the block's scale and packed signs,
@@ -165,6 +174,7 @@ void* efo_init(int64_t d, int32_t B, const int64_t* offsets, int32_t M, float mu
     o->swords.assign(o->W, 0u);
     o->sscales.assign(B, 0.f);
     o->stepped.assign(M, 0);
+    o->diag.assign(M, std::vector<double>(4 * (size_t)B, 0.0));
     return o;
 }
 
@@ -192,6 +202,15 @@ int64_t efo_worker_step(void* h, int32_t i, const float* grad, const uint32_t* h
             m[j] = std::fmaf(mu, m[j], grad[j]);             // m_t = mu m_{t-1} + g_t
             const float u = std::fmaf(mu, m[j], grad[j]);    // mu m_t + g_t
             p[j] = std::fmaf(r, e[j], u);                    // + (eta_{t-1}/eta_t) e_t
+        }
+        {   // diagnostics: plain sums over the block, independent of the compression below
+            double p1 = 0.0, p2 = 0.0, g1 = 0.0, g2 = 0.0;
+            for (int64_t j = lo; j < hi; ++j) {
+                p1 += (double)std::fabs(p[j]);      p2 += (double)p[j] * (double)p[j];
+                g1 += (double)std::fabs(grad[j]);   g2 += (double)grad[j] * (double)grad[j];
+            }
+            double* dg = o->diag[i].data() + 4 * (size_t)b;
+            dg[0] = p1; dg[1] = p2; dg[2] = g1; dg[3] = g2;
         }
         n_adopted = compress_block(p, lo, hi, &o->scales[i][b],
                                    o->words[i].data() + o->woff[b], e, nullptr, 0.f, 0.f, 0.f,
@@ -261,6 +280,8 @@ int32_t efo_set_weight_decay(void* h, float lambda)
     if (lambda > 0.f && o->mt.empty()) o->mt.assign(o->d, 0.f);
     return 0;
 }
+
+double* efo_diagnostics(void* h, int32_t i) { return static_cast<Oracle*>(h)->diag[i].data(); }
 
 float* efo_decay_momentum(void* h) { Oracle* o = static_cast<Oracle*>(h);
                                      return o->mt.empty() ? nullptr : o->mt.data(); }
