@@ -61,6 +61,8 @@ enum ef_status {
 #define EF_FLAG_FUSED_SCALE 2u     /* always complete the sums inside the main kernels */
 #define EF_FLAG_SPLIT_SCALE 4u     /* always use the follow-up kernel */
 #define EF_FLAG_WEIGHT_DECAY 8u    /* reserve the d-float decay momentum for ef_set_weight_decay */
+#define EF_FLAG_DIAGNOSTICS 16u    /* worker steps also record per-block sums (ef_worker_diagnostics);
+                                      implies the follow-up scale kernel, excludes EF_FLAG_FUSED_SCALE */
 
 /* Maximum number of simulated workers. */
 #define EF_MAX_WORKERS 4096
@@ -120,6 +122,15 @@ int ef_worker_step_host(ef_ctx* ctx, int32_t i, const float* grad /* host */);
  * Errors: BAD_STATE unless every worker has been stepped exactly once since the last
  * server step; CUDA. */
 int ef_server_step(ef_ctx* ctx);
+
+/* Diagnostics of worker i's last step (needs EF_FLAG_DIAGNOSTICS): B x 4 doubles, row b =
+ * { ||p_b||_1, ||p_b||_2^2, ||g_b||_1, ||g_b||_2^2 } accumulated in fp64 inside the worker kernel
+ * at no extra memory traffic.  From them follow the quantities of Section 3.2 / Fig. 1:
+ * phi(p) = min_b ||p_b||_1^2 / (d_b ||p_b||_2^2) (Prop. 1), the non-block compressor's
+ * delta = ||p||_1^2 / (d ||p||_2^2), and the coefficient of variation of |g| inside block b,
+ * sqrt(d_b ||g_b||_2^2 / ||g_b||_1^2 - 1).  Device pointer, valid until ef_destroy, ordered on
+ * the context's stream; NULL without the flag or on a bad index. */
+const double* ef_worker_diagnostics(ef_ctx* ctx, int32_t i);
 
 /* Stepsize of the coming iteration (Algorithms 2-4 take a stepsize sequence {eta_t}).  In that
  * iteration both the workers' and the server's residual enter rescaled by eta_{t-1}/eta_t

@@ -30,6 +30,7 @@ EF_FLAG_HOST_STAGING = 1
 EF_FLAG_FUSED_SCALE = 2
 EF_FLAG_SPLIT_SCALE = 4
 EF_FLAG_WEIGHT_DECAY = 8
+EF_FLAG_DIAGNOSTICS = 16
 EF_MAX_WORKERS = 4096
 
 _vp, _i64, _i32, _u32, _f32 = (ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_uint32,
@@ -44,6 +45,7 @@ SIGNATURES = {
     "ef_worker_step_all": (ctypes.c_int, [_vp, _vp, _i64]),
     "ef_worker_step_host": (ctypes.c_int, [_vp, _i32, _vp]),
     "ef_server_step": (ctypes.c_int, [_vp]),
+    "ef_worker_diagnostics": (_vp, [_vp, _i32]),
     "ef_set_eta": (ctypes.c_int, [_vp, _f32]),
     "ef_set_weight_decay": (ctypes.c_int, [_vp, _f32]),
     "ef_decay_momentum": (_vp, [_vp]),
@@ -131,6 +133,10 @@ def ef_worker_step_host(ctx: int, i: int, grad_host_ptr: int) -> None:
 
 def ef_server_step(ctx: int) -> None:
     _check(load_library().ef_server_step(ctx), "ef_server_step")
+
+
+def ef_worker_diagnostics(ctx: int, i: int) -> Optional[int]:
+    return load_library().ef_worker_diagnostics(ctx, i)
 
 
 def ef_set_eta(ctx: int, eta: float) -> None:

@@ -75,6 +75,10 @@ struct WorkerArgs {
     // batched launches: blockIdx.y selects the worker; its buffers lie at these strides
     long long g_stride, state_stride, word_stride, partial_stride;
     int scale_stride;      // also the stride of the ticket arrays
+    // diagnostics (DIAG instantiation only): per-CTA partial sums of p^2, |g|, g^2 in three
+    // arrays of `partial_stride` slots each, and the per-block results [B][4] (|p|, p^2, |g|, g^2)
+    double* dpartials;
+    double* diag;
 };
 
 struct ServerArgs {
@@ -103,6 +107,8 @@ struct ScaleArgs {
     float* rscale;
     long long partial_stride;   // blockIdx.y selects the buffer set (worker)
     int scale_stride;
+    double* dpartials;          // DIAG instantiation only, as in WorkerArgs
+    double* diag;
 };
 
 struct ApplyArgs {
@@ -182,21 +188,28 @@ __device__ __forceinline__ double cta_sum(double v, double* s_sum) {
 
 // Adds the partial sums of block b in a fixed order (thread k takes slots k, k+256, ...; then
 // the CTA tree) and writes the scale s_b = ||p_b||_1 / d_b (Section 3.2).  Called by a whole CTA.
-__device__ __forceinline__ void sum_partials_and_write(const Block& b, int block_id,
-                                                       const double* __restrict__ partials,
-                                                       float* __restrict__ scale_out,
-                                                       float* __restrict__ rscale,
-                                                       double* s_sum) {
+// Sum of the block's partial-sum slots in a fixed order; valid in thread 0.
+__device__ __forceinline__ double sum_slots(const Block& b, const double* __restrict__ partials,
+                                            double* s_sum) {
     const double* src = partials + (long long)b.tile_begin * kTileChunks;
     const int n = b.tile_count * kTileChunks;
     double v = 0.0;
     for (int k = threadIdx.x; k < n; k += kThreads) v += __ldcg(&src[k]);
-    const double S = cta_sum(v, s_sum);
+    return cta_sum(v, s_sum);
+}
+
+__device__ __forceinline__ double sum_partials_and_write(const Block& b, int block_id,
+                                                         const double* __restrict__ partials,
+                                                         float* __restrict__ scale_out,
+                                                         float* __restrict__ rscale,
+                                                         double* s_sum) {
+    const double S = sum_slots(b, partials, s_sum);
     if (threadIdx.x == 0) {
         const float s = (float)(S / (double)b.len);
         scale_out[block_id] = s;
         rscale[block_id] = s;
     }
+    return S;
 }
 
 // End of a CTA's work: turns its |p| sum into the block scale or a published partial sum.
@@ -243,13 +256,63 @@ __device__ __forceinline__ void finish_block(double acc, long long slot, int zer
 }
 
 // Follow-up kernel of the non-fused mode: one CTA per block that spans more than one chunk.
+// DIAG also completes the three diagnostic sums and records all four per block.
+template <bool DIAG>
 __global__ void __launch_bounds__(kThreads) ef_scale_kernel(const ScaleArgs a) {
     __shared__ double s_sum[kWarps];
     const int block_id = a.multi[blockIdx.x];
     const Block b = a.blocks[block_id];
     const long long so = (long long)blockIdx.y * a.scale_stride;
-    sum_partials_and_write(b, block_id, a.partials + blockIdx.y * a.partial_stride,
-                           a.scale_out + so, a.rscale + so, s_sum);
+    const double S = sum_partials_and_write(b, block_id, a.partials + blockIdx.y * a.partial_stride,
+                                            a.scale_out + so, a.rscale + so, s_sum);
+    if (DIAG) {
+        double* dg = a.diag + (so + block_id) * 4;
+        if (threadIdx.x == 0) dg[0] = S;
+        const double* dp = a.dpartials + blockIdx.y * (3 * a.partial_stride);
+#pragma unroll
+        for (int k = 0; k < 3; ++k) {
+            __syncthreads();
+            const double v = sum_slots(b, dp + k * a.partial_stride, s_sum);
+            if (threadIdx.x == 0) dg[1 + k] = v;
+        }
+    }
+}
+
+// Diagnostic sums of one thread: p^2, |g|, g^2 (|p| is the compressor's own sum).
+struct DiagAcc {
+    double p2 = 0.0, g1 = 0.0, g2 = 0.0;
+};
+
+// End of a CTA's work in the DIAG instantiation (always the non-fused mode): publishes the four
+// sums as partial sums, or as final per-block values when the CTA covered the whole block.
+__device__ __forceinline__ void finish_block_diag(double acc, const DiagAcc& d, long long slot,
+                                                  bool alone, int block_id, long long block_len,
+                                                  double* __restrict__ partials,
+                                                  double* __restrict__ dpartials,
+                                                  long long partial_stride,
+                                                  double* __restrict__ diag,
+                                                  float* __restrict__ scale_out,
+                                                  float* __restrict__ rscale) {
+    __shared__ double s_sum[kWarps];
+    const double in[4] = {acc, d.p2, d.g1, d.g2};
+    double r[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        r[k] = cta_sum(in[k], s_sum);
+        __syncthreads();
+    }
+    if (threadIdx.x != 0) return;
+    if (alone) {
+        const float s = (float)(r[0] / (double)block_len);
+        scale_out[block_id] = s;
+        rscale[block_id] = s;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) diag[(long long)block_id * 4 + k] = r[k];
+    } else {
+        partials[slot] = r[0];
+#pragma unroll
+        for (int k = 0; k < 3; ++k) dpartials[k * partial_stride + slot] = r[1 + k];
+    }
 }
 
 // Packs the four sign bits each lane holds (nibble, element k in bit k) into 32-bit words:
@@ -295,8 +358,9 @@ __device__ __forceinline__ Tile chunk_of(const Tile& t, int sub) {
 // ------------------------------------------------------------------ worker kernel
 // One chunk per CTA.  Warp w owns the 128*U consecutive elements starting at w*128*U; in row u
 // lane l holds elements u*128 + 4l .. +3 (a 128-bit access, 512 contiguous bytes per warp).
-template <int U, bool FULL>
-__device__ __forceinline__ double worker_rows(const WorkerArgs& a, const Tile& t, float sp) {
+template <int U, bool FULL, bool DIAG = false>
+__device__ __forceinline__ double worker_rows(const WorkerArgs& a, const Tile& t, float sp,
+                                              DiagAcc* dacc = nullptr) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int o0 = warp * (128 * U) + lane * 4;
     const float* gp = a.g + t.start + o0;
@@ -324,6 +388,15 @@ __device__ __forceinline__ double worker_rows(const WorkerArgs& a, const Tile& t
         }
         const unsigned nib = sign_nibble(p[u]);
         acc += abs_sum4(p[u]);
+        if (DIAG) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {          // g is 0 beyond the chunk's end (load4)
+                const double pd = (double)p[u][k], gd = (double)g[u][k];
+                dacc->p2 = fma(pd, pd, dacc->p2);
+                dacc->g1 += fabs(gd);
+                dacc->g2 = fma(gd, gd, dacc->g2);
+            }
+        }
         const unsigned w = pack_nibbles(nib, lane);
         store4(mp + u * 128, o, t.len, FULL, m[u]);
         store4(pp + u * 128, o, t.len, FULL, p[u]);
@@ -334,7 +407,9 @@ __device__ __forceinline__ double worker_rows(const WorkerArgs& a, const Tile& t
 
 // Fallback for chunks that do not start on a 16-byte boundary: 32-bit accesses, one ballot per
 // 32 elements.
-__device__ __forceinline__ double worker_rows_scalar(const WorkerArgs& a, const Tile& t, float sp) {
+template <bool DIAG = false>
+__device__ __forceinline__ double worker_rows_scalar(const WorkerArgs& a, const Tile& t, float sp,
+                                                     DiagAcc* dacc = nullptr) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rows = (t.len + 31) >> 5;
     double acc = 0.0;
@@ -350,6 +425,12 @@ __device__ __forceinline__ double worker_rows_scalar(const WorkerArgs& a, const 
             pv = __fmaf_rn(a.ratio, e, __fmaf_rn(a.mu, m, g));
             a.m[j] = m;
             a.pb[j] = pv;
+            if (DIAG) {
+                const double pd = (double)pv, gd = (double)g;
+                dacc->p2 = fma(pd, pd, dacc->p2);
+                dacc->g1 += fabs(gd);
+                dacc->g2 = fma(gd, gd, dacc->g2);
+            }
         }
         acc += (double)fabsf(pv);
         const unsigned w = __ballot_sync(kFull, valid && pv < 0.f);
@@ -359,11 +440,15 @@ __device__ __forceinline__ double worker_rows_scalar(const WorkerArgs& a, const 
 }
 
 // grid.x = chunks, grid.y = workers stepped by this launch (1 for ef_worker_step).
-template <int U>
+template <int U, bool DIAG>
 __global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a0) {
     WorkerArgs a = a0;
     {
         const long long wi = blockIdx.y;
+        if (DIAG) {
+            a.dpartials += wi * (3 * a.partial_stride);
+            a.diag += wi * (4LL * a.scale_stride);
+        }
         a.g += wi * a.g_stride;
         a.m += wi * a.state_stride;
         a.pb += wi * a.state_stride;
@@ -378,17 +463,22 @@ __global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a0
     const bool alone = b.len <= 1024 * U;              // the block is this single chunk
     if (t.len <= 0 && alone) return;
     double acc = 0.0;
+    DiagAcc dacc;
     if (t.len > 0) {
         const float sp = a.rscale[t.block];
         if ((t.start & 3) != 0)
-            acc = worker_rows_scalar(a, t, sp);
+            acc = worker_rows_scalar<DIAG>(a, t, sp, &dacc);
         else if (t.len == 1024 * U)
-            acc = worker_rows<U, true>(a, t, sp);
+            acc = worker_rows<U, true, DIAG>(a, t, sp, &dacc);
         else
-            acc = worker_rows<U, false>(a, t, sp);
+            acc = worker_rows<U, false, DIAG>(a, t, sp, &dacc);
     }
-    finish_block(acc, blockIdx.x, 0, alone, (unsigned)(b.tile_count * kTileChunks), t.block,
-                 a.blocks, a.partials, a.tickets, a.scale_out, a.rscale, a.fused);
+    if (DIAG)
+        finish_block_diag(acc, dacc, blockIdx.x, alone, t.block, b.len, a.partials, a.dpartials,
+                          a.partial_stride, a.diag, a.scale_out, a.rscale);
+    else
+        finish_block(acc, blockIdx.x, 0, alone, (unsigned)(b.tile_count * kTileChunks), t.block,
+                     a.blocks, a.partials, a.tickets, a.scale_out, a.rscale, a.fused);
 }
 
 // ------------------------------------------------------------------ server kernel

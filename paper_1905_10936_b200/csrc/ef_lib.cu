@@ -35,7 +35,7 @@ struct Layout {
     size_t dpad = 0, wpad = 0, bpad = 0, tpad = 0;    // padded element counts per sub-buffer
     size_t off_x = 0, off_m = 0, off_pb = 0, off_spb = 0, off_words = 0, off_scales = 0,
            off_rscale = 0, off_partials = 0, off_tickets = 0, off_tiles = 0, off_blocks = 0,
-           off_multi = 0, off_stage = 0, off_mt = 0, total = 0;
+           off_multi = 0, off_stage = 0, off_mt = 0, off_dpartials = 0, off_diag = 0, total = 0;
     int32_t num_multi = 0;                            // blocks that span more than one chunk
 };
 
@@ -52,9 +52,10 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
     int rc = check_problem(d, B, offsets, M);
     if (rc != EF_OK) return rc;
     if (flags & ~(EF_FLAG_HOST_STAGING | EF_FLAG_FUSED_SCALE | EF_FLAG_SPLIT_SCALE |
-                  EF_FLAG_WEIGHT_DECAY))
+                  EF_FLAG_WEIGHT_DECAY | EF_FLAG_DIAGNOSTICS))
         return EF_ERR_INVALID_ARG;
-    if ((flags & EF_FLAG_FUSED_SCALE) && (flags & EF_FLAG_SPLIT_SCALE)) return EF_ERR_INVALID_ARG;
+    if ((flags & EF_FLAG_FUSED_SCALE) && (flags & (EF_FLAG_SPLIT_SCALE | EF_FLAG_DIAGNOSTICS)))
+        return EF_ERR_INVALID_ARG;
     L->d = d; L->B = B; L->M = M;
     int64_t W = 0, T = 0;
     for (int32_t b = 0; b < B; ++b) {
@@ -81,6 +82,8 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
     L->off_rscale = o;   o += M1 * L->bpad * 4;
     L->off_partials = o; o += M1 * L->tpad * 8;
     L->off_tickets = o;  o += M1 * L->bpad * 4;
+    L->off_dpartials = o; if (flags & EF_FLAG_DIAGNOSTICS) o += (size_t)M * 3 * L->tpad * 8;
+    L->off_diag = o;      if (flags & EF_FLAG_DIAGNOSTICS) o += (size_t)M * 4 * L->bpad * 8;
     L->off_tiles = o;    o += align_up((size_t)T * sizeof(Tile));
     L->off_blocks = o;   o += align_up((size_t)B * sizeof(Block));
     L->off_multi = o;    o += align_up((size_t)L->num_multi * sizeof(int32_t) + 4);
@@ -129,6 +132,8 @@ struct ef_ctx {
     const Block* blocks() const { return (const Block*)(ws + L.off_blocks); }
     const int* multi() const { return (const int*)(ws + L.off_multi); }
     float* mt() const { return (float*)(ws + L.off_mt); }
+    double* dpartials(int i) const { return (double*)(ws + L.off_dpartials) + (size_t)i * 3 * L.tpad; }
+    double* diag(int i) const { return (double*)(ws + L.off_diag) + (size_t)i * 4 * L.bpad; }
     float* stage(int s) const { return (float*)(ws + L.off_stage) + (size_t)s * L.dpad; }
 };
 
@@ -154,8 +159,12 @@ int launch_scale(ef_ctx* c, int k, int count = 1) {
     a.partials = c->partials(k); a.blocks = c->blocks(); a.multi = c->multi();
     a.scale_out = c->scales(k); a.rscale = c->rscale(k);
     a.partial_stride = (long long)c->L.tpad; a.scale_stride = (int)c->L.bpad;
-    efk::ef_scale_kernel<<<dim3((unsigned)c->L.num_multi, (unsigned)count), efk::kThreads, 0,
-                           c->stream>>>(a);
+    const bool diag = (c->flags & EF_FLAG_DIAGNOSTICS) && k < c->L.M;
+    a.dpartials = diag ? c->dpartials(k) : nullptr;
+    a.diag = diag ? c->diag(k) : nullptr;
+    const dim3 grid((unsigned)c->L.num_multi, (unsigned)count);
+    if (diag) efk::ef_scale_kernel<true><<<grid, efk::kThreads, 0, c->stream>>>(a);
+    else efk::ef_scale_kernel<false><<<grid, efk::kThreads, 0, c->stream>>>(a);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
     return EF_OK;
@@ -172,8 +181,12 @@ int launch_worker(ef_ctx* c, int i, const float* grad, int count = 1, long long 
     a.g_stride = g_stride; a.state_stride = (long long)c->L.dpad;
     a.word_stride = (long long)c->L.wpad; a.partial_stride = (long long)c->L.tpad;
     a.scale_stride = (int)c->L.bpad;
-    efk::ef_worker_kernel<kU><<<dim3((unsigned)(c->L.num_tiles * efk::kTileChunks), (unsigned)count),
-                                efk::kThreads, 0, c->stream>>>(a);
+    const bool diag = (c->flags & EF_FLAG_DIAGNOSTICS) != 0;
+    a.dpartials = diag ? c->dpartials(i) : nullptr;
+    a.diag = diag ? c->diag(i) : nullptr;
+    const dim3 grid((unsigned)(c->L.num_tiles * efk::kTileChunks), (unsigned)count);
+    if (diag) efk::ef_worker_kernel<kU, true><<<grid, efk::kThreads, 0, c->stream>>>(a);
+    else efk::ef_worker_kernel<kU, false><<<grid, efk::kThreads, 0, c->stream>>>(a);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
     return launch_scale(c, i, count);
@@ -325,7 +338,7 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
     // Small grids are launch-bound: finish block scales inside the main kernels.  Large grids
     // are bandwidth-bound: the per-CTA fence of the fused form costs more than a tiny launch.
     if (flags & EF_FLAG_FUSED_SCALE) c->fused = 1;
-    else if (flags & EF_FLAG_SPLIT_SCALE) c->fused = 0;
+    else if (flags & (EF_FLAG_SPLIT_SCALE | EF_FLAG_DIAGNOSTICS)) c->fused = 0;
     else c->fused = (L.num_tiles * efk::kTileChunks <= kFusedMaxChunks) ? 1 : 0;
 
     auto fail = [&](cudaError_t e) { delete c; (void)e; return EF_ERR_CUDA; };
@@ -421,6 +434,10 @@ int ef_set_weight_decay(ef_ctx* c, float lambda) {
     if (c->pending != 0 || !(c->flags & EF_FLAG_WEIGHT_DECAY)) return EF_ERR_BAD_STATE;
     c->lambda = lambda;
     return EF_OK;
+}
+
+const double* ef_worker_diagnostics(ef_ctx* c, int32_t i) {
+    return (c && (c->flags & EF_FLAG_DIAGNOSTICS) && i >= 0 && i < c->L.M) ? c->diag(i) : nullptr;
 }
 
 float* ef_decay_momentum(ef_ctx* c) {
@@ -643,7 +660,7 @@ extern "C" int ef_worker_step_noalloc(const float* grad, float* momentum, float*
     a.w.scale_out = nullptr; a.w.rscale = nullptr; a.w.partials = nullptr; a.w.tickets = nullptr;
     a.w.tiles = nullptr; a.w.blocks = nullptr; a.w.mu = mu; a.w.ratio = 1.f; a.w.fused = 1;
     a.w.g_stride = 0; a.w.state_stride = 0; a.w.word_stride = 0; a.w.partial_stride = 0;
-    a.w.scale_stride = 0;
+    a.w.scale_stride = 0; a.w.dpartials = nullptr; a.w.diag = nullptr;
     a.rscale_io = residual_scale; a.scale_out = scale;
     a.partials = scratch;
     a.ticket = reinterpret_cast<unsigned*>(scratch + kNoAllocMaxChunks);

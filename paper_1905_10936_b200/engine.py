@@ -17,7 +17,8 @@ def _as_tensor(ptr: int, n: int, dtype: torch.dtype, device: torch.device) -> to
 
     class _Holder:
         __cuda_array_interface__ = {
-            "shape": (n,), "typestr": {torch.float32: "<f4", torch.int32: "<i4"}[dtype],
+            "shape": (n,), "typestr": {torch.float32: "<f4", torch.int32: "<i4",
+                                       torch.float64: "<f8"}[dtype],
             "data": (ptr, False), "version": 3, "strides": (itemsize,),
         }
     return torch.as_tensor(_Holder(), device=device)
@@ -27,7 +28,7 @@ class EFEngine:
     """One dist-EF-blockSGDM problem on the current CUDA device."""
 
     def __init__(self, offsets, M: int, mu: float, eta: float, host_staging: bool = False,
-                 scale_mode: str = "auto", weight_decay: bool = False, stream: Optional[torch.cuda.Stream] = None, device: Optional[torch.device] = None):
+                 scale_mode: str = "auto", weight_decay: bool = False, diagnostics: bool = False, stream: Optional[torch.cuda.Stream] = None, device: Optional[torch.device] = None):
         if not torch.cuda.is_available():
             raise RuntimeError("EFEngine needs a CUDA device (there is no CPU path)")
         self.device = torch.device(device if device is not None else f"cuda:{torch.cuda.current_device()}")
@@ -37,6 +38,7 @@ class EFEngine:
         self.M = int(M)
         flags = ef.EF_FLAG_HOST_STAGING if host_staging else 0
         flags |= ef.EF_FLAG_WEIGHT_DECAY if weight_decay else 0
+        flags |= ef.EF_FLAG_DIAGNOSTICS if diagnostics else 0
         flags |= {"auto": 0, "fused": ef.EF_FLAG_FUSED_SCALE, "split": ef.EF_FLAG_SPLIT_SCALE}[scale_mode]
         nbytes = ef.ef_workspace_bytes(self.d, self.B, self.offsets, self.M, flags)
         self.workspace_bytes = nbytes
@@ -77,6 +79,11 @@ class EFEngine:
 
     def server_step(self) -> None:
         ef.ef_server_step(self.ctx)
+
+    def worker_diagnostics(self, i: int) -> torch.Tensor:
+        """[B, 4] float64 view: ||p_b||_1, ||p_b||_2^2, ||g_b||_1, ||g_b||_2^2 of worker i's last step."""
+        return _as_tensor(ef.ef_worker_diagnostics(self.ctx, i), 4 * self.B, torch.float64,
+                          self.device).view(self.B, 4)
 
     def set_eta(self, eta: float) -> None:
         ef.ef_set_eta(self.ctx, float(eta))

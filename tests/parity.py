@@ -83,11 +83,12 @@ def run_parity(w: Workload, steps: Optional[int] = None, blocks: Optional[Sequen
                grads: Optional[List[List[torch.Tensor]]] = None, check_every_step: bool = True,
                device: str = "cuda", scale_mode: str = "auto", batched: bool = False,
                etas: Optional[Sequence[float]] = None, weight_decay: float = 0.0,
-               x0: Optional[torch.Tensor] = None):
+               x0: Optional[torch.Tensor] = None, diagnostics: bool = False):
     """Runs `steps` iterations on both sides; returns (engine, oracle, stats)."""
     steps = w.steps if steps is None else steps
     eta0 = w.eta if etas is None else etas[0]
-    eng = EFEngine(w.offsets, w.M, w.mu, eta0, scale_mode=scale_mode, weight_decay=weight_decay > 0)
+    eng = EFEngine(w.offsets, w.M, w.mu, eta0, scale_mode=scale_mode, weight_decay=weight_decay > 0,
+                   diagnostics=diagnostics)
     smp = BlockSample(w.offsets, blocks)
     orc = Oracle(smp.sub_offsets, w.M, w.mu, eta0)
     if weight_decay > 0:
@@ -129,6 +130,12 @@ def run_parity(w: Workload, steps: Optional[int] = None, blocks: Optional[Sequen
             assert_scales_close(gs, orc.scales(i), f"worker {i} step {t}")
             stats["scale_bit_mismatch"] += int((gs != orc.scales(i)).sum())
             stats["scales_compared"] += gs.size
+            if diagnostics:      # fp64 sums in a different order: 1e-11 relative
+                gd = eng.worker_diagnostics(i)[smp.block_index.to(device)].cpu().numpy()
+                od = orc.diagnostics(i)
+                assert np.all(np.abs(gd - od) <= 1e-11 * np.abs(od)), \
+                    f"worker {i} step {t}: diagnostics differ, max rel " \
+                    f"{(np.abs(gd - od) / np.maximum(np.abs(od), 1e-300)).max():.3e}"
         eng.server_step()
         gw = smp.words(eng.server_words())
         ad = orc.server_step(hint=gw)

@@ -116,6 +116,29 @@ def test_weight_decay_needs_the_flag():
     assert ef.ef_decay_momentum(e.ctx) is None
 
 
+@pytest.mark.parametrize("sizes,M,batched", [
+    ([TILE + 100, 777, 2 * BIG + 36, 3, 64], 3, False),
+    ([3, 5, 31, 33, 63, 65, 127, 129, TILE + 1], 2, True),       # scalar path
+    ([BIG, 2 * TILE, 5 * BIG + 8], 7, True),
+])
+def test_diagnostics_match_the_oracle(sizes, M, batched):
+    """Per-block ||p||_1, ||p||_2^2, ||g||_1, ||g||_2^2 recorded by the worker kernel."""
+    w = _wl("diag", sizes, M, steps=4, scale_range=(1e-3, 1.0))
+    run_parity(w, diagnostics=True, batched=batched)
+
+
+def test_diagnostics_on_the_resnet50_layout_give_phi_and_delta():
+    """phi(p) of the blockwise compressor against the non-block delta (Section 3.2, Fig. 1b)."""
+    w = wl.make_workload(3)
+    eng, orc, _ = run_parity(w, steps=2, diagnostics=True, batched=True, check_every_step=False)
+    dg = eng.worker_diagnostics(0).cpu().numpy()
+    sizes = np.asarray(w.sizes, dtype=np.float64)
+    phi = (dg[:, 0] ** 2 / (sizes * dg[:, 1])).min()
+    delta = dg[:, 0].sum() ** 2 / (sizes.sum() * dg[:, 1].sum())
+    assert 0.4 < phi < 0.7 and delta < 0.5 * phi          # Laplace-like blocks: phi ~ 1/2
+    assert ef.ef_worker_diagnostics(EFEngine(w.offsets[:2], 1, 0.9, 0.1).ctx, 0) is None
+
+
 def test_zero_gradients_and_zero_blocks():
     """All-zero blocks: scale 0, every bit 0, state stays 0 (sign(0) = +1)."""
     w = _wl("zeros", [100, TILE, 64], 2, steps=3)
