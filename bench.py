@@ -200,7 +200,8 @@ def run_ours(args) -> None:
     # all work of the context runs on this (non-default) stream, which is also made current
     stream = torch.cuda.Stream(device=dev)
     torch.cuda.set_stream(stream)
-    eng = EFEngine(w.offsets, w.M, w.mu, w.eta, stream=stream, weight_decay=args.weight_decay > 0)
+    eng = EFEngine(w.offsets, w.M, w.mu, w.eta, stream=stream, weight_decay=args.weight_decay > 0,
+                   diagnostics=args.diagnostics)
     if args.weight_decay > 0:
         eng.set_weight_decay(args.weight_decay)
     es = w.element_scales(dev)
@@ -334,7 +335,7 @@ def run_ours(args) -> None:
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
         "config": {"workload": w.name, "d": w.d, "B": w.B, "M": w.M, "mu": w.mu, "eta": w.eta,
-                   "weight_decay": args.weight_decay,
+                   "weight_decay": args.weight_decay, "diagnostics": bool(args.diagnostics),
                    "worker_calls": "ef_worker_step_all" if batched else "ef_worker_step x M",
                    "per_gpu": "each rank owns one such layout (block-range shard of an "
                               "N-times larger problem)",
@@ -404,6 +405,8 @@ def main():
                     help="step the workers with M ef_worker_step calls instead of one ef_worker_step_all")
     ap.add_argument("--weight-decay", type=float, default=0.0,
                     help="enable the weight-decay side path (adds a d-float momentum to the server call)")
+    ap.add_argument("--diagnostics", action="store_true",
+                    help="worker steps also record the per-block diagnostic sums")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--graph", action="store_true",
                     help="also time the step replayed from a CUDA graph (extra key cuda_graph)")

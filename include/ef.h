@@ -124,8 +124,9 @@ int ef_worker_step_host(ef_ctx* ctx, int32_t i, const float* grad /* host */);
 int ef_server_step(ef_ctx* ctx);
 
 /* Diagnostics of worker i's last step (needs EF_FLAG_DIAGNOSTICS): B x 4 doubles, row b =
- * { ||p_b||_1, ||p_b||_2^2, ||g_b||_1, ||g_b||_2^2 } accumulated in fp64 inside the worker kernel
- * at no extra memory traffic.  From them follow the quantities of Section 3.2 / Fig. 1:
+ * { ||p_b||_1, ||p_b||_2^2, ||g_b||_1, ||g_b||_2^2 } accumulated inside the worker kernel at no
+ * extra memory traffic (||p_b||_1 is the compressor's own fp64 sum; the other three combine four
+ * elements in fp32 before the fp64 accumulation: relative error below 1e-6).  From them follow the quantities of Section 3.2 / Fig. 1:
  * phi(p) = min_b ||p_b||_1^2 / (d_b ||p_b||_2^2) (Prop. 1), the non-block compressor's
  * delta = ||p||_1^2 / (d ||p||_2^2), and the coefficient of variation of |g| inside block b,
  * sqrt(d_b ||g_b||_2^2 / ||g_b||_1^2 - 1).  Device pointer, valid until ef_destroy, ordered on

@@ -389,13 +389,20 @@ __device__ __forceinline__ double worker_rows(const WorkerArgs& a, const Tile& t
         const unsigned nib = sign_nibble(p[u]);
         acc += abs_sum4(p[u]);
         if (DIAG) {
+            // The four elements of a lane are combined in fp32 (all terms are >= 0, so the
+            // relative error stays below 4 * 2^-24) and added to the fp64 sums once per row:
+            // diagnostics need 1e-6, not the 1e-13 of the scale.  g is 0 beyond the chunk's end.
+            float p2 = __fmul_rn(p[u][0], p[u][0]), g2 = __fmul_rn(g[u][0], g[u][0]);
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {          // g is 0 beyond the chunk's end (load4)
-                const double pd = (double)p[u][k], gd = (double)g[u][k];
-                dacc->p2 = fma(pd, pd, dacc->p2);
-                dacc->g1 += fabs(gd);
-                dacc->g2 = fma(gd, gd, dacc->g2);
+            for (int k = 1; k < 4; ++k) {
+                p2 = __fmaf_rn(p[u][k], p[u][k], p2);
+                g2 = __fmaf_rn(g[u][k], g[u][k], g2);
             }
+            const float g1 = __fadd_rn(__fadd_rn(fabsf(g[u][0]), fabsf(g[u][1])),
+                                       __fadd_rn(fabsf(g[u][2]), fabsf(g[u][3])));
+            dacc->p2 += (double)p2;
+            dacc->g1 += (double)g1;
+            dacc->g2 += (double)g2;
         }
         const unsigned w = pack_nibbles(nib, lane);
         store4(mp + u * 128, o, t.len, FULL, m[u]);

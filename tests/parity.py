@@ -130,10 +130,13 @@ def run_parity(w: Workload, steps: Optional[int] = None, blocks: Optional[Sequen
             assert_scales_close(gs, orc.scales(i), f"worker {i} step {t}")
             stats["scale_bit_mismatch"] += int((gs != orc.scales(i)).sum())
             stats["scales_compared"] += gs.size
-            if diagnostics:      # fp64 sums in a different order: 1e-11 relative
+            if diagnostics:
+                # ||p||_1 is the compressor's own fp64 sum (1e-11); the three diagnostic sums
+                # combine each lane's four elements in fp32 first: <= 4 * 2^-24 relative
                 gd = eng.worker_diagnostics(i)[smp.block_index.to(device)].cpu().numpy()
                 od = orc.diagnostics(i)
-                assert np.all(np.abs(gd - od) <= 1e-11 * np.abs(od)), \
+                tol = np.array([1e-11, 1e-6, 1e-6, 1e-6])
+                assert np.all(np.abs(gd - od) <= tol * np.abs(od)), \
                     f"worker {i} step {t}: diagnostics differ, max rel " \
                     f"{(np.abs(gd - od) / np.maximum(np.abs(od), 1e-300)).max():.3e}"
         eng.server_step()
