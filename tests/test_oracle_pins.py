@@ -480,36 +480,32 @@ def test_call_order_is_enforced():
 from hypothesis import given, settings, strategies as st
 
 
-@settings(max_examples=40, deadline=None)
+@settings(max_examples=40, deadline=None, derandomize=True)
 @given(st.lists(st.sampled_from([1, 2, 4, 8, 16, 32, 64]), min_size=1, max_size=5),
-       st.integers(1, 5), st.sampled_from([0.0, 0.25, 0.5]), st.integers(0, 2 ** 31 - 1))
+       st.sampled_from([1, 2, 4]), st.sampled_from([0.0, 0.25, 0.5]), st.integers(0, 2 ** 31 - 1))
 def test_property_two_exact_steps_on_random_dyadic_problems(sizes, M, mu, seed):
-    """Random layouts with power-of-two blocks (so every scale stays dyadic) and dyadic gradients:
-    the first worker pass of every step must equal exact rational arithmetic; everything after
-    a possibly inexact server division is compared to 1e-6."""
+    """Random layouts with power-of-two blocks and worker counts (so scales and the server
+    average stay dyadic) and dyadic gradients: every quantity of two full steps must equal exact
+    rational arithmetic.  (With other M the division by M is inexact, exact cancellations in
+    ptilde turn into +-tiny values and the sign there is legitimately not unique.)"""
     rng = np.random.default_rng(seed)
     off = [0] + list(np.cumsum(sizes))
     d = off[-1]
     o = Oracle(off, M, mu, 0.5)
     ex = ExactAlg4(off, M, Fraction(mu), Fraction(1, 2))
-    exact = True
     for t in range(2):
         grads = [rng.integers(-8, 9, size=d) / 2.0 for _ in range(M)]
         res = ex.step([[Fraction(float(v)) for v in g] for g in grads])
         for i in range(M):
             o.worker_step(i, grads[i].astype(np.float32))
             p, delta, scales = res[i]
-            if exact:
-                assert [Fraction(float(v)) for v in o.last_p] == p
-                assert [Fraction(float(v)) for v in o.scales(i)] == scales
-                assert [Fraction(v) for v in decode(o.words(i), o.scales(i), off)] == delta
-            else:
-                assert np.allclose(o.last_p, [float(v) for v in p], rtol=1e-6, atol=1e-6)
+            assert [Fraction(float(v)) for v in o.last_p] == p
+            assert [Fraction(float(v)) for v in o.scales(i)] == scales
+            assert [Fraction(v) for v in decode(o.words(i), o.scales(i), off)] == delta
+            assert [Fraction(float(v)) for v in o.residual(i)] == ex.e[i]
         o.server_step()
         p, delta, scales = res[-1]
-        exact = exact and all(Fraction(float(np.float32(float(v)))) == v for v in p) \
-            and (M & (M - 1)) == 0
-        if exact:
-            assert [Fraction(float(v)) for v in o.x] == ex.x
-        else:
-            assert np.allclose(o.x, [float(v) for v in ex.x], rtol=1e-6, atol=1e-6)
+        assert [Fraction(float(v)) for v in o.last_p] == p
+        assert [Fraction(float(v)) for v in o.scales(-1)] == scales
+        assert [Fraction(float(v)) for v in o.residual(-1)] == ex.et
+        assert [Fraction(float(v)) for v in o.x] == ex.x
