@@ -1,11 +1,13 @@
 #!/usr/bin/env python
 """Throughput of one two-way compressed dist-EF-blockSGDM step (Algorithm 4) on B200.
 
-A "step" is M calls of ef_worker_step plus one ef_server_step over one batch of synthetic
-gradients.  The default workload is the flat 2^28-parameter layout (256 blocks of 2^20,
-M = 7).  Prints ONE JSON line on rank 0.
+A "step" is the worker side of all M workers (one ef_worker_step_all launch, or M
+ef_worker_step calls with --per-worker-calls) plus one ef_server_step over one batch of
+synthetic gradients.  The default workload is the flat 2^28-parameter layout (256 blocks of
+2^20, M = 7).  Prints ONE JSON line on rank 0.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
+                  [--graph] [--per-worker-calls] [--weight-decay L] [--diagnostics] [--blocks N]
 
 With N > 1 (launched by torch.distributed.run) every rank owns its own block range of an
 N-times larger problem (blocks are independent in the method, so there is no data-path

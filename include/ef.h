@@ -4,7 +4,7 @@
  * momentum SGD with error feedback) of arXiv 1905.10936 for M simulated workers that all
  * live on one GPU.  One iteration t is
  *
- *     for each worker i in [0, M):  ef_worker_step(ctx, i, g_{t,i})
+ *     for each worker i in [0, M):  ef_worker_step(ctx, i, g_{t,i})     (or one ef_worker_step_all)
  *     ef_server_step(ctx)
  *
  * All entry points are plain C.  "device" pointers are CUDA device pointers of the current
