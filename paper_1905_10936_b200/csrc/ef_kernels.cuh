@@ -612,7 +612,8 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
         reinterpret_cast<unsigned*>(ring + (size_t)kServerStages * U * kThreads * sizeof(float4)) +
         threadIdx.x;
     double acc = 0.0;
-    unsigned c6 = 0, c7 = 0;               // bit patterns of the scaled scales of workers 6, 7
+    // bit patterns of the scaled scales of the workers the table does not cover
+    unsigned cdir[kMaxLutWorkers - kLutWorkers + 1] = {};
 
     auto issue_chunk = [&](int c) {
         if (c < nfull) {
@@ -636,21 +637,19 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
         for (int u = 0; u < U; ++u) {
             const int o = o0 + u * 128;
             const unsigned R = bf.indices(w[u]);
-            // byte offset of entry (R_k & 63) in this lane's copy: 128 * index
+            // byte offset of entry (R_k & (entries-1)) in this lane's copy: 128 * index
+            constexpr unsigned kIdxMask = (unsigned)(kLutEntries(MT) - 1) << 7;
             float avg[4];
-            avg[0] = *reinterpret_cast<const float*>(lut + ((R << 7) & 0x1F80u));
-            avg[1] = *reinterpret_cast<const float*>(lut + ((R >> 1) & 0x1F80u));
-            avg[2] = *reinterpret_cast<const float*>(lut + ((R >> 9) & 0x1F80u));
-            avg[3] = *reinterpret_cast<const float*>(lut + ((R >> 17) & 0x1F80u));
-            if (MT > 6) {                  // workers 6 and 7 follow in order
+            avg[0] = *reinterpret_cast<const float*>(lut + ((R << 7) & kIdxMask));
+            avg[1] = *reinterpret_cast<const float*>(lut + ((R >> 1) & kIdxMask));
+            avg[2] = *reinterpret_cast<const float*>(lut + ((R >> 9) & kIdxMask));
+            avg[3] = *reinterpret_cast<const float*>(lut + ((R >> 17) & kIdxMask));
+#pragma unroll
+            for (int wk = kLutWorkers; wk < MT; ++wk) {     // remaining workers follow in order
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
-                    avg[k] = __fadd_rn(avg[k], __uint_as_float(c6 ^ ((R << (25 - 8 * k)) & 0x80000000u)));
-            }
-            if (MT > 7) {
-#pragma unroll
-                for (int k = 0; k < 4; ++k)
-                    avg[k] = __fadd_rn(avg[k], __uint_as_float(c7 ^ ((R << (24 - 8 * k)) & 0x80000000u)));
+                    avg[k] = __fadd_rn(avg[k], __uint_as_float(
+                        cdir[wk - kLutWorkers] ^ ((R << (31 - wk - 8 * k)) & 0x80000000u)));
             }
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -673,8 +672,8 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
     build_scaled(a, t.block, MT, s_c);
     __syncthreads();
     build_lut<MT>(s_c, s_base, s_lut);
-    c6 = __float_as_uint(s_c[MT > 6 ? 6 : 0]);
-    c7 = __float_as_uint(s_c[MT > 7 ? 7 : 0]);
+#pragma unroll
+    for (int wk = kLutWorkers; wk < MT; ++wk) cdir[wk - kLutWorkers] = __float_as_uint(s_c[wk]);
     for (int c = 0; c < nfull; ++c) {
         issue_chunk(c + kServerStages - 1);      // reuses the slot this thread consumed at c - 1
         cp_async_wait<kServerStages - 1>();      // only the groups after chunk c may be in flight
