@@ -17,6 +17,10 @@
  * a caller may record them into a CUDA graph by capturing the stream; the host-side counters
  * and call-order checks then see the captured calls only, not the replays.
  *
+ * A context is not thread-safe: use it from one host thread at a time.  Different contexts
+ * are independent (the no-allocation entry point at the end of this file is the exception: its
+ * calls share one scratch array per device).
+ *
  * There is no CPU fallback: on a device that is not compute capability 10.x ef_init fails
  * with EF_ERR_UNSUPPORTED_DEVICE.
  *
