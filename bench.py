@@ -390,6 +390,9 @@ def load_workload(args) -> wl.Workload:
     if args.blocks and args.blocks < w.B:
         w = wl.custom_workload(f"{w.name}-first{args.blocks}blocks", w.sizes[:args.blocks], w.M,
                                w.mu, w.eta, w.steps, w.law, w.scale_range, config_id=w.config_id)
+    if args.workers and args.workers != w.M:
+        w = wl.custom_workload(f"{w.name}-M{args.workers}", w.sizes, args.workers, w.mu, w.eta,
+                               w.steps, w.law, w.scale_range, config_id=w.config_id)
     return w
 
 
@@ -401,6 +404,8 @@ def main():
     ap.add_argument("--config", type=int, default=4, help="workload 1..5 (default: flat 2^28)")
     ap.add_argument("--blocks", type=int, default=0,
                     help="use only the first N blocks of the workload (small cases for profiling)")
+    ap.add_argument("--workers", type=int, default=0,
+                    help="override the number of simulated workers M of the workload")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--per-worker-calls", action="store_true",
