@@ -492,22 +492,23 @@ __global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a0
 // a_j = sum over ascending i of (bit_i ? -c_i : +c_i), c_i = fl(scale_{i,b} / M), the first
 // term taken as is (Algorithm 4, server line: (1/M) sum_i Delta_{t,i}).
 //
-// For M <= 8 the sum over the first min(M, 6) workers is tabulated once per CTA in shared
-// memory (each entry is the same chain of fp32 additions, so the table is exact) and workers
-// 6 and 7 are added to the looked-up value directly, in order.  An element then costs one
+// For M <= 16 the sum over the first min(M, 6) workers is tabulated once per CTA in shared
+// memory (each entry is the same chain of fp32 additions, so the table is exact) and the
+// remaining workers are added to the looked-up value directly, in order.  An element then costs one
 // lookup plus at most two additions instead of M dependent additions with 2 bit operations
 // each.  The table has at most 64 entries and is stored 32 times, entry e of copy l at word
 // 32*e + l, so that lane l always reads bank l: the lookups are free of bank conflicts.
 //
 // Building the table index without per-worker work in every lane: the 8 lanes that share a
-// packed word each load the word of ONE worker (lane q -> worker kLaneWorker(q)).  Seen as an
+// packed word each load the word of ONE worker per group of 8 workers (lane q -> worker
+// kLaneWorker(q) of the group; M > 8 uses two groups, i.e. two words and two transposes).  Seen as an
 // 8x8 matrix of nibbles (row = lane that loaded it, column = lane whose 4 elements the nibble
 // belongs to), a three-stage butterfly over the lanes (xor 4: half-words, xor 2: bytes, xor 1:
 // nibbles) transposes it, so lane r ends with N = the 8 nibbles for its own 4 elements.  Two
 // delta swaps of the bit-index (4 <-> 1, 3 <-> 0) then turn N into R, whose byte k holds the 8
 // sign bits of element k; the data loaded by lane q lands at bit kLaneWorker(q), i.e. worker w
 // sits at bit w.
-constexpr int kMaxLutWorkers = 8;
+constexpr int kMaxLutWorkers = 16;      // workers the table path handles (two lane groups)
 constexpr int kLutWorkers = 6;        // workers covered by the table
 constexpr int kLutCopies = 32;        // one copy per lane
 
@@ -580,10 +581,11 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 constexpr int kServerStages = 2;
-// Dynamic shared memory of the server kernel: staging ring, then M scaled scales.
+// Dynamic shared memory of the server kernel: staging ring (per thread and stage U float4 of
+// ptilde and U words for each group of 8 workers), then M scaled scales.
 template <int U>
-__host__ __device__ constexpr size_t server_ring_bytes() {
-    return (size_t)kServerStages * U * kThreads * (sizeof(float4) + sizeof(unsigned));
+__host__ __device__ constexpr size_t server_ring_bytes(int groups) {
+    return (size_t)kServerStages * U * kThreads * (sizeof(float4) + groups * sizeof(unsigned));
 }
 
 // Table path: one CTA walks the chunks of its tile.  Full chunks are staged through a ring of
@@ -597,12 +599,17 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q = lane & 7;
     const int o0 = warp * (128 * U) + lane * 4;
-    const int wq = kLaneWorker(q);                 // the worker whose words this lane loads
-    const bool has_w = wq < MT;
+    constexpr int G = (MT + 7) / 8;                // groups of 8 workers (lane q loads one of each)
+    const int wq = kLaneWorker(q);                 // the worker (of every group) this lane loads
     const Butterfly bf(q);
     float* const pbase = a.pb + t.start + o0;
-    const uint32_t* const wbase =
-        a.wwords + (long long)(has_w ? wq : 0) * a.wstride + t.word + (o0 >> 5);
+    bool has_w[G];
+    const uint32_t* wbase[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        has_w[g] = wq + 8 * g < MT;
+        wbase[g] = a.wwords + (long long)(has_w[g] ? wq + 8 * g : 0) * a.wstride + t.word + (o0 >> 5);
+    }
     const int nfull = t.len / kChunk;              // chunks staged through shared memory
     const int tail = t.len - nfull * kChunk;       // ragged rest (only at the end of a block)
     const char* lut = reinterpret_cast<const char*>(s_lut + lane);   // this lane's copy
@@ -619,24 +626,30 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
         if (c < nfull) {
             const int s = c % kServerStages;
             const float* pp = pbase + (long long)c * kChunk;
-            const uint32_t* wp = wbase + c * (kChunk / 32);
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 cp_async16(ring_p + (s * U + u) * kThreads, pp + u * 128);
-                if (has_w) cp_async4(ring_w + (s * U + u) * kThreads, wp + u * 4);
+#pragma unroll
+                for (int g = 0; g < G; ++g)
+                    if (has_w[g])
+                        cp_async4(ring_w + ((s * U + u) * G + g) * kThreads,
+                                  wbase[g] + c * (kChunk / 32) + u * 4);
             }
         }
         cp_async_commit();                 // one (possibly empty) group per chunk index
     };
     // full_c: std::true_type for a whole chunk (no bounds checks), std::false_type for the tail
-    auto compute_chunk = [&](auto full_c, int c, int clen, float (&p)[U][4], unsigned (&w)[U]) {
+    auto compute_chunk = [&](auto full_c, int c, int clen, float (&p)[U][4], unsigned (&w)[U][G]) {
         constexpr bool full = decltype(full_c)::value;
         float* pp = pbase + (long long)c * kChunk;
         uint32_t* words = a.words + t.word + c * (kChunk / 32);
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int o = o0 + u * 128;
-            const unsigned R = bf.indices(w[u]);
+            unsigned Rg[G];                 // Rg[g]: bit 8k + i = sign of worker 8g + i, element k
+#pragma unroll
+            for (int g = 0; g < G; ++g) Rg[g] = bf.indices(w[u][g]);
+            const unsigned R = Rg[0];
             // byte offset of entry (R_k & (entries-1)) in this lane's copy: 128 * index
             constexpr unsigned kIdxMask = (unsigned)(kLutEntries(MT) - 1) << 7;
             float avg[4];
@@ -649,7 +662,8 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
                     avg[k] = __fadd_rn(avg[k], __uint_as_float(
-                        cdir[wk - kLutWorkers] ^ ((R << (31 - wk - 8 * k)) & 0x80000000u)));
+                        cdir[wk - kLutWorkers] ^
+                        ((Rg[wk / 8] << (31 - (wk % 8) - 8 * k)) & 0x80000000u)));
             }
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -666,7 +680,7 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
     };
 
     float p[U][4];
-    unsigned w[U];
+    unsigned w[U][G];
 #pragma unroll
     for (int c = 0; c < kServerStages - 1; ++c) issue_chunk(c);   // in flight while the table is built
     build_scaled(a, t.block, MT, s_c);
@@ -682,18 +696,22 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
         for (int u = 0; u < U; ++u) {
             const float4 v = ring_p[(s * U + u) * kThreads];
             p[u][0] = v.x; p[u][1] = v.y; p[u][2] = v.z; p[u][3] = v.w;
-            w[u] = has_w ? ring_w[(s * U + u) * kThreads] : 0u;
+#pragma unroll
+            for (int g = 0; g < G; ++g)
+                w[u][g] = has_w[g] ? ring_w[((s * U + u) * G + g) * kThreads] : 0u;
         }
         compute_chunk(std::true_type{}, c, kChunk, p, w);
     }
     if (tail > 0) {
         const float* pp = pbase + (long long)nfull * kChunk;
-        const uint32_t* wp = wbase + nfull * (kChunk / 32);
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int o = o0 + u * 128;
             load4(pp + u * 128, o, tail, false, p[u]);
-            w[u] = (has_w && (o & ~31) < tail) ? __ldg(wp + u * 4) : 0u;
+#pragma unroll
+            for (int g = 0; g < G; ++g)
+                w[u][g] = (has_w[g] && (o & ~31) < tail)
+                              ? __ldg(wbase[g] + nfull * (kChunk / 32) + u * 4) : 0u;
         }
         compute_chunk(std::false_type{}, nfull, tail, p, w);
     }
@@ -777,12 +795,12 @@ __device__ __forceinline__ double server_rows_scalar(const ServerArgs& a, const 
     return acc;
 }
 
-// One tile per CTA.  MT = number of workers when 1 <= M <= 8 (table path), 0 for any other M.
+// One tile per CTA.  MT = number of workers when 1 <= M <= 16 (table path), 0 for any other M.
 template <int U, int MT>
 __global__ void __launch_bounds__(kThreads) ef_server_kernel(const ServerArgs a) {
     // dynamic shared memory: [staging ring (table path only)] [M scaled worker scales]
     extern __shared__ __align__(16) unsigned char s_dyn[];
-    float* s_c = reinterpret_cast<float*>(s_dyn + (MT > 0 ? server_ring_bytes<U>() : 0));
+    float* s_c = reinterpret_cast<float*>(s_dyn + (MT > 0 ? server_ring_bytes<U>((MT + 7) / 8) : 0));
     __shared__ float s_base[MT > 0 ? kLutEntries(MT) : 1];
     __shared__ float s_lut[MT > 0 ? kLutEntries(MT) * kLutCopies : 1];
     const Tile t = a.tiles[blockIdx.x];

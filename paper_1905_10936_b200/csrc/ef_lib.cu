@@ -194,7 +194,7 @@ int launch_worker(ef_ctx* c, int i, const float* grad, int count = 1, long long 
 
 template <int MT>
 size_t server_smem_bytes(int M) {
-    return (MT > 0 ? efk::server_ring_bytes<kU>() : 0) + (size_t)M * sizeof(float);
+    return (MT > 0 ? efk::server_ring_bytes<kU>((MT + 7) / 8) : 0) + (size_t)M * sizeof(float);
 }
 
 // Raises the dynamic shared-memory limit of the server kernel this context will use.  Done once
@@ -217,6 +217,14 @@ cudaError_t prepare_server(int M) {
         case 6: return prepare_server_t<6>(M);
         case 7: return prepare_server_t<7>(M);
         case 8: return prepare_server_t<8>(M);
+        case 9: return prepare_server_t<9>(M);
+        case 10: return prepare_server_t<10>(M);
+        case 11: return prepare_server_t<11>(M);
+        case 12: return prepare_server_t<12>(M);
+        case 13: return prepare_server_t<13>(M);
+        case 14: return prepare_server_t<14>(M);
+        case 15: return prepare_server_t<15>(M);
+        case 16: return prepare_server_t<16>(M);
         default: return prepare_server_t<0>(M);
     }
 }
@@ -247,6 +255,14 @@ int launch_server(ef_ctx* c) {
         case 6: le = launch_server_t<6>(c, a); break;
         case 7: le = launch_server_t<7>(c, a); break;
         case 8: le = launch_server_t<8>(c, a); break;
+        case 9: le = launch_server_t<9>(c, a); break;
+        case 10: le = launch_server_t<10>(c, a); break;
+        case 11: le = launch_server_t<11>(c, a); break;
+        case 12: le = launch_server_t<12>(c, a); break;
+        case 13: le = launch_server_t<13>(c, a); break;
+        case 14: le = launch_server_t<14>(c, a); break;
+        case 15: le = launch_server_t<15>(c, a); break;
+        case 16: le = launch_server_t<16>(c, a); break;
         default: le = launch_server_t<0>(c, a); break;
     }
     EF_CUDA(c, le);

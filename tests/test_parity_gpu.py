@@ -28,7 +28,9 @@ def _wl(name, sizes, M, mu=0.9, eta=0.1, steps=5, law="normal", scale_range=None
     ([TILE], 2), ([TILE - 1], 2), ([TILE + 1], 2), ([TILE - 4, 8, TILE + 4], 7),
     ([2 * TILE, TILE // 2, 3 * TILE + 36, 100], 8),  # several tiles per block + ragged tails
     ([5 * TILE + 2, 3, 2 * TILE + 1, 4 * TILE], 2),  # multi-tile blocks on the scalar path
-    ([1000] * 40, 16), ([12345, 54321, 99999], 9),   # generic-M server path
+    ([1000] * 40, 16), ([12345, 54321, 99999], 9),   # two lane groups in the server table path
+    ([TILE + 3, BIG + 40, 777], 15), ([BIG + TILE + 8, 100], 13),
+    ([BIG + 5, 300, 2 * TILE], 17), ([640, TILE], 33),  # direct-sum server path (M > 16)
     ([BIG], 7), ([BIG + 1, BIG - 1], 4), ([BIG - 4, 3 * BIG + TILE + 4, 2 * BIG + 2 * TILE], 7),
     ([2 * TILE + 8, BIG + 3 * TILE, 5 * BIG + 100], 3),
 ])
