@@ -315,6 +315,9 @@ def test_denormal_range_gradients():
 def test_indexing_beyond_2_32_elements():
     """d > 2^32: one huge block followed by small ragged blocks whose flat indices need 33 bits;
     the oracle follows the small blocks (blocks are independent).  M = 1 keeps it at 86 GB."""
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     if free < 110 * 2 ** 30:
         pytest.skip("needs about 100 GB of free device memory")
