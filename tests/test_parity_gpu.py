@@ -333,6 +333,42 @@ def test_indexing_beyond_2_32_elements():
     assert int(eng.worker_words(0)[(huge // 32) - 8:(huge // 32)].ne(0).sum()) > 0
 
 
+@pytest.mark.parametrize("cid,steps", [(4, 3), (5, 2)])
+def test_error_corrected_iterate_identity_at_full_size(cid, steps):
+    """A property that holds at any size and needs no oracle (Lemma 3): after T iterations
+    x_T - eta (etilde_T + mean_i e_{T,i}) equals the iterate of uncompressed Nesterov SGDM on the
+    same gradients, here evaluated in fp64 with torch on the whole 2^28 / GPT-2-sized vector."""
+    w = wl.make_workload(cid)
+    eng = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    es = w.element_scales("cuda")
+    stride = (w.d + 3) // 4 * 4
+    gall = torch.zeros(w.M, stride, device="cuda")
+    mu, eta = float(np.float32(w.mu)), float(np.float32(w.eta))
+    m64 = torch.zeros(w.M, w.d, dtype=torch.float64, device="cuda")
+    ref = torch.zeros(w.d, dtype=torch.float64, device="cuda")
+    for t in range(steps):
+        for i in range(w.M):
+            w.draw_grad(t, i, "cuda", es, out=gall[i, :w.d])
+        eng.worker_step_all(gall)
+        eng.server_step()
+        g64 = gall[:, :w.d].double()
+        m64.mul_(mu).add_(g64)                               # m_i = mu m_i + g_i
+        ref.sub_((m64 * mu + g64).mean(dim=0), alpha=eta)    # x -= eta mean_i(mu m_i + g_i)
+        del g64
+    corrected = eng.params().double()
+    resid = eng.residual(-1).double()
+    for i in range(w.M):
+        resid.add_(eng.residual(i).double(), alpha=1.0 / w.M)
+    corrected.sub_(resid, alpha=eta)
+    off = torch.from_numpy(w.offsets).cuda()
+    err = (corrected - ref).abs()
+    # per block, relative to the block's largest reference magnitude
+    seg = torch.repeat_interleave(torch.arange(w.B, device="cuda"), off[1:] - off[:-1])
+    max_err = torch.zeros(w.B, dtype=torch.float64, device="cuda").scatter_reduce_(0, seg, err, "amax")
+    max_ref = torch.zeros(w.B, dtype=torch.float64, device="cuda").scatter_reduce_(0, seg, ref.abs(), "amax")
+    assert bool((max_err <= 2e-5 * max_ref).all()), float((max_err / max_ref).max())
+
+
 # ------------------------------------------------------------------ state access / checkpoint
 def test_checkpoint_roundtrip_is_bit_exact():
     """5 steps, export (x, m_i, e_i, etilde), import into a fresh context, 5 more steps:
