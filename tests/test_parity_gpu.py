@@ -369,6 +369,43 @@ def test_error_corrected_iterate_identity_at_full_size(cid, steps):
     assert bool((max_err <= 2e-5 * max_ref).all()), float((max_err / max_ref).max())
 
 
+def test_residual_norm_closed_form_at_full_size():
+    """Oracle-free at full size (GPT-2-sized layout): per block and worker the residual the
+    kernel keeps must satisfy ||e'_b||_2^2 = ||p_b||_2^2 - ||p_b||_1^2 / d_b (proof of Prop. 1)
+    with the sums the same launch recorded, scale_b = ||p_b||_1 / d_b, and the sign words must
+    have zero padding bits."""
+    w = wl.make_workload(5)
+    eng = EFEngine(w.offsets, w.M, w.mu, w.eta, diagnostics=True)
+    es = w.element_scales("cuda")
+    off = torch.from_numpy(w.offsets).cuda()
+    sizes = (off[1:] - off[:-1]).double()
+    seg = torch.repeat_interleave(torch.arange(w.B, device="cuda"), off[1:] - off[:-1])
+    for t in range(2):
+        for i in range(w.M):
+            eng.worker_step(i, w.draw_grad(t, i, "cuda", es))
+        eng.server_step()
+    for i in range(w.M):
+        dg = eng.worker_diagnostics(i)
+        e2 = torch.zeros(w.B, dtype=torch.float64, device="cuda").scatter_add_(
+            0, seg, eng.residual(i).double().square_())
+        expect = dg[:, 1] - dg[:, 0] ** 2 / sizes
+        assert bool(((e2 - expect).abs() <= 1e-5 * dg[:, 1]).all())
+        scale = eng.worker_scales(i).double()
+        assert bool(((scale - dg[:, 0] / sizes).abs() <= 1e-6 * scale).all())
+    # padding bits: the ResNet-50 layout has a 1000-element block (31 full words + 8 bits)
+    w3 = wl.make_workload(3)
+    e3 = EFEngine(w3.offsets, w3.M, w3.mu, w3.eta)
+    es3 = w3.element_scales("cuda")
+    for i in range(w3.M):
+        e3.worker_step(i, -w3.draw_grad(0, i, "cuda", es3).abs())     # all negative: all bits set
+    e3.server_step()
+    b = w3.sizes.index(1000)                                         # the 1000-element block
+    wbeg = sum((sz + 31) // 32 for sz in w3.sizes[:b])
+    last = int(e3.worker_words(0)[wbeg + 31].item()) & 0xFFFFFFFF
+    assert last == 0xFF and int(e3.server_words()[wbeg + 31].item()) & 0xFFFFFFFF == 0xFF
+    assert int(e3.worker_words(0)[wbeg + 30].item()) & 0xFFFFFFFF == 0xFFFFFFFF
+
+
 # ------------------------------------------------------------------ state access / checkpoint
 def test_checkpoint_roundtrip_is_bit_exact():
     """5 steps, export (x, m_i, e_i, etilde), import into a fresh context, 5 more steps:
