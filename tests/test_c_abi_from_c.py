@@ -7,6 +7,7 @@ import subprocess
 import pytest
 
 from paper_1905_10936_b200 import binding as ef
+from paper_1905_10936_b200 import build as efbuild
 from test_oracle_pins import parse_hand_case
 
 HERE = os.path.dirname(os.path.abspath(__file__))
@@ -15,6 +16,7 @@ SRC = os.path.join(HERE, "c_abi", "ef_c_driver.c")
 
 
 def _build(tmp_path):
+    efbuild.build_library()            # no-op when libef.so is up to date
     exe = str(tmp_path / "ef_c_driver")
     nvcc = os.path.join(os.environ.get("CUDA_HOME", "/usr/local/cuda"), "bin", "nvcc")
     libdir = os.path.dirname(ef.LIB_PATH)
