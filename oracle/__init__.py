@@ -60,6 +60,8 @@ def _load():
     for name in ("efo_momentum", "efo_residual", "efo_words", "efo_scales"):
         getattr(lib, name).restype = vp
         getattr(lib, name).argtypes = [vp, i32]
+    lib.efo_set_diagnostics.restype = None
+    lib.efo_set_diagnostics.argtypes = [vp, i32]
     lib.efo_diagnostics.restype = vp
     lib.efo_diagnostics.argtypes = [vp, i32]
     _lib = lib
@@ -76,7 +78,7 @@ class Oracle:
 
     ADOPT_CAP = 1 << 16
 
-    def __init__(self, offsets, M: int, mu: float, eta: float):
+    def __init__(self, offsets, M: int, mu: float, eta: float, diagnostics: bool = False):
         lib = _load()
         self._lib = lib
         self.offsets = np.ascontiguousarray(offsets, dtype=np.int64)
@@ -88,6 +90,8 @@ class Oracle:
         if not self._h:
             raise ValueError("efo_init rejected the arguments")
         self.W = int(lib.efo_num_words(self._h))
+        if diagnostics:
+            lib.efo_set_diagnostics(self._h, 1)
         self._adopt = np.zeros(self.ADOPT_CAP, dtype=np.int64)
 
     def close(self):
@@ -164,5 +168,6 @@ class Oracle:
         return _view(self._lib.efo_scales(self._h, i), self.B, np.float32)
 
     def diagnostics(self, i: int) -> np.ndarray:
-        """[B, 4] float64: ||p_b||_1, ||p_b||_2^2, ||g_b||_1, ||g_b||_2^2 of worker i's last call."""
+        """[B, 4] float64: ||p_b||_1, ||p_b||_2^2, ||g_b||_1, ||g_b||_2^2 of worker i's last call
+        (recorded only by an Oracle created with diagnostics=True)."""
         return _view(self._lib.efo_diagnostics(self._h, i), 4 * self.B, np.float64).reshape(self.B, 4)

@@ -24,8 +24,9 @@
 //   mtilde_t = mu mtilde_{t-1} + lambda x_t,   x_{t+1} = x_t - eta_t (Deltatilde_t + mu mtilde_t + lambda x_t),
 // done once here because all replicas of x are identical.
 //
-// Diagnostics (Section 3.2, Fig. 1): every worker call also records, per block, ||p_b||_1,
-// ||p_b||_2^2, ||g_b||_1 and ||g_b||_2^2 (binary64 sums), from which follow
+// Diagnostics (Section 3.2, Fig. 1), off by default and switched on by efo_set_diagnostics: a
+// worker call then also records, per block, ||p_b||_1, ||p_b||_2^2, ||g_b||_1 and ||g_b||_2^2
+// (binary64 sums; they are not part of Algorithm 4 and change none of its results), from which follow
 //   phi(p) = min_b ||p_b||_1^2 / (d_b ||p_b||_2^2)            (Prop. 1),
 //   delta of the non-block compressor = ||p||_1^2 / (d ||p||_2^2)   (Section 3.2),
 //   coefficient of variation of |g| in block b = sqrt(d_b ||g_b||_2^2 / ||g_b||_1^2 - 1).
@@ -95,6 +96,7 @@ struct Oracle {
     // Diagnostics of the last worker call of each worker (the quantities behind Fig. 1):
     // per block ||p_b||_1, ||p_b||_2^2, ||g_b||_1, ||g_b||_2^2, accumulated in binary64.
     std::vector<std::vector<double>> diag;   // [M][4*B]
+    bool want_diag = false;                  // record them (efo_set_diagnostics)
 };
 
 // Compress p[lo,hi) of block b (Section 3.2), write the block's scale and packed signs,
@@ -203,7 +205,7 @@ int64_t efo_worker_step(void* h, int32_t i, const float* grad, const uint32_t* h
             const float u = std::fmaf(mu, m[j], grad[j]);    // mu m_t + g_t
             p[j] = std::fmaf(r, e[j], u);                    // + (eta_{t-1}/eta_t) e_t
         }
-        {   // diagnostics: plain sums over the block, independent of the compression below
+        if (o->want_diag) {   // plain sums over the block, independent of the compression below
             double p1 = 0.0, p2 = 0.0, g1 = 0.0, g2 = 0.0;
             for (int64_t j = lo; j < hi; ++j) {
                 p1 += (double)std::fabs(p[j]);      p2 += (double)p[j] * (double)p[j];
@@ -280,6 +282,9 @@ int32_t efo_set_weight_decay(void* h, float lambda)
     if (lambda > 0.f && o->mt.empty()) o->mt.assign(o->d, 0.f);
     return 0;
 }
+
+// Diagnostic sums on/off (off after efo_init); they never change what Algorithm 4 computes.
+void efo_set_diagnostics(void* h, int32_t on) { static_cast<Oracle*>(h)->want_diag = on != 0; }
 
 double* efo_diagnostics(void* h, int32_t i) { return static_cast<Oracle*>(h)->diag[i].data(); }
 
