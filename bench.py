@@ -37,9 +37,13 @@ from paper_1905_10936_b200 import workloads as wl
 METRIC = "parameters/sec through one two-way compressed dist-EF-blockSGDM step (M workers)"
 UNIT = "params/s"
 
-# DRAM traffic per launch of the worker kernel measured by ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum), in bytes per parameter; see profiles/ for the capture it comes from.
-NCU_WORKER_TRAFFIC_BYTES_PER_PARAM = 20.10   # 37.766e9 bytes per 7-worker launch at d = 2^28
+# DRAM traffic of the worker kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum) on
+# the small case of the flat layout (its first 64 blocks: d = 2^26, M = 7, one launch of
+# ef_worker_step_all), in bytes per worker-parameter; traffic grows in proportion to d*M on this
+# layout (every CTA streams one 4096-element chunk), so a full launch is this figure x d x M.
+# The capture is summarised in profiles/; the figure is reported for that layout only.
+NCU_WORKER_TRAFFIC = {"workload": "C4-flat-2^28", "bytes_per_worker_param": 20.01,
+                      "captured_on": "first 64 blocks (d = 2^26), M = 7, scaled by d*M"}
 
 
 # --------------------------------------------------------------------------- byte counts
@@ -57,6 +61,16 @@ def server_call_bytes(d: int, B: int, M: int) -> float:
 
 def step_bytes(d: int, B: int, M: int) -> float:
     return M * worker_call_bytes(d, B) + server_call_bytes(d, B, M)
+
+
+def config_dict(w) -> dict:
+    """Names the workload; identical in both arms (descriptive extras go under "run")."""
+    gib = eng_state_gib(w)
+    return {"workload": w.name, "d": w.d, "B": w.B, "M": w.M, "mu": w.mu, "eta": w.eta,
+            "l2": f"no flush: state + one gradient batch = {gib:.2f} GiB per GPU vs 126 MB of L2"
+                  if gib * 2 ** 30 > 4 * 126e6 else
+                  f"no flush: state + one gradient batch = {gib * 1024:.0f} MiB per GPU fits the "
+                  "126 MB L2 (launch-latency-bound layout, reported as such)"}
 
 
 def measured_hbm_peak():
@@ -165,10 +179,13 @@ def run_reference(args) -> None:
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": s_per_step * 1e3,
+        # time one step of the WHOLE workload takes at the sampled rate (blocks are independent,
+        # the oracle's cost is linear in the number of parameters); the sample's own step time
+        # is given beside it
+        "ms_per_step": w.d / value * 1e3, "ms_per_sample_step": s_per_step * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
-        "config": {"workload": w.name, "d": w.d, "B": w.B, "M": w.M, "mu": w.mu, "eta": w.eta},
+        "config": config_dict(w),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -197,7 +214,25 @@ def run_ours(args) -> None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    w = load_workload(args)
+    def max_over_ranks(ms: float) -> float:
+        if world == 1:
+            return ms
+        tt = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        return float(tt.item())
+
+    w_full = load_workload(args)
+    if args.scaling == "strong" and world > 1:
+        # ONE layout cut into block ranges: this rank builds and steps only its own blocks
+        # (every operation of the method is per element or per block: no data-path collective)
+        b0, b1 = wl.shard_blocks(w_full.sizes, world, rank)
+        w = wl.custom_workload(f"{w_full.name}[blocks {b0}:{b1}]", w_full.sizes[b0:b1] or [4],
+                               w_full.M, w_full.mu, w_full.eta, w_full.steps, w_full.law,
+                               w_full.scale_range, config_id=1000 * w_full.config_id + rank)
+        job_params = w_full.d                       # total work is fixed as N grows
+    else:
+        w = w_full                                  # every rank owns one whole layout
+        job_params = world * w_full.d
     K, W = args.steps, args.warmup
     # all work of the context runs on this (non-default) stream, which is also made current
     stream = torch.cuda.Stream(device=dev)
@@ -208,27 +243,39 @@ def run_ours(args) -> None:
         eng.set_weight_decay(args.weight_decay)
     es = w.element_scales(dev)
     stride = (w.d + 3) // 4 * 4
-    gall = torch.zeros(w.M, stride, dtype=torch.float32, device=dev)   # pre-staged in HBM
-    grads = [w.draw_grad(0, i, dev, es, out=gall[i, :w.d]) for i in range(w.M)]
+    # Gradient batches pre-staged in HBM and rotated step by step (fresh values every step as
+    # far as memory allows: up to 3 batches within a quarter of the device memory)
+    free_b, total_b = torch.cuda.mem_get_info(dev)
+    batch_bytes = w.M * stride * 4
+    nbatch = int(max(1, min(3, args.grad_batches or 3, (total_b // 4) // max(batch_bytes, 1))))
+    galls = []
+    for bidx in range(nbatch):
+        ga = torch.zeros(w.M, stride, dtype=torch.float32, device=dev)
+        for i in range(w.M):
+            w.draw_grad(bidx, i, dev, es, out=ga[i, :w.d])
+        galls.append(ga)
     del es
     batched = not args.per_worker_calls
+    step_no = [0]
 
     def worker_calls():
+        ga = galls[step_no[0] % nbatch]
         if batched:
-            eng.worker_step_all(gall)          # all M workers in one launch
+            eng.worker_step_all(ga)            # all M workers in one launch
         else:
             for i in range(w.M):
-                eng.worker_step(i, grads[i])
+                eng.worker_step(i, ga[i, :w.d])
 
     def one_step():
         worker_calls()
         eng.server_step()
+        step_no[0] += 1
 
     for _ in range(W):
         one_step()
     barrier()
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(local_rank, period_s=0.002)
     launches0 = eng.launch_count
     sampler.start()
     barrier()
@@ -238,6 +285,7 @@ def run_ours(args) -> None:
         ev[k][1].record()
         eng.server_step()
         ev[k][2].record()
+        step_no[0] += 1
     barrier()
     clocks = sampler.stop()
     launches = eng.launch_count - launches0
@@ -245,10 +293,30 @@ def run_ours(args) -> None:
     launches_per_step_worker = 1 if batched else w.M
     worker_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / (K * launches_per_step_worker)
     server_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / K
-    if world > 1:
-        tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = max_over_ranks(total_ms)
+    if clocks.get("sm_mhz"):
+        clocks["ms_per_step_x_sm_mhz"] = total_ms / K * clocks["sm_mhz"]
+
+    # ---- sustained: many back-to-back steps (the board reaches its power limit after ~1 s)
+    sustained = None
+    if args.sustained_steps > 0:
+        Ks = args.sustained_steps
+        s_sampler = ClockSampler(local_rank, period_s=0.01)
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        s_sampler.start()
+        s0.record()
+        for _ in range(Ks):
+            one_step()
+        s1.record()
+        barrier()
+        s_clk = s_sampler.stop()
+        s_ms = max_over_ranks(s0.elapsed_time(s1))
+        sustained = {"steps": Ks, "ms_per_step": s_ms / Ks, "value": job_params * Ks / (s_ms * 1e-3),
+                     "unit": UNIT, "seconds": s_ms * 1e-3, "sm_mhz": s_clk.get("sm_mhz"),
+                     "sm_max_mhz": s_clk.get("sm_max_mhz"), "reasons": s_clk.get("reasons"),
+                     "clock_samples": s_clk.get("samples"),
+                     "step_gbs": step_bytes(w.d, w.B, w.M) / (s_ms / Ks * 1e-3) / 1e9}
 
     # ---- the same step replayed from a CUDA graph (launch gaps shrink; matters for small layouts)
     graph_info = None
@@ -265,25 +333,27 @@ def run_ours(args) -> None:
             g.replay()
         g1.record()
         barrier()
-        g_ms = g0.elapsed_time(g1)
-        if world > 1:
-            tt = torch.tensor([g_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            g_ms = float(tt.item())
-        graph_info = {"ms_per_step": g_ms / K, "value": world * w.d * K / (g_ms * 1e-3),
+        g_ms = max_over_ranks(g0.elapsed_time(g1))
+        graph_info = {"ms_per_step": g_ms / K, "value": job_params * K / (g_ms * 1e-3),
                       "unit": UNIT, "note": "one whole step captured once, replayed K times"}
         del g
+
+    # ---- ceiling of a no-compute kernel with the worker step's access mix (3 reads, 2 writes)
+    ceiling = None
+    if args.ceiling:
+        ceiling = stream_ceilings(eng, galls[0], w, stream)
 
     # ---- end to end: host gradients in, packed update out, copies inside the timed region
     e2e = None
     if not args.no_e2e:
+        hsrc = galls[0]
         del eng
         torch.cuda.empty_cache()
         eng2 = EFEngine(w.offsets, w.M, w.mu, w.eta, host_staging=True, stream=stream)
         hgrads = []
         for i in range(w.M):
             h = torch.empty(w.d, dtype=torch.float32).pin_memory()
-            h.copy_(grads[i])
+            h.copy_(hsrc[i, :w.d])
             hgrads.append(h)
         hwords = torch.empty(eng2.W, dtype=torch.int32).pin_memory()
         hscales = torch.empty(eng2.B, dtype=torch.float32).pin_memory()
@@ -306,17 +376,13 @@ def run_ours(args) -> None:
         s1.record()
         barrier()
         wall_ms = (time.perf_counter() - t0) * 1e3
-        e2e_ms = max(s0.elapsed_time(s1), 0.0)
-        if world > 1:
-            tt = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e2e_ms = float(tt.item())
-        e2e = {"value": world * w.d * Ke / (e2e_ms * 1e-3), "unit": UNIT,
+        e2e_ms = max_over_ranks(max(s0.elapsed_time(s1), 0.0))
+        e2e = {"value": job_params * Ke / (e2e_ms * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": int(w.M * w.d * 4),
                "d2h_bytes_per_step": int(eng2.W * 4 + eng2.B * 4),
                "steps": Ke, "ms_per_step": e2e_ms / Ke, "wall_ms_per_step": wall_ms / Ke,
                "note": "pinned host gradients -> ef_worker_step_host (double-buffered H2D on a "
-                       "copy stream) -> ef_server_step -> ef_read_update_host"}
+                       "copy stream) -> ef_server_step -> ef_read_update_host; PCIe-bound"}
         del eng2, hgrads
 
     if rank != 0:
@@ -329,20 +395,24 @@ def run_ours(args) -> None:
     sbytes = server_call_bytes(w.d, w.B, w.M) + (8.0 * w.d if args.weight_decay > 0 else 0.0)
     w_gbs = wbytes / (worker_ms * 1e-3) / 1e9
     s_gbs = sbytes / (server_ms * 1e-3) / 1e9
-    state_gib = eng_state_gib(w)
+    plain = (args.weight_decay == 0 and not args.diagnostics and world == 1)
+    traffic = None
+    if plain and w.name == NCU_WORKER_TRAFFIC["workload"]:
+        traffic = NCU_WORKER_TRAFFIC["bytes_per_worker_param"] * w.d * (w.M if batched else 1)
     line = {
-        "metric": METRIC, "value": world * w.d * K / (total_ms * 1e-3), "unit": UNIT,
+        "metric": METRIC, "value": job_params * K / (total_ms * 1e-3), "unit": UNIT,
         "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": total_ms / K,
         "steps_per_sec": K / (total_ms * 1e-3),
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-        "data": "synthetic",
-        "config": {"workload": w.name, "d": w.d, "B": w.B, "M": w.M, "mu": w.mu, "eta": w.eta,
-                   "weight_decay": args.weight_decay, "diagnostics": bool(args.diagnostics),
-                   "worker_calls": "ef_worker_step_all" if batched else "ef_worker_step x M",
-                   "per_gpu": "each rank owns one such layout (block-range shard of an "
-                              "N-times larger problem)",
-                   "l2": f"no flush: state+gradients {state_gib:.1f} GiB per GPU, far larger "
-                         "than the 126 MB L2"},
+        "higher_is_better": True, "scaling": args.scaling if world > 1 else "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": config_dict(w_full),
+        "run": {"weight_decay": args.weight_decay, "diagnostics": bool(args.diagnostics),
+                "worker_calls": "ef_worker_step_all" if batched else "ef_worker_step x M",
+                "gradient_batches_rotated": nbatch,
+                "per_gpu": ("every rank owns one whole layout (a block-range shard of an N-times "
+                            "larger problem); no data-path collective" if args.scaling == "weak" or world == 1
+                            else f"one layout cut into {world} block ranges (workloads.shard_blocks); "
+                                 "each rank builds and steps only its own blocks; no data-path collective")},
         "clocks": clocks,
         "e2e": e2e,
         "gpu_launches": int(launches * world),
@@ -350,22 +420,30 @@ def run_ours(args) -> None:
             "kernel": "ef_worker_kernel", "call": ("ef_worker_step_all: M workers per launch" if batched
                                                    else "ef_worker_step: one worker per launch"),
             "bound": "hbm", "achieved": w_gbs, "peak": peak,
-            "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": w_gbs / peak,
+            "peak_kind": f"of {peak_kind} (a 1:1 copy; context for a kernel that reads 60% of its bytes)",
+            "unit": "GB/s", "frac": w_gbs / peak,
             "frac_of_8000_nominal": w_gbs / 8000.0,
             "bytes_per_launch": wbytes, "ms_per_launch": worker_ms,
-            "traffic": (NCU_WORKER_TRAFFIC_BYTES_PER_PARAM * w.d * (w.M if batched else 1)
-                        if NCU_WORKER_TRAFFIC_BYTES_PER_PARAM else None),
+            "traffic": traffic,
+            "traffic_source": NCU_WORKER_TRAFFIC["captured_on"] if traffic else None,
         },
         "roofline_server": {
-            "kernel": "ef_server_kernel + ef_apply_kernel", "bound": "hbm", "achieved": s_gbs,
+            "kernel": "ef_server_kernel (+ ef_apply_kernel where the update is not fused)",
+            "bound": "hbm", "achieved": s_gbs,
             "peak": peak, "unit": "GB/s", "frac": s_gbs / peak,
             "frac_of_8000_nominal": s_gbs / 8000.0, "bytes_per_call": sbytes,
             "ms_per_call": server_ms,
         },
         "step_gbs": step_bytes(w.d, w.B, w.M) / (total_ms / K * 1e-3) / 1e9,
     }
+    if sustained is not None:
+        line["sustained"] = sustained
     if graph_info is not None:
         line["cuda_graph"] = graph_info
+    if ceiling is not None:
+        line["stream_ceiling"] = ceiling
+        line["roofline"]["frac_of_stream_ceiling"] = w_gbs / ceiling["3r2w_gbs"]
+        line["roofline_server"]["frac_of_stream_ceiling"] = s_gbs / ceiling["1r1w_gbs"]
     if world == 1 and not args.no_cpu_baseline:
         per_block = np.mean(w.sizes) * oracle_ns_per_param(w.M) * 1e-9
         steps_c = 2
@@ -379,6 +457,32 @@ def run_ours(args) -> None:
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def stream_ceilings(eng, gall: torch.Tensor, w: wl.Workload, stream) -> dict:
+    """Rates of the library's no-compute stream kernels (ef_stream_probe) on buffers of this
+    workload's size: the ceiling a kernel with the same read/write mix can reach."""
+    from paper_1905_10936_b200 import binding as ef
+    n = (w.d // 4096) * 4096
+    a = gall[0, :n]
+    b = torch.empty(n, dtype=torch.float32, device=gall.device)
+    c = torch.empty(n, dtype=torch.float32, device=gall.device)
+    out = {}
+    for mode, key, bytes_per_elem in ((ef.EF_PROBE_3R2W, "3r2w_gbs", 20.0),
+                                      (ef.EF_PROBE_1R1W, "1r1w_gbs", 8.0)):
+        reps = max(3, min(50, int(2e10 / (bytes_per_elem * n))))
+        for _ in range(3):
+            ef.ef_stream_probe(mode, a.data_ptr(), b.data_ptr(), c.data_ptr(), n, stream.cuda_stream)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            ef.ef_stream_probe(mode, a.data_ptr(), b.data_ptr(), c.data_ptr(), n, stream.cuda_stream)
+        e1.record()
+        torch.cuda.synchronize()
+        out[key] = bytes_per_elem * n * reps / (e0.elapsed_time(e1) * 1e-3) / 1e9
+    out["note"] = (f"no-compute float4 stream kernels on {n} elements per buffer, one 4096-element "
+                   "chunk per CTA: 3 reads + 2 writes (the worker step's mix) and 1 read + 1 write")
+    return out
 
 
 def eng_state_gib(w: wl.Workload) -> float:
@@ -418,6 +522,16 @@ def main():
     ap.add_argument("--graph", action="store_true",
                     help="also time the step replayed from a CUDA graph (extra key cuda_graph)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sustained-steps", type=int, default=300,
+                    help="extra back-to-back steps timed as one region with the clocks sampled "
+                         "(key `sustained`; 0 = skip)")
+    ap.add_argument("--scaling", choices=["weak", "strong"], default="weak",
+                    help="N > 1: weak = every rank owns one whole layout; strong = one layout cut "
+                         "into block ranges, each rank builds only its own")
+    ap.add_argument("--grad-batches", type=int, default=0,
+                    help="gradient batches kept in HBM and rotated (default: up to 3)")
+    ap.add_argument("--ceiling", action="store_true",
+                    help="also time the library's no-compute stream kernels (key `stream_ceiling`)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -53,7 +53,8 @@ enum ef_status {
     EF_ERR_CUDA = 5,               /* a CUDA runtime call failed; see ef_last_cuda_error */
     EF_ERR_UNSUPPORTED_DEVICE = 6, /* current device is not compute capability 10.x */
     EF_ERR_TIMEOUT = 7,            /* reserved: a bounded device-side wait gave up */
-    EF_ERR_TOO_LARGE = 8           /* ef_worker_step_noalloc: n exceeds EF_NOALLOC_MAX_ELEMS */
+    EF_ERR_TOO_LARGE = 8,          /* ef_worker_step_noalloc: n exceeds EF_NOALLOC_MAX_ELEMS */
+    EF_ERR_NO_MEMORY = 9           /* a host allocation failed (the library allocates no device memory) */
 };
 
 /* Flags for ef_workspace_bytes / ef_init. */
@@ -80,12 +81,13 @@ int ef_workspace_bytes(int64_t d, int32_t B, const int64_t* offsets /* host, B+1
 
 /* Creates a context and initialises the state of Algorithm 4 in the workspace:
  * x_0 = 0, m_{-1,i} = 0, e_{0,i} = 0, etilde_0 = 0, t = 0 (Algorithm 4, "Initialize").
- * mu in [0, 1) is the momentum parameter, eta > 0 the (constant) stepsize, so the factor
- * eta_{t-1}/eta_t of Algorithm 4 is 1 (at t = 0 it multiplies a zero residual).
+ * mu in [0, 1) is the momentum parameter, eta > 0 the stepsize eta_0.  The stepsize stays at
+ * this value until ef_set_eta changes it; while it is constant the factor eta_{t-1}/eta_t of
+ * Algorithm 4 is exactly 1 (at t = 0 it multiplies a zero residual).
  * workspace: device, 256-byte aligned, at least ef_workspace_bytes; borrowed until ef_destroy.
  * cuda_stream: a cudaStream_t (0 = default stream) on which all work of this context runs.
- * Errors: INVALID_ARG, WORKSPACE, ALIGNMENT, UNSUPPORTED_DEVICE, CUDA.  On error *out = NULL
- * and nothing was launched. */
+ * Errors: INVALID_ARG, WORKSPACE, ALIGNMENT, UNSUPPORTED_DEVICE, NO_MEMORY (host), CUDA.  On
+ * error *out = NULL and nothing was launched. */
 int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets /* host, B+1 */,
             int32_t M, float mu, float eta, uint32_t flags,
             void* workspace /* device */, size_t workspace_bytes, void* cuda_stream);
@@ -172,7 +174,12 @@ int64_t         ef_num_words(ef_ctx* ctx);/* W = sum_b ceil(d_b / 32) */
  * The residual is stored internally in a deferred form (the corrected vector p_t plus the
  * block scale); ef_get_residual writes the residual e_{t+1} = p_t - Delta_t itself.
  * ef_set_state overwrites momentum (ignored for the server, may be NULL there) and residual.
- * Errors: INVALID_ARG, ALIGNMENT, BAD_STATE (called in the middle of an iteration), CUDA. */
+ * The two getters may be called at any time, also in the middle of an iteration: they are
+ * ordered on the context's stream and return worker i's state after its last enqueued step
+ * (m_{t,i} and e_{t+1,i} once worker i has been stepped in iteration t).  ef_set_state is only
+ * allowed between iterations.
+ * Errors: INVALID_ARG, ALIGNMENT, CUDA; ef_set_state also BAD_STATE (called in the middle of an
+ * iteration). */
 int ef_get_momentum(ef_ctx* ctx, int32_t i, float* dst);
 int ef_get_residual(ef_ctx* ctx, int32_t i, float* dst);
 int ef_set_state(ef_ctx* ctx, int32_t i, const float* momentum, const float* residual);
@@ -180,6 +187,20 @@ int ef_step_count(ef_ctx* ctx, int64_t* t /* out: completed iterations */);
 
 /* Number of kernels this context has launched so far (for launch accounting). */
 int64_t ef_launch_count(ef_ctx* ctx);
+
+/* Measurement aid (the paper has no counterpart): no-compute stream kernels with the access mix
+ * of the step kernels, one 4096-element chunk per CTA and 128-bit accesses like them, so that a
+ * measured rate can be set against the ceiling of a kernel of the same shape.
+ *   EF_PROBE_3R2W  reads a, b, c and rewrites b, c in place (the worker step: g, m, e -> m, e)
+ *   EF_PROBE_1R1W  reads and rewrites b in place (the server and update passes)
+ *   EF_PROBE_COPY  c <- a
+ * a, b, c: device, n floats each, 16-byte aligned, distinct buffers; n a positive multiple of
+ * 4096.  b and c are overwritten.  Enqueued on cuda_stream, no synchronisation.
+ * Errors: INVALID_ARG, ALIGNMENT, CUDA. */
+#define EF_PROBE_3R2W 0
+#define EF_PROBE_1R1W 1
+#define EF_PROBE_COPY 2
+int ef_stream_probe(int32_t mode, const float* a, float* b, float* c, int64_t n, void* cuda_stream);
 
 /* (The paper has no counterpart for this entry point; it exists for deployment reasons.)
  * The worker step of one block for callers that must not allocate device memory where they

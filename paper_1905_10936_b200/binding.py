@@ -25,6 +25,7 @@ EF_ERR_CUDA = 5
 EF_ERR_UNSUPPORTED_DEVICE = 6
 EF_ERR_TIMEOUT = 7
 EF_ERR_TOO_LARGE = 8
+EF_ERR_NO_MEMORY = 9
 EF_NOALLOC_MAX_ELEMS = 1 << 24
 EF_FLAG_HOST_STAGING = 1
 EF_FLAG_FUSED_SCALE = 2
@@ -32,6 +33,7 @@ EF_FLAG_SPLIT_SCALE = 4
 EF_FLAG_WEIGHT_DECAY = 8
 EF_FLAG_DIAGNOSTICS = 16
 EF_MAX_WORKERS = 4096
+EF_PROBE_3R2W, EF_PROBE_1R1W, EF_PROBE_COPY = 0, 1, 2
 
 _vp, _i64, _i32, _u32, _f32 = (ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_uint32,
                                ctypes.c_float)
@@ -62,6 +64,7 @@ SIGNATURES = {
     "ef_step_count": (ctypes.c_int, [_vp, ctypes.POINTER(_i64)]),
     "ef_launch_count": (_i64, [_vp]),
     "ef_worker_step_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _f32, _vp, _vp, _vp]),
+    "ef_stream_probe": (ctypes.c_int, [_i32, _vp, _vp, _vp, _i64, _vp]),
     "ef_strerror": (ctypes.c_char_p, [ctypes.c_int]),
     "ef_last_cuda_error": (ctypes.c_int, [_vp]),
     "ef_destroy": (ctypes.c_int, [_vp]),
@@ -210,6 +213,11 @@ def ef_worker_step_noalloc(grad_ptr: int, momentum_ptr: int, residual_ptr: int,
     _check(load_library().ef_worker_step_noalloc(grad_ptr, momentum_ptr, residual_ptr,
                                                  residual_scale_ptr, n, mu, words_ptr, scale_ptr,
                                                  cuda_stream), "ef_worker_step_noalloc")
+
+
+def ef_stream_probe(mode: int, a_ptr: int, b_ptr: int, c_ptr: int, n: int, cuda_stream: int) -> None:
+    """No-compute stream kernel (measurement aid); see include/ef.h."""
+    _check(load_library().ef_stream_probe(mode, a_ptr, b_ptr, c_ptr, n, cuda_stream), "ef_stream_probe")
 
 
 def ef_last_cuda_error(ctx: int) -> int:

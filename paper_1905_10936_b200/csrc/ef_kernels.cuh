@@ -141,9 +141,14 @@ __device__ __forceinline__ void st_stream(float* p, float4 v) {
 
 // Sign convention: sign(+-0) = +1 (Appendix A maps signs to {-1,+1}), i.e. "negative" means
 // p < 0.  The kernels test the IEEE sign bit instead, which is the same predicate for every
-// value except -0.0, and -0.0 never occurs in a residual buffer: the scale s is >= +0, so
-// e = p - s*sign(p) is never -0 (x - x = +0 in round-to-nearest), hence p = u + e is never -0,
-// the buffers start at +0 and ef_set_state adds +0 to what it imports.  (NaN is unspecified.)
+// value except -0.0, so -0.0 must never be stored in a residual buffer:
+//  * constant stepsize (ratio == 1): the scale s is >= +0, so e = p - s*sign(p) is never -0
+//    (x - x = +0 in round-to-nearest); p = fl(v + e) with e != -0 is -0 only if the exact sum is
+//    zero, which rounds to +0 (a sum of two binary32 numbers never underflows);
+//  * rescaled residual (ratio != 1): p = fma(ratio, e, v) CAN underflow to -0 (e.g. ratio = 1/2,
+//    e = -2^-149, v = +0), so those paths add +0 afterwards (corrected_vector below), which maps
+//    -0 to +0 and changes nothing else;
+//  * the buffers start at +0 and ef_set_state adds +0 to what it imports.  (NaN is unspecified.)
 //
 // e_{t+1,j} = p_{t,j} - s * sign(p_{t,j})   (Algorithm 4): one rounding, as p + s or p - s.
 // It enters the next corrected vector as fma(eta_{t-1}/eta_t, e, .), which is fl(. + e) for a
@@ -151,6 +156,13 @@ __device__ __forceinline__ void st_stream(float* p, float4 v) {
 __device__ __forceinline__ float residual_of(float pb, float s) {
     const float signed_s = __uint_as_float((__float_as_uint(pb) & 0x80000000u) | __float_as_uint(s));
     return __fsub_rn(pb, signed_s);
+}
+
+// p = v + (eta_{t-1}/eta_t) e (Algorithm 4), never -0 (see above).  `rescale` is ratio != 1,
+// uniform over the launch.
+__device__ __forceinline__ float corrected_vector(float ratio, bool rescale, float e, float v) {
+    const float p = __fmaf_rn(ratio, e, v);
+    return rescale ? __fadd_rn(p, 0.0f) : p;
 }
 
 // Sign bits of four values as a nibble, element k in bit k.
@@ -374,6 +386,7 @@ __device__ __forceinline__ double worker_rows(const WorkerArgs& a, const Tile& t
         load4(pp + u * 128, o0 + u * 128, t.len, FULL, p[u]);
     }
     double acc = 0.0;
+    const bool rescale = a.ratio != 1.0f;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         const int o = o0 + u * 128;
@@ -382,7 +395,7 @@ __device__ __forceinline__ double worker_rows(const WorkerArgs& a, const Tile& t
             const float e = residual_of(p[u][k], sp);                // e_{t,i}
             m[u][k] = __fmaf_rn(a.mu, m[u][k], g[u][k]);             // m_t = mu m_{t-1} + g
             const float v = __fmaf_rn(a.mu, m[u][k], g[u][k]);       // mu m_t + g
-            float pv = __fmaf_rn(a.ratio, e, v);                     // p_t = v + (eta_{t-1}/eta_t) e
+            float pv = corrected_vector(a.ratio, rescale, e, v);     // p_t = v + (eta_{t-1}/eta_t) e
             if (!FULL && o + k >= t.len) pv = 0.f;
             p[u][k] = pv;
         }
@@ -429,7 +442,7 @@ __device__ __forceinline__ double worker_rows_scalar(const WorkerArgs& a, const 
             const float g = a.g[j];
             const float e = residual_of(a.pb[j], sp);
             const float m = __fmaf_rn(a.mu, a.m[j], g);
-            pv = __fmaf_rn(a.ratio, e, __fmaf_rn(a.mu, m, g));
+            pv = corrected_vector(a.ratio, a.ratio != 1.0f, e, __fmaf_rn(a.mu, m, g));
             a.m[j] = m;
             a.pb[j] = pv;
             if (DIAG) {
@@ -619,6 +632,7 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
         reinterpret_cast<unsigned*>(ring + (size_t)kServerStages * U * kThreads * sizeof(float4)) +
         threadIdx.x;
     double acc = 0.0;
+    const bool rescale = a.ratio != 1.0f;
     // bit patterns of the scaled scales of the workers the table does not cover
     unsigned cdir[kMaxLutWorkers - kLutWorkers + 1] = {};
 
@@ -667,7 +681,7 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
             }
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                float pv = __fmaf_rn(a.ratio, residual_of(p[u][k], sp), avg[k]);   // ptilde_t
+                float pv = corrected_vector(a.ratio, rescale, residual_of(p[u][k], sp), avg[k]);   // ptilde_t
                 if (!full && o + k >= clen) pv = 0.f;
                 p[u][k] = pv;
             }
@@ -754,7 +768,7 @@ __device__ __forceinline__ double server_rows(const ServerArgs& a, const Tile& t
         if (full || o < t.len) average4(a, s_c, t.word + (o >> 5), sh, avg);
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            float pv = __fmaf_rn(a.ratio, residual_of(p[u][k], sp), avg[k]);   // ptilde_t
+            float pv = corrected_vector(a.ratio, a.ratio != 1.0f, residual_of(p[u][k], sp), avg[k]);   // ptilde_t
             if (!full && o + k >= t.len) pv = 0.f;
             p[u][k] = pv;
         }
@@ -785,7 +799,7 @@ __device__ __forceinline__ double server_rows_scalar(const ServerArgs& a, const 
                 avg = (i == 0) ? v : __fadd_rn(avg, v);
             }
             const long long j = t.start + o;
-            pv = __fmaf_rn(a.ratio, residual_of(a.pb[j], sp), avg);
+            pv = corrected_vector(a.ratio, a.ratio != 1.0f, residual_of(a.pb[j], sp), avg);
             a.pb[j] = pv;
         }
         acc += (double)fabsf(pv);

@@ -325,10 +325,11 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
     if (major != 10) return EF_ERR_UNSUPPORTED_DEVICE;
 
     ef_ctx* c = new (std::nothrow) ef_ctx();
-    if (!c) return EF_ERR_INVALID_ARG;
+    if (!c) return EF_ERR_NO_MEMORY;
     c->L = L; c->mu = mu; c->eta = eta; c->eta_prev = eta; c->flags = flags;
     c->ws = (char*)workspace;
     c->stream = (cudaStream_t)cuda_stream;
+    try {
     c->stepped.assign(M, 0);
 
     // tile and block tables
@@ -350,6 +351,10 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
         blk.tile_count = (int)c->h_tiles.size() - blk.tile_begin;
         if (len > kChunkLen) c->h_multi.push_back(b);
         word += (len + 31) / 32;
+    }
+    } catch (const std::bad_alloc&) {
+        delete c;
+        return EF_ERR_NO_MEMORY;
     }
     // Small grids are launch-bound: finish block scales inside the main kernels.  Large grids
     // are bandwidth-bound: the per-CTA fence of the fused form costs more than a tiny launch.
@@ -541,6 +546,7 @@ const char* ef_strerror(int status) {
         case EF_ERR_UNSUPPORTED_DEVICE: return "device is not compute capability 10.x";
         case EF_ERR_TIMEOUT: return "device-side wait timed out";
         case EF_ERR_TOO_LARGE: return "size exceeds the fixed scratch of the no-allocation entry point";
+        case EF_ERR_NO_MEMORY: return "host allocation failed";
         default: return "unknown status";
     }
 }
@@ -561,11 +567,66 @@ int ef_destroy(ef_ctx* c) {
 }  // extern "C"
 
 // =============================================================================================
+// ef_stream_probe: no-compute stream kernels with the access mix of the step kernels, so that a
+// measured rate can be set against what the memory system gives a kernel of the same shape
+// (one 4096-element chunk per CTA, 128-bit accesses through L2) that does no arithmetic worth
+// the name.  A measurement aid; not part of the method.
+// =============================================================================================
+namespace {
+
+template <int MODE>
+__global__ void __launch_bounds__(efk::kThreads) ef_stream_probe_kernel(const float* __restrict__ a,
+                                                                        float* __restrict__ b,
+                                                                        float* __restrict__ c) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long base = (long long)blockIdx.x * kChunkLen + warp * (128 * kU) + lane * 4;
+    float4 A[kU], Bv[kU], C[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+        if (MODE != EF_PROBE_1R1W) A[u] = efk::ld_stream(a + base + u * 128);
+        if (MODE != EF_PROBE_COPY) Bv[u] = efk::ld_stream(b + base + u * 128);
+        if (MODE == EF_PROBE_3R2W) C[u] = efk::ld_stream(c + base + u * 128);
+    }
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+        if (MODE == EF_PROBE_3R2W) {
+            Bv[u].x += A[u].x; Bv[u].y += A[u].y; Bv[u].z += A[u].z; Bv[u].w += A[u].w;
+            C[u].x += Bv[u].x; C[u].y += Bv[u].y; C[u].z += Bv[u].z; C[u].w += Bv[u].w;
+            efk::st_stream(b + base + u * 128, Bv[u]);
+            efk::st_stream(c + base + u * 128, C[u]);
+        } else if (MODE == EF_PROBE_1R1W) {
+            Bv[u].x += 1.f; Bv[u].y -= 1.f; Bv[u].z += 1.f; Bv[u].w -= 1.f;
+            efk::st_stream(b + base + u * 128, Bv[u]);
+        } else {
+            efk::st_stream(c + base + u * 128, A[u]);
+        }
+    }
+}
+
+}  // namespace
+
+extern "C" int ef_stream_probe(int32_t mode, const float* a, float* b, float* c, int64_t n,
+                               void* cuda_stream) {
+    if (!a || !b || !c || n < kChunkLen || n % kChunkLen != 0 || n / kChunkLen > 0x7fffffffLL)
+        return EF_ERR_INVALID_ARG;
+    if (!aligned16(a) || !aligned16(b) || !aligned16(c)) return EF_ERR_ALIGNMENT;
+    const unsigned grid = (unsigned)(n / kChunkLen);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    switch (mode) {
+        case EF_PROBE_3R2W: ef_stream_probe_kernel<EF_PROBE_3R2W><<<grid, efk::kThreads, 0, st>>>(a, b, c); break;
+        case EF_PROBE_1R1W: ef_stream_probe_kernel<EF_PROBE_1R1W><<<grid, efk::kThreads, 0, st>>>(a, b, c); break;
+        case EF_PROBE_COPY: ef_stream_probe_kernel<EF_PROBE_COPY><<<grid, efk::kThreads, 0, st>>>(a, b, c); break;
+        default: return EF_ERR_INVALID_ARG;
+    }
+    return cudaGetLastError() == cudaSuccess ? EF_OK : EF_ERR_CUDA;
+}
+
+// =============================================================================================
 // ef_worker_step_noalloc: the worker step for callers that cannot allocate device memory.
 //
 // Some hosts of this library are not allowed to call cudaMalloc at the point where they step
-// the optimizer: code running inside a CUDA-graph capture or another framework's stream
-// callback, plugins that were handed a fixed arena and must not grow it, and real-time loops
+// the optimizer: code running while another framework owns the allocator or the stream,
+// plugins that were handed a fixed arena and must not grow it, and real-time loops
 // where an allocation (which may synchronise the whole device) is not tolerable.  The regular
 // entry points avoid allocation by taking a caller-sized workspace; this variant needs not even
 // that: its scratch memory (one fp64 partial sum per 4096-element chunk plus one arrival

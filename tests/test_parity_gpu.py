@@ -1,4 +1,6 @@
 """GPU parity: the CUDA path, called through the C ABI, against the CPU oracle."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -255,19 +257,44 @@ def test_config3_fused_scale_mode():
     run_parity(w, steps=3, check_every_step=False, scale_mode="fused")
 
 
-def test_config4_flat_2_28_sampled_blocks():
+ORACLE_PROCS = max(2, min(os.cpu_count() or 2, 16))
+
+
+def _assert_locked(stats):
+    """Whole-vector runs: every state element that was compared has the oracle's bit pattern
+    unless a tie-zone bit was adopted or a scale differed in its last bit (both are listed)."""
+    assert stats["adopted"] <= 3 and stats["scale_bit_mismatch"] <= 3, stats["adopted_list"]
+    if stats["adopted"] == 0 and stats["scale_bit_mismatch"] == 0:
+        assert stats["state_bit_mismatch"] == 0
+    assert stats["state_elements_compared"] > 0
+
+
+def test_config4_flat_2_28_whole_vector():
     """Full-size launch (d = 2^28, M = 7, 20 steps) in the configuration bench.py times (all
-    workers in one ef_worker_step_all launch); the oracle follows 6 of the 256 blocks."""
+    workers in one ef_worker_step_all launch).  The oracle follows ALL 256 blocks: untouched
+    single-threaded oracle instances on disjoint block ranges, one per process (blocks are
+    independent in the method).  Words are compared after every call, the state after the last
+    step, element by element."""
     w = wl.make_workload(4)
-    run_parity(w, blocks=[0, 1, 100, 127, 128, 255], check_every_step=False, batched=True)
+    eng, _, stats = run_parity(w, check_every_step=False, batched=True, oracle_procs=ORACLE_PROCS)
+    assert stats["state_elements_compared"] == (2 * w.M + 2) * w.d
+    _assert_locked(stats)
 
 
-def test_config5_gpt2_layout_sampled_blocks():
-    """Full-size launch; the oracle follows the embedding block (51M elements, 12.5k tiles),
-    the position table and one whole transformer layer, plus the last block."""
+def test_config5_gpt2_layout_whole_vector():
+    """Full-size launch of the GPT-2-medium-shaped layout (290 blocks, M = 4, 10 steps); the
+    oracle follows all blocks, including the 51M-element embedding (12.5k tiles)."""
     w = wl.make_workload(5)
-    layer7 = list(range(2 + 12 * 7, 2 + 12 * 8))
-    run_parity(w, blocks=[0, 1] + layer7 + [w.B - 1], check_every_step=False)
+    eng, _, stats = run_parity(w, check_every_step=False, oracle_procs=ORACLE_PROCS)
+    assert stats["state_elements_compared"] == (2 * w.M + 2) * w.d
+    _assert_locked(stats)
+
+
+def test_config3_whole_vector_through_the_process_pool():
+    """The pooled oracle on a layout the single oracle also follows (ResNet-50, 161 uneven blocks)."""
+    w = wl.make_workload(3)
+    eng, _, stats = run_parity(w, steps=3, check_every_step=True, batched=True, oracle_procs=4)
+    _assert_locked(stats)
 
 
 @pytest.mark.parametrize("seed", range(14))
@@ -310,6 +337,28 @@ def test_denormal_range_gradients():
     assert all((g != 0).any() and g.abs().max() < 1.2e-38 for gs in grads for g in gs)
     eng, orc, stats = run_parity(w, grads=grads)
     assert float(eng.worker_scales(0).max()) > 0.0
+
+
+def test_rescaled_residuals_that_underflow_to_negative_zero():
+    """With a stepsize change the residual enters as fma(eta_{t-1}/eta_t, e, .), which can
+    underflow to -0; sign(-0) = +1, so the bit must be 0 and the stored value must behave as +0.
+    Construction (u = 2^-149, mu = 0, M = 2): step 0 gives worker residuals of +-u and a server
+    residual of +-u; step 1 doubles the stepsize (ratio 1/2) with zero gradients, so every
+    corrected vector is +-u/2, which rounds to +-0, and every scale is 0: there is no tie zone
+    to hide a wrong bit in.  Blocks cover the vector path, a ragged tail and the scalar path."""
+    u = 2.0 ** -149
+    sizes = [64, TILE + 64, 5, 2 * TILE + 6, 33]
+    w = _wl("negzero-rescale", sizes, 2, mu=0.0, steps=4)
+    k = torch.cat([torch.arange(n) for n in sizes])          # index inside the block
+    odd = (k % 2 == 1)
+    g0 = torch.where(odd, torch.tensor(u), torch.tensor(3 * u)).float()
+    g1 = torch.where(odd, torch.tensor(-u), torch.tensor(3 * u)).float()
+    assert (g0 != 0).all() and (g1 != 0).all()
+    z = torch.zeros(w.d)
+    gen = torch.Generator().manual_seed(11)
+    tail = [[torch.randn(w.d, generator=gen) * 1e-42 for _ in range(2)] for _ in range(2)]
+    eng, orc, stats = run_parity(w, grads=[[g0, g1], [z, z]] + tail, etas=[0.1, 0.2, 0.2, 0.05])
+    assert stats["adopted"] == 0 and stats["state_bit_mismatch"] == 0
 
 
 def test_indexing_beyond_2_32_elements():

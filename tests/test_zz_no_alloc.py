@@ -1,12 +1,13 @@
-"""The no-allocation worker step (ef_worker_step_noalloc) against the regular entry point.
+"""The no-allocation worker step (ef_worker_step_noalloc) against the regular entry point and
+against the CPU oracle.
 
 Who needs it: hosts that may not call cudaMalloc where they step the optimizer (code running
 under another framework's allocator or stream, plugins with a fixed arena, latency-critical
 loops).  The variant keeps its scratch in a fixed array inside the library, so the caller passes
-only inputs and outputs.  Here it is called twice in a row through the C ABI, carrying its state
-in caller-owned tensors, and every output is compared with what ef_worker_step produces for a
-layout with one block of the same size: packed words and scale bit for bit, momentum and the
-residual within the tolerance of the other parity tests.
+only inputs and outputs.  Here it is called several times in a row through the C ABI, carrying
+its state in caller-owned tensors.  Every output must equal, bit for bit, what ef_worker_step
+produces for a layout with one block of the same size (the header promises exactly that), and
+must agree with the oracle's worker step under the tolerances of the other parity tests.
 
 This file sorts last on purpose, so that a run that stops at the first failure has already run
 every other test; it does not depend on anything the other tests leave behind.
@@ -15,6 +16,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import Oracle
 from paper_1905_10936_b200 import binding as ef
 from paper_1905_10936_b200.engine import EFEngine
 
@@ -28,35 +30,77 @@ def _materialise(p: torch.Tensor, s: torch.Tensor) -> torch.Tensor:
     return torch.where(p < 0, p + s, p - s)
 
 
+class _NoAllocState:
+    """The caller-owned state of one block for ef_worker_step_noalloc."""
+
+    def __init__(self, n, dev):
+        self.n = n
+        self.m = torch.zeros(n, device=dev)
+        self.p = torch.zeros(n, device=dev)
+        self.s_prev = torch.zeros(1, device=dev)
+        self.words = torch.empty((n + 31) // 32, dtype=torch.int32, device=dev)
+        self.scale = torch.empty(1, device=dev)
+
+    def step(self, g, mu):
+        ef.ef_worker_step_noalloc(g.data_ptr(), self.m.data_ptr(), self.p.data_ptr(),
+                                  self.s_prev.data_ptr(), self.n, mu, self.words.data_ptr(),
+                                  self.scale.data_ptr(), torch.cuda.current_stream().cuda_stream)
+
+
+def _check_call(st, eng, orc, g, mu, what):
+    eng.worker_step(0, g)
+    st.step(g, mu)
+    torch.cuda.synchronize()
+    # against the regular entry point: identical in every bit
+    assert torch.equal(st.words, eng.worker_words(0)), f"{what}: packed words differ"
+    assert st.scale.item() == eng.worker_scales(0).item(), f"{what}: scale differs"
+    assert st.s_prev.item() == st.scale.item()
+    assert torch.equal(st.m, eng.momentum(0)), f"{what}: momentum differs"
+    e = _materialise(st.p, st.s_prev)
+    assert torch.equal(e, eng.residual(0)), f"{what}: residual differs"
+    # against the oracle (one block, one worker): words bit-exact after tie-zone adoption,
+    # scale / momentum / residual within 1e-5 (of the largest magnitude for the vectors)
+    gw = st.words.cpu().numpy().view(np.uint32)
+    adopted = orc.worker_step(0, g.cpu().numpy(), hint=gw)
+    assert np.array_equal(orc.words(0), gw), f"{what}: words differ from the oracle's"
+    ref_s = float(orc.scales(0)[0])
+    assert abs(st.scale.item() - ref_s) <= RTOL * abs(ref_s)
+    for got, ref in ((st.m, orc.momentum(0)), (e, orc.residual(0))):
+        got = got.cpu().numpy()
+        assert np.abs(got - ref).max() <= RTOL * np.abs(ref).max()
+        if len(adopted) == 0 and st.scale.item() == ref_s:
+            assert np.array_equal(got.view(np.uint32), ref.view(np.uint32))
+    eng.server_step()              # closes the iteration on both reference sides (M = 1)
+    orc.server_step()
+
+
 @pytest.mark.parametrize("n", [5 * 4096 + 37, 1000, 16384 * 3, 4096])
-def test_two_calls_in_a_row_match_the_regular_worker_step(n):
+def test_two_calls_in_a_row_match_the_regular_worker_step_and_the_oracle(n):
     mu = 0.9
     dev = torch.device("cuda")
     gen = torch.Generator(device=dev); gen.manual_seed(1234 + n)
-    grads = [torch.randn(n, device=dev, generator=gen) * 0.3 for _ in range(2)]
-
     eng = EFEngine([0, n], 1, mu, 0.1)
-    m = torch.zeros(n, device=dev)
-    p = torch.zeros(n, device=dev)
-    s_prev = torch.zeros(1, device=dev)
-    words = torch.empty((n + 31) // 32, dtype=torch.int32, device=dev)
-    scale = torch.empty(1, device=dev)
-    stream = torch.cuda.current_stream().cuda_stream
+    orc = Oracle([0, n], 1, mu, 0.1)
+    st = _NoAllocState(n, dev)
+    for call in range(2):
+        g = torch.randn(n, device=dev, generator=gen) * 0.3
+        _check_call(st, eng, orc, g, mu, f"n={n} call {call}")
 
-    for call, g in enumerate(grads):
-        eng.worker_step(0, g)
-        ef.ef_worker_step_noalloc(g.data_ptr(), m.data_ptr(), p.data_ptr(), s_prev.data_ptr(), n, mu,
-                                  words.data_ptr(), scale.data_ptr(), stream)
-        torch.cuda.synchronize()
-        assert torch.equal(words, eng.worker_words(0)), f"call {call}: packed words differ"
-        ref_scale = eng.worker_scales(0)
-        assert abs(scale.item() - ref_scale.item()) <= RTOL * abs(ref_scale.item())
-        assert s_prev.item() == scale.item()
-        ref_m, ref_e = eng.momentum(0), eng.residual(0)
-        assert (m - ref_m).abs().max().item() <= RTOL * ref_m.abs().max().item()
-        e = _materialise(p, s_prev)
-        assert (e - ref_e).abs().max().item() <= RTOL * ref_e.abs().max().item()
-        eng.server_step()          # closes the iteration of the regular engine
+
+def test_a_smaller_problem_after_a_larger_one_ignores_stale_scratch():
+    """All calls share one scratch array, which keeps the previous call's partial sums: a
+    40-chunk problem leaves 40 slots behind, the 3-chunk problem after it must read only its
+    own three; then the large one again."""
+    mu = 0.5
+    dev = torch.device("cuda")
+    gen = torch.Generator(device=dev); gen.manual_seed(99)
+    sizes = [40 * 4096 + 5, 3 * 4096 - 8]
+    engs = [EFEngine([0, n], 1, mu, 0.1) for n in sizes]
+    orcs = [Oracle([0, n], 1, mu, 0.1) for n in sizes]
+    sts = [_NoAllocState(n, dev) for n in sizes]
+    for call, k in enumerate([0, 1, 0, 1]):
+        g = torch.randn(sizes[k], device=dev, generator=gen) * (10.0 if k == 0 else 0.01)
+        _check_call(sts[k], engs[k], orcs[k], g, mu, f"problem {k} call {call}")
 
 
 def test_limits_are_enforced_without_launching():
