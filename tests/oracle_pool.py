@@ -39,14 +39,15 @@ def split_blocks(sizes: Sequence[int], parts: int) -> List[Tuple[int, int]]:
 
 
 def blockwise_check(got: np.ndarray, ref: np.ndarray, sub_offsets: np.ndarray):
-    """Per block: max |got - ref| against RTOL * max |ref|.  Returns (bad, bit_mismatch):
-    bad = [(block, err, max_ref)] for the blocks out of tolerance, bit_mismatch = number of
-    elements whose binary32 patterns differ."""
+    """Per block: max |got - ref| against RTOL * max |ref|.  Returns (bad, mismatch):
+    bad = [(block, err, max_ref)] for the blocks out of tolerance, mismatch = number of
+    elements that are not the same binary32 number (+0 and -0 are the same number: the method
+    reads sign(+-0) = +1 and never divides by a state value, so the two are interchangeable)."""
     diff = np.abs(got.astype(np.float64) - ref.astype(np.float64))
     mx_d = np.maximum.reduceat(diff, sub_offsets[:-1])
     mx_r = np.maximum.reduceat(np.abs(ref).astype(np.float64), sub_offsets[:-1])
     bad = [(int(b), float(mx_d[b]), float(mx_r[b])) for b in np.nonzero(mx_d > RTOL * mx_r)[0]]
-    mism = int(np.count_nonzero(got.view(np.uint32) != ref.view(np.uint32)))
+    mism = int(np.count_nonzero(got != ref))
     return bad, mism
 
 
@@ -202,7 +203,7 @@ class OraclePool:
     # ---- comparison: the caller has filled self.state with the other side's vector -----------
     def compare(self, kind: str, i: int = -1):
         """kind: "x", "m", "e" (i = -1: server residual) or "mt".  Returns (bad blocks, number of
-        elements whose bit patterns differ)."""
+        elements that differ in value)."""
         res = self._all("cmp", kind, int(i))
         bad = [b for r in res for b in r[0]]
         return bad, sum(r[1] for r in res)

@@ -70,8 +70,9 @@ def test_pool_equals_single_oracle_bit_for_bit(nproc):
         pool.close()
 
 
-def test_blockwise_check_counts_bit_patterns():
+def test_blockwise_check_counts_values_that_differ():
     ref = np.array([1.0, -2.0, 0.0, 4.0], dtype=np.float32)
-    got = ref.copy(); got[2] = -0.0                      # equal in value, different pattern
-    bad, mism = blockwise_check(got, ref, np.array([0, 2, 4]))
-    assert bad == [] and mism == 1
+    got = ref.copy(); got[2] = -0.0                      # the two zeros are the same number
+    assert blockwise_check(got, ref, np.array([0, 2, 4])) == ([], 0)
+    got[3] = np.nextafter(np.float32(4.0), np.float32(5.0))   # one ulp off: within 1e-5, but counted
+    assert blockwise_check(got, ref, np.array([0, 2, 4])) == ([], 1)
