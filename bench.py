@@ -35,6 +35,7 @@ import torch
 from paper_1905_10936_b200 import workloads as wl
 
 METRIC = "parameters/sec through one two-way compressed dist-EF-blockSGDM step (M workers)"
+METRIC_SIGNUM = "parameters/sec through one signum-with-majority-vote step (M workers)"
 UNIT = "params/s"
 
 # DRAM traffic of the worker kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum) on
@@ -61,6 +62,16 @@ def server_call_bytes(d: int, B: int, M: int) -> float:
 
 def step_bytes(d: int, B: int, M: int) -> float:
     return M * worker_call_bytes(d, B) + server_call_bytes(d, B, M)
+
+
+def vote_worker_call_bytes(d: int, B: int) -> float:
+    """signum worker: read g, m; write m; write 1 bit per element."""
+    return 12.125 * d
+
+
+def vote_server_call_bytes(d: int, B: int, M: int) -> float:
+    """signum server: read M bits and x; write x and 1 bit per element."""
+    return (8.0 + (M + 1) / 8.0) * d
 
 
 def config_dict(w) -> dict:
@@ -138,14 +149,14 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- CPU oracle legs
-def time_oracle(w: wl.Workload, n_blocks: int, steps: int, warmup: int):
+def time_oracle(w: wl.Workload, n_blocks: int, steps: int, warmup: int, workload: str = "ef"):
     """Times the oracle, as it stands, on the first n_blocks blocks of the workload.
     Returns (params_per_s, seconds_per_step, d_sample)."""
-    from oracle import Oracle
+    from oracle import Oracle, SignumOracle
     sizes = w.sizes[:n_blocks]
     sub = wl.custom_workload(w.name + "-sample", sizes, w.M, w.mu, w.eta, steps, w.law,
                              w.scale_range, config_id=w.config_id)
-    orc = Oracle(sub.offsets, sub.M, sub.mu, sub.eta)
+    orc = (SignumOracle if workload == "signum" else Oracle)(sub.offsets, sub.M, sub.mu, sub.eta)
     es = sub.element_scales("cpu")
     grads = [sub.draw_grad(0, i, "cpu", es).numpy() for i in range(sub.M)]
     elapsed = 0.0
@@ -173,11 +184,12 @@ def run_reference(args) -> None:
     budget_s = 90.0
     per_block = np.mean(w.sizes) * oracle_ns_per_param(w.M) * 1e-9
     n_blocks = int(max(1, min(w.B, budget_s / ((args.steps + args.warmup) * per_block))))
-    value, s_per_step, d_s = time_oracle(w, n_blocks, args.steps, args.warmup)
+    value, s_per_step, d_s = time_oracle(w, n_blocks, args.steps, args.warmup, args.workload)
     sample = (f"first {n_blocks} of {w.B} blocks ({d_s} of {w.d} parameters), M={w.M}, "
               f"{args.steps} timed steps; single-threaded C++ oracle")
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+        "impl": "reference", "metric": METRIC_SIGNUM if args.workload == "signum" else METRIC,
+        "value": value, "unit": UNIT,
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         # time one step of the WHOLE workload takes at the sampled rate (blocks are independent,
         # the oracle's cost is linear in the number of parameters); the sample's own step time
@@ -257,18 +269,24 @@ def run_ours(args) -> None:
     del es
     batched = not args.per_worker_calls
     step_no = [0]
+    signum = args.workload == "signum"
+    step_all = eng.vote_worker_step_all if signum else eng.worker_step_all
+    step_one = eng.vote_worker_step if signum else eng.worker_step
+    server_call = eng.vote_server_step if signum else eng.server_step
+    w_bytes_fn = vote_worker_call_bytes if signum else worker_call_bytes
+    s_bytes_fn = vote_server_call_bytes if signum else server_call_bytes
 
     def worker_calls():
         ga = galls[step_no[0] % nbatch]
         if batched:
-            eng.worker_step_all(ga)            # all M workers in one launch
+            step_all(ga)                       # all M workers in one launch
         else:
             for i in range(w.M):
-                eng.worker_step(i, ga[i, :w.d])
+                step_one(i, ga[i, :w.d])
 
     def one_step():
         worker_calls()
-        eng.server_step()
+        server_call()
         step_no[0] += 1
 
     for _ in range(W):
@@ -283,7 +301,7 @@ def run_ours(args) -> None:
         ev[k][0].record()
         worker_calls()
         ev[k][1].record()
-        eng.server_step()
+        server_call()
         ev[k][2].record()
         step_no[0] += 1
     barrier()
@@ -316,7 +334,8 @@ def run_ours(args) -> None:
                      "unit": UNIT, "seconds": s_ms * 1e-3, "sm_mhz": s_clk.get("sm_mhz"),
                      "sm_max_mhz": s_clk.get("sm_max_mhz"), "reasons": s_clk.get("reasons"),
                      "clock_samples": s_clk.get("samples"),
-                     "step_gbs": step_bytes(w.d, w.B, w.M) / (s_ms / Ks * 1e-3) / 1e9}
+                     "step_gbs": (w.M * w_bytes_fn(w.d, w.B) + s_bytes_fn(w.d, w.B, w.M))
+                                 / (s_ms / Ks * 1e-3) / 1e9}
 
     # ---- the same step replayed from a CUDA graph (launch gaps shrink; matters for small layouts)
     graph_info = None
@@ -345,7 +364,7 @@ def run_ours(args) -> None:
 
     # ---- end to end: host gradients in, packed update out, copies inside the timed region
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not signum:
         hsrc = galls[0]
         del eng
         torch.cuda.empty_cache()
@@ -391,22 +410,23 @@ def run_ours(args) -> None:
         return
 
     peak, peak_kind = measured_hbm_peak()
-    wbytes = worker_call_bytes(w.d, w.B) * (w.M if batched else 1)
-    sbytes = server_call_bytes(w.d, w.B, w.M) + (8.0 * w.d if args.weight_decay > 0 else 0.0)
+    wbytes = w_bytes_fn(w.d, w.B) * (w.M if batched else 1)
+    sbytes = s_bytes_fn(w.d, w.B, w.M) + (8.0 * w.d if args.weight_decay > 0 else 0.0)
     w_gbs = wbytes / (worker_ms * 1e-3) / 1e9
     s_gbs = sbytes / (server_ms * 1e-3) / 1e9
-    plain = (args.weight_decay == 0 and not args.diagnostics and world == 1)
+    plain = (args.weight_decay == 0 and not args.diagnostics and world == 1 and not signum)
     traffic = None
     if plain and w.name == NCU_WORKER_TRAFFIC["workload"]:
         traffic = NCU_WORKER_TRAFFIC["bytes_per_worker_param"] * w.d * (w.M if batched else 1)
     line = {
-        "metric": METRIC, "value": job_params * K / (total_ms * 1e-3), "unit": UNIT,
+        "metric": METRIC_SIGNUM if signum else METRIC,
+        "value": job_params * K / (total_ms * 1e-3), "unit": UNIT,
         "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": total_ms / K,
         "steps_per_sec": K / (total_ms * 1e-3),
         "higher_is_better": True, "scaling": args.scaling if world > 1 else "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": config_dict(w_full),
-        "run": {"weight_decay": args.weight_decay, "diagnostics": bool(args.diagnostics),
+        "run": {"workload": args.workload, "weight_decay": args.weight_decay, "diagnostics": bool(args.diagnostics),
                 "worker_calls": "ef_worker_step_all" if batched else "ef_worker_step x M",
                 "gradient_batches_rotated": nbatch,
                 "per_gpu": ("every rank owns one whole layout (a block-range shard of an N-times "
@@ -417,8 +437,8 @@ def run_ours(args) -> None:
         "e2e": e2e,
         "gpu_launches": int(launches * world),
         "roofline": {
-            "kernel": "ef_worker_kernel", "call": ("ef_worker_step_all: M workers per launch" if batched
-                                                   else "ef_worker_step: one worker per launch"),
+            "kernel": "ef_vote_worker_kernel" if signum else "ef_worker_kernel",
+            "call": ("all M workers in one launch" if batched else "one worker per launch"),
             "bound": "hbm", "achieved": w_gbs, "peak": peak,
             "peak_kind": f"of {peak_kind} (a 1:1 copy; context for a kernel that reads 60% of its bytes)",
             "unit": "GB/s", "frac": w_gbs / peak,
@@ -428,13 +448,14 @@ def run_ours(args) -> None:
             "traffic_source": NCU_WORKER_TRAFFIC["captured_on"] if traffic else None,
         },
         "roofline_server": {
-            "kernel": "ef_server_kernel (+ ef_apply_kernel where the update is not fused)",
+            "kernel": ("ef_vote_server_kernel" if signum else
+                       "ef_server_kernel (+ ef_apply_kernel where the update is not fused)"),
             "bound": "hbm", "achieved": s_gbs,
             "peak": peak, "unit": "GB/s", "frac": s_gbs / peak,
             "frac_of_8000_nominal": s_gbs / 8000.0, "bytes_per_call": sbytes,
             "ms_per_call": server_ms,
         },
-        "step_gbs": step_bytes(w.d, w.B, w.M) / (total_ms / K * 1e-3) / 1e9,
+        "step_gbs": (w.M * w_bytes_fn(w.d, w.B) + s_bytes_fn(w.d, w.B, w.M)) / (total_ms / K * 1e-3) / 1e9,
     }
     if sustained is not None:
         line["sustained"] = sustained
@@ -448,7 +469,7 @@ def run_ours(args) -> None:
         per_block = np.mean(w.sizes) * oracle_ns_per_param(w.M) * 1e-9
         steps_c = 2
         n_blocks = int(max(1, min(w.B, 15.0 / ((steps_c + 1) * per_block))))
-        v, s_per_step, d_s = time_oracle(w, n_blocks, steps_c, 1)
+        v, s_per_step, d_s = time_oracle(w, n_blocks, steps_c, 1, args.workload)
         line["cpu_baseline"] = {
             "value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
             "sample": f"first {n_blocks} of {w.B} blocks ({d_s} of {w.d} parameters), M={w.M}, "
@@ -511,6 +532,9 @@ def main():
     ap.add_argument("--workers", type=int, default=0,
                     help="override the number of simulated workers M of the workload")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", choices=["ef", "signum"], default="ef",
+                    help="ef: dist-EF-blockSGDM (default, the headline); signum: the paper's "
+                         "comparison method, signum with majority vote, on the same layouts")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--per-worker-calls", action="store_true",
                     help="step the workers with M ef_worker_step calls instead of one ef_worker_step_all")

@@ -188,6 +188,47 @@ int ef_step_count(ef_ctx* ctx, int64_t* t /* out: completed iterations */);
 /* Number of kernels this context has launched so far (for launch accounting). */
 int64_t ef_launch_count(ef_ctx* ctx);
 
+/* ---- signum / signSGD with majority vote: the paper's comparison method (Section 1: only the
+ * 1-bit gradient sign travels between workers and server, in both directions; baselines of
+ * Sections 4.1 and 4.2; Table 1: 2Md bits per iteration).  It runs on the same context and
+ * state as the error-feedback path (momentum m_i, parameters x, the packed-word buffers, same
+ * packed layout; no scales are produced), one iteration being
+ *     for each worker i:  ef_vote_worker_step(ctx, i, g_{t,i})      (or ef_vote_worker_step_all)
+ *     ef_vote_server_step(ctx)
+ *   worker i:  m_{t,i} = mu m_{t-1,i} + g_{t,i};  message = sign(m_{t,i}), readable through
+ *              ef_worker_words (mu = 0 gives signSGD);
+ *   server:    vote = sign(sum_i sign(m_{t,i})) coordinate-wise, readable through
+ *              ef_server_words;  x_{t+1} = x_t - eta vote.
+ * Conventions where the paper is silent: sign(+-0) = +1; a tied vote (possible only for even M;
+ * Section 4.2 notes an odd M never ties) is sent as +1, the message being one bit.
+ * Arguments, ordering rules and errors are those of ef_worker_step / ef_worker_step_all /
+ * ef_server_step; in addition the worker calls of one iteration must all belong to the same
+ * method, and the server call must match them (else BAD_STATE).  The stepsize is the one set by
+ * ef_init / ef_set_eta; weight decay does not apply to this method. */
+int ef_vote_worker_step(ef_ctx* ctx, int32_t i, const float* grad /* device */);
+int ef_vote_worker_step_all(ef_ctx* ctx, const float* grads /* device, M gradients */, int64_t stride);
+int ef_vote_server_step(ef_ctx* ctx);
+
+/* ---- top-k: the second example of a delta-approximate compressor after Definition 1
+ * (Section 2): it keeps the k coordinates of largest absolute value (delta = k/d).  Together
+ * with its error-feedback residual this is the worker's compress line and residual line of
+ * Algorithm 2 with C = top-k:  Delta = C(v),  e = v - Delta.
+ *   v[n]          device, 16-byte aligned: the corrected vector to compress
+ *   idx_out[k]    device: the kept coordinates in increasing order
+ *   val_out[k]    device: their values, val_out[r] = v[idx_out[r]]
+ *   resid_out[n]  device, 16-byte aligned, or NULL: v - C(v) (exactly 0 at the kept coordinates,
+ *                 v elsewhere); may alias v
+ * Among equal magnitudes the lower index is kept (the paper does not say), +0 and -0 have the
+ * same magnitude, NaN is unspecified.  workspace: device, 256-byte aligned, at least
+ * ef_topk_workspace_bytes(n) bytes (histograms and per-chunk counts), owned by the caller and
+ * overwritten by every call; calls that share a workspace must not overlap on the GPU.
+ * Work is enqueued on cuda_stream without synchronisation; the library allocates nothing.
+ * Errors: INVALID_ARG (n < 1, k outside [1, n], null), WORKSPACE, ALIGNMENT,
+ * UNSUPPORTED_DEVICE, CUDA. */
+int ef_topk_workspace_bytes(int64_t n, size_t* bytes /* out */);
+int ef_topk_compress(const float* v, int64_t n, int64_t k, int64_t* idx_out, float* val_out,
+                     float* resid_out, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Measurement aid (the paper has no counterpart): no-compute stream kernels with the access mix
  * of the step kernels, one 4096-element chunk per CTA and 128-bit accesses like them, so that a
  * measured rate can be set against the ceiling of a kernel of the same shape.

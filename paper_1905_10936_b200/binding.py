@@ -64,6 +64,11 @@ SIGNATURES = {
     "ef_step_count": (ctypes.c_int, [_vp, ctypes.POINTER(_i64)]),
     "ef_launch_count": (_i64, [_vp]),
     "ef_worker_step_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _f32, _vp, _vp, _vp]),
+    "ef_vote_worker_step": (ctypes.c_int, [_vp, _i32, _vp]),
+    "ef_vote_worker_step_all": (ctypes.c_int, [_vp, _vp, _i64]),
+    "ef_vote_server_step": (ctypes.c_int, [_vp]),
+    "ef_topk_workspace_bytes": (ctypes.c_int, [_i64, ctypes.POINTER(ctypes.c_size_t)]),
+    "ef_topk_compress": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp, _vp, ctypes.c_size_t, _vp]),
     "ef_stream_probe": (ctypes.c_int, [_i32, _vp, _vp, _vp, _i64, _vp]),
     "ef_strerror": (ctypes.c_char_p, [ctypes.c_int]),
     "ef_last_cuda_error": (ctypes.c_int, [_vp]),
@@ -213,6 +218,30 @@ def ef_worker_step_noalloc(grad_ptr: int, momentum_ptr: int, residual_ptr: int,
     _check(load_library().ef_worker_step_noalloc(grad_ptr, momentum_ptr, residual_ptr,
                                                  residual_scale_ptr, n, mu, words_ptr, scale_ptr,
                                                  cuda_stream), "ef_worker_step_noalloc")
+
+
+def ef_vote_worker_step(ctx: int, i: int, grad_ptr: int) -> None:
+    _check(load_library().ef_vote_worker_step(ctx, i, grad_ptr), "ef_vote_worker_step")
+
+
+def ef_vote_worker_step_all(ctx: int, grads_ptr: int, stride: int) -> None:
+    _check(load_library().ef_vote_worker_step_all(ctx, grads_ptr, stride), "ef_vote_worker_step_all")
+
+
+def ef_vote_server_step(ctx: int) -> None:
+    _check(load_library().ef_vote_server_step(ctx), "ef_vote_server_step")
+
+
+def ef_topk_workspace_bytes(n: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(load_library().ef_topk_workspace_bytes(n, ctypes.byref(out)), "ef_topk_workspace_bytes")
+    return out.value
+
+
+def ef_topk_compress(v_ptr: int, n: int, k: int, idx_ptr: int, val_ptr: int, resid_ptr: Optional[int],
+                     workspace_ptr: int, workspace_bytes: int, cuda_stream: int) -> None:
+    _check(load_library().ef_topk_compress(v_ptr, n, k, idx_ptr, val_ptr, resid_ptr, workspace_ptr,
+                                           workspace_bytes, cuda_stream), "ef_topk_compress")
 
 
 def ef_stream_probe(mode: int, a_ptr: int, b_ptr: int, c_ptr: int, n: int, cuda_stream: int) -> None:

@@ -9,8 +9,9 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libef.so")
-SOURCES = [os.path.join(CSRC, "ef_lib.cu")]
-DEPS = SOURCES + [os.path.join(CSRC, "ef_kernels.cuh"), os.path.join(ROOT, "include", "ef.h")]
+SOURCES = [os.path.join(CSRC, n) for n in ("ef_lib.cu", "ef_vote.cu", "ef_topk.cu")]
+DEPS = SOURCES + [os.path.join(CSRC, "ef_kernels.cuh"), os.path.join(CSRC, "ef_internal.h"),
+                  os.path.join(ROOT, "include", "ef.h")]
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-lineinfo",

@@ -1,0 +1,123 @@
+// Internal to libef: workspace layout, the host context and small helpers shared by the
+// translation units of the library.  Not part of the interface (that is include/ef.h).
+#pragma once
+
+#include "../../include/ef.h"
+#include "ef_kernels.cuh"
+
+#include <cstddef>
+#include <cstdint>
+#include <vector>
+
+namespace efh {
+
+using efk::Block;
+using efk::Tile;
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
+
+// Rows of four elements per thread and chunk: a chunk is 1024*U elements (one CTA of the worker
+// and apply kernels), a tile is kTileChunks chunks (one CTA of the server kernel).
+constexpr int kU = 4;
+constexpr int kChunkLen = 1024 * kU;
+constexpr int kTileLen = kChunkLen * efk::kTileChunks;
+// Grids up to this many chunks (about two waves of CTAs) finalise block scales in-kernel.
+constexpr int64_t kFusedMaxChunks = 1024;
+
+struct Layout {
+    int64_t d = 0, W = 0;
+    int32_t B = 0, M = 0;
+    int64_t num_tiles = 0;
+    size_t dpad = 0, wpad = 0, bpad = 0, tpad = 0;    // padded element counts per sub-buffer
+    size_t off_x = 0, off_m = 0, off_pb = 0, off_spb = 0, off_words = 0, off_scales = 0,
+           off_rscale = 0, off_partials = 0, off_tickets = 0, off_tiles = 0, off_blocks = 0,
+           off_multi = 0, off_stage = 0, off_mt = 0, off_dpartials = 0, off_diag = 0, total = 0;
+    int32_t num_multi = 0;                            // blocks that span more than one chunk
+};
+
+}  // namespace efh
+
+struct ef_ctx {
+    efh::Layout L;
+    float mu = 0.f, eta = 0.f;
+    float eta_prev = 0.f;                  // stepsize of the last completed iteration
+    float lambda = 0.f;                    // weight decay (needs EF_FLAG_WEIGHT_DECAY)
+    uint32_t flags = 0;
+    char* ws = nullptr;
+    cudaStream_t stream = nullptr;
+    int64_t t = 0;
+    int64_t launches = 0;
+    int last_cuda = 0;
+    int pending = 0;                       // workers stepped in the current iteration
+    int mode = 0;                          // method of the current iteration (efh::kMode*)
+    std::vector<uint8_t> stepped;
+    std::vector<efk::Tile> h_tiles;             // kept alive: source of an asynchronous upload
+    std::vector<efk::Block> h_blocks;
+    std::vector<int32_t> h_multi;
+    int fused = 0;                         // block scales finalised inside the main kernels
+    // host-staging path
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_copied[2] = {nullptr, nullptr};
+    cudaEvent_t ev_free[2] = {nullptr, nullptr};
+    int64_t host_calls = 0;
+
+    float* x() const { return (float*)(ws + L.off_x); }
+    float* m(int i) const { return (float*)(ws + L.off_m) + (size_t)i * L.dpad; }
+    float* pb(int i) const {   // i == M: server
+        return i < L.M ? (float*)(ws + L.off_pb) + (size_t)i * L.dpad : (float*)(ws + L.off_spb);
+    }
+    uint32_t* words(int i) const { return (uint32_t*)(ws + L.off_words) + (size_t)i * L.wpad; }
+    float* scales(int i) const { return (float*)(ws + L.off_scales) + (size_t)i * L.bpad; }
+    float* rscale(int i) const { return (float*)(ws + L.off_rscale) + (size_t)i * L.bpad; }
+    double* partials(int i) const { return (double*)(ws + L.off_partials) + (size_t)i * L.tpad; }
+    unsigned* tickets(int i) const { return (unsigned*)(ws + L.off_tickets) + (size_t)i * L.bpad; }
+    const efk::Tile* tiles() const { return (const efk::Tile*)(ws + L.off_tiles); }
+    const efk::Block* blocks() const { return (const efk::Block*)(ws + L.off_blocks); }
+    const int* multi() const { return (const int*)(ws + L.off_multi); }
+    float* mt() const { return (float*)(ws + L.off_mt); }
+    double* dpartials(int i) const { return (double*)(ws + L.off_dpartials) + (size_t)i * 3 * L.tpad; }
+    double* diag(int i) const { return (double*)(ws + L.off_diag) + (size_t)i * 4 * L.bpad; }
+    float* stage(int s) const { return (float*)(ws + L.off_stage) + (size_t)s * L.dpad; }
+};
+
+namespace efh {
+
+// Which method the worker calls of the current iteration belong to: the two methods share the
+// context's momentum, parameter and packed-word buffers and must not be mixed inside one
+// iteration.
+enum { kModeNone = 0, kModeEF = 1, kModeVote = 2 };
+
+inline int cuda_fail(ef_ctx* c, cudaError_t e) {
+    if (c) c->last_cuda = (int)e;
+    return EF_ERR_CUDA;
+}
+#define EF_CUDA(c, call)                                         \
+    do {                                                         \
+        cudaError_t e_ = (call);                                 \
+        if (e_ != cudaSuccess) return efh::cuda_fail((c), e_);        \
+    } while (0)
+
+inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+// Common checks of a per-worker call of method `mode`.
+inline int check_worker_call(ef_ctx* c, int32_t i, const float* grad, int mode) {
+    if (!c || !grad || i < 0 || i >= c->L.M) return EF_ERR_INVALID_ARG;
+    if (c->stepped[i]) return EF_ERR_BAD_STATE;
+    if (c->pending > 0 && c->mode != mode) return EF_ERR_BAD_STATE;
+    return EF_OK;
+}
+inline void mark_stepped(ef_ctx* c, int32_t i, int mode) {
+    c->stepped[i] = 1; c->pending += 1; c->mode = mode;
+}
+inline void mark_all_stepped(ef_ctx* c, int mode) {
+    for (auto& v : c->stepped) v = 1;
+    c->pending = c->L.M; c->mode = mode;
+}
+inline void end_iteration(ef_ctx* c) {
+    for (auto& v : c->stepped) v = 0;
+    c->pending = 0; c->mode = kModeNone;
+    c->t += 1;
+}
+
+}  // namespace efh

@@ -932,7 +932,7 @@ __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
 // ------------------------------------------------------------------ residual materialisation
 // dst_j = p_j - s_b * sign(p_j): the residual e_{t+1} in its plain form (tests, checkpoints).
 // One tile per CTA.
-__global__ void __launch_bounds__(kThreads) ef_residual_kernel(const ResidualArgs a) {
+static __global__ void __launch_bounds__(kThreads) ef_residual_kernel(const ResidualArgs a) {
     const Tile t = a.tiles[blockIdx.x];
     const float s = a.rscale[t.block];
     for (int o = threadIdx.x; o < t.len; o += kThreads)
@@ -941,7 +941,7 @@ __global__ void __launch_bounds__(kThreads) ef_residual_kernel(const ResidualArg
 
 // Import of a residual (ef_set_state): adding +0 maps -0 to +0 and changes nothing else, which
 // keeps the "no -0 in a residual buffer" invariant of the sign-bit tests above.
-__global__ void __launch_bounds__(kThreads) ef_import_kernel(const float* __restrict__ src,
+static __global__ void __launch_bounds__(kThreads) ef_import_kernel(const float* __restrict__ src,
                                                              float* __restrict__ dst, long long n) {
     for (long long j = blockIdx.x * (long long)kThreads + threadIdx.x; j < n;
          j += (long long)gridDim.x * kThreads)

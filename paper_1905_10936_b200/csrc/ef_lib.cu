@@ -1,7 +1,6 @@
 // Host side of libef: argument checking, workspace layout, tile table, kernel launches.
 // The interface is documented in include/ef.h.
-#include "../../include/ef.h"
-#include "ef_kernels.cuh"
+#include "ef_internal.h"
 
 #include <algorithm>
 #include <cmath>
@@ -16,28 +15,7 @@ namespace {
 
 using efk::Block;
 using efk::Tile;
-
-constexpr size_t kAlign = 256;
-inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
-
-// Rows of four elements per thread and chunk: a chunk is 1024*U elements (one CTA of the worker
-// and apply kernels), a tile is kTileChunks chunks (one CTA of the server kernel).
-constexpr int kU = 4;
-constexpr int kChunkLen = 1024 * kU;
-constexpr int kTileLen = kChunkLen * efk::kTileChunks;
-// Grids up to this many chunks (about two waves of CTAs) finalise block scales in-kernel.
-constexpr int64_t kFusedMaxChunks = 1024;
-
-struct Layout {
-    int64_t d = 0, W = 0;
-    int32_t B = 0, M = 0;
-    int64_t num_tiles = 0;
-    size_t dpad = 0, wpad = 0, bpad = 0, tpad = 0;    // padded element counts per sub-buffer
-    size_t off_x = 0, off_m = 0, off_pb = 0, off_spb = 0, off_words = 0, off_scales = 0,
-           off_rscale = 0, off_partials = 0, off_tickets = 0, off_tiles = 0, off_blocks = 0,
-           off_multi = 0, off_stage = 0, off_mt = 0, off_dpartials = 0, off_diag = 0, total = 0;
-    int32_t num_multi = 0;                            // blocks that span more than one chunk
-};
+using namespace efh;
 
 int check_problem(int64_t d, int32_t B, const int64_t* offsets, int32_t M) {
     if (!offsets || d < 1 || B < 1 || M < 1 || M > EF_MAX_WORKERS) return EF_ERR_INVALID_ARG;
@@ -95,61 +73,7 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
 
 }  // namespace
 
-struct ef_ctx {
-    Layout L;
-    float mu = 0.f, eta = 0.f;
-    float eta_prev = 0.f;                  // stepsize of the last completed iteration
-    float lambda = 0.f;                    // weight decay (needs EF_FLAG_WEIGHT_DECAY)
-    uint32_t flags = 0;
-    char* ws = nullptr;
-    cudaStream_t stream = nullptr;
-    int64_t t = 0;
-    int64_t launches = 0;
-    int last_cuda = 0;
-    int pending = 0;                       // workers stepped in the current iteration
-    std::vector<uint8_t> stepped;
-    std::vector<Tile> h_tiles;             // kept alive: source of an asynchronous upload
-    std::vector<Block> h_blocks;
-    std::vector<int32_t> h_multi;
-    int fused = 0;                         // block scales finalised inside the main kernels
-    // host-staging path
-    cudaStream_t copy_stream = nullptr;
-    cudaEvent_t ev_copied[2] = {nullptr, nullptr};
-    cudaEvent_t ev_free[2] = {nullptr, nullptr};
-    int64_t host_calls = 0;
-
-    float* x() const { return (float*)(ws + L.off_x); }
-    float* m(int i) const { return (float*)(ws + L.off_m) + (size_t)i * L.dpad; }
-    float* pb(int i) const {   // i == M: server
-        return i < L.M ? (float*)(ws + L.off_pb) + (size_t)i * L.dpad : (float*)(ws + L.off_spb);
-    }
-    uint32_t* words(int i) const { return (uint32_t*)(ws + L.off_words) + (size_t)i * L.wpad; }
-    float* scales(int i) const { return (float*)(ws + L.off_scales) + (size_t)i * L.bpad; }
-    float* rscale(int i) const { return (float*)(ws + L.off_rscale) + (size_t)i * L.bpad; }
-    double* partials(int i) const { return (double*)(ws + L.off_partials) + (size_t)i * L.tpad; }
-    unsigned* tickets(int i) const { return (unsigned*)(ws + L.off_tickets) + (size_t)i * L.bpad; }
-    const Tile* tiles() const { return (const Tile*)(ws + L.off_tiles); }
-    const Block* blocks() const { return (const Block*)(ws + L.off_blocks); }
-    const int* multi() const { return (const int*)(ws + L.off_multi); }
-    float* mt() const { return (float*)(ws + L.off_mt); }
-    double* dpartials(int i) const { return (double*)(ws + L.off_dpartials) + (size_t)i * 3 * L.tpad; }
-    double* diag(int i) const { return (double*)(ws + L.off_diag) + (size_t)i * 4 * L.bpad; }
-    float* stage(int s) const { return (float*)(ws + L.off_stage) + (size_t)s * L.dpad; }
-};
-
 namespace {
-
-int cuda_fail(ef_ctx* c, cudaError_t e) {
-    if (c) c->last_cuda = (int)e;
-    return EF_ERR_CUDA;
-}
-#define EF_CUDA(c, call)                                         \
-    do {                                                         \
-        cudaError_t e_ = (call);                                 \
-        if (e_ != cudaSuccess) return cuda_fail((c), e_);        \
-    } while (0)
-
-inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
 // Non-fused mode: adds the partial sums of every block larger than one chunk of buffer set k
 // (worker k, or the server for k == M) after the kernel that produced them.
@@ -283,12 +207,6 @@ int launch_server(ef_ctx* c) {
     return EF_OK;
 }
 
-int check_worker_call(ef_ctx* c, int32_t i, const float* grad) {
-    if (!c || !grad || i < 0 || i >= c->L.M) return EF_ERR_INVALID_ARG;
-    if (c->stepped[i]) return EF_ERR_BAD_STATE;
-    return EF_OK;
-}
-
 }  // namespace
 
 extern "C" {
@@ -392,12 +310,12 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
 }
 
 int ef_worker_step(ef_ctx* c, int32_t i, const float* grad) {
-    int rc = check_worker_call(c, i, grad);
+    int rc = check_worker_call(c, i, grad, kModeEF);
     if (rc != EF_OK) return rc;
     if (!aligned16(grad)) return EF_ERR_ALIGNMENT;
     rc = launch_worker(c, i, grad);
     if (rc != EF_OK) return rc;
-    c->stepped[i] = 1; c->pending += 1;
+    mark_stepped(c, i, kModeEF);
     return EF_OK;
 }
 
@@ -407,13 +325,12 @@ int ef_worker_step_all(ef_ctx* c, const float* grads, int64_t stride) {
     if (c->pending != 0) return EF_ERR_BAD_STATE;
     const int rc = launch_worker(c, 0, grads, c->L.M, (long long)stride);
     if (rc != EF_OK) return rc;
-    std::fill(c->stepped.begin(), c->stepped.end(), (uint8_t)1);
-    c->pending = c->L.M;
+    mark_all_stepped(c, kModeEF);
     return EF_OK;
 }
 
 int ef_worker_step_host(ef_ctx* c, int32_t i, const float* grad) {
-    int rc = check_worker_call(c, i, grad);
+    int rc = check_worker_call(c, i, grad, kModeEF);
     if (rc != EF_OK) return rc;
     if (!(c->flags & EF_FLAG_HOST_STAGING)) return EF_ERR_BAD_STATE;
     const int s = (int)(c->host_calls & 1);
@@ -427,19 +344,17 @@ int ef_worker_step_host(ef_ctx* c, int32_t i, const float* grad) {
     if (rc != EF_OK) return rc;
     EF_CUDA(c, cudaEventRecord(c->ev_free[s], c->stream));
     c->host_calls += 1;
-    c->stepped[i] = 1; c->pending += 1;
+    mark_stepped(c, i, kModeEF);
     return EF_OK;
 }
 
 int ef_server_step(ef_ctx* c) {
     if (!c) return EF_ERR_INVALID_ARG;
-    if (c->pending != c->L.M) return EF_ERR_BAD_STATE;
+    if (c->pending != c->L.M || c->mode != kModeEF) return EF_ERR_BAD_STATE;
     const int rc = launch_server(c);
     if (rc != EF_OK) return rc;
-    std::fill(c->stepped.begin(), c->stepped.end(), (uint8_t)0);
-    c->pending = 0;
     c->eta_prev = c->eta;
-    c->t += 1;
+    end_iteration(c);
     return EF_OK;
 }
 

@@ -80,6 +80,20 @@ class EFEngine:
     def server_step(self) -> None:
         ef.ef_server_step(self.ctx)
 
+    # ---- signum with majority vote (same state, same packed layout) -------------------------
+    def vote_worker_step(self, i: int, grad: torch.Tensor) -> None:
+        assert grad.is_cuda and grad.dtype == torch.float32 and grad.numel() == self.d
+        assert grad.is_contiguous()
+        ef.ef_vote_worker_step(self.ctx, i, grad.data_ptr())
+
+    def vote_worker_step_all(self, grads: torch.Tensor) -> None:
+        assert grads.is_cuda and grads.dtype == torch.float32 and grads.dim() == 2
+        assert grads.shape[0] == self.M and grads.shape[1] >= self.d and grads.stride(1) == 1
+        ef.ef_vote_worker_step_all(self.ctx, grads.data_ptr(), grads.stride(0))
+
+    def vote_server_step(self) -> None:
+        ef.ef_vote_server_step(self.ctx)
+
     def worker_diagnostics(self, i: int) -> torch.Tensor:
         """[B, 4] float64 view: ||p_b||_1, ||p_b||_2^2, ||g_b||_1, ||g_b||_2^2 of worker i's last step."""
         return _as_tensor(ef.ef_worker_diagnostics(self.ctx, i), 4 * self.B, torch.float64,
