@@ -66,6 +66,12 @@ enum ef_status {
 #define EF_FLAG_FUSED_SCALE 2u     /* always complete the sums inside the main kernels */
 #define EF_FLAG_SPLIT_SCALE 4u     /* always use the follow-up kernel */
 #define EF_FLAG_WEIGHT_DECAY 8u    /* reserve the d-float decay momentum for ef_set_weight_decay */
+#define EF_FLAG_ONE_LOCAL_WORKER 32u /* this process is ONE worker of M (the paper's setting: one worker
+                                      per GPU) and the server of some block range: the workspace holds
+                                      the state of a single worker (index 0 in every per-worker call),
+                                      the other M-1 workers' messages arrive through
+                                      ef_server_step_range.  ef_server_step, ef_worker_step_all over M
+                                      gradients and the signum calls need all M workers locally. */
 #define EF_FLAG_DIAGNOSTICS 16u    /* worker steps also record per-block sums (ef_worker_diagnostics);
                                       implies the follow-up scale kernel, excludes EF_FLAG_FUSED_SCALE */
 
@@ -187,6 +193,45 @@ int ef_step_count(ef_ctx* ctx, int64_t* t /* out: completed iterations */);
 
 /* Number of kernels this context has launched so far (for launch accounting). */
 int64_t ef_launch_count(ef_ctx* ctx);
+
+/* ---- The parameter-server protocol in pieces (Algorithm 2 / Algorithm 4: each worker pushes
+ * Delta_{t,i} to the server and pulls Deltatilde_t; Section 4.2 sends "more parameter servers"
+ * to relieve the server and notes that sending a block's sign vector and its scale as two
+ * separate messages costs latency, and that they should be fused).  The server side of
+ * ef_server_step split by block range, plus the message format for the exchange:
+ *
+ * Fused message of a block range [b0, b1): block after block, one 32-bit unit holding the
+ * block's scale (a float) followed by the block's ceil(d_b/32) packed words; ef_message_units
+ * gives its length in 32-bit units.  Because blocks are laid out in order, the message of a
+ * sub-range is a contiguous slice of the message of a larger range: the slice for [c0, c1)
+ * starts ef_message_units(ctx, b0, c0) units into the message of [b0, b1) (0 for c0 == b0).
+ * A worker can therefore pack all its blocks once and send each server its slice; servers'
+ * update slices, concatenated in block order (an all-gather), form the whole update.
+ *
+ * ef_pack_message: writes the fused message of blocks [b0, b1) of worker `who`'s last worker
+ *   step (who = -1: of the server's last step on those blocks) to dst (device).
+ * ef_server_step_range: the server lines of Algorithm 4 on blocks [b0, b1) only:
+ *     ptilde = (1/M) sum_i Delta_i + etilde;  Deltatilde = C_B(ptilde);  etilde = ptilde - Deltatilde
+ *   msgs == NULL: the workers' messages are the context's own (all M workers local);
+ *   otherwise worker i's fused message for exactly the blocks [b0, b1) starts at
+ *   msgs + i * msg_stride (device; 32-bit units; this GPU's memory: receive buffers), i < M.
+ *   The result (words, scales of the range) is readable through ef_server_words/scales and
+ *   ef_pack_message(ctx, -1, ...).  The parameters are NOT updated.
+ * ef_apply_update: x <- x - eta Deltatilde on blocks [b0, b1) (with the weight-decay side path
+ *   if enabled); update == NULL: from the context's own server step on those blocks, otherwise
+ *   from a fused message for exactly the blocks [b0, b1) (device).
+ * Call order inside an iteration: all local workers stepped; then any sequence of
+ * ef_server_step_range on disjoint ranges and ef_apply_update on disjoint ranges; the iteration
+ * is complete (step count, stepsize bookkeeping) once ef_apply_update has covered every block.
+ * Covering [0, B) with msgs == NULL and update == NULL equals ef_server_step bit for bit.
+ * Errors: INVALID_ARG (range, null dst, msg_stride shorter than the message), BAD_STATE (workers
+ * not all stepped, a block served or applied twice in one iteration, update == NULL for a block
+ * this context has not served, msgs == NULL without all M workers local), CUDA. */
+int64_t ef_message_units(ef_ctx* ctx, int32_t b0, int32_t b1);      /* -1 on a bad range */
+int ef_pack_message(ef_ctx* ctx, int32_t who, int32_t b0, int32_t b1, uint32_t* dst /* device */);
+int ef_server_step_range(ef_ctx* ctx, int32_t b0, int32_t b1,
+                         const uint32_t* msgs /* device or NULL */, int64_t msg_stride);
+int ef_apply_update(ef_ctx* ctx, int32_t b0, int32_t b1, const uint32_t* update /* device or NULL */);
 
 /* ---- signum / signSGD with majority vote: the paper's comparison method (Section 1: only the
  * 1-bit gradient sign travels between workers and server, in both directions; baselines of

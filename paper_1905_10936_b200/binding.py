@@ -32,6 +32,7 @@ EF_FLAG_FUSED_SCALE = 2
 EF_FLAG_SPLIT_SCALE = 4
 EF_FLAG_WEIGHT_DECAY = 8
 EF_FLAG_DIAGNOSTICS = 16
+EF_FLAG_ONE_LOCAL_WORKER = 32
 EF_MAX_WORKERS = 4096
 EF_PROBE_3R2W, EF_PROBE_1R1W, EF_PROBE_COPY = 0, 1, 2
 
@@ -64,6 +65,10 @@ SIGNATURES = {
     "ef_step_count": (ctypes.c_int, [_vp, ctypes.POINTER(_i64)]),
     "ef_launch_count": (_i64, [_vp]),
     "ef_worker_step_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _f32, _vp, _vp, _vp]),
+    "ef_message_units": (_i64, [_vp, _i32, _i32]),
+    "ef_pack_message": (ctypes.c_int, [_vp, _i32, _i32, _i32, _vp]),
+    "ef_server_step_range": (ctypes.c_int, [_vp, _i32, _i32, _vp, _i64]),
+    "ef_apply_update": (ctypes.c_int, [_vp, _i32, _i32, _vp]),
     "ef_vote_worker_step": (ctypes.c_int, [_vp, _i32, _vp]),
     "ef_vote_worker_step_all": (ctypes.c_int, [_vp, _vp, _i64]),
     "ef_vote_server_step": (ctypes.c_int, [_vp]),
@@ -218,6 +223,22 @@ def ef_worker_step_noalloc(grad_ptr: int, momentum_ptr: int, residual_ptr: int,
     _check(load_library().ef_worker_step_noalloc(grad_ptr, momentum_ptr, residual_ptr,
                                                  residual_scale_ptr, n, mu, words_ptr, scale_ptr,
                                                  cuda_stream), "ef_worker_step_noalloc")
+
+
+def ef_message_units(ctx: int, b0: int, b1: int) -> int:
+    return load_library().ef_message_units(ctx, b0, b1)
+
+
+def ef_pack_message(ctx: int, who: int, b0: int, b1: int, dst_ptr: int) -> None:
+    _check(load_library().ef_pack_message(ctx, who, b0, b1, dst_ptr), "ef_pack_message")
+
+
+def ef_server_step_range(ctx: int, b0: int, b1: int, msgs_ptr: Optional[int], msg_stride: int) -> None:
+    _check(load_library().ef_server_step_range(ctx, b0, b1, msgs_ptr, msg_stride), "ef_server_step_range")
+
+
+def ef_apply_update(ctx: int, b0: int, b1: int, update_ptr: Optional[int]) -> None:
+    _check(load_library().ef_apply_update(ctx, b0, b1, update_ptr), "ef_apply_update")
 
 
 def ef_vote_worker_step(ctx: int, i: int, grad_ptr: int) -> None:

@@ -28,6 +28,8 @@ constexpr int64_t kFusedMaxChunks = 1024;
 struct Layout {
     int64_t d = 0, W = 0;
     int32_t B = 0, M = 0;
+    int32_t Ml = 0;                                   // worker state slots held here: M, or 1 with
+                                                      // EF_FLAG_ONE_LOCAL_WORKER; the server's buffers sit in slot Ml
     int64_t num_tiles = 0;
     size_t dpad = 0, wpad = 0, bpad = 0, tpad = 0;    // padded element counts per sub-buffer
     size_t off_x = 0, off_m = 0, off_pb = 0, off_spb = 0, off_words = 0, off_scales = 0,
@@ -52,6 +54,9 @@ struct ef_ctx {
     int pending = 0;                       // workers stepped in the current iteration
     int mode = 0;                          // method of the current iteration (efh::kMode*)
     std::vector<uint8_t> stepped;
+    // block-range calls (ef_server_step_range / ef_apply_update): what has been done in this iteration
+    std::vector<uint8_t> served, applied;
+    int32_t n_served = 0, n_applied = 0;
     std::vector<efk::Tile> h_tiles;             // kept alive: source of an asynchronous upload
     std::vector<efk::Block> h_blocks;
     std::vector<int32_t> h_multi;
@@ -64,8 +69,9 @@ struct ef_ctx {
 
     float* x() const { return (float*)(ws + L.off_x); }
     float* m(int i) const { return (float*)(ws + L.off_m) + (size_t)i * L.dpad; }
-    float* pb(int i) const {   // i == M: server
-        return i < L.M ? (float*)(ws + L.off_pb) + (size_t)i * L.dpad : (float*)(ws + L.off_spb);
+    int srv() const { return L.Ml; }            // slot of the server's buffers
+    float* pb(int i) const {   // i == srv(): server
+        return i < L.Ml ? (float*)(ws + L.off_pb) + (size_t)i * L.dpad : (float*)(ws + L.off_spb);
     }
     uint32_t* words(int i) const { return (uint32_t*)(ws + L.off_words) + (size_t)i * L.wpad; }
     float* scales(int i) const { return (float*)(ws + L.off_scales) + (size_t)i * L.bpad; }
@@ -102,7 +108,7 @@ inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
 // Common checks of a per-worker call of method `mode`.
 inline int check_worker_call(ef_ctx* c, int32_t i, const float* grad, int mode) {
-    if (!c || !grad || i < 0 || i >= c->L.M) return EF_ERR_INVALID_ARG;
+    if (!c || !grad || i < 0 || i >= c->L.Ml) return EF_ERR_INVALID_ARG;
     if (c->stepped[i]) return EF_ERR_BAD_STATE;
     if (c->pending > 0 && c->mode != mode) return EF_ERR_BAD_STATE;
     return EF_OK;
@@ -112,10 +118,13 @@ inline void mark_stepped(ef_ctx* c, int32_t i, int mode) {
 }
 inline void mark_all_stepped(ef_ctx* c, int mode) {
     for (auto& v : c->stepped) v = 1;
-    c->pending = c->L.M; c->mode = mode;
+    c->pending = c->L.Ml; c->mode = mode;
 }
 inline void end_iteration(ef_ctx* c) {
     for (auto& v : c->stepped) v = 0;
+    for (auto& v : c->served) v = 0;
+    for (auto& v : c->applied) v = 0;
+    c->n_served = c->n_applied = 0;
     c->pending = 0; c->mode = kModeNone;
     c->t += 1;
 }

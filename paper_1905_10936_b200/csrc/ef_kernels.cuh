@@ -97,7 +97,22 @@ struct ServerArgs {
     const Block* blocks;
     int fused;
     float ratio;             // eta_{t-1} / eta_t
+    // block-range launches: the grid covers tiles tile0 .. tile0 + gridDim.x - 1
+    int tile0;
+    // fused messages: worker i's packed words AND scales come from one buffer per worker,
+    // wwords + i*wstride, that holds the blocks from block `first` on as [scale | words] units
+    // (message_unit below); wscales is unused then
+    int fused_in;
+    long long msg_base;      // message_unit of the first block the buffers hold
 };
+
+// Fused message layout: the message of a block range [b0, b1) is, block after block, one 32-bit
+// unit holding the block's scale (a float) followed by the block's packed words.  The scale of
+// block b sits at unit (word_b + b) - (word_b0 + b0) and its words right behind it, where word_b
+// is the block's first packed word in the plain layout.
+__host__ __device__ __forceinline__ long long message_unit(long long block_word, int block) {
+    return block_word + block;
+}
 
 struct ScaleArgs {
     const double* partials;
@@ -113,9 +128,13 @@ struct ScaleArgs {
 
 struct ApplyArgs {
     float* x;
-    const uint32_t* words;   // server packed signs
-    const float* scales;     // server scales
+    const uint32_t* words;   // server packed signs (or a fused message, see ServerArgs)
+    const float* scales;     // server scales (unused with fused_in)
     const Tile* tiles;
+    const Block* blocks;
+    int tile0;
+    int fused_in;
+    long long msg_base;
     float eta;
     // weight decay kept out of the compressor (Appendix A); used by the DECAY instantiation only
     float* mt;               // decay momentum mtilde
@@ -530,9 +549,20 @@ __host__ __device__ constexpr int kLaneWorker(int q) {
 }
 __host__ __device__ constexpr int kLutEntries(int M) { return 1 << (M < kLutWorkers ? M : kLutWorkers); }
 
-__device__ __forceinline__ void build_scaled(const ServerArgs& a, int block, int M, float* s_c) {
-    for (int i = threadIdx.x; i < M; i += kThreads)
-        s_c[i] = __fdiv_rn(a.wscales[(long long)i * a.sstride + block], (float)M);
+__device__ __forceinline__ void build_scaled(const ServerArgs& a, const Tile& t, int M, float* s_c) {
+    if (a.fused_in) {
+        const long long unit = message_unit(a.blocks[t.block].word, t.block) - a.msg_base;
+        for (int i = threadIdx.x; i < M; i += kThreads)
+            s_c[i] = __fdiv_rn(__uint_as_float(__ldg(a.wwords + (long long)i * a.wstride + unit)), (float)M);
+    } else {
+        for (int i = threadIdx.x; i < M; i += kThreads)
+            s_c[i] = __fdiv_rn(a.wscales[(long long)i * a.sstride + t.block], (float)M);
+    }
+}
+
+// Where the packed words of tile t start in worker 0's buffer (plain layout, or a fused message).
+__device__ __forceinline__ const uint32_t* tile_words(const ServerArgs& a, const Tile& t) {
+    return a.wwords + (a.fused_in ? message_unit(t.word, t.block) + 1 - a.msg_base : t.word);
 }
 
 // s_base[idx] = (+-c_0) +- c_1 ... +- c_{T-1}, bit i of idx set = worker i negative, T = min(M, 6);
@@ -621,7 +651,7 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
 #pragma unroll
     for (int g = 0; g < G; ++g) {
         has_w[g] = wq + 8 * g < MT;
-        wbase[g] = a.wwords + (long long)(has_w[g] ? wq + 8 * g : 0) * a.wstride + t.word + (o0 >> 5);
+        wbase[g] = tile_words(a, t) + (long long)(has_w[g] ? wq + 8 * g : 0) * a.wstride + (o0 >> 5);
     }
     const int nfull = t.len / kChunk;              // chunks staged through shared memory
     const int tail = t.len - nfull * kChunk;       // ragged rest (only at the end of a block)
@@ -697,7 +727,7 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
     unsigned w[U][G];
 #pragma unroll
     for (int c = 0; c < kServerStages - 1; ++c) issue_chunk(c);   // in flight while the table is built
-    build_scaled(a, t.block, MT, s_c);
+    build_scaled(a, t, MT, s_c);
     __syncthreads();
     build_lut<MT>(s_c, s_base, s_lut);
 #pragma unroll
@@ -734,9 +764,8 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
 }
 
 // Direct evaluation for any M.
-__device__ __forceinline__ void average4(const ServerArgs& a, const float* s_c, long long wi,
+__device__ __forceinline__ void average4(const ServerArgs& a, const float* s_c, const uint32_t* wp,
                                          int sh, float (&avg)[4]) {
-    const uint32_t* wp = a.wwords + wi;
 #pragma unroll 4
     for (int i = 0; i < a.M; ++i) {
         const unsigned nib = __ldg(wp + (long long)i * a.wstride) >> sh;
@@ -765,7 +794,7 @@ __device__ __forceinline__ double server_rows(const ServerArgs& a, const Tile& t
     for (int u = 0; u < U; ++u) {
         const int o = o0 + u * 128;
         float avg[4] = {0.f, 0.f, 0.f, 0.f};
-        if (full || o < t.len) average4(a, s_c, t.word + (o >> 5), sh, avg);
+        if (full || o < t.len) average4(a, s_c, tile_words(a, t) + (o >> 5), sh, avg);
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             float pv = corrected_vector(a.ratio, a.ratio != 1.0f, residual_of(p[u][k], sp), avg[k]);   // ptilde_t
@@ -794,7 +823,7 @@ __device__ __forceinline__ double server_rows_scalar(const ServerArgs& a, const 
         if (valid) {
             float avg = 0.f;
             for (int i = 0; i < a.M; ++i) {
-                const unsigned w = __ldg(a.wwords + (long long)i * a.wstride + t.word + r);
+                const unsigned w = __ldg(tile_words(a, t) + (long long)i * a.wstride + r);
                 const float v = ((w >> lane) & 1u) ? -s_c[i] : s_c[i];
                 avg = (i == 0) ? v : __fadd_rn(avg, v);
             }
@@ -817,13 +846,13 @@ __global__ void __launch_bounds__(kThreads) ef_server_kernel(const ServerArgs a)
     float* s_c = reinterpret_cast<float*>(s_dyn + (MT > 0 ? server_ring_bytes<U>((MT + 7) / 8) : 0));
     __shared__ float s_base[MT > 0 ? kLutEntries(MT) : 1];
     __shared__ float s_lut[MT > 0 ? kLutEntries(MT) * kLutCopies : 1];
-    const Tile t = a.tiles[blockIdx.x];
+    const Tile t = a.tiles[blockIdx.x + a.tile0];
     const float sp = a.rscale[t.block];
     double acc = 0.0;
     if (MT > 0 && (t.start & 3) == 0) {
         acc = server_tile_lut<U, (MT > 0 ? MT : 1)>(a, t, sp, s_dyn, s_c, s_base, s_lut);
     } else {
-        build_scaled(a, t.block, a.M, s_c);
+        build_scaled(a, t, a.M, s_c);
         __syncthreads();
         if ((t.start & 3) != 0) {
             acc = server_rows_scalar(a, t, sp, s_c);
@@ -833,7 +862,7 @@ __global__ void __launch_bounds__(kThreads) ef_server_kernel(const ServerArgs a)
         }
     }
     const Block b = a.blocks[t.block];
-    finish_block(acc, (long long)blockIdx.x * kTileChunks, kTileChunks - 1, b.len <= 1024 * U,
+    finish_block(acc, (long long)(blockIdx.x + a.tile0) * kTileChunks, kTileChunks - 1, b.len <= 1024 * U,
                  (unsigned)b.tile_count, t.block, a.blocks, a.partials, a.tickets, a.scale_out,
                  a.rscale, a.fused);
 }
@@ -860,15 +889,22 @@ __device__ __forceinline__ float apply_one(const ApplyArgs& a, float x, float si
 template <int U, bool DECAY>
 __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
     constexpr int kChunk = 1024 * U;
-    const Tile t = a.tiles[blockIdx.x];
+    const Tile t = a.tiles[blockIdx.x + a.tile0];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // packed words of this tile and the block's scale: plain layout or a fused message
+    const uint32_t* const twords =
+        a.words + (a.fused_in ? message_unit(t.word, t.block) + 1 - a.msg_base : t.word);
+    const float* const scale_ptr =
+        a.fused_in ? reinterpret_cast<const float*>(a.words) +
+                         (message_unit(a.blocks[t.block].word, t.block) - a.msg_base)
+                   : a.scales + t.block;
     if ((t.start & 3) != 0) {
-        const float step = __fmul_rn(a.eta, a.scales[t.block]);
+        const float step = __fmul_rn(a.eta, *scale_ptr);
         const int rows = (t.len + 31) >> 5;
         for (int r = warp; r < rows; r += kWarps) {
             const int o = r * 32 + lane;
             if (o < t.len) {
-                const unsigned w = __ldg(a.words + t.word + r);
+                const unsigned w = __ldg(twords + r);
                 const long long j = t.start + o;
                 float mt = DECAY ? a.mt[j] : 0.f;
                 a.x[j] = apply_one<DECAY>(a, a.x[j], ((w >> lane) & 1u) ? -step : step, &mt);
@@ -881,7 +917,7 @@ __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
     const int sh = (lane & 7) * 4;
     float* const xbase = a.x + t.start + o0;
     float* const mbase = DECAY ? a.mt + t.start + o0 : nullptr;
-    const uint32_t* const wbase = a.words + t.word + (o0 >> 5);
+    const uint32_t* const wbase = twords + (o0 >> 5);
     const int nchunks = (t.len + kChunk - 1) / kChunk;
     constexpr int UM = DECAY ? U : 1;      // the decay momentum is only held when it is used
 
@@ -918,7 +954,7 @@ __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
     float xA[U][4], xB[U][4], mA[UM][4], mB[UM][4];
     unsigned nA[U], nB[U];
     load_chunk(0, xA, mA, nA);
-    step = __fmul_rn(a.eta, a.scales[t.block]);        // its latency overlaps the first loads
+    step = __fmul_rn(a.eta, *scale_ptr);               // its latency overlaps the first loads
     for (int c = 0; c < nchunks; c += 2) {
         if (c + 1 < nchunks) load_chunk(c + 1, xB, mB, nB);
         update_chunk(c, xA, mA, nA);
@@ -937,6 +973,27 @@ static __global__ void __launch_bounds__(kThreads) ef_residual_kernel(const Resi
     const float s = a.rscale[t.block];
     for (int o = threadIdx.x; o < t.len; o += kThreads)
         a.dst[t.start + o] = residual_of(a.pb[t.start + o], s);
+}
+
+// Fused message of a block range: dst gets, block after block, [scale | packed words].
+// One tile per CTA (a tile has at most kTileChunks*1024*U/32 words).
+struct PackArgs {
+    const uint32_t* words;
+    const float* scales;
+    uint32_t* dst;
+    const Tile* tiles;
+    const Block* blocks;
+    int tile0;
+    long long msg_base;
+};
+static __global__ void __launch_bounds__(kThreads) ef_pack_kernel(const PackArgs a) {
+    const Tile t = a.tiles[blockIdx.x + a.tile0];
+    const Block b = a.blocks[t.block];
+    uint32_t* dst = a.dst + (message_unit(t.word, t.block) + 1 - a.msg_base);
+    const int nwords = (t.len + 31) >> 5;
+    for (int k = threadIdx.x; k < nwords; k += kThreads) dst[k] = a.words[t.word + k];
+    if (threadIdx.x == 0 && t.start == b.start)
+        a.dst[message_unit(b.word, t.block) - a.msg_base] = __float_as_uint(a.scales[t.block]);
 }
 
 // Import of a residual (ef_set_state): adding +0 maps -0 to +0 and changes nothing else, which

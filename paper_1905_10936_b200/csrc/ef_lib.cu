@@ -30,11 +30,12 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
     int rc = check_problem(d, B, offsets, M);
     if (rc != EF_OK) return rc;
     if (flags & ~(EF_FLAG_HOST_STAGING | EF_FLAG_FUSED_SCALE | EF_FLAG_SPLIT_SCALE |
-                  EF_FLAG_WEIGHT_DECAY | EF_FLAG_DIAGNOSTICS))
+                  EF_FLAG_WEIGHT_DECAY | EF_FLAG_DIAGNOSTICS | EF_FLAG_ONE_LOCAL_WORKER))
         return EF_ERR_INVALID_ARG;
     if ((flags & EF_FLAG_FUSED_SCALE) && (flags & (EF_FLAG_SPLIT_SCALE | EF_FLAG_DIAGNOSTICS)))
         return EF_ERR_INVALID_ARG;
     L->d = d; L->B = B; L->M = M;
+    L->Ml = (flags & EF_FLAG_ONE_LOCAL_WORKER) ? 1 : M;
     int64_t W = 0, T = 0;
     for (int32_t b = 0; b < B; ++b) {
         const int64_t db = offsets[b + 1] - offsets[b];
@@ -48,11 +49,11 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
     L->wpad = align_up((size_t)W * 4) / 4;
     L->bpad = align_up((size_t)B * 4) / 4;
     L->tpad = align_up((size_t)T * efk::kTileChunks * 8) / 8;   // partial-sum slots
-    const size_t M1 = (size_t)M + 1;
+    const size_t Ml = (size_t)L->Ml, M1 = Ml + 1;
     size_t o = 0;
     L->off_x = o;        o += L->dpad * 4;
-    L->off_m = o;        o += (size_t)M * L->dpad * 4;
-    L->off_pb = o;       o += (size_t)M * L->dpad * 4;
+    L->off_m = o;        o += Ml * L->dpad * 4;
+    L->off_pb = o;       o += Ml * L->dpad * 4;
     L->off_spb = o;      o += L->dpad * 4;
     L->off_mt = o;       if (flags & EF_FLAG_WEIGHT_DECAY) o += L->dpad * 4;
     L->off_words = o;    o += M1 * L->wpad * 4;
@@ -60,8 +61,8 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
     L->off_rscale = o;   o += M1 * L->bpad * 4;
     L->off_partials = o; o += M1 * L->tpad * 8;
     L->off_tickets = o;  o += M1 * L->bpad * 4;
-    L->off_dpartials = o; if (flags & EF_FLAG_DIAGNOSTICS) o += (size_t)M * 3 * L->tpad * 8;
-    L->off_diag = o;      if (flags & EF_FLAG_DIAGNOSTICS) o += (size_t)M * 4 * L->bpad * 8;
+    L->off_dpartials = o; if (flags & EF_FLAG_DIAGNOSTICS) o += Ml * 3 * L->tpad * 8;
+    L->off_diag = o;      if (flags & EF_FLAG_DIAGNOSTICS) o += Ml * 4 * L->bpad * 8;
     L->off_tiles = o;    o += align_up((size_t)T * sizeof(Tile));
     L->off_blocks = o;   o += align_up((size_t)B * sizeof(Block));
     L->off_multi = o;    o += align_up((size_t)L->num_multi * sizeof(int32_t) + 4);
@@ -83,7 +84,7 @@ int launch_scale(ef_ctx* c, int k, int count = 1) {
     a.partials = c->partials(k); a.blocks = c->blocks(); a.multi = c->multi();
     a.scale_out = c->scales(k); a.rscale = c->rscale(k);
     a.partial_stride = (long long)c->L.tpad; a.scale_stride = (int)c->L.bpad;
-    const bool diag = (c->flags & EF_FLAG_DIAGNOSTICS) && k < c->L.M;
+    const bool diag = (c->flags & EF_FLAG_DIAGNOSTICS) && k < c->L.Ml;
     a.dpartials = diag ? c->dpartials(k) : nullptr;
     a.diag = diag ? c->diag(k) : nullptr;
     const dim3 grid((unsigned)c->L.num_multi, (unsigned)count);
@@ -153,58 +154,105 @@ cudaError_t prepare_server(int M) {
     }
 }
 
+// Range of tiles that covers the blocks [b0, b1).
+struct TileRange { int tile0; unsigned count; };
+TileRange tiles_of(const ef_ctx* c, int b0, int b1) {
+    const int t0 = c->h_blocks[b0].tile_begin;
+    const int t1 = c->h_blocks[b1 - 1].tile_begin + c->h_blocks[b1 - 1].tile_count;
+    return {t0, (unsigned)(t1 - t0)};
+}
+
 template <int MT>
-cudaError_t launch_server_t(ef_ctx* c, const efk::ServerArgs& a) {
-    efk::ef_server_kernel<kU, MT><<<(unsigned)c->L.num_tiles, efk::kThreads,
-                                    server_smem_bytes<MT>(c->L.M), c->stream>>>(a);
+cudaError_t launch_server_t(ef_ctx* c, const efk::ServerArgs& a, unsigned grid) {
+    efk::ef_server_kernel<kU, MT><<<grid, efk::kThreads, server_smem_bytes<MT>(c->L.M), c->stream>>>(a);
     return cudaGetLastError();
 }
 
-int launch_server(ef_ctx* c) {
-    const int M = c->L.M;
+// Server lines of Algorithm 4 on the blocks [b0, b1).  msgs == nullptr: the workers' words and
+// scales are the context's own; otherwise worker i's fused message for exactly this block range
+// starts at msgs + i * msg_stride.
+int launch_server_range(ef_ctx* c, int b0, int b1, const uint32_t* msgs, long long msg_stride) {
+    const int M = c->L.M, S = c->srv();
+    const TileRange tr = tiles_of(c, b0, b1);
     efk::ServerArgs a;
-    a.wwords = c->words(0); a.wstride = (long long)c->L.wpad;
+    a.wwords = msgs ? msgs : c->words(0);
+    a.wstride = msgs ? msg_stride : (long long)c->L.wpad;
     a.wscales = c->scales(0); a.sstride = (int)c->L.bpad; a.M = M;
-    a.pb = c->pb(M); a.words = c->words(M); a.scale_out = c->scales(M); a.rscale = c->rscale(M);
-    a.partials = c->partials(M); a.tickets = c->tickets(M);
+    a.pb = c->pb(S); a.words = c->words(S); a.scale_out = c->scales(S); a.rscale = c->rscale(S);
+    a.partials = c->partials(S); a.tickets = c->tickets(S);
     a.tiles = c->tiles(); a.blocks = c->blocks(); a.fused = c->fused;
     a.ratio = c->eta_prev / c->eta;
+    a.tile0 = tr.tile0;
+    a.fused_in = msgs ? 1 : 0;
+    a.msg_base = efk::message_unit(c->h_blocks[b0].word, b0);
     cudaError_t le;
     switch (M) {
-        case 1: le = launch_server_t<1>(c, a); break;
-        case 2: le = launch_server_t<2>(c, a); break;
-        case 3: le = launch_server_t<3>(c, a); break;
-        case 4: le = launch_server_t<4>(c, a); break;
-        case 5: le = launch_server_t<5>(c, a); break;
-        case 6: le = launch_server_t<6>(c, a); break;
-        case 7: le = launch_server_t<7>(c, a); break;
-        case 8: le = launch_server_t<8>(c, a); break;
-        case 9: le = launch_server_t<9>(c, a); break;
-        case 10: le = launch_server_t<10>(c, a); break;
-        case 11: le = launch_server_t<11>(c, a); break;
-        case 12: le = launch_server_t<12>(c, a); break;
-        case 13: le = launch_server_t<13>(c, a); break;
-        case 14: le = launch_server_t<14>(c, a); break;
-        case 15: le = launch_server_t<15>(c, a); break;
-        case 16: le = launch_server_t<16>(c, a); break;
-        default: le = launch_server_t<0>(c, a); break;
+        case 1: le = launch_server_t<1>(c, a, tr.count); break;
+        case 2: le = launch_server_t<2>(c, a, tr.count); break;
+        case 3: le = launch_server_t<3>(c, a, tr.count); break;
+        case 4: le = launch_server_t<4>(c, a, tr.count); break;
+        case 5: le = launch_server_t<5>(c, a, tr.count); break;
+        case 6: le = launch_server_t<6>(c, a, tr.count); break;
+        case 7: le = launch_server_t<7>(c, a, tr.count); break;
+        case 8: le = launch_server_t<8>(c, a, tr.count); break;
+        case 9: le = launch_server_t<9>(c, a, tr.count); break;
+        case 10: le = launch_server_t<10>(c, a, tr.count); break;
+        case 11: le = launch_server_t<11>(c, a, tr.count); break;
+        case 12: le = launch_server_t<12>(c, a, tr.count); break;
+        case 13: le = launch_server_t<13>(c, a, tr.count); break;
+        case 14: le = launch_server_t<14>(c, a, tr.count); break;
+        case 15: le = launch_server_t<15>(c, a, tr.count); break;
+        case 16: le = launch_server_t<16>(c, a, tr.count); break;
+        default: le = launch_server_t<0>(c, a, tr.count); break;
     }
     EF_CUDA(c, le);
     c->launches += 1;
-    {
-        const int rc = launch_scale(c, M);
-        if (rc != EF_OK) return rc;
+    if (!c->fused && c->L.num_multi > 0) {
+        // follow-up sums for the blocks of the range that span more than one chunk
+        const auto lo = std::lower_bound(c->h_multi.begin(), c->h_multi.end(), b0) - c->h_multi.begin();
+        const auto hi = std::lower_bound(c->h_multi.begin(), c->h_multi.end(), b1) - c->h_multi.begin();
+        if (hi > lo) {
+            efk::ScaleArgs sa;
+            sa.partials = c->partials(S); sa.blocks = c->blocks(); sa.multi = c->multi() + lo;
+            sa.scale_out = c->scales(S); sa.rscale = c->rscale(S);
+            sa.partial_stride = (long long)c->L.tpad; sa.scale_stride = (int)c->L.bpad;
+            sa.dpartials = nullptr; sa.diag = nullptr;
+            efk::ef_scale_kernel<false><<<dim3((unsigned)(hi - lo), 1), efk::kThreads, 0, c->stream>>>(sa);
+            EF_CUDA(c, cudaGetLastError());
+            c->launches += 1;
+        }
     }
+    return EF_OK;
+}
+
+// x_{t+1} = x_t - eta Deltatilde_t on the blocks [b0, b1); the update is the context's own
+// server message (update == nullptr) or a fused message for exactly this block range.
+int launch_apply_range(ef_ctx* c, int b0, int b1, const uint32_t* update) {
+    const int S = c->srv();
+    const TileRange tr = tiles_of(c, b0, b1);
     efk::ApplyArgs p;
-    p.x = c->x(); p.words = c->words(M); p.scales = c->scales(M); p.tiles = c->tiles();
+    p.x = c->x(); p.words = update ? update : c->words(S); p.scales = c->scales(S);
+    p.tiles = c->tiles(); p.blocks = c->blocks(); p.tile0 = tr.tile0;
+    p.fused_in = update ? 1 : 0;
+    p.msg_base = efk::message_unit(c->h_blocks[b0].word, b0);
     p.eta = c->eta; p.mu = c->mu; p.lambda = c->lambda; p.mt = c->mt();
     if (c->lambda > 0.f)
-        efk::ef_apply_kernel<kU, true><<<(unsigned)c->L.num_tiles, efk::kThreads, 0, c->stream>>>(p);
+        efk::ef_apply_kernel<kU, true><<<tr.count, efk::kThreads, 0, c->stream>>>(p);
     else
-        efk::ef_apply_kernel<kU, false><<<(unsigned)c->L.num_tiles, efk::kThreads, 0, c->stream>>>(p);
+        efk::ef_apply_kernel<kU, false><<<tr.count, efk::kThreads, 0, c->stream>>>(p);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
     return EF_OK;
+}
+
+int launch_server(ef_ctx* c) {
+    const int rc = launch_server_range(c, 0, c->L.B, nullptr, 0);
+    if (rc != EF_OK) return rc;
+    return launch_apply_range(c, 0, c->L.B, nullptr);
+}
+
+int check_block_range(const ef_ctx* c, int32_t b0, int32_t b1) {
+    return (c && b0 >= 0 && b0 < b1 && b1 <= c->L.B) ? EF_OK : EF_ERR_INVALID_ARG;
 }
 
 }  // namespace
@@ -248,7 +296,9 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
     c->ws = (char*)workspace;
     c->stream = (cudaStream_t)cuda_stream;
     try {
-    c->stepped.assign(M, 0);
+    c->stepped.assign(L.Ml, 0);
+    c->served.assign(B, 0);
+    c->applied.assign(B, 0);
 
     // tile and block tables
     c->h_tiles.reserve((size_t)L.num_tiles);
@@ -323,7 +373,7 @@ int ef_worker_step_all(ef_ctx* c, const float* grads, int64_t stride) {
     if (!c || !grads || stride < c->L.d) return EF_ERR_INVALID_ARG;
     if (!aligned16(grads) || (stride & 3) != 0) return EF_ERR_ALIGNMENT;
     if (c->pending != 0) return EF_ERR_BAD_STATE;
-    const int rc = launch_worker(c, 0, grads, c->L.M, (long long)stride);
+    const int rc = launch_worker(c, 0, grads, c->L.Ml, (long long)stride);
     if (rc != EF_OK) return rc;
     mark_all_stepped(c, kModeEF);
     return EF_OK;
@@ -350,11 +400,63 @@ int ef_worker_step_host(ef_ctx* c, int32_t i, const float* grad) {
 
 int ef_server_step(ef_ctx* c) {
     if (!c) return EF_ERR_INVALID_ARG;
-    if (c->pending != c->L.M || c->mode != kModeEF) return EF_ERR_BAD_STATE;
+    if (c->pending != c->L.M || c->L.Ml != c->L.M || c->mode != kModeEF) return EF_ERR_BAD_STATE;
+    if (c->n_served != 0 || c->n_applied != 0) return EF_ERR_BAD_STATE;   // finish the range calls instead
     const int rc = launch_server(c);
     if (rc != EF_OK) return rc;
     c->eta_prev = c->eta;
     end_iteration(c);
+    return EF_OK;
+}
+
+int64_t ef_message_units(ef_ctx* c, int32_t b0, int32_t b1) {
+    if (check_block_range(c, b0, b1) != EF_OK) return -1;
+    return efk::message_unit(c->h_blocks[b1 - 1].word + (c->h_blocks[b1 - 1].len + 31) / 32, b1) -
+           efk::message_unit(c->h_blocks[b0].word, b0);
+}
+
+int ef_pack_message(ef_ctx* c, int32_t who, int32_t b0, int32_t b1, uint32_t* dst) {
+    if (check_block_range(c, b0, b1) != EF_OK || !dst || who < -1 || who >= c->L.Ml)
+        return EF_ERR_INVALID_ARG;
+    const int k = who < 0 ? c->srv() : who;
+    const TileRange tr = tiles_of(c, b0, b1);
+    efk::PackArgs a;
+    a.words = c->words(k); a.scales = c->scales(k); a.dst = dst;
+    a.tiles = c->tiles(); a.blocks = c->blocks(); a.tile0 = tr.tile0;
+    a.msg_base = efk::message_unit(c->h_blocks[b0].word, b0);
+    efk::ef_pack_kernel<<<tr.count, efk::kThreads, 0, c->stream>>>(a);
+    EF_CUDA(c, cudaGetLastError());
+    c->launches += 1;
+    return EF_OK;
+}
+
+int ef_server_step_range(ef_ctx* c, int32_t b0, int32_t b1, const uint32_t* msgs, int64_t msg_stride) {
+    if (check_block_range(c, b0, b1) != EF_OK) return EF_ERR_INVALID_ARG;
+    if (c->pending != c->L.Ml || c->mode != kModeEF) return EF_ERR_BAD_STATE;
+    if (!msgs && c->L.Ml != c->L.M) return EF_ERR_BAD_STATE;     // the other workers' messages are needed
+    if (msgs && c->L.M > 1 && msg_stride < ef_message_units(c, b0, b1)) return EF_ERR_INVALID_ARG;
+    for (int32_t b = b0; b < b1; ++b)
+        if (c->served[b]) return EF_ERR_BAD_STATE;
+    const int rc = launch_server_range(c, b0, b1, msgs, (long long)msg_stride);
+    if (rc != EF_OK) return rc;
+    for (int32_t b = b0; b < b1; ++b) c->served[b] = 1;
+    c->n_served += b1 - b0;
+    return EF_OK;
+}
+
+int ef_apply_update(ef_ctx* c, int32_t b0, int32_t b1, const uint32_t* update) {
+    if (check_block_range(c, b0, b1) != EF_OK) return EF_ERR_INVALID_ARG;
+    if (c->pending != c->L.Ml || c->mode != kModeEF) return EF_ERR_BAD_STATE;
+    for (int32_t b = b0; b < b1; ++b)
+        if (c->applied[b] || (!update && !c->served[b])) return EF_ERR_BAD_STATE;
+    const int rc = launch_apply_range(c, b0, b1, update);
+    if (rc != EF_OK) return rc;
+    for (int32_t b = b0; b < b1; ++b) c->applied[b] = 1;
+    c->n_applied += b1 - b0;
+    if (c->n_applied == c->L.B) {        // every block has its update: the iteration is complete
+        c->eta_prev = c->eta;
+        end_iteration(c);
+    }
     return EF_OK;
 }
 
@@ -373,7 +475,7 @@ int ef_set_weight_decay(ef_ctx* c, float lambda) {
 }
 
 const double* ef_worker_diagnostics(ef_ctx* c, int32_t i) {
-    return (c && (c->flags & EF_FLAG_DIAGNOSTICS) && i >= 0 && i < c->L.M) ? c->diag(i) : nullptr;
+    return (c && (c->flags & EF_FLAG_DIAGNOSTICS) && i >= 0 && i < c->L.Ml) ? c->diag(i) : nullptr;
 }
 
 float* ef_decay_momentum(ef_ctx* c) {
@@ -382,7 +484,7 @@ float* ef_decay_momentum(ef_ctx* c) {
 
 int ef_read_update_host(ef_ctx* c, uint32_t* words, float* scales) {
     if (!c || !words || !scales) return EF_ERR_INVALID_ARG;
-    const int M = c->L.M;
+    const int M = c->srv();
     EF_CUDA(c, cudaMemcpyAsync(words, c->words(M), (size_t)c->L.W * 4, cudaMemcpyDeviceToHost,
                                c->stream));
     EF_CUDA(c, cudaMemcpyAsync(scales, c->scales(M), (size_t)c->L.B * 4, cudaMemcpyDeviceToHost,
@@ -391,18 +493,18 @@ int ef_read_update_host(ef_ctx* c, uint32_t* words, float* scales) {
 }
 
 const uint32_t* ef_worker_words(ef_ctx* c, int32_t i) {
-    return (c && i >= 0 && i < c->L.M) ? c->words(i) : nullptr;
+    return (c && i >= 0 && i < c->L.Ml) ? c->words(i) : nullptr;
 }
 const float* ef_worker_scales(ef_ctx* c, int32_t i) {
-    return (c && i >= 0 && i < c->L.M) ? c->scales(i) : nullptr;
+    return (c && i >= 0 && i < c->L.Ml) ? c->scales(i) : nullptr;
 }
-const uint32_t* ef_server_words(ef_ctx* c) { return c ? c->words(c->L.M) : nullptr; }
-const float* ef_server_scales(ef_ctx* c) { return c ? c->scales(c->L.M) : nullptr; }
+const uint32_t* ef_server_words(ef_ctx* c) { return c ? c->words(c->srv()) : nullptr; }
+const float* ef_server_scales(ef_ctx* c) { return c ? c->scales(c->srv()) : nullptr; }
 float* ef_params(ef_ctx* c) { return c ? c->x() : nullptr; }
 int64_t ef_num_words(ef_ctx* c) { return c ? c->L.W : -1; }
 
 int ef_get_momentum(ef_ctx* c, int32_t i, float* dst) {
-    if (!c || !dst || i < 0 || i >= c->L.M) return EF_ERR_INVALID_ARG;
+    if (!c || !dst || i < 0 || i >= c->L.Ml) return EF_ERR_INVALID_ARG;
     if (!aligned16(dst)) return EF_ERR_ALIGNMENT;
     EF_CUDA(c, cudaMemcpyAsync(dst, c->m(i), (size_t)c->L.d * 4, cudaMemcpyDeviceToDevice,
                                c->stream));
@@ -410,9 +512,9 @@ int ef_get_momentum(ef_ctx* c, int32_t i, float* dst) {
 }
 
 int ef_get_residual(ef_ctx* c, int32_t i, float* dst) {
-    if (!c || !dst || i < -1 || i >= c->L.M) return EF_ERR_INVALID_ARG;
+    if (!c || !dst || i < -1 || i >= c->L.Ml) return EF_ERR_INVALID_ARG;
     if (!aligned16(dst)) return EF_ERR_ALIGNMENT;
-    const int k = (i < 0) ? c->L.M : i;
+    const int k = (i < 0) ? c->srv() : i;
     efk::ResidualArgs a;
     a.pb = c->pb(k); a.rscale = c->rscale(k); a.dst = dst; a.tiles = c->tiles();
     efk::ef_residual_kernel<<<(unsigned)c->L.num_tiles, efk::kThreads, 0, c->stream>>>(a);
@@ -422,11 +524,11 @@ int ef_get_residual(ef_ctx* c, int32_t i, float* dst) {
 }
 
 int ef_set_state(ef_ctx* c, int32_t i, const float* momentum, const float* residual) {
-    if (!c || !residual || i < -1 || i >= c->L.M) return EF_ERR_INVALID_ARG;
+    if (!c || !residual || i < -1 || i >= c->L.Ml) return EF_ERR_INVALID_ARG;
     if (i >= 0 && !momentum) return EF_ERR_INVALID_ARG;
     if (!aligned16(residual) || (momentum && !aligned16(momentum))) return EF_ERR_ALIGNMENT;
     if (c->pending != 0) return EF_ERR_BAD_STATE;
-    const int k = (i < 0) ? c->L.M : i;
+    const int k = (i < 0) ? c->srv() : i;
     const size_t nbytes = (size_t)c->L.d * 4;
     if (i >= 0)
         EF_CUDA(c, cudaMemcpyAsync(c->m(i), momentum, nbytes, cudaMemcpyDeviceToDevice, c->stream));

@@ -255,7 +255,7 @@ int ef_vote_worker_step_all(ef_ctx* c, const float* grads, int64_t stride) {
     if (!c || !grads || stride < c->L.d) return EF_ERR_INVALID_ARG;
     if (!aligned16(grads) || (stride & 3) != 0) return EF_ERR_ALIGNMENT;
     if (c->pending != 0) return EF_ERR_BAD_STATE;
-    const int rc = launch_vote_worker(c, 0, grads, c->L.M, (long long)stride);
+    const int rc = launch_vote_worker(c, 0, grads, c->L.Ml, (long long)stride);
     if (rc != EF_OK) return rc;
     mark_all_stepped(c, kModeVote);
     return EF_OK;
@@ -263,12 +263,12 @@ int ef_vote_worker_step_all(ef_ctx* c, const float* grads, int64_t stride) {
 
 int ef_vote_server_step(ef_ctx* c) {
     if (!c) return EF_ERR_INVALID_ARG;
-    if (c->pending != c->L.M || c->mode != kModeVote) return EF_ERR_BAD_STATE;
+    if (c->pending != c->L.M || c->mode != kModeVote) return EF_ERR_BAD_STATE;   // needs all M workers local
     const int M = c->L.M;
     VoteServerArgs a;
     a.wwords = c->words(0); a.wstride = (long long)c->L.wpad; a.M = M;
     a.threshold = (unsigned)(M / 2 + 1);
-    a.words = c->words(M); a.x = c->x(); a.tiles = c->tiles(); a.eta = c->eta;
+    a.words = c->words(c->srv()); a.x = c->x(); a.tiles = c->tiles(); a.eta = c->eta;
     switch (planes_for(M)) {
         case 1: launch_vote_server_t<1>(c, a); break;
         case 2: launch_vote_server_t<2>(c, a); break;

@@ -28,7 +28,9 @@ class EFEngine:
     """One dist-EF-blockSGDM problem on the current CUDA device."""
 
     def __init__(self, offsets, M: int, mu: float, eta: float, host_staging: bool = False,
-                 scale_mode: str = "auto", weight_decay: bool = False, diagnostics: bool = False, stream: Optional[torch.cuda.Stream] = None, device: Optional[torch.device] = None):
+                 scale_mode: str = "auto", weight_decay: bool = False, diagnostics: bool = False,
+                 stream: Optional[torch.cuda.Stream] = None, device: Optional[torch.device] = None,
+                 one_local_worker: bool = False):
         if not torch.cuda.is_available():
             raise RuntimeError("EFEngine needs a CUDA device (there is no CPU path)")
         self.device = torch.device(device if device is not None else f"cuda:{torch.cuda.current_device()}")
@@ -39,6 +41,8 @@ class EFEngine:
         flags = ef.EF_FLAG_HOST_STAGING if host_staging else 0
         flags |= ef.EF_FLAG_WEIGHT_DECAY if weight_decay else 0
         flags |= ef.EF_FLAG_DIAGNOSTICS if diagnostics else 0
+        flags |= ef.EF_FLAG_ONE_LOCAL_WORKER if one_local_worker else 0
+        self.local_workers = 1 if one_local_worker else self.M
         flags |= {"auto": 0, "fused": ef.EF_FLAG_FUSED_SCALE, "split": ef.EF_FLAG_SPLIT_SCALE}[scale_mode]
         nbytes = ef.ef_workspace_bytes(self.d, self.B, self.offsets, self.M, flags)
         self.workspace_bytes = nbytes
@@ -79,6 +83,30 @@ class EFEngine:
 
     def server_step(self) -> None:
         ef.ef_server_step(self.ctx)
+
+    # ---- parameter-server protocol in pieces (block ranges, fused messages) -------------------
+    def message_units(self, b0: int, b1: int) -> int:
+        return ef.ef_message_units(self.ctx, b0, b1)
+
+    def pack_message(self, who: int, b0: int, b1: int, dst: torch.Tensor) -> None:
+        assert dst.is_cuda and dst.dtype == torch.int32 and dst.is_contiguous()
+        assert dst.numel() >= self.message_units(b0, b1)
+        ef.ef_pack_message(self.ctx, who, b0, b1, dst.data_ptr())
+
+    def server_step_range(self, b0: int, b1: int, msgs: Optional[torch.Tensor] = None) -> None:
+        """msgs: [M, units] int32 on this device, row i = worker i's fused message for [b0, b1)."""
+        if msgs is None:
+            ef.ef_server_step_range(self.ctx, b0, b1, None, 0)
+        else:
+            assert msgs.is_cuda and msgs.dtype == torch.int32 and msgs.dim() == 2
+            assert msgs.shape[0] == self.M and msgs.stride(1) == 1
+            ef.ef_server_step_range(self.ctx, b0, b1, msgs.data_ptr(), msgs.stride(0))
+
+    def apply_update(self, b0: int, b1: int, update: Optional[torch.Tensor] = None) -> None:
+        if update is not None:
+            assert update.is_cuda and update.dtype == torch.int32 and update.is_contiguous()
+            assert update.numel() >= self.message_units(b0, b1)
+        ef.ef_apply_update(self.ctx, b0, b1, update.data_ptr() if update is not None else None)
 
     # ---- signum with majority vote (same state, same packed layout) -------------------------
     def vote_worker_step(self, i: int, grad: torch.Tensor) -> None:
