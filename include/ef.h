@@ -52,7 +52,7 @@ enum ef_status {
     EF_ERR_ALIGNMENT = 4,          /* a device pointer is not 16-byte aligned */
     EF_ERR_CUDA = 5,               /* a CUDA runtime call failed; see ef_last_cuda_error */
     EF_ERR_UNSUPPORTED_DEVICE = 6, /* current device is not compute capability 10.x */
-    EF_ERR_TIMEOUT = 7,            /* reserved: a bounded device-side wait gave up */
+    EF_ERR_TIMEOUT = 7,            /* a bounded device-side wait gave up (reported by ef_check_status) */
     EF_ERR_TOO_LARGE = 8,          /* ef_worker_step_noalloc: n exceeds EF_NOALLOC_MAX_ELEMS */
     EF_ERR_NO_MEMORY = 9           /* a host allocation failed (the library allocates no device memory) */
 };
@@ -72,6 +72,17 @@ enum ef_status {
                                       the other M-1 workers' messages arrive through
                                       ef_server_step_range.  ef_server_step, ef_worker_step_all over M
                                       gradients and the signum calls need all M workers locally. */
+/* Variants of the server kernel.  By default the library picks what measured fastest on B200
+ * for the layout and M; these flags force a choice (for comparisons).  All variants compute the
+ * same values; only the grouping of the fp64 partial sums differs between TILES and STREAM, which
+ * can change the last bit of a scale in rare cases. */
+#define EF_FLAG_SERVER_TILES 64u     /* large layouts: one CTA per 16384-element tile */
+#define EF_FLAG_SERVER_STREAM 128u   /* large layouts: persistent one-wave kernel, each CTA walks a
+                                      balanced run of consecutive chunks (M <= 16) */
+#define EF_FLAG_SERVER_BULK 256u     /* stage the server kernel's inputs with bulk copies (TMA) where
+                                      the layout allows: every block but the last a multiple of 128
+                                      elements (M <= 16) */
+#define EF_FLAG_SERVER_NO_BULK 512u  /* stage them with per-thread asynchronous copies */
 #define EF_FLAG_DIAGNOSTICS 16u    /* worker steps also record per-block sums (ef_worker_diagnostics);
                                       implies the follow-up scale kernel, excludes EF_FLAG_FUSED_SCALE */
 
@@ -190,6 +201,16 @@ int ef_get_momentum(ef_ctx* ctx, int32_t i, float* dst);
 int ef_get_residual(ef_ctx* ctx, int32_t i, float* dst);
 int ef_set_state(ef_ctx* ctx, int32_t i, const float* momentum, const float* residual);
 int ef_step_count(ef_ctx* ctx, int64_t* t /* out: completed iterations */);
+
+/* Synchronises the context's stream and reads the device status word that kernels set when a
+ * bounded device-side wait runs out (only the bulk-staged server kernel waits at all: on an
+ * mbarrier that counts the bytes of its own copies, with an iteration limit).  Returns EF_OK,
+ * EF_ERR_TIMEOUT (the results of the affected call are undefined; the word is cleared) or
+ * EF_ERR_CUDA.  The step calls themselves never synchronise, so a caller who wants the check
+ * calls this, e.g. once per iteration or at checkpoints. */
+int ef_check_status(ef_ctx* ctx);
+uint32_t* ef_status_word(ef_ctx* ctx);   /* the word itself (device, inside the workspace): 0 = no event;
+                                            monitoring code may copy it instead of calling ef_check_status */
 
 /* Number of kernels this context has launched so far (for launch accounting). */
 int64_t ef_launch_count(ef_ctx* ctx);

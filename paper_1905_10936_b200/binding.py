@@ -33,6 +33,10 @@ EF_FLAG_SPLIT_SCALE = 4
 EF_FLAG_WEIGHT_DECAY = 8
 EF_FLAG_DIAGNOSTICS = 16
 EF_FLAG_ONE_LOCAL_WORKER = 32
+EF_FLAG_SERVER_TILES = 64
+EF_FLAG_SERVER_STREAM = 128
+EF_FLAG_SERVER_BULK = 256
+EF_FLAG_SERVER_NO_BULK = 512
 EF_MAX_WORKERS = 4096
 EF_PROBE_3R2W, EF_PROBE_1R1W, EF_PROBE_COPY = 0, 1, 2
 
@@ -63,6 +67,8 @@ SIGNATURES = {
     "ef_get_residual": (ctypes.c_int, [_vp, _i32, _vp]),
     "ef_set_state": (ctypes.c_int, [_vp, _i32, _vp, _vp]),
     "ef_step_count": (ctypes.c_int, [_vp, ctypes.POINTER(_i64)]),
+    "ef_check_status": (ctypes.c_int, [_vp]),
+    "ef_status_word": (_vp, [_vp]),
     "ef_launch_count": (_i64, [_vp]),
     "ef_worker_step_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _f32, _vp, _vp, _vp]),
     "ef_message_units": (_i64, [_vp, _i32, _i32]),
@@ -209,6 +215,14 @@ def ef_step_count(ctx: int) -> int:
     t = _i64(0)
     _check(load_library().ef_step_count(ctx, ctypes.byref(t)), "ef_step_count")
     return t.value
+
+
+def ef_check_status(ctx: int) -> None:
+    _check(load_library().ef_check_status(ctx), "ef_check_status")
+
+
+def ef_status_word(ctx: int) -> Optional[int]:
+    return load_library().ef_status_word(ctx)
 
 
 def ef_launch_count(ctx: int) -> int:

@@ -104,6 +104,7 @@ struct ServerArgs {
     // (message_unit below); wscales is unused then
     int fused_in;
     long long msg_base;      // message_unit of the first block the buffers hold
+    unsigned* status;        // the context's status word (bounded waits report here)
 };
 
 // Fused message layout: the message of a block range [b0, b1) is, block after block, one 32-bit
@@ -351,10 +352,14 @@ __device__ __forceinline__ void finish_block_diag(double acc, const DiagAcc& d, 
 // the group.
 __device__ __forceinline__ unsigned pack_nibbles(unsigned nib, int lane) {
     unsigned v = nib << ((lane & 7) * 4);
+#ifdef EF_REDUX_PACK
+    return __reduce_or_sync(0xffu << (lane & 24), v);
+#else
     v |= __shfl_xor_sync(kFull, v, 1);
     v |= __shfl_xor_sync(kFull, v, 2);
     v |= __shfl_xor_sync(kFull, v, 4);
     return v;
+#endif
 }
 
 __device__ __forceinline__ void load4(const float* p, int o, int len, bool full, float (&v)[4]) {
@@ -541,7 +546,10 @@ __global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a0
 // sign bits of element k; the data loaded by lane q lands at bit kLaneWorker(q), i.e. worker w
 // sits at bit w.
 constexpr int kMaxLutWorkers = 16;      // workers the table path handles (two lane groups)
-constexpr int kLutWorkers = 6;        // workers covered by the table
+#ifndef EF_LUT_WORKERS
+#define EF_LUT_WORKERS 6
+#endif
+constexpr int kLutWorkers = EF_LUT_WORKERS;   // workers covered by the table
 constexpr int kLutCopies = 32;        // one copy per lane
 
 __host__ __device__ constexpr int kLaneWorker(int q) {
@@ -624,20 +632,73 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 constexpr int kServerStages = 2;
-// Dynamic shared memory of the server kernel: staging ring (per thread and stage U float4 of
-// ptilde and U words for each group of 8 workers), then M scaled scales.
+
+// ---- bulk staging (TMA, 1-D): one elected thread copies a whole chunk of ptilde (16 KB) and
+// each worker's 128 packed words (512 B) into a shared-memory stage with cp.async.bulk and an
+// mbarrier that counts the bytes; the other threads only wait.  Never multicast, and only this
+// GPU's own memory is read.  Every wait is bounded: when the limit runs out the kernel records
+// kStatusWaitTimeout in the context's status word, waits (bounded again) for the copies it
+// still has in flight, and ends.
+constexpr unsigned kStatusWaitTimeout = 1u;
+constexpr int kMbarWaitLimit = 1 << 22;          // try_wait attempts (each blocks for a while itself)
+constexpr int kBulkWordStride = 1024 * 4 / 32 + 4;   // words per worker and stage: +4 keeps the
+                                                     // eight workers a warp reads in different banks
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned parity) {
+    unsigned ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+                 " selp.u32 %0, 1, 0, p;\n}" : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0u;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsigned parity) {
+    for (int it = 0; it < kMbarWaitLimit; ++it)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, unsigned bytes,
+                                          unsigned long long* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// Dynamic shared memory of the server kernel: staging ring, then M scaled scales.  A stage holds
+// either, per thread, U float4 of ptilde and U words for each group of 8 workers (per-thread
+// cp.async), or one chunk of ptilde in memory order and kBulkWordStride words per worker (bulk).
 template <int U>
-__host__ __device__ constexpr size_t server_ring_bytes(int groups) {
-    return (size_t)kServerStages * U * kThreads * (sizeof(float4) + groups * sizeof(unsigned));
+__host__ __device__ constexpr size_t server_stage_bytes(int M) {
+    const size_t per_thread = (size_t)U * kThreads * (sizeof(float4) + ((M + 7) / 8) * sizeof(unsigned));
+    const size_t bulk = (size_t)1024 * U * sizeof(float) + (size_t)M * kBulkWordStride * sizeof(unsigned);
+    return ((per_thread > bulk ? per_thread : bulk) + 127) / 128 * 128;
+}
+template <int U>
+__host__ __device__ constexpr size_t server_ring_bytes(int M) {
+    return (size_t)kServerStages * server_stage_bytes<U>(M);
 }
 
 // Table path: one CTA walks the chunks of its tile.  Full chunks are staged through a ring of
 // kServerStages shared-memory slots filled two chunks ahead with cp.async, so loads stay in
 // flight during the lookups without costing registers; a ragged last chunk is loaded directly.
-template <int U, int MT>
+//
+// BULK: the stages are filled by thread 0 with cp.async.bulk instead (see above); `full` are the
+// stages' mbarriers, `phase` their parities (bit s), both kept across calls by the caller.
+// Returns the thread's sum of |ptilde|; sets *failed when a bounded wait ran out.
+template <int U, int MT, bool BULK>
 __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Tile& t, float sp,
                                                   unsigned char* ring, float* s_c, float* s_base,
-                                                  float* s_lut) {
+                                                  float* s_lut, unsigned long long* full,
+                                                  unsigned& phase, bool* failed) {
     constexpr int kChunk = 1024 * U;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q = lane & 7;
@@ -656,11 +717,12 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
     const int nfull = t.len / kChunk;              // chunks staged through shared memory
     const int tail = t.len - nfull * kChunk;       // ragged rest (only at the end of a block)
     const char* lut = reinterpret_cast<const char*>(s_lut + lane);   // this lane's copy
-    // slot (stage s, row u) of this thread: consecutive threads are 16 (4) bytes apart
+    constexpr size_t kStage = server_stage_bytes<U>(MT);
+    // per-thread staging: slot (stage s, row u) of this thread, consecutive threads 16 (4) bytes apart
     float4* const ring_p = reinterpret_cast<float4*>(ring) + threadIdx.x;
     unsigned* const ring_w =
-        reinterpret_cast<unsigned*>(ring + (size_t)kServerStages * U * kThreads * sizeof(float4)) +
-        threadIdx.x;
+        reinterpret_cast<unsigned*>(ring + (size_t)U * kThreads * sizeof(float4)) + threadIdx.x;
+    constexpr int kStageP4 = (int)(kStage / sizeof(float4)), kStageW = (int)(kStage / sizeof(unsigned));
     double acc = 0.0;
     const bool rescale = a.ratio != 1.0f;
     // bit patterns of the scaled scales of the workers the table does not cover
@@ -672,15 +734,28 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
             const float* pp = pbase + (long long)c * kChunk;
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                cp_async16(ring_p + (s * U + u) * kThreads, pp + u * 128);
+                cp_async16(ring_p + s * kStageP4 + u * kThreads, pp + u * 128);
 #pragma unroll
                 for (int g = 0; g < G; ++g)
                     if (has_w[g])
-                        cp_async4(ring_w + ((s * U + u) * G + g) * kThreads,
+                        cp_async4(ring_w + s * kStageW + (u * G + g) * kThreads,
                                   wbase[g] + c * (kChunk / 32) + u * 4);
             }
         }
         cp_async_commit();                 // one (possibly empty) group per chunk index
+    };
+    // bulk staging, thread 0 only: chunk c of ptilde in memory order, then 128 words per worker
+    auto issue_chunk_bulk = [&](int c) {
+        const int s = c % kServerStages;
+        unsigned char* stage = ring + s * kStage;
+        mbar_expect_tx(&full[s], (unsigned)(kChunk * sizeof(float) + MT * (kChunk / 32) * sizeof(unsigned)));
+        bulk_load(stage, a.pb + t.start + (long long)c * kChunk, kChunk * sizeof(float), &full[s]);
+        const uint32_t* wsrc = tile_words(a, t) + c * (kChunk / 32);
+        unsigned* wdst = reinterpret_cast<unsigned*>(stage + kChunk * sizeof(float));
+#pragma unroll
+        for (int i = 0; i < MT; ++i)
+            bulk_load(wdst + i * kBulkWordStride, wsrc + (long long)i * a.wstride,
+                      (kChunk / 32) * sizeof(unsigned), &full[s]);
     };
     // full_c: std::true_type for a whole chunk (no bounds checks), std::false_type for the tail
     auto compute_chunk = [&](auto full_c, int c, int clen, float (&p)[U][4], unsigned (&w)[U][G]) {
@@ -725,24 +800,63 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
 
     float p[U][4];
     unsigned w[U][G];
+    if (BULK) {
+        if (threadIdx.x == 0) {
+            fence_proxy_async();                 // the stages were last read through ordinary loads
+            for (int c = 0; c < kServerStages && c < nfull; ++c) issue_chunk_bulk(c);
+        }
+    } else {
 #pragma unroll
-    for (int c = 0; c < kServerStages - 1; ++c) issue_chunk(c);   // in flight while the table is built
+        for (int c = 0; c < kServerStages - 1; ++c) issue_chunk(c);   // in flight while the table is built
+    }
     build_scaled(a, t, MT, s_c);
     __syncthreads();
     build_lut<MT>(s_c, s_base, s_lut);
 #pragma unroll
     for (int wk = kLutWorkers; wk < MT; ++wk) cdir[wk - kLutWorkers] = __float_as_uint(s_c[wk]);
     for (int c = 0; c < nfull; ++c) {
-        issue_chunk(c + kServerStages - 1);      // reuses the slot this thread consumed at c - 1
-        cp_async_wait<kServerStages - 1>();      // only the groups after chunk c may be in flight
         const int s = c % kServerStages;
+        if (BULK) {
+            const bool ok = mbar_wait_bounded(&full[s], (phase >> s) & 1u);
+            phase ^= 1u << s;
+            const float4* sp4 = reinterpret_cast<const float4*>(ring + s * kStage) + warp * (32 * U) + lane;
+            const unsigned* sw = reinterpret_cast<const unsigned*>(ring + s * kStage + kChunk * sizeof(float)) +
+                                 warp * (4 * U) + (lane >> 3);
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const float4 v = ring_p[(s * U + u) * kThreads];
-            p[u][0] = v.x; p[u][1] = v.y; p[u][2] = v.z; p[u][3] = v.w;
+            for (int u = 0; u < U; ++u) {
+                const float4 v = sp4[u * 32];
+                p[u][0] = v.x; p[u][1] = v.y; p[u][2] = v.z; p[u][3] = v.w;
 #pragma unroll
-            for (int g = 0; g < G; ++g)
-                w[u][g] = has_w[g] ? ring_w[((s * U + u) * G + g) * kThreads] : 0u;
+                for (int g = 0; g < G; ++g)
+                    w[u][g] = has_w[g] ? sw[(wq + 8 * g) * kBulkWordStride + u * 4] : 0u;
+            }
+            // everyone has read stage s (it may be refilled) -- and did every wait succeed?
+            if (__syncthreads_or(!ok)) {
+                if (threadIdx.x == 0) atomicOr(a.status, kStatusWaitTimeout);
+                // chunks c+1 .. are still in flight into the other stages: let them land
+                for (int c2 = c + 1; c2 < nfull && c2 < c + kServerStages; ++c2) {
+                    const int s2 = c2 % kServerStages;
+                    mbar_wait_bounded(&full[s2], (phase >> s2) & 1u);
+                    phase ^= 1u << s2;
+                }
+                *failed = true;
+                return acc;
+            }
+            if (threadIdx.x == 0 && c + kServerStages < nfull) {
+                fence_proxy_async();
+                issue_chunk_bulk(c + kServerStages);
+            }
+        } else {
+            issue_chunk(c + kServerStages - 1);      // reuses the slot this thread consumed at c - 1
+            cp_async_wait<kServerStages - 1>();      // only the groups after chunk c may be in flight
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const float4 v = ring_p[s * kStageP4 + u * kThreads];
+                p[u][0] = v.x; p[u][1] = v.y; p[u][2] = v.z; p[u][3] = v.w;
+#pragma unroll
+                for (int g = 0; g < G; ++g)
+                    w[u][g] = has_w[g] ? ring_w[s * kStageW + (u * G + g) * kThreads] : 0u;
+            }
         }
         compute_chunk(std::true_type{}, c, kChunk, p, w);
     }
@@ -759,7 +873,7 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
         }
         compute_chunk(std::false_type{}, nfull, tail, p, w);
     }
-    cp_async_wait<0>();
+    if (!BULK) cp_async_wait<0>();
     return acc;
 }
 
@@ -839,18 +953,32 @@ __device__ __forceinline__ double server_rows_scalar(const ServerArgs& a, const 
 }
 
 // One tile per CTA.  MT = number of workers when 1 <= M <= 16 (table path), 0 for any other M.
-template <int U, int MT>
+// BULK (table path, layouts whose packed words are 16-byte aligned per chunk only): stages are
+// filled with cp.async.bulk.
+template <int U, int MT, bool BULK>
 __global__ void __launch_bounds__(kThreads) ef_server_kernel(const ServerArgs a) {
     // dynamic shared memory: [staging ring (table path only)] [M scaled worker scales]
-    extern __shared__ __align__(16) unsigned char s_dyn[];
-    float* s_c = reinterpret_cast<float*>(s_dyn + (MT > 0 ? server_ring_bytes<U>((MT + 7) / 8) : 0));
+    extern __shared__ __align__(128) unsigned char s_dyn[];
+    float* s_c = reinterpret_cast<float*>(s_dyn + (MT > 0 ? server_ring_bytes<U>(MT) : 0));
     __shared__ float s_base[MT > 0 ? kLutEntries(MT) : 1];
     __shared__ float s_lut[MT > 0 ? kLutEntries(MT) * kLutCopies : 1];
+    __shared__ unsigned long long s_full[kServerStages];
+    unsigned phase = 0u;
+    bool failed = false;
+    if (BULK) {
+        if (threadIdx.x == 0) {
+            for (int s = 0; s < kServerStages; ++s) mbar_init(&s_full[s], 1u);
+            mbar_fence_init();
+        }
+        __syncthreads();
+    }
     const Tile t = a.tiles[blockIdx.x + a.tile0];
     const float sp = a.rscale[t.block];
     double acc = 0.0;
     if (MT > 0 && (t.start & 3) == 0) {
-        acc = server_tile_lut<U, (MT > 0 ? MT : 1)>(a, t, sp, s_dyn, s_c, s_base, s_lut);
+        acc = server_tile_lut<U, (MT > 0 ? MT : 1), BULK>(a, t, sp, s_dyn, s_c, s_base, s_lut, s_full,
+                                                          phase, &failed);
+        if (BULK && failed) return;
     } else {
         build_scaled(a, t, a.M, s_c);
         __syncthreads();
@@ -865,6 +993,81 @@ __global__ void __launch_bounds__(kThreads) ef_server_kernel(const ServerArgs a)
     finish_block(acc, (long long)(blockIdx.x + a.tile0) * kTileChunks, kTileChunks - 1, b.len <= 1024 * U,
                  (unsigned)b.tile_count, t.block, a.blocks, a.partials, a.tickets, a.scale_out,
                  a.rscale, a.fused);
+}
+
+// Persistent form of the table path for large grids.  CTA r owns a run of consecutive chunks
+// given by plan[r] = (first block, first chunk inside that block, number of chunks); the host
+// balances the runs by element count (plus a constant per block start).  The CTA walks its run
+// block by block: inside one block its chunks are handled exactly like a tile of the kernel
+// above (server_tile_lut), so the scaled scales and the table are built once per block and CTA
+// instead of once per 4 chunks, the staging ring never drains inside a block, and the grid is
+// one wave by construction (no tail wave).  Per block the CTA publishes ONE partial sum, in the
+// partial-sum slot of its first chunk of that block, and zeroes the slots of its other chunks,
+// so ef_scale_kernel finds every slot of a block defined; it runs after this kernel (split
+// mode only: there is no arrival ticket here).
+struct __align__(16) RunPlan {
+    int block, chunk, count, pad;
+};
+
+template <int U, int MT, bool BULK>
+__global__ void __launch_bounds__(kThreads, 4) ef_server_stream_kernel(const ServerArgs a,
+                                                                    const RunPlan* __restrict__ plan) {
+    constexpr int kChunk = 1024 * U;
+    extern __shared__ __align__(128) unsigned char s_dyn[];
+    float* s_c = reinterpret_cast<float*>(s_dyn + server_ring_bytes<U>(MT));
+    __shared__ float s_base[kLutEntries(MT)];
+    __shared__ float s_lut[kLutEntries(MT) * kLutCopies];
+    __shared__ double s_sum[kWarps];
+    __shared__ unsigned long long s_full[kServerStages];
+    unsigned phase = 0u;
+    bool failed = false;
+    if (BULK) {
+        if (threadIdx.x == 0) {
+            for (int s = 0; s < kServerStages; ++s) mbar_init(&s_full[s], 1u);
+            mbar_fence_init();
+        }
+        __syncthreads();
+    }
+    const RunPlan pl = plan[blockIdx.x];
+    int blk = pl.block, k = pl.chunk, remaining = pl.count;
+    while (remaining > 0) {
+        const Block b = a.blocks[blk];
+        const int nch = (int)((b.len + kChunk - 1) / kChunk);
+        const int kend = min(nch, k + remaining);
+        Tile t;
+        t.start = b.start + (long long)k * kChunk;
+        t.word = b.word + (long long)k * (kChunk / 32);
+        t.len = (int)min((long long)(kend - k) * kChunk, b.len - (long long)k * kChunk);
+        t.block = blk; t.pad0 = 0; t.pad1 = 0;
+        const float sp = a.rscale[blk];
+        double acc;
+        if ((t.start & 3) == 0) {
+            acc = server_tile_lut<U, MT, BULK>(a, t, sp, s_dyn, s_c, s_base, s_lut, s_full, phase, &failed);
+            if (BULK && failed) return;
+        } else {
+            build_scaled(a, t, a.M, s_c);
+            __syncthreads();
+            acc = server_rows_scalar(a, t, sp, s_c);
+        }
+        const double S = cta_sum(acc, s_sum);                 // valid in thread 0
+        double* slots = a.partials + (long long)b.tile_begin * kTileChunks;
+        if (nch == 1) {                                       // the block is this single chunk
+            if (threadIdx.x == 0) {
+                const float s = (float)(S / (double)b.len);
+                a.scale_out[blk] = s;
+                a.rscale[blk] = s;
+            }
+        } else {
+            if (threadIdx.x == 0) slots[k] = S;
+            for (int z = k + 1 + threadIdx.x; z < kend; z += kThreads) slots[z] = 0.0;
+            if (kend == nch)                                  // slots of the last tile beyond the block's end
+                for (int z = nch + threadIdx.x; z < b.tile_count * kTileChunks; z += kThreads) slots[z] = 0.0;
+        }
+        __syncthreads();              // s_sum, s_c and the table are rewritten by the next block
+        remaining -= kend - k;
+        blk += 1;
+        k = 0;
+    }
 }
 
 // ------------------------------------------------------------------ parameter update

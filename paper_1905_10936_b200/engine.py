@@ -30,7 +30,7 @@ class EFEngine:
     def __init__(self, offsets, M: int, mu: float, eta: float, host_staging: bool = False,
                  scale_mode: str = "auto", weight_decay: bool = False, diagnostics: bool = False,
                  stream: Optional[torch.cuda.Stream] = None, device: Optional[torch.device] = None,
-                 one_local_worker: bool = False):
+                 one_local_worker: bool = False, extra_flags: int = 0):
         if not torch.cuda.is_available():
             raise RuntimeError("EFEngine needs a CUDA device (there is no CPU path)")
         self.device = torch.device(device if device is not None else f"cuda:{torch.cuda.current_device()}")
@@ -42,6 +42,7 @@ class EFEngine:
         flags |= ef.EF_FLAG_WEIGHT_DECAY if weight_decay else 0
         flags |= ef.EF_FLAG_DIAGNOSTICS if diagnostics else 0
         flags |= ef.EF_FLAG_ONE_LOCAL_WORKER if one_local_worker else 0
+        flags |= int(extra_flags)
         self.local_workers = 1 if one_local_worker else self.M
         flags |= {"auto": 0, "fused": ef.EF_FLAG_FUSED_SCALE, "split": ef.EF_FLAG_SPLIT_SCALE}[scale_mode]
         nbytes = ef.ef_workspace_bytes(self.d, self.B, self.offsets, self.M, flags)

@@ -72,7 +72,7 @@ def test_init_validates_before_using_the_device():
         ef.ef_init(128, 2, off, 2, 0.9, 0.1, 0, 264, 1 << 30, 0)
     assert ei.value.status == ef.EF_ERR_ALIGNMENT
     with pytest.raises(ef.EFError) as ei:
-        ef.ef_init(128, 2, off, 2, 0.9, 0.1, 64, 256, 1 << 30, 0)    # unknown flag
+        ef.ef_init(128, 2, off, 2, 0.9, 0.1, 1 << 20, 256, 1 << 30, 0)    # unknown flag
     assert ei.value.status == ef.EF_ERR_INVALID_ARG
     for bad in (ef.EF_FLAG_FUSED_SCALE | ef.EF_FLAG_SPLIT_SCALE,          # contradictory flags
                 ef.EF_FLAG_FUSED_SCALE | ef.EF_FLAG_DIAGNOSTICS):

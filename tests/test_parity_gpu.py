@@ -79,6 +79,47 @@ def test_batched_and_per_worker_calls_are_bit_identical():
     assert ei.value.status == ef.EF_ERR_BAD_STATE
 
 
+@pytest.mark.parametrize("variant", ["tiles", "stream", "tiles+bulk", "stream+bulk"])
+@pytest.mark.parametrize("sizes,M", [
+    ([BIG, 2 * TILE, 5 * BIG + 128, 3 * TILE + 256, 640], 7),       # every block a multiple of 128: bulk-eligible
+    ([8 * BIG + 3 * TILE, 128, 2 * BIG], 15),                       # two lane groups
+    ([6 * BIG, TILE + 384], 16), ([3 * BIG + 1152], 1), ([2 * BIG, 9 * TILE], 8),
+    ([BIG + 4, 777, 2 * BIG + 36, 3, 5 * TILE + 1], 7),             # not eligible: bulk falls back
+    ([3, 5, 31, 33, 63, 65, 127, 129, 4 * BIG + 5], 3),             # unaligned starts: scalar path in a run
+    ([1000] * 40, 16), ([BIG + 5, 300, 2 * TILE], 17),              # many small blocks; M > 16 (no table path)
+])
+def test_server_kernel_variants(sizes, M, variant):
+    """The server kernel's variants (one CTA per tile / persistent runs, per-thread / bulk
+    staging), forced by flags, all against the oracle; the follow-up scale kernel is forced too,
+    because the persistent kernel exists in that mode only."""
+    flags = {"tiles": ef.EF_FLAG_SERVER_TILES, "stream": ef.EF_FLAG_SERVER_STREAM,
+             "tiles+bulk": ef.EF_FLAG_SERVER_TILES | ef.EF_FLAG_SERVER_BULK,
+             "stream+bulk": ef.EF_FLAG_SERVER_STREAM | ef.EF_FLAG_SERVER_BULK}[variant]
+    w = _wl("variants", sizes, M, steps=5, scale_range=(1e-3, 1.0))
+    factory = lambda *a, **kw: EFEngine(*a, extra_flags=flags, **kw)
+    eng, orc, stats = run_parity(w, scale_mode="split", engine_factory=factory, batched=True,
+                                 etas=[0.1, 0.1, 0.05, 0.2, 0.2])
+    ef.ef_check_status(eng.ctx)                 # no bounded wait ran out
+    assert stats["adopted"] <= 2
+
+
+def test_status_word_maps_to_the_timeout_code():
+    """ef_check_status turns the device status word into EF_ERR_TIMEOUT and clears it.  The word
+    is written from the host side here (through ef_status_word); no kernel is made to wait."""
+    from paper_1905_10936_b200.engine import _as_tensor
+    w = _wl("status", [TILE, 64], 2)
+    e = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    ef.ef_check_status(e.ctx)
+    word = _as_tensor(ef.ef_status_word(e.ctx), 1, torch.int32, e.device)
+    assert int(word.item()) == 0
+    word.fill_(1)
+    with pytest.raises(ef.EFError) as ei:
+        ef.ef_check_status(e.ctx)
+    assert ei.value.status == ef.EF_ERR_TIMEOUT
+    ef.ef_check_status(e.ctx)                   # cleared
+    assert "wait" in ef.ef_strerror(ef.EF_ERR_TIMEOUT)
+
+
 @pytest.mark.parametrize("mu,eta", [(0.0, 0.1), (0.5, 1.0), (0.99, 1e-3)])
 def test_hyper_parameters(mu, eta):
     w = _wl("hp", [TILE + 100, 777, 2 * TILE], 3, mu=mu, eta=eta, steps=6, scale_range=(1e-3, 1.0))
