@@ -72,17 +72,11 @@ enum ef_status {
                                       the other M-1 workers' messages arrive through
                                       ef_server_step_range.  ef_server_step, ef_worker_step_all over M
                                       gradients and the signum calls need all M workers locally. */
-/* Variants of the server kernel.  By default the library picks what measured fastest on B200
- * for the layout and M; these flags force a choice (for comparisons).  All variants compute the
- * same values; only the grouping of the fp64 partial sums differs between TILES and STREAM, which
- * can change the last bit of a scale in rare cases. */
-#define EF_FLAG_SERVER_TILES 64u     /* large layouts: one CTA per 16384-element tile */
-#define EF_FLAG_SERVER_STREAM 128u   /* large layouts: persistent one-wave kernel, each CTA walks a
-                                      balanced run of consecutive chunks (M <= 16) */
-#define EF_FLAG_SERVER_BULK 256u     /* stage the server kernel's inputs with bulk copies (TMA) where
-                                      the layout allows: every block but the last a multiple of 128
-                                      elements (M <= 16) */
-#define EF_FLAG_SERVER_NO_BULK 512u  /* stage them with per-thread asynchronous copies */
+#define EF_FLAG_SERVER_NO_BULK 512u  /* The server kernel stages its inputs in shared memory with bulk
+                                      copies (TMA) when the layout allows it (every block but the last a
+                                      multiple of 128 elements, M <= 16) and with per-thread asynchronous
+                                      copies otherwise; this flag forces the latter (for comparisons;
+                                      results are identical). */
 #define EF_FLAG_DIAGNOSTICS 16u    /* worker steps also record per-block sums (ef_worker_diagnostics);
                                       implies the follow-up scale kernel, excludes EF_FLAG_FUSED_SCALE */
 

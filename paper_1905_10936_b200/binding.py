@@ -33,9 +33,6 @@ EF_FLAG_SPLIT_SCALE = 4
 EF_FLAG_WEIGHT_DECAY = 8
 EF_FLAG_DIAGNOSTICS = 16
 EF_FLAG_ONE_LOCAL_WORKER = 32
-EF_FLAG_SERVER_TILES = 64
-EF_FLAG_SERVER_STREAM = 128
-EF_FLAG_SERVER_BULK = 256
 EF_FLAG_SERVER_NO_BULK = 512
 EF_MAX_WORKERS = 4096
 EF_PROBE_3R2W, EF_PROBE_1R1W, EF_PROBE_COPY = 0, 1, 2

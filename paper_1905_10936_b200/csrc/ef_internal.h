@@ -24,16 +24,6 @@ constexpr int kChunkLen = 1024 * kU;
 constexpr int kTileLen = kChunkLen * efk::kTileChunks;
 // Grids up to this many chunks (about two waves of CTAs) finalise block scales in-kernel.
 constexpr int64_t kFusedMaxChunks = 1024;
-// Largest grid of the persistent server kernel (CTAs per SM x SMs, with room to spare).
-constexpr int kMaxStreamGrid = 4096;
-// Defaults of the server kernel's two options, from measurements on B200 (see the profile
-// summaries): the persistent one-wave kernel pays off from this many workers on; bulk staging
-// is used where the layout allows it if kDefaultBulk.
-constexpr int kStreamMinWorkers = 9;
-constexpr bool kDefaultBulk = false;
-// Cost of starting a block inside a run of the persistent server kernel, in elements: loading
-// the workers' scales, building the table, the closing reduction.
-constexpr int64_t kBlockStartCost = 4096;
 
 struct Layout {
     int64_t d = 0, W = 0;
@@ -44,7 +34,7 @@ struct Layout {
     size_t dpad = 0, wpad = 0, bpad = 0, tpad = 0;    // padded element counts per sub-buffer
     size_t off_x = 0, off_m = 0, off_pb = 0, off_spb = 0, off_words = 0, off_scales = 0,
            off_rscale = 0, off_partials = 0, off_tickets = 0, off_tiles = 0, off_blocks = 0,
-           off_multi = 0, off_stage = 0, off_mt = 0, off_dpartials = 0, off_diag = 0, off_plan = 0,
+           off_multi = 0, off_stage = 0, off_mt = 0, off_dpartials = 0, off_diag = 0,
            off_status = 0, total = 0;
     int32_t num_multi = 0;                            // blocks that span more than one chunk
 };
@@ -72,13 +62,7 @@ struct ef_ctx {
     std::vector<efk::Block> h_blocks;
     std::vector<int32_t> h_multi;
     int fused = 0;                         // block scales finalised inside the main kernels
-    // persistent server kernel: run plans (one entry per CTA) for the whole block list and for
-    // the block range of the last ef_server_step_range call
-    int stream_grid = 0;                   // CTAs of the persistent server kernel; 0: not used
-    bool use_stream = false;               // large grids run the persistent server kernel
     bool use_bulk = false;                 // the server kernel stages its inputs with cp.async.bulk
-    std::vector<efk::RunPlan> h_plan_full, h_plan_range;
-    int plan_range_b0 = -1, plan_range_b1 = -1, plan_full_ctas = 0, plan_range_ctas = 0;
     // host-staging path
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t ev_copied[2] = {nullptr, nullptr};
@@ -104,7 +88,6 @@ struct ef_ctx {
     double* diag(int i) const { return (double*)(ws + L.off_diag) + (size_t)i * 4 * L.bpad; }
     float* stage(int s) const { return (float*)(ws + L.off_stage) + (size_t)s * L.dpad; }
     unsigned* status() const { return (unsigned*)(ws + L.off_status); }
-    efk::RunPlan* plan(int which) const { return (efk::RunPlan*)(ws + L.off_plan) + (size_t)which * efh::kMaxStreamGrid; }
 };
 
 namespace efh {

@@ -692,7 +692,7 @@ __host__ __device__ constexpr size_t server_ring_bytes(int M) {
 // flight during the lookups without costing registers; a ragged last chunk is loaded directly.
 //
 // BULK: the stages are filled by thread 0 with cp.async.bulk instead (see above); `full` are the
-// stages' mbarriers, `phase` their parities (bit s), both kept across calls by the caller.
+// stages' mbarriers, `phase` their parities (bit s).
 // Returns the thread's sum of |ptilde|; sets *failed when a bounded wait ran out.
 template <int U, int MT, bool BULK>
 __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Tile& t, float sp,
@@ -993,81 +993,6 @@ __global__ void __launch_bounds__(kThreads) ef_server_kernel(const ServerArgs a)
     finish_block(acc, (long long)(blockIdx.x + a.tile0) * kTileChunks, kTileChunks - 1, b.len <= 1024 * U,
                  (unsigned)b.tile_count, t.block, a.blocks, a.partials, a.tickets, a.scale_out,
                  a.rscale, a.fused);
-}
-
-// Persistent form of the table path for large grids.  CTA r owns a run of consecutive chunks
-// given by plan[r] = (first block, first chunk inside that block, number of chunks); the host
-// balances the runs by element count (plus a constant per block start).  The CTA walks its run
-// block by block: inside one block its chunks are handled exactly like a tile of the kernel
-// above (server_tile_lut), so the scaled scales and the table are built once per block and CTA
-// instead of once per 4 chunks, the staging ring never drains inside a block, and the grid is
-// one wave by construction (no tail wave).  Per block the CTA publishes ONE partial sum, in the
-// partial-sum slot of its first chunk of that block, and zeroes the slots of its other chunks,
-// so ef_scale_kernel finds every slot of a block defined; it runs after this kernel (split
-// mode only: there is no arrival ticket here).
-struct __align__(16) RunPlan {
-    int block, chunk, count, pad;
-};
-
-template <int U, int MT, bool BULK>
-__global__ void __launch_bounds__(kThreads, 4) ef_server_stream_kernel(const ServerArgs a,
-                                                                    const RunPlan* __restrict__ plan) {
-    constexpr int kChunk = 1024 * U;
-    extern __shared__ __align__(128) unsigned char s_dyn[];
-    float* s_c = reinterpret_cast<float*>(s_dyn + server_ring_bytes<U>(MT));
-    __shared__ float s_base[kLutEntries(MT)];
-    __shared__ float s_lut[kLutEntries(MT) * kLutCopies];
-    __shared__ double s_sum[kWarps];
-    __shared__ unsigned long long s_full[kServerStages];
-    unsigned phase = 0u;
-    bool failed = false;
-    if (BULK) {
-        if (threadIdx.x == 0) {
-            for (int s = 0; s < kServerStages; ++s) mbar_init(&s_full[s], 1u);
-            mbar_fence_init();
-        }
-        __syncthreads();
-    }
-    const RunPlan pl = plan[blockIdx.x];
-    int blk = pl.block, k = pl.chunk, remaining = pl.count;
-    while (remaining > 0) {
-        const Block b = a.blocks[blk];
-        const int nch = (int)((b.len + kChunk - 1) / kChunk);
-        const int kend = min(nch, k + remaining);
-        Tile t;
-        t.start = b.start + (long long)k * kChunk;
-        t.word = b.word + (long long)k * (kChunk / 32);
-        t.len = (int)min((long long)(kend - k) * kChunk, b.len - (long long)k * kChunk);
-        t.block = blk; t.pad0 = 0; t.pad1 = 0;
-        const float sp = a.rscale[blk];
-        double acc;
-        if ((t.start & 3) == 0) {
-            acc = server_tile_lut<U, MT, BULK>(a, t, sp, s_dyn, s_c, s_base, s_lut, s_full, phase, &failed);
-            if (BULK && failed) return;
-        } else {
-            build_scaled(a, t, a.M, s_c);
-            __syncthreads();
-            acc = server_rows_scalar(a, t, sp, s_c);
-        }
-        const double S = cta_sum(acc, s_sum);                 // valid in thread 0
-        double* slots = a.partials + (long long)b.tile_begin * kTileChunks;
-        if (nch == 1) {                                       // the block is this single chunk
-            if (threadIdx.x == 0) {
-                const float s = (float)(S / (double)b.len);
-                a.scale_out[blk] = s;
-                a.rscale[blk] = s;
-            }
-        } else {
-            if (threadIdx.x == 0) slots[k] = S;
-            for (int z = k + 1 + threadIdx.x; z < kend; z += kThreads) slots[z] = 0.0;
-            if (kend == nch)                                  // slots of the last tile beyond the block's end
-                for (int z = nch + threadIdx.x; z < b.tile_count * kTileChunks; z += kThreads) slots[z] = 0.0;
-        }
-        __syncthreads();              // s_sum, s_c and the table are rewritten by the next block
-        remaining -= kend - k;
-        blk += 1;
-        k = 0;
-    }
 }
 
 // ------------------------------------------------------------------ parameter update

@@ -31,11 +31,7 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
     if (rc != EF_OK) return rc;
     if (flags & ~(EF_FLAG_HOST_STAGING | EF_FLAG_FUSED_SCALE | EF_FLAG_SPLIT_SCALE |
                   EF_FLAG_WEIGHT_DECAY | EF_FLAG_DIAGNOSTICS | EF_FLAG_ONE_LOCAL_WORKER |
-                  EF_FLAG_SERVER_TILES | EF_FLAG_SERVER_STREAM | EF_FLAG_SERVER_BULK |
                   EF_FLAG_SERVER_NO_BULK))
-        return EF_ERR_INVALID_ARG;
-    if (((flags & EF_FLAG_SERVER_TILES) && (flags & EF_FLAG_SERVER_STREAM)) ||
-        ((flags & EF_FLAG_SERVER_BULK) && (flags & EF_FLAG_SERVER_NO_BULK)))
         return EF_ERR_INVALID_ARG;
     if ((flags & EF_FLAG_FUSED_SCALE) && (flags & (EF_FLAG_SPLIT_SCALE | EF_FLAG_DIAGNOSTICS)))
         return EF_ERR_INVALID_ARG;
@@ -71,7 +67,6 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
     L->off_tiles = o;    o += align_up((size_t)T * sizeof(Tile));
     L->off_blocks = o;   o += align_up((size_t)B * sizeof(Block));
     L->off_multi = o;    o += align_up((size_t)L->num_multi * sizeof(int32_t) + 4);
-    L->off_plan = o;     o += align_up(2 * (size_t)kMaxStreamGrid * sizeof(efk::RunPlan));
     L->off_status = o;   o += kAlign;
     L->off_stage = o;
     if (flags & EF_FLAG_HOST_STAGING) o += 2 * L->dpad * 4;
@@ -132,80 +127,36 @@ size_t server_smem_bytes(int M) {
 // Raises the dynamic shared-memory limit of the server kernel this context will use.  Done once
 // in ef_init so that the step calls themselves only enqueue work.
 template <int MT>
-cudaError_t prepare_server_t(int M, int* stream_ctas_per_sm) {
+cudaError_t prepare_server_t(int M) {
     const size_t smem = server_smem_bytes<MT>(M);
-    *stream_ctas_per_sm = 0;
-    cudaError_t e = cudaSuccess;
-    if (smem > 16 * 1024)                         // else static + dynamic stays far below the 48 KB default
-        e = cudaFuncSetAttribute(efk::ef_server_kernel<kU, MT, false>,
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (smem <= 16 * 1024) return cudaSuccess;    // static + dynamic stays far below the 48 KB default
+    cudaError_t e = cudaFuncSetAttribute(efk::ef_server_kernel<kU, MT, false>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess || MT == 0) return e;
-    constexpr int MS = MT > 0 ? MT : 1;
-    if ((e = cudaFuncSetAttribute(efk::ef_server_kernel<kU, MS, true>,
-                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess ||
-        (e = cudaFuncSetAttribute(efk::ef_server_stream_kernel<kU, MS, false>,
-                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess ||
-        (e = cudaFuncSetAttribute(efk::ef_server_stream_kernel<kU, MS, true>,
-                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
-        return e;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(stream_ctas_per_sm,
-                                                         efk::ef_server_stream_kernel<kU, MS, false>,
-                                                         efk::kThreads, smem);
+    return cudaFuncSetAttribute(efk::ef_server_kernel<kU, (MT > 0 ? MT : 1), true>,
+                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
 }
 
-cudaError_t prepare_server(int M, int* ctas) {
+cudaError_t prepare_server(int M) {
     switch (M) {
-        case 1: return prepare_server_t<1>(M, ctas);
-        case 2: return prepare_server_t<2>(M, ctas);
-        case 3: return prepare_server_t<3>(M, ctas);
-        case 4: return prepare_server_t<4>(M, ctas);
-        case 5: return prepare_server_t<5>(M, ctas);
-        case 6: return prepare_server_t<6>(M, ctas);
-        case 7: return prepare_server_t<7>(M, ctas);
-        case 8: return prepare_server_t<8>(M, ctas);
-        case 9: return prepare_server_t<9>(M, ctas);
-        case 10: return prepare_server_t<10>(M, ctas);
-        case 11: return prepare_server_t<11>(M, ctas);
-        case 12: return prepare_server_t<12>(M, ctas);
-        case 13: return prepare_server_t<13>(M, ctas);
-        case 14: return prepare_server_t<14>(M, ctas);
-        case 15: return prepare_server_t<15>(M, ctas);
-        case 16: return prepare_server_t<16>(M, ctas);
-        default: return prepare_server_t<0>(M, ctas);
+        case 1: return prepare_server_t<1>(M);
+        case 2: return prepare_server_t<2>(M);
+        case 3: return prepare_server_t<3>(M);
+        case 4: return prepare_server_t<4>(M);
+        case 5: return prepare_server_t<5>(M);
+        case 6: return prepare_server_t<6>(M);
+        case 7: return prepare_server_t<7>(M);
+        case 8: return prepare_server_t<8>(M);
+        case 9: return prepare_server_t<9>(M);
+        case 10: return prepare_server_t<10>(M);
+        case 11: return prepare_server_t<11>(M);
+        case 12: return prepare_server_t<12>(M);
+        case 13: return prepare_server_t<13>(M);
+        case 14: return prepare_server_t<14>(M);
+        case 15: return prepare_server_t<15>(M);
+        case 16: return prepare_server_t<16>(M);
+        default: return prepare_server_t<0>(M);
     }
-}
-
-// Cuts the chunks of blocks [b0, b1) into at most `ctas` runs of similar cost (elements plus a
-// constant per block start) for the persistent server kernel.
-void build_run_plan(const ef_ctx* c, int b0, int b1, int ctas, std::vector<efk::RunPlan>* out) {
-    out->clear();
-    long long total = 0, chunks = 0;
-    for (int b = b0; b < b1; ++b) {
-        total += c->h_blocks[b].len + kBlockStartCost;
-        chunks += (c->h_blocks[b].len + kChunkLen - 1) / kChunkLen;
-    }
-    ctas = (int)std::max<long long>(1, std::min<long long>(ctas, chunks));
-    long long done = 0;          // cost handed out so far
-    int r = 0;                   // run being filled
-    efk::RunPlan cur{b0, 0, 0, 0};
-    for (int b = b0; b < b1; ++b) {
-        const long long len = c->h_blocks[b].len;
-        const int nch = (int)((len + kChunkLen - 1) / kChunkLen);
-        for (int k = 0; k < nch; ++k) {
-            const long long cost = std::min<long long>(kChunkLen, len - (long long)k * kChunkLen) +
-                                   (k == 0 ? kBlockStartCost : 0);
-            // close the current run when this chunk would carry it past its share
-            if (cur.count > 0 && r + 1 < ctas && done + cost / 2 >= total * (r + 1) / ctas) {
-                out->push_back(cur);
-                r += 1;
-                cur = efk::RunPlan{b, k, 0, 0};
-            }
-            if (cur.count == 0) { cur.block = b; cur.chunk = k; }
-            cur.count += 1;
-            done += cost;
-        }
-    }
-    if (cur.count > 0) out->push_back(cur);
 }
 
 // Range of tiles that covers the blocks [b0, b1).
@@ -217,18 +168,11 @@ TileRange tiles_of(const ef_ctx* c, int b0, int b1) {
 }
 
 template <int MT>
-cudaError_t launch_server_t(ef_ctx* c, const efk::ServerArgs& a, unsigned grid,
-                            const efk::RunPlan* plan, unsigned plan_ctas, bool bulk) {
+cudaError_t launch_server_t(ef_ctx* c, const efk::ServerArgs& a, unsigned grid, bool bulk) {
     constexpr int MS = MT > 0 ? MT : 1;
     const size_t smem = server_smem_bytes<MT>(c->L.M);
-    if (MT > 0 && plan != nullptr) {
-        if (bulk) efk::ef_server_stream_kernel<kU, MS, true><<<plan_ctas, efk::kThreads, smem, c->stream>>>(a, plan);
-        else efk::ef_server_stream_kernel<kU, MS, false><<<plan_ctas, efk::kThreads, smem, c->stream>>>(a, plan);
-    } else if (MT > 0 && bulk) {
-        efk::ef_server_kernel<kU, MS, true><<<grid, efk::kThreads, smem, c->stream>>>(a);
-    } else {
-        efk::ef_server_kernel<kU, MT, false><<<grid, efk::kThreads, smem, c->stream>>>(a);
-    }
+    if (MT > 0 && bulk) efk::ef_server_kernel<kU, MS, true><<<grid, efk::kThreads, smem, c->stream>>>(a);
+    else efk::ef_server_kernel<kU, MT, false><<<grid, efk::kThreads, smem, c->stream>>>(a);
     return cudaGetLastError();
 }
 
@@ -252,44 +196,25 @@ int launch_server_range(ef_ctx* c, int b0, int b1, const uint32_t* msgs, long lo
     a.status = c->status();
     // bulk staging needs every chunk's packed words on a 16-byte boundary: plain layout only
     const bool bulk = c->use_bulk && !msgs;
-    // large grids: the persistent kernel with a balanced run plan (whole block list: built at
-    // init; a block range: built and uploaded when the range changes)
-    const efk::RunPlan* plan = nullptr;
-    unsigned plan_ctas = 0;
-    if (c->stream_grid > 0 && !c->fused && c->use_stream) {
-        if (b0 == 0 && b1 == c->L.B) {
-            plan = c->plan(0); plan_ctas = (unsigned)c->plan_full_ctas;
-        } else {
-            if (b0 != c->plan_range_b0 || b1 != c->plan_range_b1) {
-                build_run_plan(c, b0, b1, c->stream_grid, &c->h_plan_range);
-                EF_CUDA(c, cudaMemcpyAsync(c->plan(1), c->h_plan_range.data(),
-                                           c->h_plan_range.size() * sizeof(efk::RunPlan),
-                                           cudaMemcpyHostToDevice, c->stream));
-                c->plan_range_b0 = b0; c->plan_range_b1 = b1;
-                c->plan_range_ctas = (int)c->h_plan_range.size();
-            }
-            plan = c->plan(1); plan_ctas = (unsigned)c->plan_range_ctas;
-        }
-    }
     cudaError_t le;
     switch (M) {
-        case 1: le = launch_server_t<1>(c, a, tr.count, plan, plan_ctas, bulk); break;
-        case 2: le = launch_server_t<2>(c, a, tr.count, plan, plan_ctas, bulk); break;
-        case 3: le = launch_server_t<3>(c, a, tr.count, plan, plan_ctas, bulk); break;
-        case 4: le = launch_server_t<4>(c, a, tr.count, plan, plan_ctas, bulk); break;
-        case 5: le = launch_server_t<5>(c, a, tr.count, plan, plan_ctas, bulk); break;
-        case 6: le = launch_server_t<6>(c, a, tr.count, plan, plan_ctas, bulk); break;
-        case 7: le = launch_server_t<7>(c, a, tr.count, plan, plan_ctas, bulk); break;
-        case 8: le = launch_server_t<8>(c, a, tr.count, plan, plan_ctas, bulk); break;
-        case 9: le = launch_server_t<9>(c, a, tr.count, plan, plan_ctas, bulk); break;
-        case 10: le = launch_server_t<10>(c, a, tr.count, plan, plan_ctas, bulk); break;
-        case 11: le = launch_server_t<11>(c, a, tr.count, plan, plan_ctas, bulk); break;
-        case 12: le = launch_server_t<12>(c, a, tr.count, plan, plan_ctas, bulk); break;
-        case 13: le = launch_server_t<13>(c, a, tr.count, plan, plan_ctas, bulk); break;
-        case 14: le = launch_server_t<14>(c, a, tr.count, plan, plan_ctas, bulk); break;
-        case 15: le = launch_server_t<15>(c, a, tr.count, plan, plan_ctas, bulk); break;
-        case 16: le = launch_server_t<16>(c, a, tr.count, plan, plan_ctas, bulk); break;
-        default: le = launch_server_t<0>(c, a, tr.count, plan, plan_ctas, bulk); break;
+        case 1: le = launch_server_t<1>(c, a, tr.count, bulk); break;
+        case 2: le = launch_server_t<2>(c, a, tr.count, bulk); break;
+        case 3: le = launch_server_t<3>(c, a, tr.count, bulk); break;
+        case 4: le = launch_server_t<4>(c, a, tr.count, bulk); break;
+        case 5: le = launch_server_t<5>(c, a, tr.count, bulk); break;
+        case 6: le = launch_server_t<6>(c, a, tr.count, bulk); break;
+        case 7: le = launch_server_t<7>(c, a, tr.count, bulk); break;
+        case 8: le = launch_server_t<8>(c, a, tr.count, bulk); break;
+        case 9: le = launch_server_t<9>(c, a, tr.count, bulk); break;
+        case 10: le = launch_server_t<10>(c, a, tr.count, bulk); break;
+        case 11: le = launch_server_t<11>(c, a, tr.count, bulk); break;
+        case 12: le = launch_server_t<12>(c, a, tr.count, bulk); break;
+        case 13: le = launch_server_t<13>(c, a, tr.count, bulk); break;
+        case 14: le = launch_server_t<14>(c, a, tr.count, bulk); break;
+        case 15: le = launch_server_t<15>(c, a, tr.count, bulk); break;
+        case 16: le = launch_server_t<16>(c, a, tr.count, bulk); break;
+        default: le = launch_server_t<0>(c, a, tr.count, bulk); break;
     }
     EF_CUDA(c, le);
     c->launches += 1;
@@ -430,30 +355,14 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
         (ce = cudaMemcpyAsync(c->ws + L.off_multi, c->h_multi.data(),
                               c->h_multi.size() * sizeof(int32_t), cudaMemcpyHostToDevice,
                               c->stream)) != cudaSuccess) return fail(ce);
+    if ((ce = prepare_server(M)) != cudaSuccess) return fail(ce);
     {
-        int ctas_per_sm = 0, sms = 0;
-        if ((ce = prepare_server(M, &ctas_per_sm)) != cudaSuccess) return fail(ce);
-        if ((ce = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
-            return fail(ce);
         // bulk staging: every block but the last must hold a multiple of 128 elements (so that
         // every chunk's 128 packed words start on a 16-byte boundary) and start 16-byte aligned
         bool aligned = (L.wpad % 4) == 0;
         for (int32_t b = 0; b < B && aligned; ++b)
             aligned = (c->h_blocks[b].word % 4) == 0 && (c->h_blocks[b].start % 4) == 0;
-        c->use_bulk = aligned && M <= 16 && kDefaultBulk;
-        if (flags & EF_FLAG_SERVER_BULK) c->use_bulk = aligned && M <= 16;
-        if (flags & EF_FLAG_SERVER_NO_BULK) c->use_bulk = false;
-        c->use_stream = M >= kStreamMinWorkers;
-        if (flags & EF_FLAG_SERVER_STREAM) c->use_stream = true;
-        if (flags & EF_FLAG_SERVER_TILES) c->use_stream = false;
-        if (ctas_per_sm > 0 && !c->fused && c->use_stream) {
-            c->stream_grid = std::min(kMaxStreamGrid, ctas_per_sm * sms);
-            build_run_plan(c, 0, B, c->stream_grid, &c->h_plan_full);
-            c->plan_full_ctas = (int)c->h_plan_full.size();
-            if ((ce = cudaMemcpyAsync(c->plan(0), c->h_plan_full.data(),
-                                      c->h_plan_full.size() * sizeof(efk::RunPlan),
-                                      cudaMemcpyHostToDevice, c->stream)) != cudaSuccess) return fail(ce);
-        }
+        c->use_bulk = aligned && M <= 16 && !(flags & EF_FLAG_SERVER_NO_BULK);
     }
     if (flags & EF_FLAG_HOST_STAGING) {
         if ((ce = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking)) != cudaSuccess)

@@ -79,7 +79,7 @@ def test_batched_and_per_worker_calls_are_bit_identical():
     assert ei.value.status == ef.EF_ERR_BAD_STATE
 
 
-@pytest.mark.parametrize("variant", ["tiles", "stream", "tiles+bulk", "stream+bulk"])
+@pytest.mark.parametrize("variant", ["bulk where eligible", "per-thread"])
 @pytest.mark.parametrize("sizes,M", [
     ([BIG, 2 * TILE, 5 * BIG + 128, 3 * TILE + 256, 640], 7),       # every block a multiple of 128: bulk-eligible
     ([8 * BIG + 3 * TILE, 128, 2 * BIG], 15),                       # two lane groups
@@ -89,16 +89,14 @@ def test_batched_and_per_worker_calls_are_bit_identical():
     ([1000] * 40, 16), ([BIG + 5, 300, 2 * TILE], 17),              # many small blocks; M > 16 (no table path)
 ])
 def test_server_kernel_variants(sizes, M, variant):
-    """The server kernel's variants (one CTA per tile / persistent runs, per-thread / bulk
-    staging), forced by flags, all against the oracle; the follow-up scale kernel is forced too,
-    because the persistent kernel exists in that mode only."""
-    flags = {"tiles": ef.EF_FLAG_SERVER_TILES, "stream": ef.EF_FLAG_SERVER_STREAM,
-             "tiles+bulk": ef.EF_FLAG_SERVER_TILES | ef.EF_FLAG_SERVER_BULK,
-             "stream+bulk": ef.EF_FLAG_SERVER_STREAM | ef.EF_FLAG_SERVER_BULK}[variant]
+    """The two ways the server kernel stages its inputs (bulk copies with an mbarrier where the
+    layout is eligible, per-thread asynchronous copies otherwise or when forced), both against
+    the oracle, in both scale modes."""
+    flags = {"bulk where eligible": 0, "per-thread": ef.EF_FLAG_SERVER_NO_BULK}[variant]
     w = _wl("variants", sizes, M, steps=5, scale_range=(1e-3, 1.0))
     factory = lambda *a, **kw: EFEngine(*a, extra_flags=flags, **kw)
-    eng, orc, stats = run_parity(w, scale_mode="split", engine_factory=factory, batched=True,
-                                 etas=[0.1, 0.1, 0.05, 0.2, 0.2])
+    eng, orc, stats = run_parity(w, scale_mode="split" if M % 2 else "fused", engine_factory=factory,
+                                 batched=True, etas=[0.1, 0.1, 0.05, 0.2, 0.2])
     ef.ef_check_status(eng.ctx)                 # no bounded wait ran out
     assert stats["adopted"] <= 2
 
