@@ -556,6 +556,23 @@ __host__ __device__ constexpr int kLaneWorker(int q) {
     return 4 * (q & 1) + 2 * ((q >> 2) & 1) + ((q >> 1) & 1);
 }
 __host__ __device__ constexpr int kLutEntries(int M) { return 1 << (M < kLutWorkers ? M : kLutWorkers); }
+// M > 8 (two lane groups): ONE table, not replicated, over the first min(M, 10 or 11) workers, indexed by
+// the element's sign byte of workers 0-7 and the low bits of its sign byte of workers 8-15.  Its
+// lookups do collide in the banks (about 3.4 lanes per bank on random indices), which is still
+// far cheaper than three instructions per element for each worker added outside a table.
+// The table size is set by occupancy: the kernel is latency-bound and loses a third of its rate
+// at three CTAs per SM instead of four, so ring + table must stay within a quarter of the SM's
+// shared memory: 11 workers (8 KB) next to the bulk-staged ring for M <= 15, 10 (4 KB) next to
+// the slightly larger per-thread ring and for M = 16.
+__host__ __device__ constexpr int kWideLutWorkers(int M, bool bulk) { return (bulk && M <= 15) ? 11 : 10; }
+__host__ __device__ constexpr int kWideLutBits(int M, bool bulk) {
+    return M < kWideLutWorkers(M, bulk) ? M : kWideLutWorkers(M, bulk);
+}
+__host__ __device__ constexpr bool kUseWideLut(int M) { return M > 8; }
+// floats of static shared memory the table path needs
+__host__ __device__ constexpr int kLutFloats(int M, bool bulk) {
+    return kUseWideLut(M) ? (1 << kWideLutBits(M, bulk)) : kLutEntries(M) * kLutCopies;
+}
 
 __device__ __forceinline__ void build_scaled(const ServerArgs& a, const Tile& t, int M, float* s_c) {
     if (a.fused_in) {
@@ -589,6 +606,35 @@ __device__ __forceinline__ void build_lut(const float* s_c, float* s_base, float
     for (int e = threadIdx.x; e < (1 << T) * kLutCopies; e += kThreads)
         s_lut[e] = s_base[e / kLutCopies];
     __syncthreads();
+}
+
+// Wide table (M > 8): entry idx = (+-c_0) +- c_1 ... +- c_{T-1}, T = kWideLutBits, bit i of idx set =
+// worker i negative; every entry is the same chain of fp32 additions as the direct evaluation.
+// Built by doubling: thread k first forms entry k over the workers 0..7 (256 entries), then
+// worker i = 8, 9, ... turns every entry e < 2^i (a sum over workers 0..i-1) into the two entries
+// e (+c_i) and e + 2^i (-c_i): one addition per entry instead of T.  Ends with a barrier.
+template <int MT, bool BULK>
+__device__ __forceinline__ void build_wide_lut(const float* s_c, float* s_lut) {
+    constexpr int T = kWideLutBits(MT, BULK);
+    static_assert(T >= 8 && kThreads == 256, "the first level fills 256 entries, one per thread");
+    {
+        const int idx = threadIdx.x;
+        float v = (idx & 1) ? -s_c[0] : s_c[0];
+#pragma unroll
+        for (int i = 1; i < 8; ++i) v = __fadd_rn(v, ((idx >> i) & 1) ? -s_c[i] : s_c[i]);
+        s_lut[idx] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 8; i < T; ++i) {
+        const float ci = s_c[i];
+        for (int e = threadIdx.x; e < (1 << i); e += kThreads) {
+            const float v = s_lut[e];
+            s_lut[e] = __fadd_rn(v, ci);
+            s_lut[e + (1 << i)] = __fadd_rn(v, -ci);
+        }
+        __syncthreads();
+    }
 }
 
 __device__ __forceinline__ unsigned delta_swap(unsigned x, int d, unsigned mask) {
@@ -677,14 +723,14 @@ __device__ __forceinline__ void fence_proxy_async() {
 // either, per thread, U float4 of ptilde and U words for each group of 8 workers (per-thread
 // cp.async), or one chunk of ptilde in memory order and kBulkWordStride words per worker (bulk).
 template <int U>
-__host__ __device__ constexpr size_t server_stage_bytes(int M) {
+__host__ __device__ constexpr size_t server_stage_bytes(int M, bool bulk) {
     const size_t per_thread = (size_t)U * kThreads * (sizeof(float4) + ((M + 7) / 8) * sizeof(unsigned));
-    const size_t bulk = (size_t)1024 * U * sizeof(float) + (size_t)M * kBulkWordStride * sizeof(unsigned);
-    return ((per_thread > bulk ? per_thread : bulk) + 127) / 128 * 128;
+    const size_t bulk_bytes = (size_t)1024 * U * sizeof(float) + (size_t)M * kBulkWordStride * sizeof(unsigned);
+    return ((bulk ? bulk_bytes : per_thread) + 127) / 128 * 128;
 }
 template <int U>
-__host__ __device__ constexpr size_t server_ring_bytes(int M) {
-    return (size_t)kServerStages * server_stage_bytes<U>(M);
+__host__ __device__ constexpr size_t server_ring_bytes(int M, bool bulk) {
+    return (size_t)kServerStages * server_stage_bytes<U>(M, bulk);
 }
 
 // Table path: one CTA walks the chunks of its tile.  Full chunks are staged through a ring of
@@ -717,7 +763,7 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
     const int nfull = t.len / kChunk;              // chunks staged through shared memory
     const int tail = t.len - nfull * kChunk;       // ragged rest (only at the end of a block)
     const char* lut = reinterpret_cast<const char*>(s_lut + lane);   // this lane's copy
-    constexpr size_t kStage = server_stage_bytes<U>(MT);
+    constexpr size_t kStage = server_stage_bytes<U>(MT, BULK);
     // per-thread staging: slot (stage s, row u) of this thread, consecutive threads 16 (4) bytes apart
     float4* const ring_p = reinterpret_cast<float4*>(ring) + threadIdx.x;
     unsigned* const ring_w =
@@ -769,15 +815,28 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
 #pragma unroll
             for (int g = 0; g < G; ++g) Rg[g] = bf.indices(w[u][g]);
             const unsigned R = Rg[0];
-            // byte offset of entry (R_k & (entries-1)) in this lane's copy: 128 * index
-            constexpr unsigned kIdxMask = (unsigned)(kLutEntries(MT) - 1) << 7;
             float avg[4];
-            avg[0] = *reinterpret_cast<const float*>(lut + ((R << 7) & kIdxMask));
-            avg[1] = *reinterpret_cast<const float*>(lut + ((R >> 1) & kIdxMask));
-            avg[2] = *reinterpret_cast<const float*>(lut + ((R >> 9) & kIdxMask));
-            avg[3] = *reinterpret_cast<const float*>(lut + ((R >> 17) & kIdxMask));
+            if constexpr (kUseWideLut(MT)) {
+                // byte offset 4 * (byte k of R | low bits of byte k of Rg[1] << 8) in the one table
+                constexpr int kT = kWideLutBits(MT, BULK);
+                constexpr unsigned kHiMask = ((1u << (kT > 8 ? kT - 8 : 0)) - 1u) << 10;
+                const unsigned R1 = Rg[G - 1];
+                const char* wl = reinterpret_cast<const char*>(s_lut);
+                avg[0] = *reinterpret_cast<const float*>(wl + (((R << 2) & 0x3FCu) | ((R1 << 10) & kHiMask)));
+                avg[1] = *reinterpret_cast<const float*>(wl + (((R >> 6) & 0x3FCu) | ((R1 << 2) & kHiMask)));
+                avg[2] = *reinterpret_cast<const float*>(wl + (((R >> 14) & 0x3FCu) | ((R1 >> 6) & kHiMask)));
+                avg[3] = *reinterpret_cast<const float*>(wl + (((R >> 22) & 0x3FCu) | ((R1 >> 14) & kHiMask)));
+            } else {
+                // byte offset of entry (R_k & (entries-1)) in this lane's copy: 128 * index
+                constexpr unsigned kIdxMask = (unsigned)(kLutEntries(MT) - 1) << 7;
+                avg[0] = *reinterpret_cast<const float*>(lut + ((R << 7) & kIdxMask));
+                avg[1] = *reinterpret_cast<const float*>(lut + ((R >> 1) & kIdxMask));
+                avg[2] = *reinterpret_cast<const float*>(lut + ((R >> 9) & kIdxMask));
+                avg[3] = *reinterpret_cast<const float*>(lut + ((R >> 17) & kIdxMask));
+            }
+            constexpr int kFirstDirect = kUseWideLut(MT) ? kWideLutBits(MT, BULK) : kLutWorkers;
 #pragma unroll
-            for (int wk = kLutWorkers; wk < MT; ++wk) {     // remaining workers follow in order
+            for (int wk = kFirstDirect; wk < MT; ++wk) {    // remaining workers follow in order
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
                     avg[k] = __fadd_rn(avg[k], __uint_as_float(
@@ -811,7 +870,8 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
     }
     build_scaled(a, t, MT, s_c);
     __syncthreads();
-    build_lut<MT>(s_c, s_base, s_lut);
+    if constexpr (kUseWideLut(MT)) build_wide_lut<MT, BULK>(s_c, s_lut);
+    else build_lut<MT>(s_c, s_base, s_lut);
 #pragma unroll
     for (int wk = kLutWorkers; wk < MT; ++wk) cdir[wk - kLutWorkers] = __float_as_uint(s_c[wk]);
     for (int c = 0; c < nfull; ++c) {
@@ -959,9 +1019,9 @@ template <int U, int MT, bool BULK>
 __global__ void __launch_bounds__(kThreads) ef_server_kernel(const ServerArgs a) {
     // dynamic shared memory: [staging ring (table path only)] [M scaled worker scales]
     extern __shared__ __align__(128) unsigned char s_dyn[];
-    float* s_c = reinterpret_cast<float*>(s_dyn + (MT > 0 ? server_ring_bytes<U>(MT) : 0));
-    __shared__ float s_base[MT > 0 ? kLutEntries(MT) : 1];
-    __shared__ float s_lut[MT > 0 ? kLutEntries(MT) * kLutCopies : 1];
+    float* s_c = reinterpret_cast<float*>(s_dyn + (MT > 0 ? server_ring_bytes<U>(MT, BULK) : 0));
+    __shared__ float s_base[(MT > 0 && !kUseWideLut(MT)) ? kLutEntries(MT) : 1];
+    __shared__ float s_lut[MT > 0 ? kLutFloats(MT, BULK) : 1];
     __shared__ unsigned long long s_full[kServerStages];
     unsigned phase = 0u;
     bool failed = false;

@@ -120,21 +120,22 @@ int launch_worker(ef_ctx* c, int i, const float* grad, int count = 1, long long 
 }
 
 template <int MT>
-size_t server_smem_bytes(int M) {
-    return (MT > 0 ? efk::server_ring_bytes<kU>(MT) : 0) + (size_t)M * sizeof(float);
+size_t server_smem_bytes(int M, bool bulk) {
+    return (MT > 0 ? efk::server_ring_bytes<kU>(MT, bulk) : 0) + (size_t)M * sizeof(float);
 }
 
 // Raises the dynamic shared-memory limit of the server kernel this context will use.  Done once
 // in ef_init so that the step calls themselves only enqueue work.
 template <int MT>
 cudaError_t prepare_server_t(int M) {
-    const size_t smem = server_smem_bytes<MT>(M);
+    const size_t smem = server_smem_bytes<MT>(M, false);
     if (smem <= 16 * 1024) return cudaSuccess;    // static + dynamic stays far below the 48 KB default
     cudaError_t e = cudaFuncSetAttribute(efk::ef_server_kernel<kU, MT, false>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess || MT == 0) return e;
     return cudaFuncSetAttribute(efk::ef_server_kernel<kU, (MT > 0 ? MT : 1), true>,
-                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                                cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)server_smem_bytes<MT>(M, true));
 }
 
 cudaError_t prepare_server(int M) {
@@ -170,9 +171,10 @@ TileRange tiles_of(const ef_ctx* c, int b0, int b1) {
 template <int MT>
 cudaError_t launch_server_t(ef_ctx* c, const efk::ServerArgs& a, unsigned grid, bool bulk) {
     constexpr int MS = MT > 0 ? MT : 1;
-    const size_t smem = server_smem_bytes<MT>(c->L.M);
-    if (MT > 0 && bulk) efk::ef_server_kernel<kU, MS, true><<<grid, efk::kThreads, smem, c->stream>>>(a);
-    else efk::ef_server_kernel<kU, MT, false><<<grid, efk::kThreads, smem, c->stream>>>(a);
+    if (MT > 0 && bulk)
+        efk::ef_server_kernel<kU, MS, true><<<grid, efk::kThreads, server_smem_bytes<MT>(c->L.M, true), c->stream>>>(a);
+    else
+        efk::ef_server_kernel<kU, MT, false><<<grid, efk::kThreads, server_smem_bytes<MT>(c->L.M, false), c->stream>>>(a);
     return cudaGetLastError();
 }
 
