@@ -54,7 +54,9 @@ enum ef_status {
     EF_ERR_UNSUPPORTED_DEVICE = 6, /* current device is not compute capability 10.x */
     EF_ERR_TIMEOUT = 7,            /* a bounded device-side wait gave up (reported by ef_check_status) */
     EF_ERR_TOO_LARGE = 8,          /* ef_worker_step_noalloc: n exceeds EF_NOALLOC_MAX_ELEMS */
-    EF_ERR_NO_MEMORY = 9           /* a host allocation failed (the library allocates no device memory) */
+    EF_ERR_NO_MEMORY = 9,          /* a host allocation failed (the library allocates no device memory) */
+    EF_ERR_BOUNDS = 10             /* checked build only: a kernel refused a work item that reached
+                                      outside its arrays (reported by ef_check_status) */
 };
 
 /* Flags for ef_workspace_bytes / ef_init. */
@@ -205,6 +207,17 @@ int ef_step_count(ef_ctx* ctx, int64_t* t /* out: completed iterations */);
 int ef_check_status(ef_ctx* ctx);
 uint32_t* ef_status_word(ef_ctx* ctx);   /* the word itself (device, inside the workspace): 0 = no event;
                                             monitoring code may copy it instead of calling ef_check_status */
+
+/* Checked build.  Compiled with -DEF_DEBUG, every kernel validates its work item (tile or chunk
+ * descriptor: block id, length, element and word ranges) against the problem's sizes before it
+ * touches memory; an item that reaches outside is skipped and EF_ERR_BOUNDS is reported by
+ * ef_check_status.  Nothing traps or asserts, so the context and the device stay usable.  (A
+ * memory checker for the device is not always available; this is the library's own net.)
+ * ef_debug_build: 1 if this library is the checked build.  ef_debug_shift_tile: test hook of the
+ * checked build only (EF_ERR_BAD_STATE otherwise): moves the start of one tile descriptor by
+ * `delta` elements, between iterations, so that a test can see the check refuse it. */
+int ef_debug_build(void);
+int ef_debug_shift_tile(ef_ctx* ctx, int64_t tile, int64_t delta);
 
 /* Number of kernels this context has launched so far (for launch accounting). */
 int64_t ef_launch_count(ef_ctx* ctx);

@@ -26,6 +26,7 @@ EF_ERR_UNSUPPORTED_DEVICE = 6
 EF_ERR_TIMEOUT = 7
 EF_ERR_TOO_LARGE = 8
 EF_ERR_NO_MEMORY = 9
+EF_ERR_BOUNDS = 10
 EF_NOALLOC_MAX_ELEMS = 1 << 24
 EF_FLAG_HOST_STAGING = 1
 EF_FLAG_FUSED_SCALE = 2
@@ -66,6 +67,8 @@ SIGNATURES = {
     "ef_step_count": (ctypes.c_int, [_vp, ctypes.POINTER(_i64)]),
     "ef_check_status": (ctypes.c_int, [_vp]),
     "ef_status_word": (_vp, [_vp]),
+    "ef_debug_build": (ctypes.c_int, []),
+    "ef_debug_shift_tile": (ctypes.c_int, [_vp, _i64, _i64]),
     "ef_launch_count": (_i64, [_vp]),
     "ef_worker_step_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _vp, _i64, _f32, _vp, _vp, _vp]),
     "ef_message_units": (_i64, [_vp, _i32, _i32]),
@@ -86,8 +89,18 @@ SIGNATURES = {
 _lib = None
 
 
+def use_library(path: Optional[str] = None) -> None:
+    """Selects the shared library the binding calls from now on (None: the regular libef.so);
+    used to run the checked build (libef_debug.so).  Contexts of one library must not be
+    passed to another."""
+    global _lib, LIB_PATH
+    LIB_PATH = path if path is not None else os.path.join(_PKG, "libef.so")
+    _lib = None
+
+
 def load_library() -> ctypes.CDLL:
-    """Loads libef.so from the package directory; raises if it has not been built."""
+    """Loads the selected library (libef.so in the package directory unless use_library chose
+    another); raises if it has not been built."""
     global _lib
     if _lib is None:
         if not os.path.exists(LIB_PATH):
@@ -216,6 +229,14 @@ def ef_step_count(ctx: int) -> int:
 
 def ef_check_status(ctx: int) -> None:
     _check(load_library().ef_check_status(ctx), "ef_check_status")
+
+
+def ef_debug_build() -> bool:
+    return bool(load_library().ef_debug_build())
+
+
+def ef_debug_shift_tile(ctx: int, tile: int, delta: int) -> None:
+    _check(load_library().ef_debug_shift_tile(ctx, tile, delta), "ef_debug_shift_tile")
 
 
 def ef_status_word(ctx: int) -> Optional[int]:

@@ -9,6 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libef.so")
+DEBUG_LIB = os.path.join(PKG, "libef_debug.so")      # the checked build (-DEF_DEBUG)
 SOURCES = [os.path.join(CSRC, n) for n in ("ef_lib.cu", "ef_vote.cu", "ef_topk.cu")]
 DEPS = SOURCES + [os.path.join(CSRC, "ef_kernels.cuh"), os.path.join(CSRC, "ef_internal.h"),
                   os.path.join(ROOT, "include", "ef.h")]
@@ -26,19 +27,23 @@ def nvcc_path() -> str:
     return cand if os.path.exists(cand) else "nvcc"
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    if not force and os.path.exists(LIB):
+def build_library(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Builds libef.so, or with debug=True the checked build libef_debug.so (every kernel
+    validates its work item against the problem's sizes)."""
+    lib = DEBUG_LIB if debug else LIB
+    if not force and os.path.exists(lib):
         newest = max(os.path.getmtime(p) for p in DEPS)
-        if os.path.getmtime(LIB) >= newest:
-            return LIB
-    cmd = [nvcc_path()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB] + SOURCES
+        if os.path.getmtime(lib) >= newest:
+            return lib
+    cmd = ([nvcc_path()] + NVCC_FLAGS + (["-DEF_DEBUG"] if debug else [])
+           + (["-Xptxas", "-v"] if verbose else []) + ["-o", lib] + SOURCES)
     res = subprocess.run(cmd, capture_output=True, text=True)
     if verbose:
         sys.stderr.write(res.stderr)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":
-    print(build_library(force=True, verbose="-v" in sys.argv))
+    print(build_library(force=True, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

@@ -88,6 +88,7 @@ struct ef_ctx {
     double* diag(int i) const { return (double*)(ws + L.off_diag) + (size_t)i * 4 * L.bpad; }
     float* stage(int s) const { return (float*)(ws + L.off_stage) + (size_t)s * L.dpad; }
     unsigned* status() const { return (unsigned*)(ws + L.off_status); }
+    efk::DebugLimits limits() const { return efk::DebugLimits{L.d, L.W, L.B, status()}; }
 };
 
 namespace efh {

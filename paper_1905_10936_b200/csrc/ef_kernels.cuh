@@ -58,6 +58,29 @@ struct __align__(16) Block {
 };
 static_assert(sizeof(Block) == 32, "Block must be 32 bytes");
 
+// Limits of the problem, carried by every launch.  A build with -DEF_DEBUG checks each CTA's
+// work item (tile or chunk descriptor) against them before touching memory: a descriptor that
+// reaches outside its arrays is not used; the CTA records kStatusBounds in the status word and
+// ends (no trap, no assert: the context stays usable and ef_check_status reports it).
+struct DebugLimits {
+    long long d, W;      // elements, packed words
+    int B;               // blocks
+    unsigned* status;
+};
+constexpr unsigned kStatusBounds = 2u;
+__device__ __forceinline__ bool work_item_ok(const Tile& t, const DebugLimits& lim, int max_len) {
+#ifdef EF_DEBUG
+    const long long len = t.len > 0 ? t.len : 0;      // an empty item touches no element
+    const bool ok = t.block >= 0 && t.block < lim.B && t.len <= max_len &&
+                    (len == 0 || (t.start >= 0 && t.start + len <= lim.d && t.word >= 0 &&
+                                  t.word + (len + 31) / 32 <= lim.W));
+    if (!ok && threadIdx.x == 0) atomicOr(lim.status, kStatusBounds);
+    return ok;
+#else
+    return true;
+#endif
+}
+
 struct WorkerArgs {
     const float* g;        // gradient g_{t,i}
     float* m;              // momentum m_i (in/out)
@@ -79,6 +102,7 @@ struct WorkerArgs {
     // arrays of `partial_stride` slots each, and the per-block results [B][4] (|p|, p^2, |g|, g^2)
     double* dpartials;
     double* diag;
+    DebugLimits lim;
 };
 
 struct ServerArgs {
@@ -105,6 +129,7 @@ struct ServerArgs {
     int fused_in;
     long long msg_base;      // message_unit of the first block the buffers hold
     unsigned* status;        // the context's status word (bounded waits report here)
+    DebugLimits lim;
 };
 
 // Fused message layout: the message of a block range [b0, b1) is, block after block, one 32-bit
@@ -140,6 +165,7 @@ struct ApplyArgs {
     // weight decay kept out of the compressor (Appendix A); used by the DECAY instantiation only
     float* mt;               // decay momentum mtilde
     float mu, lambda;
+    DebugLimits lim;
 };
 
 struct ResidualArgs {
@@ -147,6 +173,7 @@ struct ResidualArgs {
     const float* rscale;
     float* dst;
     const Tile* tiles;
+    DebugLimits lim;
 };
 
 // ------------------------------------------------------------------ small helpers
@@ -503,6 +530,7 @@ __global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a0
         a.tickets += wi * a.scale_stride;
     }
     const Tile t = chunk_of<U>(a.tiles[blockIdx.x / kTileChunks], blockIdx.x % kTileChunks);
+    if (!work_item_ok(t, a.lim, 1024 * U)) return;
     const Block b = a.blocks[t.block];
     const bool alone = b.len <= 1024 * U;              // the block is this single chunk
     if (t.len <= 0 && alone) return;
@@ -1033,6 +1061,7 @@ __global__ void __launch_bounds__(kThreads) ef_server_kernel(const ServerArgs a)
         __syncthreads();
     }
     const Tile t = a.tiles[blockIdx.x + a.tile0];
+    if (!work_item_ok(t, a.lim, kTileChunks * 1024 * U)) return;
     const float sp = a.rscale[t.block];
     double acc = 0.0;
     if (MT > 0 && (t.start & 3) == 0) {
@@ -1078,6 +1107,7 @@ template <int U, bool DECAY>
 __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
     constexpr int kChunk = 1024 * U;
     const Tile t = a.tiles[blockIdx.x + a.tile0];
+    if (!work_item_ok(t, a.lim, kTileChunks * kChunk)) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // packed words of this tile and the block's scale: plain layout or a fused message
     const uint32_t* const twords =
@@ -1158,6 +1188,7 @@ __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
 // One tile per CTA.
 static __global__ void __launch_bounds__(kThreads) ef_residual_kernel(const ResidualArgs a) {
     const Tile t = a.tiles[blockIdx.x];
+    if (!work_item_ok(t, a.lim, 1 << 30)) return;
     const float s = a.rscale[t.block];
     for (int o = threadIdx.x; o < t.len; o += kThreads)
         a.dst[t.start + o] = residual_of(a.pb[t.start + o], s);
@@ -1173,9 +1204,11 @@ struct PackArgs {
     const Block* blocks;
     int tile0;
     long long msg_base;
+    DebugLimits lim;
 };
 static __global__ void __launch_bounds__(kThreads) ef_pack_kernel(const PackArgs a) {
     const Tile t = a.tiles[blockIdx.x + a.tile0];
+    if (!work_item_ok(t, a.lim, 1 << 30)) return;
     const Block b = a.blocks[t.block];
     uint32_t* dst = a.dst + (message_unit(t.word, t.block) + 1 - a.msg_base);
     const int nwords = (t.len + 31) >> 5;

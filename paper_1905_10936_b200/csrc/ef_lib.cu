@@ -111,6 +111,7 @@ int launch_worker(ef_ctx* c, int i, const float* grad, int count = 1, long long 
     const bool diag = (c->flags & EF_FLAG_DIAGNOSTICS) != 0;
     a.dpartials = diag ? c->dpartials(i) : nullptr;
     a.diag = diag ? c->diag(i) : nullptr;
+    a.lim = c->limits();
     const dim3 grid((unsigned)(c->L.num_tiles * efk::kTileChunks), (unsigned)count);
     if (diag) efk::ef_worker_kernel<kU, true><<<grid, efk::kThreads, 0, c->stream>>>(a);
     else efk::ef_worker_kernel<kU, false><<<grid, efk::kThreads, 0, c->stream>>>(a);
@@ -196,6 +197,7 @@ int launch_server_range(ef_ctx* c, int b0, int b1, const uint32_t* msgs, long lo
     a.fused_in = msgs ? 1 : 0;
     a.msg_base = efk::message_unit(c->h_blocks[b0].word, b0);
     a.status = c->status();
+    a.lim = c->limits();
     // bulk staging needs every chunk's packed words on a 16-byte boundary: plain layout only
     const bool bulk = c->use_bulk && !msgs;
     cudaError_t le;
@@ -249,6 +251,7 @@ int launch_apply_range(ef_ctx* c, int b0, int b1, const uint32_t* update) {
     p.fused_in = update ? 1 : 0;
     p.msg_base = efk::message_unit(c->h_blocks[b0].word, b0);
     p.eta = c->eta; p.mu = c->mu; p.lambda = c->lambda; p.mt = c->mt();
+    p.lim = c->limits();
     if (c->lambda > 0.f)
         efk::ef_apply_kernel<kU, true><<<tr.count, efk::kThreads, 0, c->stream>>>(p);
     else
@@ -446,6 +449,7 @@ int ef_pack_message(ef_ctx* c, int32_t who, int32_t b0, int32_t b1, uint32_t* ds
     a.words = c->words(k); a.scales = c->scales(k); a.dst = dst;
     a.tiles = c->tiles(); a.blocks = c->blocks(); a.tile0 = tr.tile0;
     a.msg_base = efk::message_unit(c->h_blocks[b0].word, b0);
+    a.lim = c->limits();
     efk::ef_pack_kernel<<<tr.count, efk::kThreads, 0, c->stream>>>(a);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
@@ -539,6 +543,7 @@ int ef_get_residual(ef_ctx* c, int32_t i, float* dst) {
     const int k = (i < 0) ? c->srv() : i;
     efk::ResidualArgs a;
     a.pb = c->pb(k); a.rscale = c->rscale(k); a.dst = dst; a.tiles = c->tiles();
+    a.lim = c->limits();
     efk::ef_residual_kernel<<<(unsigned)c->L.num_tiles, efk::kThreads, 0, c->stream>>>(a);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
@@ -579,7 +584,29 @@ int ef_check_status(ef_ctx* c) {
     EF_CUDA(c, cudaStreamSynchronize(c->stream));
     if (word == 0) return EF_OK;
     EF_CUDA(c, cudaMemsetAsync(c->status(), 0, sizeof(word), c->stream));
+    if (word & efk::kStatusBounds) return EF_ERR_BOUNDS;
     return (word & efk::kStatusWaitTimeout) ? EF_ERR_TIMEOUT : EF_ERR_CUDA;
+}
+
+int ef_debug_build(void) {
+#ifdef EF_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+int ef_debug_shift_tile(ef_ctx* c, int64_t tile, int64_t delta) {
+#ifdef EF_DEBUG
+    if (!c || tile < 0 || tile >= c->L.num_tiles || c->pending != 0) return EF_ERR_INVALID_ARG;
+    c->h_tiles[(size_t)tile].start += delta;
+    EF_CUDA(c, cudaMemcpyAsync(c->ws + c->L.off_tiles + (size_t)tile * sizeof(Tile), &c->h_tiles[(size_t)tile],
+                               sizeof(Tile), cudaMemcpyHostToDevice, c->stream));
+    return EF_OK;
+#else
+    (void)c; (void)tile; (void)delta;
+    return EF_ERR_BAD_STATE;
+#endif
 }
 
 uint32_t* ef_status_word(ef_ctx* c) { return c ? (uint32_t*)c->status() : nullptr; }
@@ -598,6 +625,7 @@ const char* ef_strerror(int status) {
         case EF_ERR_TIMEOUT: return "device-side wait timed out";
         case EF_ERR_TOO_LARGE: return "size exceeds the fixed scratch of the no-allocation entry point";
         case EF_ERR_NO_MEMORY: return "host allocation failed";
+        case EF_ERR_BOUNDS: return "a work item reached outside its arrays (checked build)";
         default: return "unknown status";
     }
 }

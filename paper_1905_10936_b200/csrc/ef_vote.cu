@@ -31,6 +31,7 @@ struct VoteWorkerArgs {
     const Tile* tiles;
     float mu;
     long long g_stride, state_stride, word_stride;   // blockIdx.y selects the worker
+    efk::DebugLimits lim;
 };
 
 struct VoteServerArgs {
@@ -42,6 +43,7 @@ struct VoteServerArgs {
     float* x;
     const Tile* tiles;
     float eta;
+    efk::DebugLimits lim;
 };
 
 // Sign bits (value < 0, so that -0 counts as +1) of four values as a nibble, element k in bit k.
@@ -104,7 +106,7 @@ __global__ void __launch_bounds__(kThreads) ef_vote_worker_kernel(const VoteWork
     a.m += wi * a.state_stride;
     a.words += wi * a.word_stride;
     const Tile t = efk::chunk_of<U>(a.tiles[blockIdx.x / efk::kTileChunks], blockIdx.x % efk::kTileChunks);
-    if (t.len <= 0) return;
+    if (t.len <= 0 || !efk::work_item_ok(t, a.lim, 1024 * U)) return;
     if ((t.start & 3) != 0) vote_worker_rows_scalar(a, t);
     else if (t.len == 1024 * U) vote_worker_rows<U, true>(a, t);
     else vote_worker_rows<U, false>(a, t);
@@ -170,6 +172,7 @@ template <int U, int P>
 __global__ void __launch_bounds__(kThreads) ef_vote_server_kernel(const VoteServerArgs a) {
     constexpr int kChunk = 1024 * U;
     const Tile t = a.tiles[blockIdx.x];
+    if (!efk::work_item_ok(t, a.lim, efk::kTileChunks * kChunk)) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if ((t.start & 3) != 0) {                   // block does not start on a 16-byte boundary
         const int rows = (t.len + 31) >> 5;
@@ -230,6 +233,7 @@ int launch_vote_worker(ef_ctx* c, int i, const float* grad, int count, long long
     VoteWorkerArgs a;
     a.g = grad; a.m = c->m(i); a.words = c->words(i); a.tiles = c->tiles(); a.mu = c->mu;
     a.g_stride = g_stride; a.state_stride = (long long)c->L.dpad; a.word_stride = (long long)c->L.wpad;
+    a.lim = c->limits();
     const dim3 grid((unsigned)(c->L.num_tiles * efk::kTileChunks), (unsigned)count);
     ef_vote_worker_kernel<kU><<<grid, kThreads, 0, c->stream>>>(a);
     EF_CUDA(c, cudaGetLastError());
@@ -269,6 +273,7 @@ int ef_vote_server_step(ef_ctx* c) {
     a.wwords = c->words(0); a.wstride = (long long)c->L.wpad; a.M = M;
     a.threshold = (unsigned)(M / 2 + 1);
     a.words = c->words(c->srv()); a.x = c->x(); a.tiles = c->tiles(); a.eta = c->eta;
+    a.lim = c->limits();
     switch (planes_for(M)) {
         case 1: launch_vote_server_t<1>(c, a); break;
         case 2: launch_vote_server_t<2>(c, a); break;

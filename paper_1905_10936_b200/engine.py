@@ -30,7 +30,8 @@ class EFEngine:
     def __init__(self, offsets, M: int, mu: float, eta: float, host_staging: bool = False,
                  scale_mode: str = "auto", weight_decay: bool = False, diagnostics: bool = False,
                  stream: Optional[torch.cuda.Stream] = None, device: Optional[torch.device] = None,
-                 one_local_worker: bool = False, extra_flags: int = 0):
+                 one_local_worker: bool = False, extra_flags: int = 0,
+                 workspace: Optional[torch.Tensor] = None):
         if not torch.cuda.is_available():
             raise RuntimeError("EFEngine needs a CUDA device (there is no CPU path)")
         self.device = torch.device(device if device is not None else f"cuda:{torch.cuda.current_device()}")
@@ -48,7 +49,11 @@ class EFEngine:
         nbytes = ef.ef_workspace_bytes(self.d, self.B, self.offsets, self.M, flags)
         self.workspace_bytes = nbytes
         with torch.cuda.device(self.device):
-            self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            if workspace is None:
+                workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            assert workspace.is_cuda and workspace.dtype == torch.uint8 and workspace.is_contiguous()
+            assert workspace.numel() >= nbytes and workspace.data_ptr() % 256 == 0
+            self.workspace = workspace
             self.stream = stream if stream is not None else torch.cuda.current_stream()
             self.ctx = ef.ef_init(self.d, self.B, self.offsets, self.M, float(mu), float(eta), flags,
                                   self.workspace.data_ptr(), nbytes, self.stream.cuda_stream)
