@@ -250,7 +250,7 @@ def run_ours(args) -> None:
     stream = torch.cuda.Stream(device=dev)
     torch.cuda.set_stream(stream)
     eng = EFEngine(w.offsets, w.M, w.mu, w.eta, stream=stream, weight_decay=args.weight_decay > 0,
-                   diagnostics=args.diagnostics)
+                   diagnostics=args.diagnostics, extra_flags=args.library_flags)
     if args.weight_decay > 0:
         eng.set_weight_decay(args.weight_decay)
     es = w.element_scales(dev)
@@ -426,7 +426,8 @@ def run_ours(args) -> None:
         "higher_is_better": True, "scaling": args.scaling if world > 1 else "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": config_dict(w_full),
-        "run": {"workload": args.workload, "weight_decay": args.weight_decay, "diagnostics": bool(args.diagnostics),
+        "run": {"workload": args.workload, "library_flags": args.library_flags,
+                "weight_decay": args.weight_decay, "diagnostics": bool(args.diagnostics),
                 "worker_calls": "ef_worker_step_all" if batched else "ef_worker_step x M",
                 "gradient_batches_rotated": nbatch,
                 "per_gpu": ("every rank owns one whole layout (a block-range shard of an N-times "
@@ -546,6 +547,9 @@ def main():
     ap.add_argument("--graph", action="store_true",
                     help="also time the step replayed from a CUDA graph (extra key cuda_graph)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--library-flags", type=int, default=0,
+                    help="extra EF_FLAG_* bits for ef_init (A/B comparisons: 512 = per-thread staging in "
+                         "the server kernel, 1024 = programmatic instead of ordinary launches)")
     ap.add_argument("--sustained-steps", type=int, default=300,
                     help="extra back-to-back steps timed as one region with the clocks sampled "
                          "(key `sustained`; 0 = skip)")

@@ -79,6 +79,11 @@ enum ef_status {
                                       multiple of 128 elements, M <= 16) and with per-thread asynchronous
                                       copies otherwise; this flag forces the latter (for comparisons;
                                       results are identical). */
+#define EF_FLAG_PROGRAMMATIC_LAUNCH 1024u /* Launch the kernels with programmatic stream serialization: each
+                                      may be scheduled while its predecessor on the stream drains and waits
+                                      on the device for the predecessor's results.  Off by default: on B200
+                                      it did not shorten the launch-bound small layouts (results are
+                                      identical either way). */
 #define EF_FLAG_DIAGNOSTICS 16u    /* worker steps also record per-block sums (ef_worker_diagnostics);
                                       implies the follow-up scale kernel, excludes EF_FLAG_FUSED_SCALE */
 
@@ -214,8 +219,9 @@ uint32_t* ef_status_word(ef_ctx* ctx);   /* the word itself (device, inside the 
  * ef_check_status.  Nothing traps or asserts, so the context and the device stay usable.  (A
  * memory checker for the device is not always available; this is the library's own net.)
  * ef_debug_build: 1 if this library is the checked build.  ef_debug_shift_tile: test hook of the
- * checked build only (EF_ERR_BAD_STATE otherwise): moves the start of one tile descriptor by
- * `delta` elements, between iterations, so that a test can see the check refuse it. */
+ * checked build only (EF_ERR_BAD_STATE otherwise): moves the start of one tile descriptor
+ * (tile = -1: the last one) by `delta` elements, between iterations, so that a test can see the
+ * check refuse it. */
 int ef_debug_build(void);
 int ef_debug_shift_tile(ef_ctx* ctx, int64_t tile, int64_t delta);
 

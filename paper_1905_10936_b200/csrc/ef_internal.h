@@ -7,6 +7,7 @@
 
 #include <cstddef>
 #include <cstdint>
+#include <utility>
 #include <vector>
 
 namespace efh {
@@ -21,7 +22,6 @@ inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a
 // and apply kernels), a tile is kTileChunks chunks (one CTA of the server kernel).
 constexpr int kU = 4;
 constexpr int kChunkLen = 1024 * kU;
-constexpr int kTileLen = kChunkLen * efk::kTileChunks;
 // Grids up to this many chunks (about two waves of CTAs) finalise block scales in-kernel.
 constexpr int64_t kFusedMaxChunks = 1024;
 
@@ -31,6 +31,7 @@ struct Layout {
     int32_t Ml = 0;                                   // worker state slots held here: M, or 1 with
                                                       // EF_FLAG_ONE_LOCAL_WORKER; the server's buffers sit in slot Ml
     int64_t num_tiles = 0;
+    int32_t tile_chunks = 0;                          // chunks per tile: 1 for launch-bound layouts, else kTileChunks
     size_t dpad = 0, wpad = 0, bpad = 0, tpad = 0;    // padded element counts per sub-buffer
     size_t off_x = 0, off_m = 0, off_pb = 0, off_spb = 0, off_words = 0, off_scales = 0,
            off_rscale = 0, off_partials = 0, off_tickets = 0, off_tiles = 0, off_blocks = 0,
@@ -63,6 +64,7 @@ struct ef_ctx {
     std::vector<int32_t> h_multi;
     int fused = 0;                         // block scales finalised inside the main kernels
     bool use_bulk = false;                 // the server kernel stages its inputs with cp.async.bulk
+    bool pdl = false;                      // kernels are launched with programmatic stream serialization
     // host-staging path
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t ev_copied[2] = {nullptr, nullptr};
@@ -88,7 +90,7 @@ struct ef_ctx {
     double* diag(int i) const { return (double*)(ws + L.off_diag) + (size_t)i * 4 * L.bpad; }
     float* stage(int s) const { return (float*)(ws + L.off_stage) + (size_t)s * L.dpad; }
     unsigned* status() const { return (unsigned*)(ws + L.off_status); }
-    efk::DebugLimits limits() const { return efk::DebugLimits{L.d, L.W, L.B, status()}; }
+    efk::DebugLimits limits() const { return efk::DebugLimits{L.d, L.W, L.B, L.tile_chunks, status()}; }
 };
 
 namespace efh {
@@ -109,6 +111,25 @@ inline int cuda_fail(ef_ctx* c, cudaError_t e) {
     } while (0)
 
 inline bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+// Launches one of the library's kernels (all take their arguments by value and run kThreads
+// threads per CTA) on the context's stream.  With programmatic stream serialization the kernel
+// may be scheduled while its predecessor on the stream drains; every kernel begins with
+// efk::pdl_enter(), which holds it back until the predecessor's results are complete.
+template <typename... KArgs, typename... Args>
+inline void launch_kernel(ef_ctx* c, void (*kernel)(KArgs...), dim3 grid, size_t smem, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(efk::kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = c->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = c->pdl ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 // Common checks of a per-worker call of method `mode`.
 inline int check_worker_call(ef_ctx* c, int32_t i, const float* grad, int mode) {

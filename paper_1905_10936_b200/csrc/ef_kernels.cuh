@@ -15,7 +15,8 @@
 // whereas a device-wide fence in every CTA costs about 8% of the streaming rate) or, for small
 // launch-bound grids, by the last CTA to finish the block (one atomic ticket, no waiting).
 //
-// Work decomposition.  The flat vector is cut into tiles of at most kTileChunks chunks of
+// Work decomposition.  The flat vector is cut into tiles of at most `tc` chunks (tc = kTileChunks
+// for bandwidth-bound layouts, 1 for small launch-bound ones, where more and shorter CTAs win) of
 // 1024*U elements; a tile never crosses a block boundary.  The worker kernel runs one CTA per
 // chunk (three read and two write streams of 16 KB each per CTA keep enough bytes in flight).
 // The server and apply kernels have one read and one write stream only, so one CTA walks all
@@ -35,7 +36,7 @@ namespace efk {
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr unsigned kFull = 0xffffffffu;
-constexpr int kTileChunks = 4;        // chunks per tile; also partial-sum slots per tile
+constexpr int kTileChunks = 4;        // most chunks per tile; partial-sum slots per tile = the layout's tc
 
 // A tile is a run of at most kTileChunks*1024*U consecutive elements inside one block.  Tiles
 // of a block start at multiples of the tile length from the block's first element, so tiles
@@ -58,13 +59,14 @@ struct __align__(16) Block {
 };
 static_assert(sizeof(Block) == 32, "Block must be 32 bytes");
 
-// Limits of the problem, carried by every launch.  A build with -DEF_DEBUG checks each CTA's
+// Sizes of the problem, carried by every launch.  A build with -DEF_DEBUG checks each CTA's
 // work item (tile or chunk descriptor) against them before touching memory: a descriptor that
 // reaches outside its arrays is not used; the CTA records kStatusBounds in the status word and
 // ends (no trap, no assert: the context stays usable and ef_check_status reports it).
 struct DebugLimits {
     long long d, W;      // elements, packed words
     int B;               // blocks
+    int tc;              // chunks per tile of this layout (1 or kTileChunks)
     unsigned* status;
 };
 constexpr unsigned kStatusBounds = 2u;
@@ -150,6 +152,7 @@ struct ScaleArgs {
     int scale_stride;
     double* dpartials;          // DIAG instantiation only, as in WorkerArgs
     double* diag;
+    int tc;                     // chunks (= partial-sum slots) per tile
 };
 
 struct ApplyArgs {
@@ -175,6 +178,18 @@ struct ResidualArgs {
     const Tile* tiles;
     DebugLimits lim;
 };
+
+// ------------------------------------------------------------------ programmatic dependent launch
+// Every kernel of the library starts with pdl_enter(): it waits until the kernel launched before
+// it on the stream has completed and its writes are visible (a no-op for an ordinary launch),
+// then lets the kernel launched after it be scheduled as soon as SM resources free up.  With the
+// launch attribute set on the host side this overlaps each kernel's launch latency and ramp-up
+// with its predecessor's tail; the data dependence is still enforced by the wait, so nothing
+// may touch global memory before pdl_enter().
+__device__ __forceinline__ void pdl_enter() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 
 // ------------------------------------------------------------------ small helpers
 // Streaming accesses go through L2 only (.cg): every byte is used once per launch, and on
@@ -249,9 +264,9 @@ __device__ __forceinline__ double cta_sum(double v, double* s_sum) {
 // the CTA tree) and writes the scale s_b = ||p_b||_1 / d_b (Section 3.2).  Called by a whole CTA.
 // Sum of the block's partial-sum slots in a fixed order; valid in thread 0.
 __device__ __forceinline__ double sum_slots(const Block& b, const double* __restrict__ partials,
-                                            double* s_sum) {
-    const double* src = partials + (long long)b.tile_begin * kTileChunks;
-    const int n = b.tile_count * kTileChunks;
+                                            double* s_sum, int tc) {
+    const double* src = partials + (long long)b.tile_begin * tc;
+    const int n = b.tile_count * tc;
     double v = 0.0;
     for (int k = threadIdx.x; k < n; k += kThreads) v += __ldcg(&src[k]);
     return cta_sum(v, s_sum);
@@ -261,8 +276,8 @@ __device__ __forceinline__ double sum_partials_and_write(const Block& b, int blo
                                                          const double* __restrict__ partials,
                                                          float* __restrict__ scale_out,
                                                          float* __restrict__ rscale,
-                                                         double* s_sum) {
-    const double S = sum_slots(b, partials, s_sum);
+                                                         double* s_sum, int tc) {
+    const double S = sum_slots(b, partials, s_sum, tc);
     if (threadIdx.x == 0) {
         const float s = (float)(S / (double)b.len);
         scale_out[block_id] = s;
@@ -284,7 +299,7 @@ __device__ __forceinline__ void finish_block(double acc, long long slot, int zer
                                              double* __restrict__ partials,
                                              unsigned* __restrict__ tickets,
                                              float* __restrict__ scale_out,
-                                             float* __restrict__ rscale, int fused) {
+                                             float* __restrict__ rscale, int fused, int tc) {
     __shared__ double s_sum[kWarps];
     __shared__ int s_last;
     const double S = cta_sum(acc, s_sum);
@@ -310,7 +325,7 @@ __device__ __forceinline__ void finish_block(double acc, long long slot, int zer
     if (!s_last) return;
     __threadfence();
     const Block b = blocks[block_id];
-    sum_partials_and_write(b, block_id, partials, scale_out, rscale, s_sum);
+    sum_partials_and_write(b, block_id, partials, scale_out, rscale, s_sum, tc);
     if (threadIdx.x == 0) tickets[block_id] = 0u;      // ready for the next launch
 }
 
@@ -319,11 +334,12 @@ __device__ __forceinline__ void finish_block(double acc, long long slot, int zer
 template <bool DIAG>
 __global__ void __launch_bounds__(kThreads) ef_scale_kernel(const ScaleArgs a) {
     __shared__ double s_sum[kWarps];
+    pdl_enter();
     const int block_id = a.multi[blockIdx.x];
     const Block b = a.blocks[block_id];
     const long long so = (long long)blockIdx.y * a.scale_stride;
     const double S = sum_partials_and_write(b, block_id, a.partials + blockIdx.y * a.partial_stride,
-                                            a.scale_out + so, a.rscale + so, s_sum);
+                                            a.scale_out + so, a.rscale + so, s_sum, a.tc);
     if (DIAG) {
         double* dg = a.diag + (so + block_id) * 4;
         if (threadIdx.x == 0) dg[0] = S;
@@ -331,7 +347,7 @@ __global__ void __launch_bounds__(kThreads) ef_scale_kernel(const ScaleArgs a) {
 #pragma unroll
         for (int k = 0; k < 3; ++k) {
             __syncthreads();
-            const double v = sum_slots(b, dp + k * a.partial_stride, s_sum);
+            const double v = sum_slots(b, dp + k * a.partial_stride, s_sum, a.tc);
             if (threadIdx.x == 0) dg[1 + k] = v;
         }
     }
@@ -513,6 +529,7 @@ __device__ __forceinline__ double worker_rows_scalar(const WorkerArgs& a, const 
 // grid.x = chunks, grid.y = workers stepped by this launch (1 for ef_worker_step).
 template <int U, bool DIAG>
 __global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a0) {
+    pdl_enter();
     WorkerArgs a = a0;
     {
         const long long wi = blockIdx.y;
@@ -529,7 +546,7 @@ __global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a0
         a.rscale += wi * a.scale_stride;
         a.tickets += wi * a.scale_stride;
     }
-    const Tile t = chunk_of<U>(a.tiles[blockIdx.x / kTileChunks], blockIdx.x % kTileChunks);
+    const Tile t = chunk_of<U>(a.tiles[blockIdx.x / a.lim.tc], blockIdx.x % a.lim.tc);
     if (!work_item_ok(t, a.lim, 1024 * U)) return;
     const Block b = a.blocks[t.block];
     const bool alone = b.len <= 1024 * U;              // the block is this single chunk
@@ -549,8 +566,8 @@ __global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a0
         finish_block_diag(acc, dacc, blockIdx.x, alone, t.block, b.len, a.partials, a.dpartials,
                           a.partial_stride, a.diag, a.scale_out, a.rscale);
     else
-        finish_block(acc, blockIdx.x, 0, alone, (unsigned)(b.tile_count * kTileChunks), t.block,
-                     a.blocks, a.partials, a.tickets, a.scale_out, a.rscale, a.fused);
+        finish_block(acc, blockIdx.x, 0, alone, (unsigned)(b.tile_count * a.lim.tc), t.block,
+                     a.blocks, a.partials, a.tickets, a.scale_out, a.rscale, a.fused, a.lim.tc);
 }
 
 // ------------------------------------------------------------------ server kernel
@@ -1060,8 +1077,9 @@ __global__ void __launch_bounds__(kThreads) ef_server_kernel(const ServerArgs a)
         }
         __syncthreads();
     }
+    pdl_enter();                       // the barrier set-up above overlaps the previous kernel's tail
     const Tile t = a.tiles[blockIdx.x + a.tile0];
-    if (!work_item_ok(t, a.lim, kTileChunks * 1024 * U)) return;
+    if (!work_item_ok(t, a.lim, a.lim.tc * 1024 * U)) return;
     const float sp = a.rscale[t.block];
     double acc = 0.0;
     if (MT > 0 && (t.start & 3) == 0) {
@@ -1079,9 +1097,9 @@ __global__ void __launch_bounds__(kThreads) ef_server_kernel(const ServerArgs a)
         }
     }
     const Block b = a.blocks[t.block];
-    finish_block(acc, (long long)(blockIdx.x + a.tile0) * kTileChunks, kTileChunks - 1, b.len <= 1024 * U,
+    finish_block(acc, (long long)(blockIdx.x + a.tile0) * a.lim.tc, a.lim.tc - 1, b.len <= 1024 * U,
                  (unsigned)b.tile_count, t.block, a.blocks, a.partials, a.tickets, a.scale_out,
-                 a.rscale, a.fused);
+                 a.rscale, a.fused, a.lim.tc);
 }
 
 // ------------------------------------------------------------------ parameter update
@@ -1106,8 +1124,9 @@ __device__ __forceinline__ float apply_one(const ApplyArgs& a, float x, float si
 template <int U, bool DECAY>
 __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
     constexpr int kChunk = 1024 * U;
+    pdl_enter();
     const Tile t = a.tiles[blockIdx.x + a.tile0];
-    if (!work_item_ok(t, a.lim, kTileChunks * kChunk)) return;
+    if (!work_item_ok(t, a.lim, a.lim.tc * kChunk)) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // packed words of this tile and the block's scale: plain layout or a fused message
     const uint32_t* const twords =
@@ -1187,6 +1206,7 @@ __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
 // dst_j = p_j - s_b * sign(p_j): the residual e_{t+1} in its plain form (tests, checkpoints).
 // One tile per CTA.
 static __global__ void __launch_bounds__(kThreads) ef_residual_kernel(const ResidualArgs a) {
+    pdl_enter();
     const Tile t = a.tiles[blockIdx.x];
     if (!work_item_ok(t, a.lim, 1 << 30)) return;
     const float s = a.rscale[t.block];
@@ -1207,6 +1227,7 @@ struct PackArgs {
     DebugLimits lim;
 };
 static __global__ void __launch_bounds__(kThreads) ef_pack_kernel(const PackArgs a) {
+    pdl_enter();
     const Tile t = a.tiles[blockIdx.x + a.tile0];
     if (!work_item_ok(t, a.lim, 1 << 30)) return;
     const Block b = a.blocks[t.block];
@@ -1221,6 +1242,7 @@ static __global__ void __launch_bounds__(kThreads) ef_pack_kernel(const PackArgs
 // keeps the "no -0 in a residual buffer" invariant of the sign-bit tests above.
 static __global__ void __launch_bounds__(kThreads) ef_import_kernel(const float* __restrict__ src,
                                                              float* __restrict__ dst, long long n) {
+    pdl_enter();
     for (long long j = blockIdx.x * (long long)kThreads + threadIdx.x; j < n;
          j += (long long)gridDim.x * kThreads)
         dst[j] = __fadd_rn(src[j], 0.0f);

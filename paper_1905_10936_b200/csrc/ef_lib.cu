@@ -31,25 +31,32 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
     if (rc != EF_OK) return rc;
     if (flags & ~(EF_FLAG_HOST_STAGING | EF_FLAG_FUSED_SCALE | EF_FLAG_SPLIT_SCALE |
                   EF_FLAG_WEIGHT_DECAY | EF_FLAG_DIAGNOSTICS | EF_FLAG_ONE_LOCAL_WORKER |
-                  EF_FLAG_SERVER_NO_BULK))
+                  EF_FLAG_SERVER_NO_BULK | EF_FLAG_PROGRAMMATIC_LAUNCH))
         return EF_ERR_INVALID_ARG;
     if ((flags & EF_FLAG_FUSED_SCALE) && (flags & (EF_FLAG_SPLIT_SCALE | EF_FLAG_DIAGNOSTICS)))
         return EF_ERR_INVALID_ARG;
     L->d = d; L->B = B; L->M = M;
     L->Ml = (flags & EF_FLAG_ONE_LOCAL_WORKER) ? 1 : M;
-    int64_t W = 0, T = 0;
+    int64_t W = 0, chunks = 0;
     for (int32_t b = 0; b < B; ++b) {
         const int64_t db = offsets[b + 1] - offsets[b];
         W += (db + 31) / 32;
-        T += (db + kTileLen - 1) / kTileLen;
+        chunks += (db + kChunkLen - 1) / kChunkLen;
         if (db > kChunkLen) L->num_multi += 1;
     }
-    if (T * efk::kTileChunks > 0x7fffffffLL) return EF_ERR_INVALID_ARG;
+    // Small layouts are launch-bound: one chunk per tile gives the server and update kernels
+    // four times as many (and shorter) CTAs.  Large ones amortise the per-tile set-up over
+    // kTileChunks chunks.
+    L->tile_chunks = (chunks <= kFusedMaxChunks) ? 1 : efk::kTileChunks;
+    const int64_t tile_len = (int64_t)kChunkLen * L->tile_chunks;
+    int64_t T = 0;
+    for (int32_t b = 0; b < B; ++b) T += (offsets[b + 1] - offsets[b] + tile_len - 1) / tile_len;
+    if (T * L->tile_chunks > 0x7fffffffLL) return EF_ERR_INVALID_ARG;
     L->W = W; L->num_tiles = T;
     L->dpad = align_up((size_t)d * 4) / 4;
     L->wpad = align_up((size_t)W * 4) / 4;
     L->bpad = align_up((size_t)B * 4) / 4;
-    L->tpad = align_up((size_t)T * efk::kTileChunks * 8) / 8;   // partial-sum slots
+    L->tpad = align_up((size_t)T * L->tile_chunks * 8) / 8;     // partial-sum slots
     const size_t Ml = (size_t)L->Ml, M1 = Ml + 1;
     size_t o = 0;
     L->off_x = o;        o += L->dpad * 4;
@@ -86,12 +93,13 @@ int launch_scale(ef_ctx* c, int k, int count = 1) {
     a.partials = c->partials(k); a.blocks = c->blocks(); a.multi = c->multi();
     a.scale_out = c->scales(k); a.rscale = c->rscale(k);
     a.partial_stride = (long long)c->L.tpad; a.scale_stride = (int)c->L.bpad;
+    a.tc = c->L.tile_chunks;
     const bool diag = (c->flags & EF_FLAG_DIAGNOSTICS) && k < c->L.Ml;
     a.dpartials = diag ? c->dpartials(k) : nullptr;
     a.diag = diag ? c->diag(k) : nullptr;
     const dim3 grid((unsigned)c->L.num_multi, (unsigned)count);
-    if (diag) efk::ef_scale_kernel<true><<<grid, efk::kThreads, 0, c->stream>>>(a);
-    else efk::ef_scale_kernel<false><<<grid, efk::kThreads, 0, c->stream>>>(a);
+    if (diag) launch_kernel(c, efk::ef_scale_kernel<true>, grid, 0, a);
+    else launch_kernel(c, efk::ef_scale_kernel<false>, grid, 0, a);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
     return EF_OK;
@@ -112,9 +120,9 @@ int launch_worker(ef_ctx* c, int i, const float* grad, int count = 1, long long 
     a.dpartials = diag ? c->dpartials(i) : nullptr;
     a.diag = diag ? c->diag(i) : nullptr;
     a.lim = c->limits();
-    const dim3 grid((unsigned)(c->L.num_tiles * efk::kTileChunks), (unsigned)count);
-    if (diag) efk::ef_worker_kernel<kU, true><<<grid, efk::kThreads, 0, c->stream>>>(a);
-    else efk::ef_worker_kernel<kU, false><<<grid, efk::kThreads, 0, c->stream>>>(a);
+    const dim3 grid((unsigned)(c->L.num_tiles * c->L.tile_chunks), (unsigned)count);
+    if (diag) launch_kernel(c, efk::ef_worker_kernel<kU, true>, grid, 0, a);
+    else launch_kernel(c, efk::ef_worker_kernel<kU, false>, grid, 0, a);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
     return launch_scale(c, i, count);
@@ -173,9 +181,9 @@ template <int MT>
 cudaError_t launch_server_t(ef_ctx* c, const efk::ServerArgs& a, unsigned grid, bool bulk) {
     constexpr int MS = MT > 0 ? MT : 1;
     if (MT > 0 && bulk)
-        efk::ef_server_kernel<kU, MS, true><<<grid, efk::kThreads, server_smem_bytes<MT>(c->L.M, true), c->stream>>>(a);
+        launch_kernel(c, efk::ef_server_kernel<kU, MS, true>, dim3(grid), server_smem_bytes<MT>(c->L.M, true), a);
     else
-        efk::ef_server_kernel<kU, MT, false><<<grid, efk::kThreads, server_smem_bytes<MT>(c->L.M, false), c->stream>>>(a);
+        launch_kernel(c, efk::ef_server_kernel<kU, MT, false>, dim3(grid), server_smem_bytes<MT>(c->L.M, false), a);
     return cudaGetLastError();
 }
 
@@ -231,8 +239,8 @@ int launch_server_range(ef_ctx* c, int b0, int b1, const uint32_t* msgs, long lo
             sa.partials = c->partials(S); sa.blocks = c->blocks(); sa.multi = c->multi() + lo;
             sa.scale_out = c->scales(S); sa.rscale = c->rscale(S);
             sa.partial_stride = (long long)c->L.tpad; sa.scale_stride = (int)c->L.bpad;
-            sa.dpartials = nullptr; sa.diag = nullptr;
-            efk::ef_scale_kernel<false><<<dim3((unsigned)(hi - lo), 1), efk::kThreads, 0, c->stream>>>(sa);
+            sa.dpartials = nullptr; sa.diag = nullptr; sa.tc = c->L.tile_chunks;
+            launch_kernel(c, efk::ef_scale_kernel<false>, dim3((unsigned)(hi - lo), 1), 0, sa);
             EF_CUDA(c, cudaGetLastError());
             c->launches += 1;
         }
@@ -253,9 +261,9 @@ int launch_apply_range(ef_ctx* c, int b0, int b1, const uint32_t* update) {
     p.eta = c->eta; p.mu = c->mu; p.lambda = c->lambda; p.mt = c->mt();
     p.lim = c->limits();
     if (c->lambda > 0.f)
-        efk::ef_apply_kernel<kU, true><<<tr.count, efk::kThreads, 0, c->stream>>>(p);
+        launch_kernel(c, efk::ef_apply_kernel<kU, true>, dim3(tr.count), 0, p);
     else
-        efk::ef_apply_kernel<kU, false><<<tr.count, efk::kThreads, 0, c->stream>>>(p);
+        launch_kernel(c, efk::ef_apply_kernel<kU, false>, dim3(tr.count), 0, p);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
     return EF_OK;
@@ -311,6 +319,7 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
     c->L = L; c->mu = mu; c->eta = eta; c->eta_prev = eta; c->flags = flags;
     c->ws = (char*)workspace;
     c->stream = (cudaStream_t)cuda_stream;
+    c->pdl = (flags & EF_FLAG_PROGRAMMATIC_LAUNCH) != 0;
     try {
     c->stepped.assign(L.Ml, 0);
     c->served.assign(B, 0);
@@ -325,10 +334,11 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
         Block& blk = c->h_blocks[b];
         blk.start = start; blk.len = len; blk.word = word;
         blk.tile_begin = (int)c->h_tiles.size();
-        for (int64_t o = 0; o < len; o += kTileLen) {
+        const int64_t tile_len = (int64_t)kChunkLen * L.tile_chunks;
+        for (int64_t o = 0; o < len; o += tile_len) {
             Tile t;
             t.start = start + o; t.word = word + o / 32;
-            t.len = (int)((len - o < kTileLen) ? (len - o) : kTileLen);
+            t.len = (int)((len - o < tile_len) ? (len - o) : tile_len);
             t.block = b; t.pad0 = 0; t.pad1 = 0;
             c->h_tiles.push_back(t);
         }
@@ -344,7 +354,7 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
     // are bandwidth-bound: the per-CTA fence of the fused form costs more than a tiny launch.
     if (flags & EF_FLAG_FUSED_SCALE) c->fused = 1;
     else if (flags & (EF_FLAG_SPLIT_SCALE | EF_FLAG_DIAGNOSTICS)) c->fused = 0;
-    else c->fused = (L.num_tiles * efk::kTileChunks <= kFusedMaxChunks) ? 1 : 0;
+    else c->fused = (L.tile_chunks == 1) ? 1 : 0;
 
     auto fail = [&](cudaError_t e) { delete c; (void)e; return EF_ERR_CUDA; };
     // Algorithm 4 "Initialize": x_0, m, e, etilde = 0; also words, scales, tickets, partials.
@@ -450,7 +460,7 @@ int ef_pack_message(ef_ctx* c, int32_t who, int32_t b0, int32_t b1, uint32_t* ds
     a.tiles = c->tiles(); a.blocks = c->blocks(); a.tile0 = tr.tile0;
     a.msg_base = efk::message_unit(c->h_blocks[b0].word, b0);
     a.lim = c->limits();
-    efk::ef_pack_kernel<<<tr.count, efk::kThreads, 0, c->stream>>>(a);
+    launch_kernel(c, efk::ef_pack_kernel, dim3(tr.count), 0, a);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
     return EF_OK;
@@ -544,7 +554,7 @@ int ef_get_residual(ef_ctx* c, int32_t i, float* dst) {
     efk::ResidualArgs a;
     a.pb = c->pb(k); a.rscale = c->rscale(k); a.dst = dst; a.tiles = c->tiles();
     a.lim = c->limits();
-    efk::ef_residual_kernel<<<(unsigned)c->L.num_tiles, efk::kThreads, 0, c->stream>>>(a);
+    launch_kernel(c, efk::ef_residual_kernel, dim3((unsigned)c->L.num_tiles), 0, a);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
     return EF_OK;
@@ -563,7 +573,7 @@ int ef_set_state(ef_ctx* c, int32_t i, const float* momentum, const float* resid
     {
         const long long n = c->L.d;
         const unsigned grid = (unsigned)std::min<long long>((n + efk::kThreads - 1) / efk::kThreads, 148 * 16);
-        efk::ef_import_kernel<<<grid, efk::kThreads, 0, c->stream>>>(residual, c->pb(k), n);
+        launch_kernel(c, efk::ef_import_kernel, dim3(grid), 0, residual, c->pb(k), n);
         EF_CUDA(c, cudaGetLastError());
         c->launches += 1;
     }
@@ -598,6 +608,7 @@ int ef_debug_build(void) {
 
 int ef_debug_shift_tile(ef_ctx* c, int64_t tile, int64_t delta) {
 #ifdef EF_DEBUG
+    if (c && tile == -1) tile = c->L.num_tiles - 1;          // -1 names the last tile
     if (!c || tile < 0 || tile >= c->L.num_tiles || c->pending != 0) return EF_ERR_INVALID_ARG;
     c->h_tiles[(size_t)tile].start += delta;
     EF_CUDA(c, cudaMemcpyAsync(c->ws + c->L.off_tiles + (size_t)tile * sizeof(Tile), &c->h_tiles[(size_t)tile],

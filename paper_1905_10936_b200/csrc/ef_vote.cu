@@ -100,12 +100,13 @@ __device__ __forceinline__ void vote_worker_rows_scalar(const VoteWorkerArgs& a,
 
 template <int U>
 __global__ void __launch_bounds__(kThreads) ef_vote_worker_kernel(const VoteWorkerArgs a0) {
+    efk::pdl_enter();
     VoteWorkerArgs a = a0;
     const long long wi = blockIdx.y;
     a.g += wi * a.g_stride;
     a.m += wi * a.state_stride;
     a.words += wi * a.word_stride;
-    const Tile t = efk::chunk_of<U>(a.tiles[blockIdx.x / efk::kTileChunks], blockIdx.x % efk::kTileChunks);
+    const Tile t = efk::chunk_of<U>(a.tiles[blockIdx.x / a.lim.tc], blockIdx.x % a.lim.tc);
     if (t.len <= 0 || !efk::work_item_ok(t, a.lim, 1024 * U)) return;
     if ((t.start & 3) != 0) vote_worker_rows_scalar(a, t);
     else if (t.len == 1024 * U) vote_worker_rows<U, true>(a, t);
@@ -171,8 +172,9 @@ __device__ __forceinline__ void vote_apply4(float (&x)[4], unsigned nib, float e
 template <int U, int P>
 __global__ void __launch_bounds__(kThreads) ef_vote_server_kernel(const VoteServerArgs a) {
     constexpr int kChunk = 1024 * U;
+    efk::pdl_enter();
     const Tile t = a.tiles[blockIdx.x];
-    if (!efk::work_item_ok(t, a.lim, efk::kTileChunks * kChunk)) return;
+    if (!efk::work_item_ok(t, a.lim, a.lim.tc * kChunk)) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if ((t.start & 3) != 0) {                   // block does not start on a 16-byte boundary
         const int rows = (t.len + 31) >> 5;
@@ -226,7 +228,7 @@ int planes_for(int M) {
 
 template <int P>
 void launch_vote_server_t(ef_ctx* c, const VoteServerArgs& a) {
-    ef_vote_server_kernel<kU, P><<<(unsigned)c->L.num_tiles, kThreads, 0, c->stream>>>(a);
+    launch_kernel(c, ef_vote_server_kernel<kU, P>, dim3((unsigned)c->L.num_tiles), 0, a);
 }
 
 int launch_vote_worker(ef_ctx* c, int i, const float* grad, int count, long long g_stride) {
@@ -234,8 +236,8 @@ int launch_vote_worker(ef_ctx* c, int i, const float* grad, int count, long long
     a.g = grad; a.m = c->m(i); a.words = c->words(i); a.tiles = c->tiles(); a.mu = c->mu;
     a.g_stride = g_stride; a.state_stride = (long long)c->L.dpad; a.word_stride = (long long)c->L.wpad;
     a.lim = c->limits();
-    const dim3 grid((unsigned)(c->L.num_tiles * efk::kTileChunks), (unsigned)count);
-    ef_vote_worker_kernel<kU><<<grid, kThreads, 0, c->stream>>>(a);
+    const dim3 grid((unsigned)(c->L.num_tiles * c->L.tile_chunks), (unsigned)count);
+    launch_kernel(c, ef_vote_worker_kernel<kU>, grid, 0, a);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
     return EF_OK;

@@ -141,16 +141,15 @@ def test_checked_build_refuses_a_descriptor_past_the_end(checked_library):
     eng.worker_step(0, g); eng.worker_step(1, g); eng.server_step()
     ef.ef_check_status(eng.ctx)                              # a valid problem reports nothing
     x_before = eng.params().clone()
-    # last tile of the last block, moved TILE elements to the right: it now ends past d, but
-    # still inside the workspace (the next array follows x directly)
-    last_tile = sum((s + BIG - 1) // BIG for s in sizes) - 1
-    ef.ef_debug_shift_tile(eng.ctx, last_tile, TILE)
+    # the last tile (the last TILE elements of this small layout), moved TILE elements to the
+    # right: it now ends past d, but still inside the workspace (the next array follows x directly)
+    ef.ef_debug_shift_tile(eng.ctx, -1, TILE)
     eng.worker_step(0, g); eng.worker_step(1, g); eng.server_step()
     with pytest.raises(ef.EFError) as ei:
         ef.ef_check_status(eng.ctx)
     assert ei.value.status == ef.EF_ERR_BOUNDS
     # the refused tile was not processed: its parameters are unchanged
-    lo = int(w.offsets[-1]) - (2 * BIG - BIG)                # start of the last tile
+    lo = int(w.offsets[-1]) - TILE                           # start of the last tile
     assert torch.equal(eng.params()[lo:], x_before[lo:])
     assert ws.intact()
     ef.ef_check_status(eng.ctx)                              # the word was cleared

@@ -79,7 +79,7 @@ def test_batched_and_per_worker_calls_are_bit_identical():
     assert ei.value.status == ef.EF_ERR_BAD_STATE
 
 
-@pytest.mark.parametrize("variant", ["bulk where eligible", "per-thread"])
+@pytest.mark.parametrize("variant", ["bulk where eligible", "per-thread", "programmatic launches"])
 @pytest.mark.parametrize("sizes,M", [
     ([BIG, 2 * TILE, 5 * BIG + 128, 3 * TILE + 256, 640], 7),       # every block a multiple of 128: bulk-eligible
     ([8 * BIG + 3 * TILE, 128, 2 * BIG], 15),                       # two lane groups
@@ -90,9 +90,10 @@ def test_batched_and_per_worker_calls_are_bit_identical():
 ])
 def test_server_kernel_variants(sizes, M, variant):
     """The two ways the server kernel stages its inputs (bulk copies with an mbarrier where the
-    layout is eligible, per-thread asynchronous copies otherwise or when forced), both against
-    the oracle, in both scale modes."""
-    flags = {"bulk where eligible": 0, "per-thread": ef.EF_FLAG_SERVER_NO_BULK}[variant]
+    layout is eligible, per-thread asynchronous copies otherwise or when forced) and the optional
+    programmatic launches, all against the oracle, in both scale modes."""
+    flags = {"bulk where eligible": 0, "per-thread": ef.EF_FLAG_SERVER_NO_BULK,
+             "programmatic launches": ef.EF_FLAG_PROGRAMMATIC_LAUNCH}[variant]
     w = _wl("variants", sizes, M, steps=5, scale_range=(1e-3, 1.0))
     factory = lambda *a, **kw: EFEngine(*a, extra_flags=flags, **kw)
     eng, orc, stats = run_parity(w, scale_mode="split" if M % 2 else "fused", engine_factory=factory,
