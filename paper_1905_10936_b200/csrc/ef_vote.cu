@@ -10,8 +10,9 @@
 // bit (8 + (M+1)/8 bytes per element).  The vote itself is computed on whole 32-bit words: the
 // M packed words of a group of 32 elements are added into bit-sliced counters (plane p holds
 // bit p of every element's count of negative votes) with a ripple of half adders, and the
-// comparison count >= floor(M/2)+1 is evaluated on the planes, so a word of 32 votes costs
-// about 2 log2(M) logic operations per worker word and no per-element work at all.
+// comparison count >= floor(M/2)+1 is evaluated on the planes.  For M <= 16 the counters come
+// from a carry-save adder network (M = 7: eight logic operations for the 32 votes of a word),
+// for larger M from a ripple of half adders; either way there is no per-element work at all.
 #include "ef_internal.h"
 
 #include <algorithm>
@@ -114,48 +115,108 @@ __global__ void __launch_bounds__(kThreads) ef_vote_worker_kernel(const VoteWork
 }
 
 // ------------------------------------------------------------------ server
-// Majority of M packed words, bit-parallel, for R independent word positions at once (the R
-// positions' loads are issued together, eight workers at a time, so that up to 8 R loads are in
-// flight per thread).  P = number of counter planes (2^P > M).  Word position r of worker i is
-// w0[r * rstride + i * wstride]; positions with active[r] == false are not read and vote 0.
-template <int P, int R>
+// Majority of M packed words, bit-parallel.  Two forms:
+//  * M known at compile time (1..16): a carry-save adder network.  Words of equal weight are
+//    compressed three at a time by full adders (sum = x^y^z stays, carry = maj(x,y,z) moves one
+//    weight up: two logic operations for three words) until one word per weight is left: the
+//    planes of the count.  M = 7 takes 4 full adders, M = 15 takes 12.
+//  * any M: a ripple of half adders into P counter planes (2^P > M), eight workers' words loaded
+//    at a time.
+// Then count >= threshold is evaluated on the planes.
+template <int N>
+struct CsaLevel {     // a[0..N): words of one weight -> a[0]; the floor(N/2) carries go to up[0..)
+    __device__ __forceinline__ static void run(unsigned* a, unsigned* up) {
+        if constexpr (N >= 3) {
+            constexpr int F = N / 3, R = N % 3;
+            unsigned s[F + R];
+#pragma unroll
+            for (int i = 0; i < F; ++i) {
+                const unsigned x = a[3 * i], y = a[3 * i + 1], z = a[3 * i + 2];
+                s[i] = x ^ y ^ z;
+                up[i] = (x & y) | (z & (x ^ y));
+            }
+#pragma unroll
+            for (int i = 0; i < R; ++i) s[F + i] = a[3 * F + i];
+#pragma unroll
+            for (int i = 0; i < F + R; ++i) a[i] = s[i];
+            CsaLevel<F + R>::run(a, up + F);
+        } else if constexpr (N == 2) {
+            const unsigned x = a[0], y = a[1];
+            a[0] = x ^ y;
+            up[0] = x & y;
+        }
+    }
+};
+template <int N, int PLANE>
+struct CsaCount {     // a[0..N) of weight 2^PLANE -> planes[PLANE..]
+    __device__ __forceinline__ static void run(unsigned* a, unsigned* planes) {
+        unsigned up[N / 2 + 1];
+        CsaLevel<N>::run(a, up);
+        planes[PLANE] = a[0];
+        if constexpr (N / 2 > 0) CsaCount<N / 2, PLANE + 1>::run(up, planes);
+    }
+};
+__host__ __device__ constexpr int planes_of(int M) { int p = 1; while ((1 << p) <= M) ++p; return p; }
+
+// count >= threshold, from the least significant plane up:
+//   ge_p = (c_p > t_p) | ((c_p == t_p) & ge_{p-1}),  ge_{-1} = 1
+template <int P>
+__device__ __forceinline__ unsigned planes_ge(const unsigned (&c)[P], unsigned threshold) {
+    unsigned ge = 0xffffffffu;
+#pragma unroll
+    for (int p = 0; p < P; ++p) ge = ((threshold >> p) & 1u) ? (ge & c[p]) : (ge | c[p]);
+    return ge;
+}
+
+// MT > 0: M = MT at compile time; MT == 0: any M with P planes.  Word position r (of R) of
+// worker i is w0[r * rstride + i * wstride]; positions with active[r] == false are not read and
+// vote 0.
+template <int MT, int P, int R>
 __device__ __forceinline__ void majority_words(const uint32_t* __restrict__ w0, int rstride,
                                                long long wstride, int M, unsigned threshold,
                                                const bool (&active)[R], unsigned (&out)[R]) {
-    unsigned c[R][P];
+    if constexpr (MT > 0) {
+        unsigned w[R][MT];
 #pragma unroll
-    for (int r = 0; r < R; ++r)
-#pragma unroll
-        for (int p = 0; p < P; ++p) c[r][p] = 0u;
-    for (int i0 = 0; i0 < M; i0 += 8) {
-        unsigned w[R][8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k)
+        for (int i = 0; i < MT; ++i)
 #pragma unroll
             for (int r = 0; r < R; ++r)
-                w[r][k] = (i0 + k < M && active[r])
-                              ? __ldg(w0 + r * rstride + (long long)(i0 + k) * wstride) : 0u;
+                w[r][i] = active[r] ? __ldg(w0 + r * rstride + (long long)i * wstride) : 0u;
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
+        for (int r = 0; r < R; ++r) {
+            unsigned planes[planes_of(MT)];
+            CsaCount<MT, 0>::run(w[r], planes);
+            out[r] = planes_ge<planes_of(MT)>(planes, (unsigned)(MT / 2 + 1));
+        }
+    } else {
+        unsigned c[R][P];
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                unsigned carry = w[r][k];          // count += word, one half adder per plane
+        for (int r = 0; r < R; ++r)
 #pragma unroll
-                for (int p = 0; p < P; ++p) {
-                    const unsigned t = c[r][p] & carry;
-                    c[r][p] ^= carry;
-                    carry = t;
+            for (int p = 0; p < P; ++p) c[r][p] = 0u;
+        for (int i0 = 0; i0 < M; i0 += 8) {
+            unsigned w[R][8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+                    w[r][k] = (i0 + k < M && active[r])
+                                  ? __ldg(w0 + r * rstride + (long long)(i0 + k) * wstride) : 0u;
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    unsigned carry = w[r][k];          // count += word, one half adder per plane
+#pragma unroll
+                    for (int p = 0; p < P; ++p) {
+                        const unsigned t = c[r][p] & carry;
+                        c[r][p] ^= carry;
+                        carry = t;
+                    }
                 }
-            }
-    }
-    // count >= threshold, from the least significant plane up:
-    //   ge_p = (c_p > t_p) | ((c_p == t_p) & ge_{p-1}),  ge_{-1} = 1
+        }
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-        unsigned ge = 0xffffffffu;
-#pragma unroll
-        for (int p = 0; p < P; ++p) ge = ((threshold >> p) & 1u) ? (ge & c[r][p]) : (ge | c[r][p]);
-        out[r] = ge;
+        for (int r = 0; r < R; ++r) out[r] = planes_ge<P>(c[r], threshold);
     }
 }
 
@@ -168,9 +229,10 @@ __device__ __forceinline__ void vote_apply4(float (&x)[4], unsigned nib, float e
     }
 }
 
-// One tile per CTA; the CTA walks the tile's chunks.
-template <int U, int P>
-__global__ void __launch_bounds__(kThreads) ef_vote_server_kernel(const VoteServerArgs a) {
+// One tile per CTA; the CTA walks the tile's chunks, one or two rows of 128 elements at a time.
+// MT = M for 1 <= M <= 16 (adder network), else 0 with P counter planes.
+template <int U, int MT, int P>
+__global__ void __launch_bounds__(kThreads, 4) ef_vote_server_kernel(const VoteServerArgs a) {
     constexpr int kChunk = 1024 * U;
     efk::pdl_enter();
     const Tile t = a.tiles[blockIdx.x];
@@ -181,7 +243,7 @@ __global__ void __launch_bounds__(kThreads) ef_vote_server_kernel(const VoteServ
         for (int r = warp; r < rows; r += kWarps) {
             const bool one[1] = {true};
             unsigned vv[1];
-            majority_words<P, 1>(a.wwords + t.word + r, 0, a.wstride, a.M, a.threshold, one, vv);
+            majority_words<MT, P, 1>(a.wwords + t.word + r, 0, a.wstride, a.M, a.threshold, one, vv);
             const unsigned v = vv[0];
             const int o = r * 32 + lane;
             if (o < t.len) {
@@ -200,35 +262,34 @@ __global__ void __launch_bounds__(kThreads) ef_vote_server_kernel(const VoteServ
         const bool full = clen == kChunk;
         float* xp = a.x + t.start + (long long)c * kChunk + o0;
         const long long wbase = t.word + c * (kChunk / 32) + (o0 >> 5);
+        // rows per batch: all of a batch's worker words are loaded before any is used
+        constexpr int RB = (MT > 0 && MT <= 8) ? 2 : 1;
+        static_assert(U % RB == 0, "rows are handled in batches");
         float x[U][4];
-        bool active[U];                                     // false: the 32-element group is past the end
-        unsigned v[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            efk::load4(xp + u * 128, o0 + u * 128, clen, full, x[u]);
-            active[u] = full || ((o0 + u * 128) & ~31) < clen;
-        }
-        majority_words<P, U>(a.wwords + wbase, 4, a.wstride, a.M, a.threshold, active, v);
+        for (int u = 0; u < U; ++u) efk::load4(xp + u * 128, o0 + u * 128, clen, full, x[u]);
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int o = o0 + u * 128;
-            if (!active[u]) continue;
-            vote_apply4(x[u], v[u] >> sh, a.eta);
-            efk::store4(xp + u * 128, o, clen, full, x[u]);
-            if ((lane & 7) == 0) a.words[wbase + u * 4] = v[u];
+        for (int u0 = 0; u0 < U; u0 += RB) {
+            bool active[RB];                                // false: the 32-element group is past the end
+            unsigned v[RB];
+#pragma unroll
+            for (int r = 0; r < RB; ++r) active[r] = full || ((o0 + (u0 + r) * 128) & ~31) < clen;
+            majority_words<MT, P, RB>(a.wwords + wbase + u0 * 4, 4, a.wstride, a.M, a.threshold, active, v);
+#pragma unroll
+            for (int r = 0; r < RB; ++r) {
+                const int u = u0 + r, o = o0 + u * 128;
+                if (!active[r]) continue;
+                vote_apply4(x[u], v[r] >> sh, a.eta);
+                efk::store4(xp + u * 128, o, clen, full, x[u]);
+                if ((lane & 7) == 0) a.words[wbase + u * 4] = v[r];
+            }
         }
     }
 }
 
-int planes_for(int M) {
-    int p = 1;
-    while ((1 << p) <= M) ++p;
-    return p;
-}
-
-template <int P>
+template <int MT, int P>
 void launch_vote_server_t(ef_ctx* c, const VoteServerArgs& a) {
-    launch_kernel(c, ef_vote_server_kernel<kU, P>, dim3((unsigned)c->L.num_tiles), 0, a);
+    launch_kernel(c, ef_vote_server_kernel<kU, MT, P>, dim3((unsigned)c->L.num_tiles), 0, a);
 }
 
 int launch_vote_worker(ef_ctx* c, int i, const float* grad, int count, long long g_stride) {
@@ -276,20 +337,32 @@ int ef_vote_server_step(ef_ctx* c) {
     a.threshold = (unsigned)(M / 2 + 1);
     a.words = c->words(c->srv()); a.x = c->x(); a.tiles = c->tiles(); a.eta = c->eta;
     a.lim = c->limits();
-    switch (planes_for(M)) {
-        case 1: launch_vote_server_t<1>(c, a); break;
-        case 2: launch_vote_server_t<2>(c, a); break;
-        case 3: launch_vote_server_t<3>(c, a); break;
-        case 4: launch_vote_server_t<4>(c, a); break;
-        case 5: launch_vote_server_t<5>(c, a); break;
-        case 6: launch_vote_server_t<6>(c, a); break;
-        case 7: launch_vote_server_t<7>(c, a); break;
-        case 8: launch_vote_server_t<8>(c, a); break;
-        case 9: launch_vote_server_t<9>(c, a); break;
-        case 10: launch_vote_server_t<10>(c, a); break;
-        case 11: launch_vote_server_t<11>(c, a); break;
-        case 12: launch_vote_server_t<12>(c, a); break;
-        default: launch_vote_server_t<13>(c, a); break;     // M <= EF_MAX_WORKERS = 4096 < 2^13
+    switch (M <= 16 ? M : 16 + planes_of(M)) {
+        case 1: launch_vote_server_t<1, 1>(c, a); break;
+        case 2: launch_vote_server_t<2, 1>(c, a); break;
+        case 3: launch_vote_server_t<3, 1>(c, a); break;
+        case 4: launch_vote_server_t<4, 1>(c, a); break;
+        case 5: launch_vote_server_t<5, 1>(c, a); break;
+        case 6: launch_vote_server_t<6, 1>(c, a); break;
+        case 7: launch_vote_server_t<7, 1>(c, a); break;
+        case 8: launch_vote_server_t<8, 1>(c, a); break;
+        case 9: launch_vote_server_t<9, 1>(c, a); break;
+        case 10: launch_vote_server_t<10, 1>(c, a); break;
+        case 11: launch_vote_server_t<11, 1>(c, a); break;
+        case 12: launch_vote_server_t<12, 1>(c, a); break;
+        case 13: launch_vote_server_t<13, 1>(c, a); break;
+        case 14: launch_vote_server_t<14, 1>(c, a); break;
+        case 15: launch_vote_server_t<15, 1>(c, a); break;
+        case 16: launch_vote_server_t<16, 1>(c, a); break;
+        case 16 + 5: launch_vote_server_t<0, 5>(c, a); break;      // 17 <= M < 32
+        case 16 + 6: launch_vote_server_t<0, 6>(c, a); break;
+        case 16 + 7: launch_vote_server_t<0, 7>(c, a); break;
+        case 16 + 8: launch_vote_server_t<0, 8>(c, a); break;
+        case 16 + 9: launch_vote_server_t<0, 9>(c, a); break;
+        case 16 + 10: launch_vote_server_t<0, 10>(c, a); break;
+        case 16 + 11: launch_vote_server_t<0, 11>(c, a); break;
+        case 16 + 12: launch_vote_server_t<0, 12>(c, a); break;
+        default: launch_vote_server_t<0, 13>(c, a); break;         // M <= EF_MAX_WORKERS = 4096 < 2^13
     }
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
