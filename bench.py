@@ -234,11 +234,13 @@ def run_ours(args) -> None:
         return float(tt.item())
 
     w_full = load_workload(args)
-    if args.scaling == "strong" and world > 1:
-        # ONE layout cut into block ranges: this rank builds and steps only its own blocks
-        # (every operation of the method is per element or per block: no data-path collective)
-        b0, b1 = wl.shard_blocks(w_full.sizes, world, rank)
-        w = wl.custom_workload(f"{w_full.name}[blocks {b0}:{b1}]", w_full.sizes[b0:b1] or [4],
+    strong = args.scaling == "strong" and world > 1
+    if strong:
+        # ONE layout cut into equal element ranges (blocks are cut where a rank's share ends
+        # inside one): this rank builds and steps only its own range.  The only data-path
+        # exchange is an all-reduce of B doubles per call, and only if some block is cut.
+        sh = wl.shard_elements(w_full.sizes, world, rank)
+        w = wl.custom_workload(f"{w_full.name}[elements {sh.elem_lo}:{sh.elem_hi}]", sh.local_sizes or [4],
                                w_full.M, w_full.mu, w_full.eta, w_full.steps, w_full.law,
                                w_full.scale_range, config_id=1000 * w_full.config_id + rank)
         job_params = w_full.d                       # total work is fixed as N grows
@@ -249,8 +251,15 @@ def run_ours(args) -> None:
     # all work of the context runs on this (non-default) stream, which is also made current
     stream = torch.cuda.Stream(device=dev)
     torch.cuda.set_stream(stream)
-    eng = EFEngine(w.offsets, w.M, w.mu, w.eta, stream=stream, weight_decay=args.weight_decay > 0,
-                   diagnostics=args.diagnostics, extra_flags=args.library_flags)
+    dshard = None
+    if strong:
+        from paper_1905_10936_b200.sharded import DistributedShard
+        dshard = DistributedShard(w_full.sizes, w.M, w.mu, w.eta, rank, world, stream=stream,
+                                  weight_decay=args.weight_decay > 0, extra_flags=args.library_flags)
+        eng = dshard.eng
+    else:
+        eng = EFEngine(w.offsets, w.M, w.mu, w.eta, stream=stream, weight_decay=args.weight_decay > 0,
+                       diagnostics=args.diagnostics, extra_flags=args.library_flags)
     if args.weight_decay > 0:
         eng.set_weight_decay(args.weight_decay)
     es = w.element_scales(dev)
@@ -273,6 +282,9 @@ def run_ours(args) -> None:
     step_all = eng.vote_worker_step_all if signum else eng.worker_step_all
     step_one = eng.vote_worker_step if signum else eng.worker_step
     server_call = eng.vote_server_step if signum else eng.server_step
+    if dshard is not None:              # cut layout: the step calls go through the exchange
+        assert not signum and batched, "--scaling strong runs the default workload with batched worker calls"
+        step_all, server_call = dshard.worker_step_all, dshard.server_step
     w_bytes_fn = vote_worker_call_bytes if signum else worker_call_bytes
     s_bytes_fn = vote_server_call_bytes if signum else server_call_bytes
 
@@ -432,8 +444,9 @@ def run_ours(args) -> None:
                 "gradient_batches_rotated": nbatch,
                 "per_gpu": ("every rank owns one whole layout (a block-range shard of an N-times "
                             "larger problem); no data-path collective" if args.scaling == "weak" or world == 1
-                            else f"one layout cut into {world} block ranges (workloads.shard_blocks); "
-                                 "each rank builds and steps only its own blocks; no data-path collective")},
+                            else f"one layout cut into {world} equal element ranges (workloads.shard_elements, "
+                                 "blocks cut where needed); each rank builds and steps only its own range; "
+                                 "one all-reduce of B doubles per call if a block is cut")},
         "clocks": clocks,
         "e2e": e2e,
         "gpu_launches": int(launches * world),

@@ -267,6 +267,28 @@ int ef_server_step_range(ef_ctx* ctx, int32_t b0, int32_t b1,
                          const uint32_t* msgs /* device or NULL */, int64_t msg_stride);
 int ef_apply_update(ef_ctx* ctx, int32_t b0, int32_t b1, const uint32_t* update /* device or NULL */);
 
+/* ---- Blocks cut across devices.  The method is per element except for one number per block,
+ * ||p_b||_1 (Section 3.2), so a layout may be cut inside a block (e.g. an embedding larger than a
+ * device's share): each device holds a piece as a block of its own context and the only exchange
+ * is the sum of the pieces' fp64 L1 sums, one number per cut block and call.
+ * ef_set_block_divisors: full_len[b] (host, B entries) is the size d_b of the whole block that
+ *   local block b belongs to; full_len[b] > the local length marks a piece.  Before the first
+ *   iteration only; not together with EF_FLAG_DIAGNOSTICS.
+ * After a worker step (and after ef_server_step_range) the scales of pieces are open:
+ *   ef_block_sums writes, for who = worker index or -1 = server, the B per-block sums to dst
+ *   (device, B doubles; 0 for blocks held whole); the caller adds them up over the devices (an
+ *   all-reduce) and hands the totals to ef_complete_scales, which forms scale_b = total_b / d_b
+ *   for the pieces.  Until then the packed words of the step are valid but the scales of the
+ *   pieces are not, and calls that need them (the next worker step of that worker,
+ *   ef_pack_message, ef_server_step_range on local messages, ef_apply_update from the own server
+ *   step) return EF_ERR_BAD_STATE.  ef_server_step is not available on such a layout: use
+ *   ef_server_step_range(0, B) -> ef_block_sums(-1) -> reduce -> ef_complete_scales(-1) ->
+ *   ef_apply_update(0, B).
+ * Errors: INVALID_ARG, BAD_STATE, CUDA. */
+int ef_set_block_divisors(ef_ctx* ctx, const int64_t* full_len /* host, B */);
+int ef_block_sums(ef_ctx* ctx, int32_t who, double* dst /* device, B */);
+int ef_complete_scales(ef_ctx* ctx, int32_t who, const double* totals /* device, B */);
+
 /* ---- signum / signSGD with majority vote: the paper's comparison method (Section 1: only the
  * 1-bit gradient sign travels between workers and server, in both directions; baselines of
  * Sections 4.1 and 4.2; Table 1: 2Md bits per iteration).  It runs on the same context and

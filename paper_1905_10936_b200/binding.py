@@ -76,6 +76,9 @@ SIGNATURES = {
     "ef_pack_message": (ctypes.c_int, [_vp, _i32, _i32, _i32, _vp]),
     "ef_server_step_range": (ctypes.c_int, [_vp, _i32, _i32, _vp, _i64]),
     "ef_apply_update": (ctypes.c_int, [_vp, _i32, _i32, _vp]),
+    "ef_set_block_divisors": (ctypes.c_int, [_vp, _vp]),
+    "ef_block_sums": (ctypes.c_int, [_vp, _i32, _vp]),
+    "ef_complete_scales": (ctypes.c_int, [_vp, _i32, _vp]),
     "ef_vote_worker_step": (ctypes.c_int, [_vp, _i32, _vp]),
     "ef_vote_worker_step_all": (ctypes.c_int, [_vp, _vp, _i64]),
     "ef_vote_server_step": (ctypes.c_int, [_vp]),
@@ -272,6 +275,19 @@ def ef_server_step_range(ctx: int, b0: int, b1: int, msgs_ptr: Optional[int], ms
 
 def ef_apply_update(ctx: int, b0: int, b1: int, update_ptr: Optional[int]) -> None:
     _check(load_library().ef_apply_update(ctx, b0, b1, update_ptr), "ef_apply_update")
+
+
+def ef_set_block_divisors(ctx: int, full_len) -> None:
+    arr = np.ascontiguousarray(full_len, dtype=np.int64)
+    _check(load_library().ef_set_block_divisors(ctx, arr.ctypes.data), "ef_set_block_divisors")
+
+
+def ef_block_sums(ctx: int, who: int, dst_ptr: int) -> None:
+    _check(load_library().ef_block_sums(ctx, who, dst_ptr), "ef_block_sums")
+
+
+def ef_complete_scales(ctx: int, who: int, totals_ptr: int) -> None:
+    _check(load_library().ef_complete_scales(ctx, who, totals_ptr), "ef_complete_scales")
 
 
 def ef_vote_worker_step(ctx: int, i: int, grad_ptr: int) -> None:

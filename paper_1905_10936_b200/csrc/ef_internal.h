@@ -63,6 +63,10 @@ struct ef_ctx {
     std::vector<efk::Block> h_blocks;
     std::vector<int32_t> h_multi;
     int fused = 0;                         // block scales finalised inside the main kernels
+    // blocks cut across devices (ef_set_block_divisors): slot k's scales of the pieces are still
+    // to be completed from the sum over all pieces (ef_complete_scales)
+    bool has_partial = false;
+    std::vector<uint8_t> scales_open;
     bool use_bulk = false;                 // the server kernel stages its inputs with cp.async.bulk
     bool pdl = false;                      // kernels are launched with programmatic stream serialization
     // host-staging path

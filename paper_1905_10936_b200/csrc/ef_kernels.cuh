@@ -52,12 +52,32 @@ static_assert(sizeof(Tile) == 32, "Tile must be 32 bytes");
 
 struct __align__(16) Block {
     long long start;   // flat index of the first element
-    long long len;     // d_b
+    long long len;     // elements of the block held here
     long long word;    // index of the block's first packed word
     int tile_begin;    // first tile of this block
     int tile_count;    // number of tiles
+    long long div;     // d_b, the divisor of the scale: len, or the whole block's size when this
+                       // context holds only a piece of a block that is cut across devices
+    int partial;       // 1: such a piece.  Its scale cannot be formed here: the kernels leave the
+                       // piece's fp64 sum of |p| in the block's first partial-sum slot instead, and
+                       // ef_complete_scales forms the scale from the sum over all pieces
+    int pad;
 };
-static_assert(sizeof(Block) == 32, "Block must be 32 bytes");
+static_assert(sizeof(Block) == 48, "Block must be 48 bytes");
+
+// The scale of block b from its L1 sum S (Section 3.2: ||p_b||_1 / d_b), or, for a piece of a
+// cut block, the sum itself for ef_complete_scales.  One thread.
+__device__ __forceinline__ void publish_scale(const Block& b, int block_id, double S,
+                                              double* __restrict__ partials, int tc,
+                                              float* __restrict__ scale_out, float* __restrict__ rscale) {
+    if (b.partial) {
+        partials[(long long)b.tile_begin * tc] = S;
+    } else {
+        const float s = (float)(S / (double)b.div);
+        scale_out[block_id] = s;
+        rscale[block_id] = s;
+    }
+}
 
 // Sizes of the problem, carried by every launch.  A build with -DEF_DEBUG checks each CTA's
 // work item (tile or chunk descriptor) against them before touching memory: a descriptor that
@@ -143,7 +163,7 @@ __host__ __device__ __forceinline__ long long message_unit(long long block_word,
 }
 
 struct ScaleArgs {
-    const double* partials;
+    double* partials;
     const Block* blocks;
     const int* multi;        // ids of the blocks that span more than one chunk
     float* scale_out;
@@ -273,16 +293,12 @@ __device__ __forceinline__ double sum_slots(const Block& b, const double* __rest
 }
 
 __device__ __forceinline__ double sum_partials_and_write(const Block& b, int block_id,
-                                                         const double* __restrict__ partials,
+                                                         double* __restrict__ partials,
                                                          float* __restrict__ scale_out,
                                                          float* __restrict__ rscale,
                                                          double* s_sum, int tc) {
     const double S = sum_slots(b, partials, s_sum, tc);
-    if (threadIdx.x == 0) {
-        const float s = (float)(S / (double)b.len);
-        scale_out[block_id] = s;
-        rscale[block_id] = s;
-    }
+    if (threadIdx.x == 0) publish_scale(b, block_id, S, partials, tc, scale_out, rscale);
     return S;
 }
 
@@ -306,9 +322,7 @@ __device__ __forceinline__ void finish_block(double acc, long long slot, int zer
     if (threadIdx.x == 0) {
         int last = 0;
         if (alone) {
-            const float s = (float)(S / (double)blocks[block_id].len);
-            scale_out[block_id] = s;
-            rscale[block_id] = s;
+            publish_scale(blocks[block_id], block_id, S, partials, tc, scale_out, rscale);
         } else {
             partials[slot] = S;
             for (int z = 1; z <= zero_slots; ++z) partials[slot + z] = 0.0;
@@ -1236,6 +1250,28 @@ static __global__ void __launch_bounds__(kThreads) ef_pack_kernel(const PackArgs
     for (int k = threadIdx.x; k < nwords; k += kThreads) dst[k] = a.words[t.word + k];
     if (threadIdx.x == 0 && t.start == b.start)
         a.dst[message_unit(b.word, t.block) - a.msg_base] = __float_as_uint(a.scales[t.block]);
+}
+
+// Cut blocks: dst[b] = the piece's fp64 sum of |p| (0 for blocks held whole), and the scale of
+// such a block from the sum over all pieces.  One thread per block.
+static __global__ void __launch_bounds__(kThreads) ef_block_sums_kernel(const Block* __restrict__ blocks,
+                                                                        const double* __restrict__ partials,
+                                                                        int tc, int B, double* __restrict__ dst) {
+    pdl_enter();
+    const int b = blockIdx.x * kThreads + threadIdx.x;
+    if (b < B) dst[b] = blocks[b].partial ? partials[(long long)blocks[b].tile_begin * tc] : 0.0;
+}
+static __global__ void __launch_bounds__(kThreads) ef_complete_scales_kernel(const Block* __restrict__ blocks,
+                                                                             const double* __restrict__ totals,
+                                                                             int B, float* __restrict__ scale_out,
+                                                                             float* __restrict__ rscale) {
+    pdl_enter();
+    const int b = blockIdx.x * kThreads + threadIdx.x;
+    if (b < B && blocks[b].partial) {
+        const float s = (float)(totals[b] / (double)blocks[b].div);
+        scale_out[b] = s;
+        rscale[b] = s;
+    }
 }
 
 // Import of a residual (ef_set_state): adding +0 maps -0 to +0 and changes nothing else, which

@@ -324,6 +324,7 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
     c->stepped.assign(L.Ml, 0);
     c->served.assign(B, 0);
     c->applied.assign(B, 0);
+    c->scales_open.assign(L.Ml + 1, 0);
 
     // tile and block tables
     c->h_tiles.reserve((size_t)L.num_tiles);
@@ -333,6 +334,7 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
         const int64_t start = offsets[b], len = offsets[b + 1] - offsets[b];
         Block& blk = c->h_blocks[b];
         blk.start = start; blk.len = len; blk.word = word;
+        blk.div = len; blk.partial = 0; blk.pad = 0;
         blk.tile_begin = (int)c->h_tiles.size();
         const int64_t tile_len = (int64_t)kChunkLen * L.tile_chunks;
         for (int64_t o = 0; o < len; o += tile_len) {
@@ -398,9 +400,11 @@ int ef_worker_step(ef_ctx* c, int32_t i, const float* grad) {
     int rc = check_worker_call(c, i, grad, kModeEF);
     if (rc != EF_OK) return rc;
     if (!aligned16(grad)) return EF_ERR_ALIGNMENT;
+    if (c->scales_open[i]) return EF_ERR_BAD_STATE;      // the last step's cut-block scales are not complete
     rc = launch_worker(c, i, grad);
     if (rc != EF_OK) return rc;
     mark_stepped(c, i, kModeEF);
+    if (c->has_partial) c->scales_open[i] = 1;
     return EF_OK;
 }
 
@@ -408,16 +412,19 @@ int ef_worker_step_all(ef_ctx* c, const float* grads, int64_t stride) {
     if (!c || !grads || stride < c->L.d) return EF_ERR_INVALID_ARG;
     if (!aligned16(grads) || (stride & 3) != 0) return EF_ERR_ALIGNMENT;
     if (c->pending != 0) return EF_ERR_BAD_STATE;
+    for (int i = 0; i < c->L.Ml; ++i)
+        if (c->scales_open[i]) return EF_ERR_BAD_STATE;
     const int rc = launch_worker(c, 0, grads, c->L.Ml, (long long)stride);
     if (rc != EF_OK) return rc;
     mark_all_stepped(c, kModeEF);
+    if (c->has_partial) std::fill(c->scales_open.begin(), c->scales_open.begin() + c->L.Ml, (uint8_t)1);
     return EF_OK;
 }
 
 int ef_worker_step_host(ef_ctx* c, int32_t i, const float* grad) {
     int rc = check_worker_call(c, i, grad, kModeEF);
     if (rc != EF_OK) return rc;
-    if (!(c->flags & EF_FLAG_HOST_STAGING)) return EF_ERR_BAD_STATE;
+    if (!(c->flags & EF_FLAG_HOST_STAGING) || c->scales_open[i]) return EF_ERR_BAD_STATE;
     const int s = (int)(c->host_calls & 1);
     // the staging slot is free once the kernel that last read it has finished
     if (c->host_calls >= 2) EF_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->ev_free[s], 0));
@@ -430,6 +437,7 @@ int ef_worker_step_host(ef_ctx* c, int32_t i, const float* grad) {
     EF_CUDA(c, cudaEventRecord(c->ev_free[s], c->stream));
     c->host_calls += 1;
     mark_stepped(c, i, kModeEF);
+    if (c->has_partial) c->scales_open[i] = 1;
     return EF_OK;
 }
 
@@ -437,6 +445,7 @@ int ef_server_step(ef_ctx* c) {
     if (!c) return EF_ERR_INVALID_ARG;
     if (c->pending != c->L.M || c->L.Ml != c->L.M || c->mode != kModeEF) return EF_ERR_BAD_STATE;
     if (c->n_served != 0 || c->n_applied != 0) return EF_ERR_BAD_STATE;   // finish the range calls instead
+    if (c->has_partial) return EF_ERR_BAD_STATE;        // cut blocks: range calls with ef_complete_scales between
     const int rc = launch_server(c);
     if (rc != EF_OK) return rc;
     c->eta_prev = c->eta;
@@ -454,6 +463,7 @@ int ef_pack_message(ef_ctx* c, int32_t who, int32_t b0, int32_t b1, uint32_t* ds
     if (check_block_range(c, b0, b1) != EF_OK || !dst || who < -1 || who >= c->L.Ml)
         return EF_ERR_INVALID_ARG;
     const int k = who < 0 ? c->srv() : who;
+    if (c->scales_open[k]) return EF_ERR_BAD_STATE;
     const TileRange tr = tiles_of(c, b0, b1);
     efk::PackArgs a;
     a.words = c->words(k); a.scales = c->scales(k); a.dst = dst;
@@ -470,6 +480,10 @@ int ef_server_step_range(ef_ctx* c, int32_t b0, int32_t b1, const uint32_t* msgs
     if (check_block_range(c, b0, b1) != EF_OK) return EF_ERR_INVALID_ARG;
     if (c->pending != c->L.Ml || c->mode != kModeEF) return EF_ERR_BAD_STATE;
     if (!msgs && c->L.Ml != c->L.M) return EF_ERR_BAD_STATE;     // the other workers' messages are needed
+    if (!msgs)
+        for (int i = 0; i < c->L.Ml; ++i)
+            if (c->scales_open[i]) return EF_ERR_BAD_STATE;      // workers' cut-block scales not complete
+    if (c->scales_open[c->srv()]) return EF_ERR_BAD_STATE;
     if (msgs && c->L.M > 1 && msg_stride < ef_message_units(c, b0, b1)) return EF_ERR_INVALID_ARG;
     for (int32_t b = b0; b < b1; ++b)
         if (c->served[b]) return EF_ERR_BAD_STATE;
@@ -477,6 +491,7 @@ int ef_server_step_range(ef_ctx* c, int32_t b0, int32_t b1, const uint32_t* msgs
     if (rc != EF_OK) return rc;
     for (int32_t b = b0; b < b1; ++b) c->served[b] = 1;
     c->n_served += b1 - b0;
+    if (c->has_partial) c->scales_open[c->srv()] = 1;
     return EF_OK;
 }
 
@@ -485,6 +500,7 @@ int ef_apply_update(ef_ctx* c, int32_t b0, int32_t b1, const uint32_t* update) {
     if (c->pending != c->L.Ml || c->mode != kModeEF) return EF_ERR_BAD_STATE;
     for (int32_t b = b0; b < b1; ++b)
         if (c->applied[b] || (!update && !c->served[b])) return EF_ERR_BAD_STATE;
+    if (!update && c->scales_open[c->srv()]) return EF_ERR_BAD_STATE;
     const int rc = launch_apply_range(c, b0, b1, update);
     if (rc != EF_OK) return rc;
     for (int32_t b = b0; b < b1; ++b) c->applied[b] = 1;
@@ -493,6 +509,45 @@ int ef_apply_update(ef_ctx* c, int32_t b0, int32_t b1, const uint32_t* update) {
         c->eta_prev = c->eta;
         end_iteration(c);
     }
+    return EF_OK;
+}
+
+int ef_set_block_divisors(ef_ctx* c, const int64_t* full_len) {
+    if (!c || !full_len) return EF_ERR_INVALID_ARG;
+    if (c->t != 0 || c->pending != 0 || (c->flags & EF_FLAG_DIAGNOSTICS)) return EF_ERR_BAD_STATE;
+    for (int32_t b = 0; b < c->L.B; ++b)
+        if (full_len[b] < c->h_blocks[b].len) return EF_ERR_INVALID_ARG;
+    c->has_partial = false;
+    for (int32_t b = 0; b < c->L.B; ++b) {
+        c->h_blocks[b].div = full_len[b];
+        c->h_blocks[b].partial = full_len[b] > c->h_blocks[b].len ? 1 : 0;
+        c->has_partial = c->has_partial || c->h_blocks[b].partial;
+    }
+    EF_CUDA(c, cudaMemcpyAsync(c->ws + c->L.off_blocks, c->h_blocks.data(),
+                               c->h_blocks.size() * sizeof(Block), cudaMemcpyHostToDevice, c->stream));
+    return EF_OK;
+}
+
+int ef_block_sums(ef_ctx* c, int32_t who, double* dst) {
+    if (!c || !dst || who < -1 || who >= c->L.Ml) return EF_ERR_INVALID_ARG;
+    const int k = who < 0 ? c->srv() : who;
+    launch_kernel(c, efk::ef_block_sums_kernel, dim3((unsigned)((c->L.B + efk::kThreads - 1) / efk::kThreads)), 0,
+                  c->blocks(), (const double*)c->partials(k), (int)c->L.tile_chunks, (int)c->L.B, dst);
+    EF_CUDA(c, cudaGetLastError());
+    c->launches += 1;
+    return EF_OK;
+}
+
+int ef_complete_scales(ef_ctx* c, int32_t who, const double* totals) {
+    if (!c || !totals || who < -1 || who >= c->L.Ml) return EF_ERR_INVALID_ARG;
+    const int k = who < 0 ? c->srv() : who;
+    if (!c->scales_open[k]) return EF_ERR_BAD_STATE;
+    launch_kernel(c, efk::ef_complete_scales_kernel,
+                  dim3((unsigned)((c->L.B + efk::kThreads - 1) / efk::kThreads)), 0, c->blocks(), totals,
+                  (int)c->L.B, c->scales(k), c->rscale(k));
+    EF_CUDA(c, cudaGetLastError());
+    c->launches += 1;
+    c->scales_open[k] = 0;
     return EF_OK;
 }
 

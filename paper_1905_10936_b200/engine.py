@@ -114,6 +114,20 @@ class EFEngine:
             assert update.numel() >= self.message_units(b0, b1)
         ef.ef_apply_update(self.ctx, b0, b1, update.data_ptr() if update is not None else None)
 
+    # ---- blocks cut across devices ------------------------------------------------------------
+    def set_block_divisors(self, full_len) -> None:
+        assert len(full_len) == self.B
+        ef.ef_set_block_divisors(self.ctx, full_len)
+
+    def block_sums(self, who: int, dst: torch.Tensor) -> None:
+        assert dst.is_cuda and dst.dtype == torch.float64 and dst.is_contiguous() and dst.numel() >= self.B
+        ef.ef_block_sums(self.ctx, who, dst.data_ptr())
+
+    def complete_scales(self, who: int, totals: torch.Tensor) -> None:
+        assert totals.is_cuda and totals.dtype == torch.float64 and totals.is_contiguous()
+        assert totals.numel() >= self.B
+        ef.ef_complete_scales(self.ctx, who, totals.data_ptr())
+
     # ---- signum with majority vote (same state, same packed layout) -------------------------
     def vote_worker_step(self, i: int, grad: torch.Tensor) -> None:
         assert grad.is_cuda and grad.dtype == torch.float32 and grad.numel() == self.d

@@ -207,3 +207,53 @@ def shard_blocks(sizes: Sequence[int], world_size: int, rank: int) -> Tuple[int,
         cuts.append(b)
     cuts.append(len(sizes))
     return cuts[rank], cuts[rank + 1]
+
+
+@dataclass
+class ElementShard:
+    """One rank's share of a layout cut by ELEMENT count (blocks may be cut): the pieces it
+    holds, as a layout of its own."""
+    elem_lo: int                   # first element (flat index in the whole vector)
+    elem_hi: int
+    local_sizes: List[int]         # sizes of the local blocks (whole blocks and pieces)
+    full_sizes: List[int]          # size of the whole block each local block belongs to
+    global_block: List[int]        # index of that block in the whole layout
+    offset_in_block: List[int]     # where the local block starts inside it
+
+
+def shard_elements(sizes: Sequence[int], world_size: int, rank: int, granule: int = 4096) -> ElementShard:
+    """Contiguous element range owned by `rank` when the flat vector is cut into `world_size`
+    nearly equal parts.  A cut may fall inside a block, but only at a multiple of `granule`
+    elements from the block's start (granule must be a multiple of 32, so that every piece
+    starts on a packed-word boundary of the whole block's message).  The ranges tile [0, d).
+
+    A rank then holds each block it intersects as a local block of its own; for a piece the
+    scale needs the sum of all pieces' L1 norms (one number per cut block, see
+    ef_set_block_divisors / ef_block_sums / ef_complete_scales)."""
+    if not (0 <= rank < world_size):
+        raise ValueError("rank out of range")
+    if granule % 32 != 0 or granule <= 0:
+        raise ValueError("granule must be a positive multiple of 32")
+    off = _offsets(sizes)
+    d = int(off[-1])
+
+    def cut(r: int) -> int:
+        if r <= 0:
+            return 0
+        if r >= world_size:
+            return d
+        target = d * r // world_size
+        b = int(np.searchsorted(off, target, side="right")) - 1      # block that holds the target
+        b = min(max(b, 0), len(sizes) - 1)
+        return int(off[b]) + (target - int(off[b])) // granule * granule
+
+    lo, hi = cut(rank), cut(rank + 1)
+    shard = ElementShard(lo, hi, [], [], [], [])
+    for b, size in enumerate(sizes):
+        s, e = max(lo, int(off[b])), min(hi, int(off[b + 1]))
+        if e > s:
+            shard.local_sizes.append(e - s)
+            shard.full_sizes.append(int(size))
+            shard.global_block.append(b)
+            shard.offset_in_block.append(s - int(off[b]))
+    return shard
