@@ -9,8 +9,8 @@
 // Method (all integer work on the bit pattern of |v_j|, which orders like the magnitude):
 //   1. radix select of the k-th largest key in three passes over v (11 + 11 + 9 bits): each pass
 //      histograms one digit of the keys that still match the prefix found so far (shared-memory
-//      histogram per CTA, merged into a global one), then one thread walks the 2048 bins from
-//      the top and fixes the next digit.  Result: the threshold key T and how many keys equal
+//      histogram per CTA, merged into a global one), then one CTA finds the bin, from the top,
+//      in which the count reaches what is still to keep, and fixes the next digit.  Result: the threshold key T and how many keys equal
 //      to T have to be kept (need_eq).
 //   2. a counting pass: per 4096-element chunk the number of keys > T and == T;
 //   3. a scan of those counts over the chunks (one CTA);
@@ -110,20 +110,37 @@ __global__ void __launch_bounds__(kThreads) ef_topk_hist_kernel(const float* __r
         if (s_hist[b]) atomicAdd(&hist[b], (unsigned long long)s_hist[b]);
 }
 
-// One thread fixes the next digit: walks the bins from the largest digit down until the keys
-// seen so far reach `remaining`.
+// One CTA fixes the next digit: it finds, from the largest digit down, the bin in which the
+// count of keys seen so far reaches `remaining`.  Thread t adds up bins 8t .. 8t+7; thread 0
+// walks the 256 sums from the top and then the eight bins of the group it stops in.
 template <int PASS>
-__global__ void ef_topk_select_kernel(const unsigned long long* __restrict__ hist, TopkState* st,
-                                      unsigned long long k) {
-    if (threadIdx.x != 0 || blockIdx.x != 0) return;
-    constexpr int bits = pass_bits(PASS);
+__global__ void __launch_bounds__(kThreads) ef_topk_select_kernel(const unsigned long long* __restrict__ hist,
+                                                                  TopkState* st, unsigned long long k) {
+    constexpr int bits = pass_bits(PASS), nbins = 1 << bits, per = kBins / kThreads;
+    __shared__ unsigned long long s_bin[kBins], s_grp[kThreads];
+    unsigned long long g = 0;
+#pragma unroll
+    for (int j = 0; j < per; ++j) {
+        const int b = threadIdx.x * per + j;
+        const unsigned long long v = b < nbins ? hist[b] : 0ull;
+        s_bin[b] = v;
+        g += v;
+    }
+    s_grp[threadIdx.x] = g;
+    __syncthreads();
+    if (threadIdx.x != 0) return;
     unsigned long long remaining = PASS == 0 ? k : st->remaining;
     const unsigned prefix = PASS == 0 ? 0u : st->prefix;
     unsigned long long above = 0;
-    int b = (1 << bits) - 1;
-    for (; b > 0; --b) {
-        if (above + hist[b] >= remaining) break;
-        above += hist[b];
+    int grp = kThreads - 1;
+    for (; grp > 0; --grp) {
+        if (above + s_grp[grp] >= remaining) break;
+        above += s_grp[grp];
+    }
+    int b = grp * per + per - 1;
+    for (; b > grp * per; --b) {
+        if (above + s_bin[b] >= remaining) break;
+        above += s_bin[b];
     }
     remaining -= above;                       // still to keep among the keys of bin b
     st->prefix = (prefix << bits) | (unsigned)b;
@@ -156,9 +173,10 @@ __global__ void __launch_bounds__(kThreads) ef_topk_count_kernel(const float* __
             eq += (in[k] && key == T) ? 1u : 0u;
         }
     }
-    gt = __reduce_add_sync(kFull, gt);
-    eq = __reduce_add_sync(kFull, eq);
-    if (lane == 0) { s_gt[warp] = gt; s_eq[warp] = eq; }
+    unsigned both = gt | (eq << 16);          // at most 512 elements per warp each: two 16-bit fields
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) both += __shfl_xor_sync(kFull, both, o);
+    if (lane == 0) { s_gt[warp] = both & 0xffffu; s_eq[warp] = both >> 16; }
     __syncthreads();
     if (threadIdx.x == 0) {
         unsigned a = 0, b = 0;
@@ -170,28 +188,37 @@ __global__ void __launch_bounds__(kThreads) ef_topk_count_kernel(const float* __
 
 // ---- 3. exclusive prefix sums of the two count arrays over the chunks (one CTA)
 constexpr int kScanThreads = 1024;
+__device__ __forceinline__ unsigned long long warp_inclusive_scan(unsigned long long v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long u = __shfl_up_sync(kFull, v, o);
+        if (lane >= o) v += u;
+    }
+    return v;
+}
 __global__ void __launch_bounds__(kScanThreads) ef_topk_scan_kernel(const unsigned* __restrict__ cgt,
                                                                     const unsigned* __restrict__ ceq,
                                                                     unsigned long long* __restrict__ pgt,
                                                                     unsigned long long* __restrict__ peq,
                                                                     long long chunks) {
-    __shared__ unsigned long long s_a[kScanThreads], s_b[kScanThreads];
+    __shared__ unsigned long long s_a[32], s_b[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long per = (chunks + kScanThreads - 1) / kScanThreads;
     const long long lo = min(chunks, (long long)threadIdx.x * per), hi = min(chunks, lo + per);
     unsigned long long a = 0, b = 0;
     for (long long c = lo; c < hi; ++c) { a += cgt[c]; b += ceq[c]; }
-    s_a[threadIdx.x] = a; s_b[threadIdx.x] = b;
+    // exclusive scan of the per-thread totals over the CTA: warps, then the warps' totals
+    const unsigned long long ia = warp_inclusive_scan(a, lane), ib = warp_inclusive_scan(b, lane);
+    if (lane == 31) { s_a[warp] = ia; s_b[warp] = ib; }
     __syncthreads();
-    if (threadIdx.x == 0) {                    // 1024 serial additions: negligible
-        unsigned long long ra = 0, rb = 0;
-        for (int t = 0; t < kScanThreads; ++t) {
-            const unsigned long long ta = s_a[t], tb = s_b[t];
-            s_a[t] = ra; s_b[t] = rb;
-            ra += ta; rb += tb;
-        }
+    if (warp == 0) {
+        const unsigned long long wa = warp_inclusive_scan(s_a[lane], lane), wb = warp_inclusive_scan(s_b[lane], lane);
+        s_a[lane] = wa - s_a[lane];            // exclusive
+        s_b[lane] = wb - s_b[lane];
     }
     __syncthreads();
-    a = s_a[threadIdx.x]; b = s_b[threadIdx.x];
+    a = s_a[warp] + ia - a;
+    b = s_b[warp] + ib - b;
     for (long long c = lo; c < hi; ++c) {
         pgt[c] = a; peq[c] = b;
         a += cgt[c]; b += ceq[c];
@@ -215,6 +242,7 @@ __global__ void __launch_bounds__(kThreads) ef_topk_scatter_kernel(const float* 
     const unsigned lt_mask = (1u << lane) - 1u;
     float x[kU][4]; bool in[kU][4];
     unsigned feq[kU], fgt[kU];                 // nibbles of flags
+    unsigned eq_lanes_before[kU], gt_lanes_before[kU], eq_row[kU], gt_row[kU];
     unsigned weq = 0, wgt = 0;                 // this warp's totals
 #pragma unroll
     for (int u = 0; u < kU; ++u) {
@@ -232,8 +260,19 @@ __global__ void __launch_bounds__(kThreads) ef_topk_scatter_kernel(const float* 
 #pragma unroll
             for (int k = 0; k < 4; ++k) { in[u][k] = false; x[u][k] = 0.f; }
         }
-        weq += __reduce_add_sync(kFull, (unsigned)__popc(feq[u]));
-        wgt += __reduce_add_sync(kFull, (unsigned)__popc(fgt[u]));
+        // keys of this row before this lane, and in the whole row: one ballot per element position
+        eq_lanes_before[u] = gt_lanes_before[u] = eq_row[u] = gt_row[u] = 0u;
+        if (__any_sync(kFull, (feq[u] | fgt[u]) != 0u)) {      // most rows keep nothing
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const unsigned be = __ballot_sync(kFull, (feq[u] >> k) & 1u);
+                const unsigned bg = __ballot_sync(kFull, (fgt[u] >> k) & 1u);
+                eq_lanes_before[u] += __popc(be & lt_mask); eq_row[u] += __popc(be);
+                gt_lanes_before[u] += __popc(bg & lt_mask); gt_row[u] += __popc(bg);
+            }
+        }
+        weq += eq_row[u];
+        wgt += gt_row[u];
     }
     if (lane == 0) { s_eq[warp] = weq; s_gt[warp] = wgt; }
     __syncthreads();
@@ -242,17 +281,8 @@ __global__ void __launch_bounds__(kThreads) ef_topk_scatter_kernel(const float* 
 #pragma unroll
     for (int u = 0; u < kU; ++u) {
         const long long base = (long long)blockIdx.x * kChunkLen + warp * (128 * kU) + u * 128 + lane * 4;
-        // equal keys of this row before this lane: per element position k one ballot
-        unsigned eq_lanes_before = 0, gt_lanes_before = 0, eq_row = 0, gt_row = 0;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const unsigned be = __ballot_sync(kFull, (feq[u] >> k) & 1u);
-            const unsigned bg = __ballot_sync(kFull, (fgt[u] >> k) & 1u);
-            eq_lanes_before += __popc(be & lt_mask); eq_row += __popc(be);
-            gt_lanes_before += __popc(bg & lt_mask); gt_row += __popc(bg);
-        }
-        unsigned long long eq_rank = eq_before + eq_lanes_before;     // equal keys before element 0 of this lane
-        unsigned long long gt_rank = gt_before + gt_lanes_before;
+        unsigned long long eq_rank = eq_before + eq_lanes_before[u];     // equal keys before element 0 of this lane
+        unsigned long long gt_rank = gt_before + gt_lanes_before[u];
         float r[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
@@ -275,8 +305,8 @@ __global__ void __launch_bounds__(kThreads) ef_topk_scatter_kernel(const float* 
             else
                 for (int k = 0; k < 4; ++k) if (in[u][k]) resid[base + k] = r[k];
         }
-        eq_before += eq_row;
-        gt_before += gt_row;
+        eq_before += eq_row[u];
+        gt_before += gt_row[u];
     }
 }
 
@@ -315,11 +345,11 @@ int ef_topk_compress(const float* v, int64_t n, int64_t k, int64_t* idx_out, flo
     const unsigned hgrid = (unsigned)std::min<long long>(L.chunks, 148 * 8);
     const unsigned long long kk = (unsigned long long)k;
     ef_topk_hist_kernel<0><<<hgrid, kThreads, 0, st>>>(v, n, L.chunks, state, hist);
-    ef_topk_select_kernel<0><<<1, 32, 0, st>>>(hist, state, kk);
+    ef_topk_select_kernel<0><<<1, kThreads, 0, st>>>(hist, state, kk);
     ef_topk_hist_kernel<1><<<hgrid, kThreads, 0, st>>>(v, n, L.chunks, state, hist + kBins);
-    ef_topk_select_kernel<1><<<1, 32, 0, st>>>(hist + kBins, state, kk);
+    ef_topk_select_kernel<1><<<1, kThreads, 0, st>>>(hist + kBins, state, kk);
     ef_topk_hist_kernel<2><<<hgrid, kThreads, 0, st>>>(v, n, L.chunks, state, hist + 2 * kBins);
-    ef_topk_select_kernel<2><<<1, 32, 0, st>>>(hist + 2 * kBins, state, kk);
+    ef_topk_select_kernel<2><<<1, kThreads, 0, st>>>(hist + 2 * kBins, state, kk);
     ef_topk_count_kernel<<<(unsigned)L.chunks, kThreads, 0, st>>>(v, n, state, cgt, ceq);
     ef_topk_scan_kernel<<<1, kScanThreads, 0, st>>>(cgt, ceq, pgt, peq, L.chunks);
     ef_topk_scatter_kernel<<<(unsigned)L.chunks, kThreads, 0, st>>>(v, n, state, pgt, peq,
