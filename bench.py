@@ -3,15 +3,22 @@
 
 A "step" is the worker side of all M workers (one ef_worker_step_all launch, or M
 ef_worker_step calls with --per-worker-calls) plus one ef_server_step over one batch of
-synthetic gradients.  The default workload is the flat 2^28-parameter layout (256 blocks of
-2^20, M = 7).  Prints ONE JSON line on rank 0.
+synthetic gradients (up to three batches are kept in HBM and rotated).  The default workload is
+the flat 2^28-parameter layout (256 blocks of 2^20, M = 7).  Prints ONE JSON line on rank 0.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
-                  [--graph] [--per-worker-calls] [--weight-decay L] [--diagnostics] [--blocks N]
+                  [--workload ef|signum|topk] [--scaling weak|strong] [--graph] [--ceiling]
+                  [--per-worker-calls] [--weight-decay L] [--diagnostics] [--blocks N] [--workers M]
 
-With N > 1 (launched by torch.distributed.run) every rank owns its own block range of an
-N-times larger problem (blocks are independent in the method, so there is no data-path
-collective): weak scaling, value = parameters processed by all ranks per second.
+Keys beyond the common ones: `roofline` (worker launch), `roofline_server` (server call),
+`sustained` (300 more back-to-back steps with the clocks sampled), `e2e` (host gradients in, packed
+update out), `cpu_baseline` (the oracle on one host core), `cuda_graph` (--graph) and
+`stream_ceiling` (--ceiling: no-compute kernels with the step kernels' access mix).
+
+With N > 1 (launched by torch.distributed.run): --scaling weak (default) gives every rank one
+whole layout (a block-range shard of an N-times larger problem; no data-path collective);
+--scaling strong cuts ONE layout into N equal element ranges, blocks included, and all-reduces
+one fp64 sum per cut block and call.
 
 --impl reference times the CPU oracle (plain single-threaded C++) on a bounded sample of the
 same workload; it is a deliberately slow program, reported for context.
@@ -520,6 +527,70 @@ def stream_ceilings(eng, gall: torch.Tensor, w: wl.Workload, stream) -> dict:
     return out
 
 
+def run_topk(args) -> None:
+    """The top-k compressor (ef_topk_compress) on a vector of the workload's size: one "step" is
+    one call (threshold search, ordered scatter of k index/value pairs, residual)."""
+    from paper_1905_10936_b200 import binding as ef
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    w = load_workload(args)
+    n, k = w.d, max(1, int(w.d * args.topk_fraction))
+    K, W = args.steps, args.warmup
+    if args.impl == "reference":
+        from oracle import topk_compress
+        ns = min(n, 1 << 22)
+        v = w.draw_grad(0, 0, "cpu")[:ns].numpy()
+        t0 = time.perf_counter()
+        for _ in range(K):
+            topk_compress(v, max(1, int(ns * args.topk_fraction)))
+        value = ns * K / (time.perf_counter() - t0)
+        line = {"impl": "reference", "metric": "elements/sec through the top-k compressor", "value": value,
+                "unit": "elements/s", "n_gpus": args.gpus, "steps": K, "warmup": W, "ms_per_step": n / value * 1e3,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": config_dict(w),
+                "cpu_baseline": {"value": value, "unit": "elements/s", "cores": 1, "kind": "oracle",
+                                 "sample": f"first {ns} of {n} elements, sort-based definition"},
+                "e2e": {"value": value, "unit": "elements/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line), flush=True)
+        return
+    torch.cuda.set_device(0)
+    v = w.draw_grad(0, 0, "cuda", w.element_scales("cuda"))
+    ws = torch.empty(ef.ef_topk_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    idx = torch.empty(k, dtype=torch.int64, device="cuda")
+    val = torch.empty(k, device="cuda")
+    resid = torch.empty(n, device="cuda")
+    st = torch.cuda.current_stream().cuda_stream
+
+    def call():
+        ef.ef_topk_compress(v.data_ptr(), n, k, idx.data_ptr(), val.data_ptr(), resid.data_ptr(),
+                            ws.data_ptr(), ws.numel(), st)
+    for _ in range(W):
+        call()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0, period_s=0.002)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    e0.record()
+    for _ in range(K):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / K
+    peak, kind = measured_hbm_peak()
+    nbytes = 24.0 * n + 12.0 * k           # five reads of v, one write of the residual, k pairs
+    line = {"metric": "elements/sec through the top-k compressor", "value": n / (ms * 1e-3), "unit": "elements/s",
+            "n_gpus": 1, "steps": K, "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config_dict(w),
+            "run": {"workload": "topk", "n": n, "k": k}, "clocks": clocks, "e2e": None, "gpu_launches": 9 * K,
+            "roofline": {"kernel": "ef_topk_* (9 launches per call)", "bound": "hbm",
+                         "achieved": nbytes / (ms * 1e-3) / 1e9, "peak": peak, "peak_kind": f"of {kind}",
+                         "unit": "GB/s", "frac": nbytes / (ms * 1e-3) / 1e9 / peak, "traffic": None,
+                         "bytes_per_launch": nbytes}}
+    print(json.dumps(line), flush=True)
+
+
 def eng_state_gib(w: wl.Workload) -> float:
     return (w.d * 4.0 * (2 * w.M + 2) + w.d * 4.0 * w.M) / 2 ** 30
 
@@ -546,9 +617,11 @@ def main():
     ap.add_argument("--workers", type=int, default=0,
                     help="override the number of simulated workers M of the workload")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=["ef", "signum"], default="ef",
+    ap.add_argument("--workload", choices=["ef", "signum", "topk"], default="ef",
                     help="ef: dist-EF-blockSGDM (default, the headline); signum: the paper's "
-                         "comparison method, signum with majority vote, on the same layouts")
+                         "comparison method, signum with majority vote, on the same layouts; "
+                         "topk: the top-k compressor on one vector of the layout's size")
+    ap.add_argument("--topk-fraction", type=float, default=0.01, help="k / n for --workload topk")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--per-worker-calls", action="store_true",
                     help="step the workers with M ef_worker_step calls instead of one ef_worker_step_all")
@@ -576,7 +649,9 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    if args.impl == "reference":
+    if args.workload == "topk":
+        run_topk(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
