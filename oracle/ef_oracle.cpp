@@ -48,9 +48,13 @@
 //   * blocks are contiguous index ranges given by B+1 offsets, every d_b >= 1;
 //   * packed layout: block b owns ceil(d_b/32) words; element k of the block is bit (k mod 32)
 //     (LSB = bit 0) of word floor(k/32); bit = 1 means negative (decodes to -1); unused high
-//     bits of the last word are 0.  PARITY UNPINNED BY THE PAPER for this layout (bit polarity,
-//     bit order, word alignment) and for the order of the server average: they are pinned
-//     only by worked examples that follow this header.
+//     bits of the last word are 0.
+// PARITY UNPINNED BY THE PAPER for: this packed layout (bit polarity, bit order, word alignment),
+// the order of the server average, the binary64 accumulation of the block sums, the single
+// rounding of the rescaled residual (one fma rather than a product and a sum), and the operation
+// order of the weight-decay update.  The paper is silent on all five; they are pinned, as
+// conventions of this repository, only by worked examples and by hand-built cases in which the
+// alternative gives a different binary32 result.
 //
 // "Hint" protocol (for step-locked comparison with another implementation): an element whose
 // |p| is below 1e-6 times its block's scale may legitimately round to either sign when two

@@ -401,6 +401,19 @@ def test_rescaled_residuals_that_underflow_to_negative_zero():
     assert stats["adopted"] == 0 and stats["state_value_mismatch"] == 0
 
 
+def test_rounding_conventions_on_the_gpu():
+    """The hand-built cases that separate the rounding conventions (binary64 block sums;
+    ascending worker order in the server sum), run through the CUDA path."""
+    w = _wl("sum64", [4], 1, mu=0.0, steps=1)
+    g = torch.tensor([2.0 ** 24, -1.0, 1.0, -1.0])
+    eng, orc, _ = run_parity(w, grads=[[g]])
+    assert eng.worker_scales(0).item() == float(np.float32((2.0 ** 24 + 3) / 4))
+    w = _wl("order", [2], 3, mu=0.0, eta=0.5, steps=1)
+    grads = [[torch.full((2,), s) for s in (3 * 2.0 ** 24, 3.0, 3.0)]]
+    eng, orc, _ = run_parity(w, grads=grads)
+    assert eng.server_scales().item() == 2.0 ** 24          # ((2^24 + 1) + 1) in binary32, not 2^24 + 2
+
+
 def test_indexing_beyond_2_32_elements():
     """d > 2^32: one huge block followed by small ragged blocks whose flat indices need 33 bits;
     the oracle follows the small blocks (blocks are independent).  M = 1 keeps it at 86 GB."""
