@@ -591,6 +591,80 @@ def run_topk(args) -> None:
     print(json.dumps(line), flush=True)
 
 
+def run_ps(args) -> None:
+    """The paper's setting in pieces on ONE GPU: G ranks (rank r = worker r + the server of one
+    block range) stepped one after the other, the exchange replaced by device copies.  Times the
+    pieces a real rank would run between its collectives; the exchange itself cannot be measured
+    on one device and is given analytically (bytes per rank and phase)."""
+    from paper_1905_10936_b200 import ps
+    from paper_1905_10936_b200.engine import EFEngine
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    w = load_workload(args)
+    G, K, W = w.M, args.steps, args.warmup
+    torch.cuda.set_device(0)
+    ranks = [ps.Rank(EFEngine(w.offsets, G, w.mu, w.eta, one_local_worker=True), w.sizes, r, G) for r in range(G)]
+    es = w.element_scales("cuda")
+    grads = [w.draw_grad(0, i, "cuda", es) for i in range(G)]
+    names = ["worker_step", "pack_message", "server_step_range", "pack_update", "apply_update"]
+    acc = {n: 0.0 for n in names}
+
+    def timed(name, fn, record):
+        if not record:
+            fn()
+            return
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); fn(); e1.record()
+        pending.append((name, e0, e1))
+
+    for it in range(W + K):
+        rec = it >= W
+        pending = []
+        for rk, g in zip(ranks, grads):
+            timed("worker_step", lambda: rk.engine.worker_step(0, g), rec)
+            timed("pack_message", lambda: rk.engine.pack_message(0, 0, rk.B, rk.send), rec)
+        for dst in ranks:                                   # stands in for the all-to-all
+            m = dst.mine
+            for src in ranks:
+                if m.units:
+                    dst.recv[src.rank, :m.units].copy_(src.send[m.unit0:m.unit0 + m.units])
+        for rk in ranks:
+            m = rk.mine
+            if m.b1 > m.b0:
+                timed("server_step_range", lambda: rk.engine.server_step_range(m.b0, m.b1, rk.recv), rec)
+                timed("pack_update", lambda: rk.engine.pack_message(-1, m.b0, m.b1,
+                                                                    rk.update[m.unit0:m.unit0 + m.units]), rec)
+        for dst in ranks:                                   # stands in for the all-gather
+            for src in ranks:
+                p = src.mine
+                if src is not dst and p.units:
+                    dst.update[p.unit0:p.unit0 + p.units].copy_(src.update[p.unit0:p.unit0 + p.units])
+        for rk in ranks:
+            timed("apply_update", lambda: rk.engine.apply_update(0, rk.B, rk.update), rec)
+        torch.cuda.synchronize()
+        for name, e0, e1 in pending:
+            acc[name] += e0.elapsed_time(e1)
+    per_rank_ms = {n: acc[n] / (K * G) for n in names}      # average over ranks and steps
+    total_ms = sum(per_rank_ms.values())
+    units = ranks[0].total_units
+    line = {"metric": "parameters/sec per rank through one iteration of the sharded parameter-server "
+                      "protocol (compute pieces only; ranks emulated one after the other on one GPU)",
+            "value": w.d / (total_ms * 1e-3), "unit": "params/s", "n_gpus": 1, "steps": K, "warmup": W,
+            "ms_per_step": total_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic", "config": config_dict(w),
+            "run": {"workload": "ps", "ranks": G, "ms_per_rank": per_rank_ms,
+                    "bytes_per_rank": {"worker_step": worker_call_bytes(w.d, w.B),
+                                       "server_step_range": (8.0 + (G + 1) / 8.0) * w.d / G,
+                                       "apply_update": 8.125 * w.d},
+                    "exchange_bytes_per_rank": {"all_to_all_out": 4 * units * (G - 1) // G,
+                                                "all_gather_in": 4 * units * (G - 1) // G},
+                    "note": "the exchange is not timed: on NVLink at the pool's measured 770 GB/s per "
+                            "direction the two phases would take "
+                            f"{2 * 4 * units * (G - 1) / G / 770e9 * 1e6:.0f} us per iteration"},
+            "e2e": None, "gpu_launches": int(sum(rk.engine.launch_count for rk in ranks))}
+    print(json.dumps(line), flush=True)
+
+
 def eng_state_gib(w: wl.Workload) -> float:
     return (w.d * 4.0 * (2 * w.M + 2) + w.d * 4.0 * w.M) / 2 ** 30
 
@@ -617,10 +691,12 @@ def main():
     ap.add_argument("--workers", type=int, default=0,
                     help="override the number of simulated workers M of the workload")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=["ef", "signum", "topk"], default="ef",
+    ap.add_argument("--workload", choices=["ef", "signum", "topk", "ps"], default="ef",
                     help="ef: dist-EF-blockSGDM (default, the headline); signum: the paper's "
                          "comparison method, signum with majority vote, on the same layouts; "
-                         "topk: the top-k compressor on one vector of the layout's size")
+                         "topk: the top-k compressor on one vector of the layout's size; "
+                         "ps: the one-worker-per-rank protocol with a block-sharded server, its "
+                         "compute pieces timed with the M ranks emulated on one GPU")
     ap.add_argument("--topk-fraction", type=float, default=0.01, help="k / n for --workload topk")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--per-worker-calls", action="store_true",
@@ -651,6 +727,8 @@ def main():
         args.warmup = 3
     if args.workload == "topk":
         run_topk(args)
+    elif args.workload == "ps":
+        run_ps(args)
     elif args.impl == "reference":
         run_reference(args)
     else:
