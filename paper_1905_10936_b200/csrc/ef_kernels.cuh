@@ -20,8 +20,12 @@
 // 1024*U elements; a tile never crosses a block boundary.  The worker kernel runs one CTA per
 // chunk (three read and two write streams of 16 KB each per CTA keep enough bytes in flight).
 // The server and apply kernels have one read and one write stream only, so one CTA walks all
-// chunks of a tile: the server kernel stages them two chunks ahead through shared memory with
-// cp.async, the apply kernel loads chunk c+1 into a second register set while it updates c.
+// chunks of a tile: the server kernel stages them ahead through a two-stage shared-memory ring
+// (bulk copies issued by one thread and an mbarrier where the layout is 16-byte aligned per
+// chunk, per-thread cp.async otherwise), the apply kernel loads chunk c+1 into a second
+// register set while it updates c.  The server kernel is the one kernel bound by latency and
+// instruction issue rather than by HBM: it needs four CTAs per SM, which fixes how much shared
+// memory its sign-pattern tables may take.
 //
 // Arithmetic is IEEE binary32 with explicit round-to-nearest intrinsics in a fixed order so
 // that results do not depend on compiler contraction; block sums are binary64.

@@ -88,3 +88,35 @@ def test_null_context_is_rejected():
     assert lib.ef_destroy(None) == ef.EF_OK
     assert lib.ef_params(None) is None
     assert ef.ef_strerror(ef.EF_ERR_BAD_STATE) == "call order violated"
+
+
+def test_later_entry_points_check_their_arguments_without_a_device():
+    """Argument checks of the entry points that do not belong to the core path come before any
+    device use, so they can be exercised without a GPU."""
+    lib = ef.load_library()
+    null = ctypes.c_void_p(None)
+    for name, args in [
+        ("ef_vote_worker_step", (null, 0, null)), ("ef_vote_worker_step_all", (null, null, 0)),
+        ("ef_vote_server_step", (null,)), ("ef_server_step_range", (null, 0, 1, null, 0)),
+        ("ef_apply_update", (null, 0, 1, null)), ("ef_pack_message", (null, 0, 0, 1, null)),
+        ("ef_set_block_divisors", (null, null)), ("ef_block_sums", (null, 0, null)),
+        ("ef_complete_scales", (null, 0, null)), ("ef_check_status", (null,)),
+        ("ef_debug_shift_tile", (null, 0, 0)),
+    ]:
+        rc = getattr(lib, name)(*args)
+        assert rc in (ef.EF_ERR_INVALID_ARG, ef.EF_ERR_BAD_STATE), (name, rc)
+    assert lib.ef_message_units(null, 0, 1) == -1 and lib.ef_status_word(null) is None
+    assert lib.ef_debug_build() in (0, 1)
+    # top-k: sizes and null pointers
+    out = ctypes.c_size_t(0)
+    assert lib.ef_topk_workspace_bytes(0, ctypes.byref(out)) == ef.EF_ERR_INVALID_ARG
+    assert lib.ef_topk_workspace_bytes(1 << 20, ctypes.byref(out)) == ef.EF_OK and out.value >= 3 * 2048 * 8
+    assert lib.ef_topk_compress(null, 16, 4, null, null, null, null, 0, null) == ef.EF_ERR_INVALID_ARG
+    buf = 4096                                                   # any non-null, 256-byte aligned value
+    assert lib.ef_topk_compress(buf, 16, 17, buf, buf, None, buf, 1 << 20, None) == ef.EF_ERR_INVALID_ARG
+    assert lib.ef_topk_compress(buf, 16, 4, buf, buf, None, buf, 8, None) == ef.EF_ERR_WORKSPACE
+    # stream probe: n must be a positive multiple of 4096, pointers 16-byte aligned
+    assert lib.ef_stream_probe(0, buf, buf, buf, 1000, None) == ef.EF_ERR_INVALID_ARG
+    assert lib.ef_stream_probe(7, buf, buf, buf, 4096, None) == ef.EF_ERR_INVALID_ARG
+    assert lib.ef_stream_probe(0, buf + 4, buf, buf, 4096, None) == ef.EF_ERR_ALIGNMENT
+    assert lib.ef_worker_step_noalloc(buf, buf, buf, buf, (1 << 24) + 1, 0.9, buf, buf, None) == ef.EF_ERR_TOO_LARGE

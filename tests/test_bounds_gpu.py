@@ -161,3 +161,25 @@ def test_regular_build_has_no_shift_hook():
     with pytest.raises(ef.EFError) as ei:
         ef.ef_debug_shift_tile(eng.ctx, 0, 4)
     assert ei.value.status == ef.EF_ERR_BAD_STATE
+
+
+def test_stream_probe_kernels_do_what_the_header_says():
+    """The no-compute stream kernels behind bench.py --ceiling, inside guard bands."""
+    n = 3 * TILE
+    a, b, c = (Guarded(4 * n, torch.float32) for _ in range(3))
+    gen = torch.Generator(device="cuda").manual_seed(4)
+    a.view.copy_(torch.randn(n, device="cuda", generator=gen))
+    b.view.copy_(torch.randn(n, device="cuda", generator=gen))
+    c.view.copy_(torch.randn(n, device="cuda", generator=gen))
+    a0, b0, c0 = a.view.clone(), b.view.clone(), c.view.clone()
+    st = torch.cuda.current_stream().cuda_stream
+    ef.ef_stream_probe(ef.EF_PROBE_3R2W, a.view.data_ptr(), b.view.data_ptr(), c.view.data_ptr(), n, st)
+    assert torch.equal(a.view, a0) and torch.equal(b.view, b0 + a0) and torch.equal(c.view, c0 + (b0 + a0))
+    b1 = b.view.clone()
+    ef.ef_stream_probe(ef.EF_PROBE_1R1W, a.view.data_ptr(), b.view.data_ptr(), c.view.data_ptr(), n, st)
+    pattern = torch.tensor([1.0, -1.0, 1.0, -1.0], device="cuda").repeat(n // 4)
+    assert torch.equal(b.view, b1 + pattern)
+    ef.ef_stream_probe(ef.EF_PROBE_COPY, a.view.data_ptr(), b.view.data_ptr(), c.view.data_ptr(), n, st)
+    assert torch.equal(c.view, a0)
+    torch.cuda.synchronize()
+    assert a.intact() and b.intact() and c.intact()
