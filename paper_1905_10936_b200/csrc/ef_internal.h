@@ -22,6 +22,10 @@ inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a
 // and apply kernels), a tile is kTileChunks chunks (one CTA of the server kernel).
 constexpr int kU = 4;
 constexpr int kChunkLen = 1024 * kU;
+// ef_server_step on large layouts: blocks of up to this many tiles get their scale from the
+// update kernel itself (every CTA adds the block's <= 4 * 256 partial sums, 8 KB from L2),
+// larger ones from ef_scale_kernel.
+constexpr int kSelfScaleTiles = 256;
 // Grids up to this many chunks (about two waves of CTAs) finalise block scales in-kernel.
 constexpr int64_t kFusedMaxChunks = 1024;
 
@@ -35,9 +39,10 @@ struct Layout {
     size_t dpad = 0, wpad = 0, bpad = 0, tpad = 0;    // padded element counts per sub-buffer
     size_t off_x = 0, off_m = 0, off_pb = 0, off_spb = 0, off_words = 0, off_scales = 0,
            off_rscale = 0, off_partials = 0, off_tickets = 0, off_tiles = 0, off_blocks = 0,
-           off_multi = 0, off_stage = 0, off_mt = 0, off_dpartials = 0, off_diag = 0,
-           off_status = 0, total = 0;
+           off_multi = 0, off_multi_big = 0, off_stage = 0, off_mt = 0, off_dpartials = 0,
+           off_diag = 0, off_status = 0, total = 0;
     int32_t num_multi = 0;                            // blocks that span more than one chunk
+    int32_t num_multi_big = 0;                        // ... and more than kSelfScaleTiles tiles
 };
 
 }  // namespace efh
@@ -61,7 +66,7 @@ struct ef_ctx {
     int32_t n_served = 0, n_applied = 0;
     std::vector<efk::Tile> h_tiles;             // kept alive: source of an asynchronous upload
     std::vector<efk::Block> h_blocks;
-    std::vector<int32_t> h_multi;
+    std::vector<int32_t> h_multi, h_multi_big;
     int fused = 0;                         // block scales finalised inside the main kernels
     // blocks cut across devices (ef_set_block_divisors): slot k's scales of the pieces are still
     // to be completed from the sum over all pieces (ef_complete_scales)
@@ -89,6 +94,7 @@ struct ef_ctx {
     const efk::Tile* tiles() const { return (const efk::Tile*)(ws + L.off_tiles); }
     const efk::Block* blocks() const { return (const efk::Block*)(ws + L.off_blocks); }
     const int* multi() const { return (const int*)(ws + L.off_multi); }
+    const int* multi_big() const { return (const int*)(ws + L.off_multi_big); }
     float* mt() const { return (float*)(ws + L.off_mt); }
     double* dpartials(int i) const { return (double*)(ws + L.off_dpartials) + (size_t)i * 3 * L.tpad; }
     double* diag(int i) const { return (double*)(ws + L.off_diag) + (size_t)i * 4 * L.bpad; }

@@ -193,6 +193,14 @@ struct ApplyArgs {
     float* mt;               // decay momentum mtilde
     float mu, lambda;
     DebugLimits lim;
+    // Scales completed here (ef_server_step, large layouts): for a block of more than one chunk
+    // and at most `self_scale_tiles` tiles (0: never) every CTA adds the block's partial sums
+    // itself, in ef_scale_kernel's order, instead of waiting for a launch of that kernel; the
+    // CTA of the block's first tile also records the scale.  Saves a launch per server step.
+    const double* partials;
+    float* scale_out;
+    float* rscale;
+    int self_scale_tiles;
 };
 
 struct ResidualArgs {
@@ -1153,8 +1161,30 @@ __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
         a.fused_in ? reinterpret_cast<const float*>(a.words) +
                          (message_unit(a.blocks[t.block].word, t.block) - a.msg_base)
                    : a.scales + t.block;
+    // The block's scale: read, or formed here from the block's partial sums (uniform per CTA).
+    auto block_scale = [&]() -> float {
+        if (a.self_scale_tiles > 0) {
+            const Block b = a.blocks[t.block];
+            if (b.len > kChunk && b.tile_count <= a.self_scale_tiles) {
+                __shared__ double s_sum[kWarps];
+                __shared__ float s_scale;
+                const double S = sum_slots(b, a.partials, s_sum, a.lim.tc);     // valid in thread 0
+                if (threadIdx.x == 0) {
+                    const float s = (float)(S / (double)b.div);
+                    s_scale = s;
+                    if (t.start == b.start) {
+                        a.scale_out[t.block] = s;
+                        a.rscale[t.block] = s;
+                    }
+                }
+                __syncthreads();
+                return s_scale;
+            }
+        }
+        return *scale_ptr;
+    };
     if ((t.start & 3) != 0) {
-        const float step = __fmul_rn(a.eta, *scale_ptr);
+        const float step = __fmul_rn(a.eta, block_scale());
         const int rows = (t.len + 31) >> 5;
         for (int r = warp; r < rows; r += kWarps) {
             const int o = r * 32 + lane;
@@ -1209,7 +1239,7 @@ __global__ void __launch_bounds__(kThreads) ef_apply_kernel(const ApplyArgs a) {
     float xA[U][4], xB[U][4], mA[UM][4], mB[UM][4];
     unsigned nA[U], nB[U];
     load_chunk(0, xA, mA, nA);
-    step = __fmul_rn(a.eta, *scale_ptr);               // its latency overlaps the first loads
+    step = __fmul_rn(a.eta, block_scale());            // its latency overlaps the first loads
     for (int c = 0; c < nchunks; c += 2) {
         if (c + 1 < nchunks) load_chunk(c + 1, xB, mB, nB);
         update_chunk(c, xA, mA, nA);

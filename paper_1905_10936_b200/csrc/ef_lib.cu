@@ -50,7 +50,11 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
     L->tile_chunks = (chunks <= kFusedMaxChunks) ? 1 : efk::kTileChunks;
     const int64_t tile_len = (int64_t)kChunkLen * L->tile_chunks;
     int64_t T = 0;
-    for (int32_t b = 0; b < B; ++b) T += (offsets[b + 1] - offsets[b] + tile_len - 1) / tile_len;
+    for (int32_t b = 0; b < B; ++b) {
+        const int64_t tiles_b = (offsets[b + 1] - offsets[b] + tile_len - 1) / tile_len;
+        T += tiles_b;
+        if (tiles_b > kSelfScaleTiles) L->num_multi_big += 1;
+    }
     if (T * L->tile_chunks > 0x7fffffffLL) return EF_ERR_INVALID_ARG;
     L->W = W; L->num_tiles = T;
     L->dpad = align_up((size_t)d * 4) / 4;
@@ -74,6 +78,7 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
     L->off_tiles = o;    o += align_up((size_t)T * sizeof(Tile));
     L->off_blocks = o;   o += align_up((size_t)B * sizeof(Block));
     L->off_multi = o;    o += align_up((size_t)L->num_multi * sizeof(int32_t) + 4);
+    L->off_multi_big = o; o += align_up((size_t)L->num_multi_big * sizeof(int32_t) + 4);
     L->off_status = o;   o += kAlign;
     L->off_stage = o;
     if (flags & EF_FLAG_HOST_STAGING) o += 2 * L->dpad * 4;
@@ -190,7 +195,10 @@ cudaError_t launch_server_t(ef_ctx* c, const efk::ServerArgs& a, unsigned grid, 
 // Server lines of Algorithm 4 on the blocks [b0, b1).  msgs == nullptr: the workers' words and
 // scales are the context's own; otherwise worker i's fused message for exactly this block range
 // starts at msgs + i * msg_stride.
-int launch_server_range(ef_ctx* c, int b0, int b1, const uint32_t* msgs, long long msg_stride) {
+// defer_scales: the caller applies the update right away with launch_apply_range(.., self_scale):
+// only the blocks too large for that get their scale from ef_scale_kernel here.
+int launch_server_range(ef_ctx* c, int b0, int b1, const uint32_t* msgs, long long msg_stride,
+                        bool defer_scales = false) {
     const int M = c->L.M, S = c->srv();
     const TileRange tr = tiles_of(c, b0, b1);
     efk::ServerArgs a;
@@ -230,13 +238,15 @@ int launch_server_range(ef_ctx* c, int b0, int b1, const uint32_t* msgs, long lo
     }
     EF_CUDA(c, le);
     c->launches += 1;
-    if (!c->fused && c->L.num_multi > 0) {
+    const std::vector<int32_t>& list = defer_scales ? c->h_multi_big : c->h_multi;
+    if (!c->fused && !list.empty()) {
         // follow-up sums for the blocks of the range that span more than one chunk
-        const auto lo = std::lower_bound(c->h_multi.begin(), c->h_multi.end(), b0) - c->h_multi.begin();
-        const auto hi = std::lower_bound(c->h_multi.begin(), c->h_multi.end(), b1) - c->h_multi.begin();
+        const auto lo = std::lower_bound(list.begin(), list.end(), b0) - list.begin();
+        const auto hi = std::lower_bound(list.begin(), list.end(), b1) - list.begin();
         if (hi > lo) {
             efk::ScaleArgs sa;
-            sa.partials = c->partials(S); sa.blocks = c->blocks(); sa.multi = c->multi() + lo;
+            sa.partials = c->partials(S); sa.blocks = c->blocks();
+            sa.multi = (defer_scales ? c->multi_big() : c->multi()) + lo;
             sa.scale_out = c->scales(S); sa.rscale = c->rscale(S);
             sa.partial_stride = (long long)c->L.tpad; sa.scale_stride = (int)c->L.bpad;
             sa.dpartials = nullptr; sa.diag = nullptr; sa.tc = c->L.tile_chunks;
@@ -250,7 +260,7 @@ int launch_server_range(ef_ctx* c, int b0, int b1, const uint32_t* msgs, long lo
 
 // x_{t+1} = x_t - eta Deltatilde_t on the blocks [b0, b1); the update is the context's own
 // server message (update == nullptr) or a fused message for exactly this block range.
-int launch_apply_range(ef_ctx* c, int b0, int b1, const uint32_t* update) {
+int launch_apply_range(ef_ctx* c, int b0, int b1, const uint32_t* update, bool self_scale = false) {
     const int S = c->srv();
     const TileRange tr = tiles_of(c, b0, b1);
     efk::ApplyArgs p;
@@ -260,6 +270,8 @@ int launch_apply_range(ef_ctx* c, int b0, int b1, const uint32_t* update) {
     p.msg_base = efk::message_unit(c->h_blocks[b0].word, b0);
     p.eta = c->eta; p.mu = c->mu; p.lambda = c->lambda; p.mt = c->mt();
     p.lim = c->limits();
+    p.partials = c->partials(S); p.scale_out = c->scales(S); p.rscale = c->rscale(S);
+    p.self_scale_tiles = self_scale ? kSelfScaleTiles : 0;
     if (c->lambda > 0.f)
         launch_kernel(c, efk::ef_apply_kernel<kU, true>, dim3(tr.count), 0, p);
     else
@@ -270,9 +282,11 @@ int launch_apply_range(ef_ctx* c, int b0, int b1, const uint32_t* update) {
 }
 
 int launch_server(ef_ctx* c) {
-    const int rc = launch_server_range(c, 0, c->L.B, nullptr, 0);
+    // Large layouts: the update kernel completes the scales of all but the largest blocks itself.
+    const bool self_scale = !c->fused;
+    const int rc = launch_server_range(c, 0, c->L.B, nullptr, 0, self_scale);
     if (rc != EF_OK) return rc;
-    return launch_apply_range(c, 0, c->L.B, nullptr);
+    return launch_apply_range(c, 0, c->L.B, nullptr, self_scale);
 }
 
 int check_block_range(const ef_ctx* c, int32_t b0, int32_t b1) {
@@ -346,6 +360,7 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
         }
         blk.tile_count = (int)c->h_tiles.size() - blk.tile_begin;
         if (len > kChunkLen) c->h_multi.push_back(b);
+        if (blk.tile_count > kSelfScaleTiles) c->h_multi_big.push_back(b);
         word += (len + 31) / 32;
     }
     } catch (const std::bad_alloc&) {
@@ -371,6 +386,10 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
     if (!c->h_multi.empty() &&
         (ce = cudaMemcpyAsync(c->ws + L.off_multi, c->h_multi.data(),
                               c->h_multi.size() * sizeof(int32_t), cudaMemcpyHostToDevice,
+                              c->stream)) != cudaSuccess) return fail(ce);
+    if (!c->h_multi_big.empty() &&
+        (ce = cudaMemcpyAsync(c->ws + L.off_multi_big, c->h_multi_big.data(),
+                              c->h_multi_big.size() * sizeof(int32_t), cudaMemcpyHostToDevice,
                               c->stream)) != cudaSuccess) return fail(ce);
     if ((ce = prepare_server(M)) != cudaSuccess) return fail(ce);
     {

@@ -87,6 +87,8 @@ def test_batched_and_per_worker_calls_are_bit_identical():
     ([BIG + 4, 777, 2 * BIG + 36, 3, 5 * TILE + 1], 7),             # not eligible: bulk falls back
     ([3, 5, 31, 33, 63, 65, 127, 129, 4 * BIG + 5], 3),             # unaligned starts: scalar path in a run
     ([1000] * 40, 16), ([BIG + 5, 300, 2 * TILE], 17),              # many small blocks; M > 16 (no table path)
+    ([300 * BIG + 128, 3 * BIG, TILE], 2),                          # a block of more than 256 tiles: its scale
+                                                                    # comes from the scale kernel, the others' from the update kernel
 ])
 def test_server_kernel_variants(sizes, M, variant):
     """The two ways the server kernel stages its inputs (bulk copies with an mbarrier where the
