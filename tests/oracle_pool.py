@@ -7,15 +7,17 @@ child process owns a contiguous range of whole blocks and runs the plain `oracle
 The oracle itself is neither threaded nor changed.  It lets the full-size layouts (2^28 and
 3.5e8 parameters) be followed element by element within the time a test may take.
 
-The parent and the children exchange vectors through three shared-memory buffers (one gradient,
-one set of packed words, one state vector); small results travel over pipes.  This module
+The parent and the children exchange vectors through three shared buffers (one gradient, one
+set of packed words, one state vector: files mapped by every process, in /dev/shm when it has
+the room); small results travel over pipes.  This module
 imports no torch and no CUDA: the children are spawned, not forked, and never touch a device.
 """
 from __future__ import annotations
 
 import multiprocessing as mp
 import os
-from multiprocessing import shared_memory
+import shutil
+import tempfile
 from typing import List, Optional, Sequence, Tuple
 
 import numpy as np
@@ -51,16 +53,28 @@ def blockwise_check(got: np.ndarray, ref: np.ndarray, sub_offsets: np.ndarray):
     return bad, mism
 
 
-def _attach(name: str, n: int, dtype):
-    shm = shared_memory.SharedMemory(name=name)
-    return shm, np.ndarray((n,), dtype=dtype, buffer=shm.buf)
+def _attach(path: str, n: int, dtype):
+    return np.memmap(path, dtype=dtype, mode="r+", shape=(max(n, 1),))[:n]
+
+
+def _shared_dir(nbytes: int) -> str:
+    """A directory for the shared buffers: memory-backed /dev/shm when it has the room, else the
+    ordinary temporary directory (slower, but it cannot run out of space under a write)."""
+    for base in ("/dev/shm", tempfile.gettempdir()):
+        try:
+            st = os.statvfs(base)
+            if st.f_bavail * st.f_frsize > nbytes + (64 << 20):
+                return tempfile.mkdtemp(prefix="oracle_pool_", dir=base)
+        except OSError:
+            pass
+    return tempfile.mkdtemp(prefix="oracle_pool_")
 
 
 def _child(conn, names, d, W, offsets, woffsets, b0, b1, M, mu, eta):
     from oracle import Oracle
-    shm_g, g = _attach(names[0], d, np.float32)
-    shm_h, hint = _attach(names[1], W, np.uint32)
-    shm_b, buf = _attach(names[2], d, np.float32)
+    g = _attach(names[0], d, np.float32)
+    hint = _attach(names[1], W, np.uint32)
+    buf = _attach(names[2], d, np.float32)
     lo, hi = int(offsets[b0]), int(offsets[b1])
     wlo, whi = int(woffsets[b0]), int(woffsets[b1])
     sub = np.ascontiguousarray(offsets[b0:b1 + 1] - offsets[b0])
@@ -98,8 +112,6 @@ def _child(conn, names, d, W, offsets, woffsets, b0, b1, M, mu, eta):
     finally:
         orc.close()
         del g, hint, buf
-        for s in (shm_g, shm_h, shm_b):
-            s.close()
 
 
 class OraclePool:
@@ -118,14 +130,16 @@ class OraclePool:
         self.W = int(self.woffsets[-1])
         nproc = nproc or min(os.cpu_count() or 1, 16)
         self.ranges = split_blocks(sizes, nproc)
-        self._shms = [shared_memory.SharedMemory(create=True, size=max(4, n * 4))
-                      for n in (self.d, self.W, self.d)]
-        self.grad = np.ndarray((self.d,), dtype=np.float32, buffer=self._shms[0].buf)
-        self.hint = np.ndarray((self.W,), dtype=np.uint32, buffer=self._shms[1].buf)
-        self.state = np.ndarray((self.d,), dtype=np.float32, buffer=self._shms[2].buf)
+        self._dir = _shared_dir(4 * (2 * self.d + self.W))
+        names = [os.path.join(self._dir, n) for n in ("grad", "hint", "state")]
+        for path, n in zip(names, (self.d, self.W, self.d)):
+            with open(path, "wb") as f:
+                f.truncate(4 * max(n, 1))
+        self.grad = _attach(names[0], self.d, np.float32)
+        self.hint = _attach(names[1], self.W, np.uint32)
+        self.state = _attach(names[2], self.d, np.float32)
         ctx = mp.get_context("spawn")
         self._procs, self._conns = [], []
-        names = [s.name for s in self._shms]
         for (b0, b1) in self.ranges:
             parent, child = ctx.Pipe()
             p = ctx.Process(target=_child, args=(child, names, self.d, self.W, self.offsets,
@@ -159,12 +173,7 @@ class OraclePool:
                     p.terminate()          # the exact child this pool started
             self._conns, self._procs = [], []
             self.grad = self.hint = self.state = None
-            for s in self._shms:
-                try:
-                    s.close(); s.unlink()
-                except Exception:
-                    pass
-            self._shms = []
+            shutil.rmtree(self._dir, ignore_errors=True)
 
     def __del__(self):
         self.close()
