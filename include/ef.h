@@ -7,6 +7,12 @@
  *     for each worker i in [0, M):  ef_worker_step(ctx, i, g_{t,i})     (or one ef_worker_step_all)
  *     ef_server_step(ctx)
  *
+ * Further down: the stepsize sequence and the weight-decay side path, per-block diagnostics,
+ * the same iteration in pieces for one worker per GPU with a block-sharded server (fused
+ * messages), layouts cut inside blocks, the paper's comparison compressors (signum with
+ * majority vote, top-k), and a few entry points without a counterpart in the paper
+ * (measurement aid, checked build, no-allocation worker step).
+ *
  * All entry points are plain C.  "device" pointers are CUDA device pointers of the current
  * device, "host" pointers are ordinary host pointers.  The library never allocates device
  * memory: the caller hands over one workspace (size from ef_workspace_bytes) and keeps
@@ -68,6 +74,8 @@ enum ef_status {
 #define EF_FLAG_FUSED_SCALE 2u     /* always complete the sums inside the main kernels */
 #define EF_FLAG_SPLIT_SCALE 4u     /* always use the follow-up kernel */
 #define EF_FLAG_WEIGHT_DECAY 8u    /* reserve the d-float decay momentum for ef_set_weight_decay */
+#define EF_FLAG_DIAGNOSTICS 16u    /* worker steps also record per-block sums (ef_worker_diagnostics);
+                                      implies the follow-up scale kernel, excludes EF_FLAG_FUSED_SCALE */
 #define EF_FLAG_ONE_LOCAL_WORKER 32u /* this process is ONE worker of M (the paper's setting: one worker
                                       per GPU) and the server of some block range: the workspace holds
                                       the state of a single worker (index 0 in every per-worker call),
@@ -84,8 +92,6 @@ enum ef_status {
                                       on the device for the predecessor's results.  Off by default: on B200
                                       it did not shorten the launch-bound small layouts (results are
                                       identical either way). */
-#define EF_FLAG_DIAGNOSTICS 16u    /* worker steps also record per-block sums (ef_worker_diagnostics);
-                                      implies the follow-up scale kernel, excludes EF_FLAG_FUSED_SCALE */
 
 /* Maximum number of simulated workers. */
 #define EF_MAX_WORKERS 4096
