@@ -420,15 +420,12 @@ __device__ __forceinline__ void finish_block_diag(double acc, const DiagAcc& d, 
 // lanes 8q..8q+7 together hold 32 consecutive elements.  Returns the word in every lane of
 // the group.
 __device__ __forceinline__ unsigned pack_nibbles(unsigned nib, int lane) {
+    // three xor-shuffles; a single __reduce_or_sync over the 8-lane group measured slower
     unsigned v = nib << ((lane & 7) * 4);
-#ifdef EF_REDUX_PACK
-    return __reduce_or_sync(0xffu << (lane & 24), v);
-#else
     v |= __shfl_xor_sync(kFull, v, 1);
     v |= __shfl_xor_sync(kFull, v, 2);
     v |= __shfl_xor_sync(kFull, v, 4);
     return v;
-#endif
 }
 
 __device__ __forceinline__ void load4(const float* p, int o, int len, bool full, float (&v)[4]) {
@@ -617,10 +614,7 @@ __global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a0
 // sign bits of element k; the data loaded by lane q lands at bit kLaneWorker(q), i.e. worker w
 // sits at bit w.
 constexpr int kMaxLutWorkers = 16;      // workers the table path handles (two lane groups)
-#ifndef EF_LUT_WORKERS
-#define EF_LUT_WORKERS 6
-#endif
-constexpr int kLutWorkers = EF_LUT_WORKERS;   // workers covered by the table
+constexpr int kLutWorkers = 6;        // workers covered by the replicated table (7 would cost a CTA per SM)
 constexpr int kLutCopies = 32;        // one copy per lane
 
 __host__ __device__ constexpr int kLaneWorker(int q) {
