@@ -595,7 +595,10 @@ def run_ps(args) -> None:
     """The paper's setting in pieces on ONE GPU: G ranks (rank r = worker r + the server of one
     block range) stepped one after the other, the exchange replaced by device copies.  Times the
     pieces a real rank would run between its collectives; the exchange itself cannot be measured
-    on one device and is given analytically (bytes per rank and phase)."""
+    on one device and is given analytically (bytes per rank and phase).  --push times the push
+    variant instead: the worker kernel stores its message into the servers' receive buffers and
+    the servers store their update slices into every rank's update buffer (here all on one
+    device, so the stores that would cross NVLink are local)."""
     from paper_1905_10936_b200 import ps
     from paper_1905_10936_b200.engine import EFEngine
     if int(os.environ.get("RANK", "0")) != 0:
@@ -606,7 +609,10 @@ def run_ps(args) -> None:
     ranks = [ps.Rank(EFEngine(w.offsets, G, w.mu, w.eta, one_local_worker=True), w.sizes, r, G) for r in range(G)]
     es = w.element_scales("cuda")
     grads = [w.draw_grad(0, i, "cuda", es) for i in range(G)]
-    names = ["worker_step", "pack_message", "server_step_range", "pack_update", "apply_update"]
+    names = (["worker_step_push", "server_step_range", "push_update", "apply_update"] if args.push else
+             ["worker_step", "pack_message", "server_step_range", "pack_update", "apply_update"])
+    if args.push:
+        ps.connect_emulated(ranks)
     acc = {n: 0.0 for n in names}
 
     def timed(name, fn, record):
@@ -620,6 +626,20 @@ def run_ps(args) -> None:
     for it in range(W + K):
         rec = it >= W
         pending = []
+        if args.push:
+            for rk, g in zip(ranks, grads):
+                timed("worker_step_push", lambda: rk.engine.worker_step_push(0, g, rk.block_dst), rec)
+            for rk in ranks:
+                m = rk.mine
+                if m.b1 > m.b0:
+                    timed("server_step_range", lambda: rk.engine.server_step_range(m.b0, m.b1, rk.recv), rec)
+                    timed("push_update", lambda: rk.engine.push_message(-1, m.b0, m.b1, rk.update_dst), rec)
+            for rk in ranks:
+                timed("apply_update", lambda: rk.engine.apply_update(0, rk.B, rk.update), rec)
+            torch.cuda.synchronize()
+            for name, e0, e1 in pending:
+                acc[name] += e0.elapsed_time(e1)
+            continue
         for rk, g in zip(ranks, grads):
             timed("worker_step", lambda: rk.engine.worker_step(0, g), rec)
             timed("pack_message", lambda: rk.engine.pack_message(0, 0, rk.B, rk.send), rec)
@@ -652,7 +672,8 @@ def run_ps(args) -> None:
             "value": w.d / (total_ms * 1e-3), "unit": "params/s", "n_gpus": 1, "steps": K, "warmup": W,
             "ms_per_step": total_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic", "config": config_dict(w),
-            "run": {"workload": "ps", "ranks": G, "ms_per_rank": per_rank_ms,
+            "run": {"workload": "ps", "variant": "push" if args.push else "collective", "ranks": G,
+                    "ms_per_rank": per_rank_ms,
                     "bytes_per_rank": {"worker_step": worker_call_bytes(w.d, w.B),
                                        "server_step_range": (8.0 + (G + 1) / 8.0) * w.d / G,
                                        "apply_update": 8.125 * w.d},
@@ -697,6 +718,8 @@ def main():
                          "topk: the top-k compressor on one vector of the layout's size; "
                          "ps: the one-worker-per-rank protocol with a block-sharded server, its "
                          "compute pieces timed with the M ranks emulated on one GPU")
+    ap.add_argument("--push", action="store_true",
+                    help="--workload ps: the push variant (messages stored where their readers are)")
     ap.add_argument("--topk-fraction", type=float, default=0.01, help="k / n for --workload topk")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--per-worker-calls", action="store_true",

@@ -273,6 +273,32 @@ int ef_server_step_range(ef_ctx* ctx, int32_t b0, int32_t b1,
                          const uint32_t* msgs /* device or NULL */, int64_t msg_stride);
 int ef_apply_update(ef_ctx* ctx, int32_t b0, int32_t b1, const uint32_t* update /* device or NULL */);
 
+/* ---- The same protocol with the messages stored where their readers are (Section 4.2's remedy
+ * for the server bottleneck is to spread the blocks over several servers; a worker's message
+ * then has one destination per block).  Instead of packing a message and handing it to a
+ * collective, the kernels store it directly: into this device's memory or, with peer access
+ * enabled by the caller, into another device's receive buffer.  The library only stores through
+ * the pointers it is given; making the stores visible to the reader (end of the stream's work
+ * plus whatever barrier the caller uses between devices) is the caller's business.
+ *
+ * ef_worker_step_push: ef_worker_step, except that the packed words go to the destinations
+ *   instead of the context's word buffer: block b's fused message, [scale | ceil(d_b/32) words]
+ *   as above, is written at block_dst[b].  block_dst is a DEVICE array of B device pointers
+ *   (4-byte aligned targets; the array is read by the enqueued kernels and must stay unchanged
+ *   until they have run).  The scales are also kept in the context (ef_worker_scales);
+ *   ef_worker_words(i) is NOT written, so until worker i's next plain step ef_pack_message(i)
+ *   and the calls that read the workers' own words (ef_server_step, ef_server_step_range with
+ *   msgs == NULL) answer BAD_STATE.  Not for contexts with cut blocks (BAD_STATE).
+ * ef_push_message: ef_pack_message with n_dst destinations (1..64): the message of blocks
+ *   [b0, b1) is written to each dst[q], a HOST array of n_dst device pointers (read during the
+ *   call).  With the servers' update slices pushed into every worker's update buffer this is the
+ *   pull of Algorithm 4 without a separate gather.
+ * Errors: INVALID_ARG (null pointers, index, range, n_dst), ALIGNMENT (grad), BAD_STATE, CUDA. */
+int ef_worker_step_push(ef_ctx* ctx, int32_t i, const float* grad /* device */,
+                        uint32_t* const* block_dst /* device array of B device pointers */);
+int ef_push_message(ef_ctx* ctx, int32_t who, int32_t b0, int32_t b1, int32_t n_dst,
+                    uint32_t* const* dst /* host array of n_dst device pointers */);
+
 /* ---- Blocks cut across devices.  The method is per element except for one number per block,
  * ||p_b||_1 (Section 3.2), so a layout may be cut inside a block (e.g. an embedding larger than a
  * device's share): each device holds a piece as a block of its own context and the only exchange

@@ -75,6 +75,8 @@ SIGNATURES = {
     "ef_message_units": (_i64, [_vp, _i32, _i32]),
     "ef_pack_message": (ctypes.c_int, [_vp, _i32, _i32, _i32, _vp]),
     "ef_server_step_range": (ctypes.c_int, [_vp, _i32, _i32, _vp, _i64]),
+    "ef_worker_step_push": (ctypes.c_int, [_vp, _i32, _vp, _vp]),
+    "ef_push_message": (ctypes.c_int, [_vp, _i32, _i32, _i32, _i32, _vp]),
     "ef_apply_update": (ctypes.c_int, [_vp, _i32, _i32, _vp]),
     "ef_set_block_divisors": (ctypes.c_int, [_vp, _vp]),
     "ef_block_sums": (ctypes.c_int, [_vp, _i32, _vp]),
@@ -267,6 +269,17 @@ def ef_message_units(ctx: int, b0: int, b1: int) -> int:
 
 def ef_pack_message(ctx: int, who: int, b0: int, b1: int, dst_ptr: int) -> None:
     _check(load_library().ef_pack_message(ctx, who, b0, b1, dst_ptr), "ef_pack_message")
+
+
+def ef_worker_step_push(ctx: int, i: int, grad_ptr: int, block_dst_ptr: int) -> None:
+    """block_dst_ptr: device array of B device pointers (one destination per block)."""
+    _check(load_library().ef_worker_step_push(ctx, i, grad_ptr, block_dst_ptr), "ef_worker_step_push")
+
+
+def ef_push_message(ctx: int, who: int, b0: int, b1: int, dst_ptrs) -> None:
+    """dst_ptrs: sequence of device addresses; the message is written to each of them."""
+    arr = (ctypes.c_void_p * len(dst_ptrs))(*[int(p) for p in dst_ptrs])
+    _check(load_library().ef_push_message(ctx, who, b0, b1, len(dst_ptrs), arr), "ef_push_message")
 
 
 def ef_server_step_range(ctx: int, b0: int, b1: int, msgs_ptr: Optional[int], msg_stride: int) -> None:

@@ -72,6 +72,8 @@ struct ef_ctx {
     // to be completed from the sum over all pieces (ef_complete_scales)
     bool has_partial = false;
     std::vector<uint8_t> scales_open;
+    // worker i's last step stored its packed words at the caller's destinations, not in words(i)
+    std::vector<uint8_t> pushed;
     bool use_bulk = false;                 // the server kernel stages its inputs with cp.async.bulk
     bool pdl = false;                      // kernels are launched with programmatic stream serialization
     // host-staging path

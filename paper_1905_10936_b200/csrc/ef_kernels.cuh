@@ -69,17 +69,24 @@ struct __align__(16) Block {
 };
 static_assert(sizeof(Block) == 48, "Block must be 48 bytes");
 
+// Push table of a worker launch (null: none).  Entry b is where block b's fused message
+// [scale | packed words] is to be written: any memory this device can store to, e.g. the receive
+// buffer of the block's server on another device.
+using PushTable = uint32_t* const*;
+
 // The scale of block b from its L1 sum S (Section 3.2: ||p_b||_1 / d_b), or, for a piece of a
 // cut block, the sum itself for ef_complete_scales.  One thread.
 __device__ __forceinline__ void publish_scale(const Block& b, int block_id, double S,
                                               double* __restrict__ partials, int tc,
-                                              float* __restrict__ scale_out, float* __restrict__ rscale) {
+                                              float* __restrict__ scale_out, float* __restrict__ rscale,
+                                              PushTable push = nullptr) {
     if (b.partial) {
         partials[(long long)b.tile_begin * tc] = S;
     } else {
         const float s = (float)(S / (double)b.div);
         scale_out[block_id] = s;
         rscale[block_id] = s;
+        if (push) push[block_id][0] = __float_as_uint(s);      // first unit of the block's message
     }
 }
 
@@ -128,6 +135,7 @@ struct WorkerArgs {
     // arrays of `partial_stride` slots each, and the per-block results [B][4] (|p|, p^2, |g|, g^2)
     double* dpartials;
     double* diag;
+    PushTable push;        // not null: the message goes there instead of to `words` (single-worker launches)
     DebugLimits lim;
 };
 
@@ -177,6 +185,7 @@ struct ScaleArgs {
     double* dpartials;          // DIAG instantiation only, as in WorkerArgs
     double* diag;
     int tc;                     // chunks (= partial-sum slots) per tile
+    PushTable push;             // as in WorkerArgs
 };
 
 struct ApplyArgs {
@@ -308,9 +317,9 @@ __device__ __forceinline__ double sum_partials_and_write(const Block& b, int blo
                                                          double* __restrict__ partials,
                                                          float* __restrict__ scale_out,
                                                          float* __restrict__ rscale,
-                                                         double* s_sum, int tc) {
+                                                         double* s_sum, int tc, PushTable push = nullptr) {
     const double S = sum_slots(b, partials, s_sum, tc);
-    if (threadIdx.x == 0) publish_scale(b, block_id, S, partials, tc, scale_out, rscale);
+    if (threadIdx.x == 0) publish_scale(b, block_id, S, partials, tc, scale_out, rscale, push);
     return S;
 }
 
@@ -327,14 +336,15 @@ __device__ __forceinline__ void finish_block(double acc, long long slot, int zer
                                              double* __restrict__ partials,
                                              unsigned* __restrict__ tickets,
                                              float* __restrict__ scale_out,
-                                             float* __restrict__ rscale, int fused, int tc) {
+                                             float* __restrict__ rscale, int fused, int tc,
+                                             PushTable push = nullptr) {
     __shared__ double s_sum[kWarps];
     __shared__ int s_last;
     const double S = cta_sum(acc, s_sum);
     if (threadIdx.x == 0) {
         int last = 0;
         if (alone) {
-            publish_scale(blocks[block_id], block_id, S, partials, tc, scale_out, rscale);
+            publish_scale(blocks[block_id], block_id, S, partials, tc, scale_out, rscale, push);
         } else {
             partials[slot] = S;
             for (int z = 1; z <= zero_slots; ++z) partials[slot + z] = 0.0;
@@ -351,7 +361,7 @@ __device__ __forceinline__ void finish_block(double acc, long long slot, int zer
     if (!s_last) return;
     __threadfence();
     const Block b = blocks[block_id];
-    sum_partials_and_write(b, block_id, partials, scale_out, rscale, s_sum, tc);
+    sum_partials_and_write(b, block_id, partials, scale_out, rscale, s_sum, tc, push);
     if (threadIdx.x == 0) tickets[block_id] = 0u;      // ready for the next launch
 }
 
@@ -365,7 +375,7 @@ __global__ void __launch_bounds__(kThreads) ef_scale_kernel(const ScaleArgs a) {
     const Block b = a.blocks[block_id];
     const long long so = (long long)blockIdx.y * a.scale_stride;
     const double S = sum_partials_and_write(b, block_id, a.partials + blockIdx.y * a.partial_stride,
-                                            a.scale_out + so, a.rscale + so, s_sum, a.tc);
+                                            a.scale_out + so, a.rscale + so, s_sum, a.tc, a.push);
     if (DIAG) {
         double* dg = a.diag + (so + block_id) * 4;
         if (threadIdx.x == 0) dg[0] = S;
@@ -393,7 +403,7 @@ __device__ __forceinline__ void finish_block_diag(double acc, const DiagAcc& d, 
                                                   long long partial_stride,
                                                   double* __restrict__ diag,
                                                   float* __restrict__ scale_out,
-                                                  float* __restrict__ rscale) {
+                                                  float* __restrict__ rscale, PushTable push) {
     __shared__ double s_sum[kWarps];
     const double in[4] = {acc, d.p2, d.g1, d.g2};
     double r[4];
@@ -407,6 +417,7 @@ __device__ __forceinline__ void finish_block_diag(double acc, const DiagAcc& d, 
         const float s = (float)(r[0] / (double)block_len);
         scale_out[block_id] = s;
         rscale[block_id] = s;
+        if (push) push[block_id][0] = __float_as_uint(s);
 #pragma unroll
         for (int k = 0; k < 4; ++k) diag[(long long)block_id * 4 + k] = r[k];
     } else {
@@ -574,6 +585,8 @@ __global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a0
     const Block b = a.blocks[t.block];
     const bool alone = b.len <= 1024 * U;              // the block is this single chunk
     if (t.len <= 0 && alone) return;
+    // word w of the layout is word w - b.word of its block: unit 1 + w - b.word of the block's message
+    if (a.push) a.words = a.push[t.block] + 1 - b.word;
     double acc = 0.0;
     DiagAcc dacc;
     if (t.len > 0) {
@@ -587,10 +600,10 @@ __global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a0
     }
     if (DIAG)
         finish_block_diag(acc, dacc, blockIdx.x, alone, t.block, b.len, a.partials, a.dpartials,
-                          a.partial_stride, a.diag, a.scale_out, a.rscale);
+                          a.partial_stride, a.diag, a.scale_out, a.rscale, a.push);
     else
         finish_block(acc, blockIdx.x, 0, alone, (unsigned)(b.tile_count * a.lim.tc), t.block,
-                     a.blocks, a.partials, a.tickets, a.scale_out, a.rscale, a.fused, a.lim.tc);
+                     a.blocks, a.partials, a.tickets, a.scale_out, a.rscale, a.fused, a.lim.tc, a.push);
 }
 
 // ------------------------------------------------------------------ server kernel
@@ -1258,10 +1271,12 @@ static __global__ void __launch_bounds__(kThreads) ef_residual_kernel(const Resi
 
 // Fused message of a block range: dst gets, block after block, [scale | packed words].
 // One tile per CTA (a tile has at most kTileChunks*1024*U/32 words).
+constexpr int kMaxPackTargets = 64;
 struct PackArgs {
     const uint32_t* words;
     const float* scales;
-    uint32_t* dst;
+    uint32_t* dst[kMaxPackTargets];   // n_dst copies of the message are written (own or peer memory)
+    int n_dst;
     const Tile* tiles;
     const Block* blocks;
     int tile0;
@@ -1273,11 +1288,16 @@ static __global__ void __launch_bounds__(kThreads) ef_pack_kernel(const PackArgs
     const Tile t = a.tiles[blockIdx.x + a.tile0];
     if (!work_item_ok(t, a.lim, 1 << 30)) return;
     const Block b = a.blocks[t.block];
-    uint32_t* dst = a.dst + (message_unit(t.word, t.block) + 1 - a.msg_base);
+    const long long unit = message_unit(t.word, t.block) + 1 - a.msg_base;
     const int nwords = (t.len + 31) >> 5;
-    for (int k = threadIdx.x; k < nwords; k += kThreads) dst[k] = a.words[t.word + k];
-    if (threadIdx.x == 0 && t.start == b.start)
-        a.dst[message_unit(b.word, t.block) - a.msg_base] = __float_as_uint(a.scales[t.block]);
+    for (int k = threadIdx.x; k < nwords; k += kThreads) {
+        const uint32_t w = a.words[t.word + k];
+        for (int q = 0; q < a.n_dst; ++q) a.dst[q][unit + k] = w;
+    }
+    if (threadIdx.x == 0 && t.start == b.start) {
+        const uint32_t s = __float_as_uint(a.scales[t.block]);
+        for (int q = 0; q < a.n_dst; ++q) a.dst[q][message_unit(b.word, t.block) - a.msg_base] = s;
+    }
 }
 
 // Cut blocks: dst[b] = the piece's fp64 sum of |p| (0 for blocks held whole), and the scale of

@@ -92,9 +92,10 @@ namespace {
 
 // Non-fused mode: adds the partial sums of every block larger than one chunk of buffer set k
 // (worker k, or the server for k == M) after the kernel that produced them.
-int launch_scale(ef_ctx* c, int k, int count = 1) {
+int launch_scale(ef_ctx* c, int k, int count = 1, efk::PushTable push = nullptr) {
     if (c->fused || c->L.num_multi == 0) return EF_OK;
     efk::ScaleArgs a;
+    a.push = push;
     a.partials = c->partials(k); a.blocks = c->blocks(); a.multi = c->multi();
     a.scale_out = c->scales(k); a.rscale = c->rscale(k);
     a.partial_stride = (long long)c->L.tpad; a.scale_stride = (int)c->L.bpad;
@@ -111,8 +112,11 @@ int launch_scale(ef_ctx* c, int k, int count = 1) {
 }
 
 // Steps workers i .. i+count-1; worker i+k reads its gradient at grad + k*g_stride.
-int launch_worker(ef_ctx* c, int i, const float* grad, int count = 1, long long g_stride = 0) {
+// With a push table (single worker only) the packed words and a copy of the scales go there.
+int launch_worker(ef_ctx* c, int i, const float* grad, int count = 1, long long g_stride = 0,
+                  efk::PushTable push = nullptr) {
     efk::WorkerArgs a;
+    a.push = push;
     a.g = grad; a.m = c->m(i); a.pb = c->pb(i); a.words = c->words(i);
     a.scale_out = c->scales(i); a.rscale = c->rscale(i);
     a.partials = c->partials(i); a.tickets = c->tickets(i);
@@ -130,7 +134,8 @@ int launch_worker(ef_ctx* c, int i, const float* grad, int count = 1, long long 
     else launch_kernel(c, efk::ef_worker_kernel<kU, false>, grid, 0, a);
     EF_CUDA(c, cudaGetLastError());
     c->launches += 1;
-    return launch_scale(c, i, count);
+    for (int k = i; k < i + count; ++k) c->pushed[k] = push != nullptr;
+    return launch_scale(c, i, count, push);
 }
 
 template <int MT>
@@ -339,6 +344,7 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
     c->served.assign(B, 0);
     c->applied.assign(B, 0);
     c->scales_open.assign(L.Ml + 1, 0);
+    c->pushed.assign(L.Ml + 1, 0);
 
     // tile and block tables
     c->h_tiles.reserve((size_t)L.num_tiles);
@@ -427,6 +433,18 @@ int ef_worker_step(ef_ctx* c, int32_t i, const float* grad) {
     return EF_OK;
 }
 
+int ef_worker_step_push(ef_ctx* c, int32_t i, const float* grad, uint32_t* const* block_dst) {
+    int rc = check_worker_call(c, i, grad, kModeEF);
+    if (rc != EF_OK) return rc;
+    if (!block_dst) return EF_ERR_INVALID_ARG;
+    if (!aligned16(grad)) return EF_ERR_ALIGNMENT;
+    if (c->has_partial) return EF_ERR_BAD_STATE;         // a piece's scale is not known inside the step
+    rc = launch_worker(c, i, grad, 1, 0, block_dst);
+    if (rc != EF_OK) return rc;
+    mark_stepped(c, i, kModeEF);
+    return EF_OK;
+}
+
 int ef_worker_step_all(ef_ctx* c, const float* grads, int64_t stride) {
     if (!c || !grads || stride < c->L.d) return EF_ERR_INVALID_ARG;
     if (!aligned16(grads) || (stride & 3) != 0) return EF_ERR_ALIGNMENT;
@@ -465,6 +483,8 @@ int ef_server_step(ef_ctx* c) {
     if (c->pending != c->L.M || c->L.Ml != c->L.M || c->mode != kModeEF) return EF_ERR_BAD_STATE;
     if (c->n_served != 0 || c->n_applied != 0) return EF_ERR_BAD_STATE;   // finish the range calls instead
     if (c->has_partial) return EF_ERR_BAD_STATE;        // cut blocks: range calls with ef_complete_scales between
+    for (int i = 0; i < c->L.Ml; ++i)
+        if (c->pushed[i]) return EF_ERR_BAD_STATE;      // that worker's words are not in the context
     const int rc = launch_server(c);
     if (rc != EF_OK) return rc;
     c->eta_prev = c->eta;
@@ -479,13 +499,22 @@ int64_t ef_message_units(ef_ctx* c, int32_t b0, int32_t b1) {
 }
 
 int ef_pack_message(ef_ctx* c, int32_t who, int32_t b0, int32_t b1, uint32_t* dst) {
-    if (check_block_range(c, b0, b1) != EF_OK || !dst || who < -1 || who >= c->L.Ml)
+    return ef_push_message(c, who, b0, b1, 1, &dst);
+}
+
+int ef_push_message(ef_ctx* c, int32_t who, int32_t b0, int32_t b1, int32_t n_dst, uint32_t* const* dst) {
+    if (check_block_range(c, b0, b1) != EF_OK || !dst || who < -1 || who >= c->L.Ml ||
+        n_dst < 1 || n_dst > efk::kMaxPackTargets)
         return EF_ERR_INVALID_ARG;
+    for (int q = 0; q < n_dst; ++q)
+        if (!dst[q]) return EF_ERR_INVALID_ARG;
     const int k = who < 0 ? c->srv() : who;
-    if (c->scales_open[k]) return EF_ERR_BAD_STATE;
+    if (c->scales_open[k] || (who >= 0 && c->pushed[k])) return EF_ERR_BAD_STATE;
     const TileRange tr = tiles_of(c, b0, b1);
     efk::PackArgs a;
-    a.words = c->words(k); a.scales = c->scales(k); a.dst = dst;
+    a.words = c->words(k); a.scales = c->scales(k);
+    a.n_dst = n_dst;
+    for (int q = 0; q < efk::kMaxPackTargets; ++q) a.dst[q] = q < n_dst ? dst[q] : nullptr;
     a.tiles = c->tiles(); a.blocks = c->blocks(); a.tile0 = tr.tile0;
     a.msg_base = efk::message_unit(c->h_blocks[b0].word, b0);
     a.lim = c->limits();
@@ -500,8 +529,8 @@ int ef_server_step_range(ef_ctx* c, int32_t b0, int32_t b1, const uint32_t* msgs
     if (c->pending != c->L.Ml || c->mode != kModeEF) return EF_ERR_BAD_STATE;
     if (!msgs && c->L.Ml != c->L.M) return EF_ERR_BAD_STATE;     // the other workers' messages are needed
     if (!msgs)
-        for (int i = 0; i < c->L.Ml; ++i)
-            if (c->scales_open[i]) return EF_ERR_BAD_STATE;      // workers' cut-block scales not complete
+        for (int i = 0; i < c->L.Ml; ++i)      // workers' cut-block scales not complete, or words not here
+            if (c->scales_open[i] || c->pushed[i]) return EF_ERR_BAD_STATE;
     if (c->scales_open[c->srv()]) return EF_ERR_BAD_STATE;
     if (msgs && c->L.M > 1 && msg_stride < ef_message_units(c, b0, b1)) return EF_ERR_INVALID_ARG;
     for (int32_t b = b0; b < b1; ++b)

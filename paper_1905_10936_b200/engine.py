@@ -99,6 +99,18 @@ class EFEngine:
         assert dst.numel() >= self.message_units(b0, b1)
         ef.ef_pack_message(self.ctx, who, b0, b1, dst.data_ptr())
 
+    def worker_step_push(self, i: int, grad: torch.Tensor, block_dst: torch.Tensor) -> None:
+        """block_dst: int64 tensor of B device addresses on this device; block b's fused message
+        [scale | words] is stored at block_dst[b] (own or peer-mapped memory)."""
+        assert grad.is_cuda and grad.dtype == torch.float32 and grad.is_contiguous() and grad.numel() == self.d
+        assert block_dst.is_cuda and block_dst.dtype == torch.int64 and block_dst.is_contiguous()
+        assert block_dst.numel() == self.B
+        ef.ef_worker_step_push(self.ctx, i, grad.data_ptr(), block_dst.data_ptr())
+
+    def push_message(self, who: int, b0: int, b1: int, dst_ptrs) -> None:
+        """The fused message of blocks [b0, b1) written to every device address in dst_ptrs."""
+        ef.ef_push_message(self.ctx, who, b0, b1, list(dst_ptrs))
+
     def server_step_range(self, b0: int, b1: int, msgs: Optional[torch.Tensor] = None) -> None:
         """msgs: [M, units] int32 on this device, row i = worker i's fused message for [b0, b1)."""
         if msgs is None:

@@ -18,6 +18,24 @@ that live in the receiving rank's own memory) and calls the engine; every arithm
 inside the engine.  The same orchestration runs (a) over a real process group (NCCL on GPUs,
 gloo on CPU with a stand-in engine in the tests) and (b) with all ranks emulated one after the
 other in a single process, where the "collectives" are slice copies between the ranks' buffers.
+
+Push variant (no pack kernel, no collective on the data path): the kernels store the messages
+where their readers are.  Every rank's receive and update buffers are mapped into its peers
+(symmetric memory); the worker kernel writes block b's [scale | words] straight into the
+receive buffer of the rank that serves b, and each server writes its update slice into every
+rank's update buffer:
+
+    engine.worker_step_push(0, grad, block_dst)       block_dst[b] = address inside server(b)'s recv
+    barrier                                           all messages have landed
+    engine.server_step_range(b0, b1, recv)
+    engine.push_message(-1, b0, b1, update_dst)       the slice, stored into every rank's update
+    barrier
+    engine.apply_update(0, B, update)
+
+Only plain stores cross the links; the barrier is a one-element all-reduce on the same stream
+(no kernel of this package ever waits for another device).  Two barriers per iteration also
+order the buffers' reuse: a rank starts its next worker step only after the second barrier,
+i.e. after every server has finished reading the receive buffers of this iteration.
 """
 from __future__ import annotations
 
@@ -60,8 +78,12 @@ class Rank:
     """One worker + one server shard.  `engine` is an EFEngine created with
     one_local_worker=True and M = world (or any object with the same methods)."""
 
-    def __init__(self, engine, sizes: Sequence[int], rank: int, world: int, device=None):
+    def __init__(self, engine, sizes: Sequence[int], rank: int, world: int, device=None,
+                 recv: Optional[torch.Tensor] = None, update: Optional[torch.Tensor] = None):
+        """recv / update: buffers to use instead of fresh ones (e.g. symmetric memory), of
+        recv_units(plan, rank) resp. total units int32 elements."""
         self.engine, self.rank, self.world = engine, rank, world
+        self.sizes = [int(v) for v in sizes]
         self.B = len(sizes)
         self.plan = make_plan(sizes, world)
         self.mine = self.plan[rank]
@@ -69,8 +91,16 @@ class Rank:
         dev = device if device is not None else getattr(engine, "device", "cpu")
         i32 = dict(dtype=torch.int32, device=dev)
         self.send = torch.zeros(self.total_units, **i32)                   # my message, all blocks
-        self.recv = torch.zeros(world, max(self.mine.units, 1), **i32)     # every worker's slice for my range
-        self.update = torch.zeros(self.total_units, **i32)                 # the whole update
+        width = recv_stride(self.plan, rank)
+        if recv is None:
+            recv = torch.zeros(world * width, **i32)
+        if update is None:
+            update = torch.zeros(self.total_units, **i32)
+        assert recv.numel() >= world * width and update.numel() >= self.total_units
+        self.recv = recv[:world * width].view(world, width)                # every worker's slice for my range
+        self.update = update[:self.total_units]                            # the whole update
+        self.block_dst = None      # push variant: device table of B addresses (connect_*)
+        self.update_dst = None     # ... and where my update slice goes on every rank
         if engine is not None and self.mine.units > 0:
             assert engine.message_units(self.mine.b0, self.mine.b1) == self.mine.units
             assert engine.message_units(0, self.B) == self.total_units
@@ -88,6 +118,41 @@ class Rank:
 
     def apply(self) -> None:
         self.engine.apply_update(0, self.B, self.update)
+
+    # ---- push variant ------------------------------------------------------------------------
+    def connect(self, recv_ptrs: Sequence[int], update_ptrs: Sequence[int]) -> None:
+        """recv_ptrs[q] / update_ptrs[q]: address, valid on THIS device, of rank q's receive /
+        update buffer (its own memory for q == rank, a peer mapping otherwise)."""
+        table = push_table(self.sizes, self.plan, self.rank, recv_ptrs)
+        self.block_dst = torch.from_numpy(table).to(self.update.device)
+        self.update_dst = [int(p) + 4 * self.mine.unit0 for p in update_ptrs]
+
+    def work_push(self, grad) -> None:
+        self.engine.worker_step_push(0, grad, self.block_dst)
+
+    def serve_push(self) -> None:
+        m = self.mine
+        if m.b1 > m.b0:
+            self.engine.server_step_range(m.b0, m.b1, self.recv)
+            self.engine.push_message(-1, m.b0, m.b1, self.update_dst)
+
+
+def recv_stride(plan: List[RangePlan], q: int) -> int:
+    """Row length (32-bit units) of rank q's receive buffer: row i holds worker i's slice."""
+    return max(plan[q].units, 1)
+
+
+def push_table(sizes: Sequence[int], plan: List[RangePlan], rank: int,
+               recv_ptrs: Sequence[int]) -> np.ndarray:
+    """dst[b] = where worker `rank` stores block b's fused message: row `rank` of the receive
+    buffer of the rank that serves b, at the block's place in that rank's range (bytes)."""
+    unit = message_unit_offsets(sizes)
+    dst = np.zeros(len(sizes), dtype=np.int64)
+    for q, p in enumerate(plan):
+        row = int(recv_ptrs[q]) + 4 * rank * recv_stride(plan, q)
+        for b in range(p.b0, p.b1):
+            dst[b] = row + 4 * int(unit[b] - unit[p.b0])
+    return dst
 
 
 # ---------------------------------------------------------------------------- real process group
@@ -124,7 +189,60 @@ def step(rk: Rank, grad, group=None) -> None:
     rk.apply()
 
 
+def symmetric_buffers(sizes: Sequence[int], rank: int, world: int, device, group=None):
+    """Receive and update buffers of one rank in symmetric memory (every rank allocates the same
+    size and maps its peers' copies).  Returns (recv, update, recv_ptrs, update_ptrs) for
+    Rank(..., recv=, update=) and Rank.connect.  Fails loudly where symmetric memory is not
+    available; the collective variant (step) needs none."""
+    import torch.distributed as dist
+    import torch.distributed._symmetric_memory as symm
+    plan = make_plan(sizes, world)
+    total = int(message_unit_offsets(sizes)[-1])
+    n_recv = (world * max(recv_stride(plan, q) for q in range(world)) + 3) // 4 * 4
+    buf = symm.empty(n_recv + total, dtype=torch.int32, device=device)
+    handle = symm.rendezvous(buf, dist.group.WORLD if group is None else group)
+    buf.zero_()
+    base = [int(p) for p in handle.buffer_ptrs]
+    assert len(base) == world and base[rank] == buf.data_ptr()
+    return buf[:n_recv], buf[n_recv:], base, [p + 4 * n_recv for p in base]
+
+
+def stream_barrier(flag: torch.Tensor, group=None) -> None:
+    """Every rank's work enqueued so far has finished before anything enqueued after this call
+    starts on any rank: a one-element all-reduce on the current stream."""
+    import torch.distributed as dist
+    dist.all_reduce(flag, group=group)
+
+
+def step_push(rk: Rank, grad, flag: torch.Tensor, group=None) -> None:
+    """One iteration of rank `rk.rank` inside a process group, push variant (rk.connect first)."""
+    rk.work_push(grad)
+    stream_barrier(flag, group)
+    rk.serve_push()
+    stream_barrier(flag, group)
+    rk.apply()
+
+
 # ---------------------------------------------------------------------------- one-process emulation
+def connect_emulated(ranks: List[Rank]) -> None:
+    """Push variant with all ranks on one device: the peers' buffers are ordinary local tensors."""
+    recv_ptrs = [r.recv.data_ptr() for r in ranks]
+    update_ptrs = [r.update.data_ptr() for r in ranks]
+    for r in ranks:
+        r.connect(recv_ptrs, update_ptrs)
+
+
+def step_emulated_push(ranks: List[Rank], grads: Sequence) -> None:
+    """One iteration of all ranks, push variant, one after the other on one stream (stream order
+    stands in for the barriers)."""
+    for rk, g in zip(ranks, grads):
+        rk.work_push(g)
+    for rk in ranks:
+        rk.serve_push()
+    for rk in ranks:
+        rk.apply()
+
+
 def step_emulated(ranks: List[Rank], grads: Sequence) -> None:
     """The same iteration with all ranks held by ONE process and run one after the other; the
     collectives become slice copies between the ranks' buffers (no rank ever waits for another,

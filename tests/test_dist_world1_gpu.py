@@ -78,3 +78,32 @@ def test_distributed_shard_through_nccl(nccl_world1):
     ref.worker_step_all(gall); ref.server_step()
     ds.worker_step_all(gall); ds.server_step()
     assert torch.equal(ds.eng.params(), ref.params())
+
+
+def test_push_variant_over_symmetric_memory(nccl_world1):
+    """The push variant as a multi-device run sets it up: buffers in symmetric memory, peer
+    addresses from the rendezvous, barriers as all-reduces.  With one rank the only peer is the
+    rank itself."""
+    try:
+        import torch.distributed._symmetric_memory  # noqa: F401
+    except ImportError:
+        pytest.skip("this torch build has no symmetric memory")
+    sizes = [3 * TILE + 5, 640, 10, 4 * TILE]
+    w = wl.custom_workload("ps-symm", sizes, 1, steps=3, scale_range=(1e-2, 1.0), config_id=702)
+    ref = EFEngine(w.offsets, 1, w.mu, w.eta)
+    recv, update, recv_ptrs, update_ptrs = ps.symmetric_buffers(w.sizes, 0, 1, torch.device("cuda", 0))
+    rk = ps.Rank(EFEngine(w.offsets, 1, w.mu, w.eta, one_local_worker=True), w.sizes, 0, 1,
+                 recv=recv, update=update)
+    rk.connect(recv_ptrs, update_ptrs)
+    flag = torch.zeros(1, device="cuda")
+    es = w.element_scales("cuda")
+    for t in range(w.steps):
+        g = w.draw_grad(t, 0, "cuda", es)
+        ref.worker_step(0, g)
+        ref.server_step()
+        ps.step_push(rk, g, flag)
+        assert torch.equal(rk.engine.params(), ref.params())
+        assert torch.equal(rk.engine.residual(-1), ref.residual(-1))
+    sc, wd = ps.unpack_message(rk.update.cpu().numpy(), w.sizes, 0, w.B)
+    assert np.array_equal(sc, ref.server_scales().cpu().numpy())
+    assert np.array_equal(wd, ref.server_words().cpu().numpy().view(np.uint32))
