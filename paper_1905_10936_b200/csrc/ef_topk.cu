@@ -7,17 +7,26 @@
 // Among equal magnitudes the lower index is kept, so the result is unique and reproducible.
 //
 // Method (all integer work on the bit pattern of |v_j|, which orders like the magnitude):
-//   1. radix select of the k-th largest key in three passes over v (11 + 11 + 9 bits): each pass
-//      histograms one digit of the keys that still match the prefix found so far (shared-memory
-//      histogram per CTA, merged into a global one), then one CTA finds the bin, from the top,
-//      in which the count reaches what is still to keep, and fixes the next digit.  Result: the threshold key T and how many keys equal
-//      to T have to be kept (need_eq).
-//   2. a counting pass: per 4096-element chunk the number of keys > T and == T;
+//   1. radix select of the k-th largest key T, three digits of 11 + 11 + 9 bits:
+//      a. histogram of the first digit over v; one CTA finds the bin P0, from the top, in which
+//         the count reaches k.  Keys above that bin are kept for sure, keys below never; only the
+//         keys IN the bin (the candidates, typically a few per cent of n) still matter.
+//      b. second pass over v: histogram of the second digit of the candidates, the number of
+//         sure keys per 4096-element chunk, and the candidates' keys copied to a compact list
+//         (one segment per chunk; the order inside a segment is arbitrary and nothing depends
+//         on it).  The third digit is then histogrammed over the list, not over v.
+//      Result: T and how many keys equal to T have to be kept (need_eq).
+//   2. per chunk the number of keys > T and == T, from the chunk's sure count and its segment
+//      of the list (no pass over v);
 //   3. a scan of those counts over the chunks (one CTA);
 //   4. a scatter pass: every chunk recomputes its flags, ranks its kept elements in index order
-//      (ballots + population counts, no sorting) and writes idx, val and the residual.
-// Traffic: five reads of v, one write of the residual, k index/value pairs: about 24 bytes per
-// element.  Nothing waits on another CTA; kernel boundaries order the passes.
+//      (a shuffle scan of per-lane counts, no sorting) and writes idx, val and the residual.
+// Traffic: three reads of v, one write of the residual, k index/value pairs: about 16 bytes per
+// element (the definition needs 8).  The list has room for n/8 candidates; when the bin holds
+// more (e.g. a vector whose magnitudes are all equal) steps 1b's list is skipped and the third
+// digit and the counts are taken from v itself (two more reads of v).  Which way a call goes is
+// decided on the device; the kernels of the other way end at once.
+// Nothing waits on another CTA; kernel boundaries order the passes.
 #include "ef_internal.h"
 
 #include <algorithm>
@@ -39,30 +48,49 @@ struct TopkState {                 // lives in the workspace; written by the sel
     unsigned prefix;               // digits fixed so far (high bits of the threshold key)
     unsigned threshold;            // final: the k-th largest key T
     unsigned long long need_eq;    // final: number of keys == T to keep (lowest indices first)
+    unsigned long long ncand;      // keys in the first digit's bin
+    unsigned long long cursor;     // next free entry of the candidate list
+    unsigned compact;              // 1: the candidates fit the list
 };
 
+constexpr int kTileOfChunks = 32;     // chunks per tile of the count scan
+constexpr int kScatterChunks = 8;     // chunks per CTA of the scatter pass (divides kTileOfChunks)
+static_assert(kTileOfChunks == 32 && kTileOfChunks % kScatterChunks == 0, "one warp adds a tile's counts");
+
 struct TopkLayout {
-    size_t off_hist = 0, off_state = 0, off_cgt = 0, off_ceq = 0, off_pgt = 0, off_peq = 0, total = 0;
-    long long chunks = 0;
+    size_t off_hist = 0, off_state = 0, off_tgt = 0, off_teq = 0, off_cgt = 0, off_ceq = 0, off_pgt = 0,
+           off_peq = 0, off_seg_start = 0, off_seg_cnt = 0, off_cand = 0, total = 0;
+    long long chunks = 0, tiles = 0;
+    unsigned long long cap = 0;    // entries of the candidate list
 };
 
 TopkLayout topk_layout(int64_t n) {
     TopkLayout L;
     L.chunks = (n + kChunkLen - 1) / kChunkLen;
+    L.tiles = (L.chunks + kTileOfChunks - 1) / kTileOfChunks;
+    // room for an eighth of the vector; short vectors always fit
+    L.cap = (unsigned long long)std::max<int64_t>(n / 8, std::min<int64_t>(n, 65536));
     size_t o = 0;
+    // zeroed at the start of every call: histograms, state, per-tile totals
     L.off_hist = o;  o += align_up(sizeof(unsigned long long) * kBins * kPasses);
     L.off_state = o; o += align_up(sizeof(TopkState));
+    L.off_tgt = o;   o += align_up(sizeof(unsigned) * (size_t)L.tiles);
+    L.off_teq = o;   o += align_up(sizeof(unsigned) * (size_t)L.tiles);
+    // written before they are read
     L.off_cgt = o;   o += align_up(sizeof(unsigned) * (size_t)L.chunks);
     L.off_ceq = o;   o += align_up(sizeof(unsigned) * (size_t)L.chunks);
-    L.off_pgt = o;   o += align_up(sizeof(unsigned long long) * (size_t)L.chunks);
-    L.off_peq = o;   o += align_up(sizeof(unsigned long long) * (size_t)L.chunks);
+    L.off_pgt = o;   o += align_up(sizeof(unsigned long long) * (size_t)L.tiles);
+    L.off_peq = o;   o += align_up(sizeof(unsigned long long) * (size_t)L.tiles);
+    L.off_seg_start = o; o += align_up(sizeof(unsigned long long) * (size_t)L.chunks);
+    L.off_seg_cnt = o;   o += align_up(sizeof(unsigned) * (size_t)L.chunks);
+    L.off_cand = o;  o += align_up(sizeof(unsigned) * (size_t)L.cap);
     L.total = o;
     return L;
 }
 
 __device__ __forceinline__ unsigned key_of(float v) { return __float_as_uint(v) & 0x7fffffffu; }
 
-// Loads the four elements of this lane's row; elements past n read as a key that is never kept.
+// Loads the four elements of this lane's row; elements past n are flagged.
 __device__ __forceinline__ void load_keys(const float* __restrict__ v, long long base, long long n,
                                           float (&x)[4], bool (&in)[4]) {
     if (base + 4 <= n) {
@@ -78,13 +106,24 @@ __device__ __forceinline__ void load_keys(const float* __restrict__ v, long long
     }
 }
 
-// ---- 1. one radix pass: histogram of digit PASS over the keys that match the prefix so far
+__device__ __forceinline__ unsigned warp_inclusive_scan32(unsigned v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned u = __shfl_up_sync(kFull, v, o);
+        if (lane >= o) v += u;
+    }
+    return v;
+}
+
+// ---- 1a / fallback of 1b: histogram of digit PASS over the keys of v that match the prefix so far.
+// PASS 2 is the fallback (the candidates did not fit the list) and ends at once otherwise.
 template <int PASS>
 __global__ void __launch_bounds__(kThreads) ef_topk_hist_kernel(const float* __restrict__ v, long long n,
                                                                 long long chunks,
                                                                 const TopkState* __restrict__ st,
                                                                 unsigned long long* __restrict__ hist) {
     __shared__ unsigned s_hist[kBins];
+    if (PASS == 2 && st->compact) return;
     for (int b = threadIdx.x; b < kBins; b += kThreads) s_hist[b] = 0u;
     __syncthreads();
     constexpr int shift = pass_shift(PASS), bits = pass_bits(PASS);
@@ -110,12 +149,140 @@ __global__ void __launch_bounds__(kThreads) ef_topk_hist_kernel(const float* __r
         if (s_hist[b]) atomicAdd(&hist[b], (unsigned long long)s_hist[b]);
 }
 
+// ---- 1b. second pass over v.  Per chunk: histogram of the second digit of the candidates (keys
+// whose first digit is P0), the number of sure keys (first digit > P0) into cgt, and -- if the
+// candidates fit the list -- the candidates' keys as one segment of the list.
+// A CTA walks its chunks with the next chunk's loads issued before it waits for the list
+// position of the current one (one atomic on the global cursor per chunk), and with two
+// shared-memory lists used in turn, so that a chunk costs two barriers.
+__device__ __forceinline__ void load_chunk_keys(const float* __restrict__ v, long long n, long long c,
+                                                int warp, int lane, float (&x)[kU][4], unsigned& fin) {
+    fin = 0u;
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+        const long long base = c * kChunkLen + warp * (128 * kU) + u * 128 + lane * 4;
+        bool in[4];
+        if (base < n) load_keys(v, base, n, x[u], in);
+        else {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) { in[k] = false; x[u][k] = 0.f; }
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) fin |= in[k] ? 1u << (4 * u + k) : 0u;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) ef_topk_candidates_kernel(const float* __restrict__ v, long long n,
+                                                                      long long chunks, TopkState* st,
+                                                                      unsigned long long* __restrict__ hist,
+                                                                      unsigned* __restrict__ cgt,
+                                                                      unsigned long long* __restrict__ seg_start,
+                                                                      unsigned* __restrict__ seg_cnt,
+                                                                      unsigned* __restrict__ cand) {
+    __shared__ unsigned s_hist[kBins];
+    __shared__ unsigned s_list[2][kChunkLen];
+    __shared__ unsigned s_gt[2][kWarps];
+    __shared__ unsigned s_cnt[2];
+    __shared__ unsigned long long s_base;
+    for (int b = threadIdx.x; b < kBins; b += kThreads) s_hist[b] = 0u;
+    if (threadIdx.x == 0) { s_cnt[0] = 0u; s_cnt[1] = 0u; }
+    const unsigned P0 = st->prefix;
+    const bool compact = st->compact != 0u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float x[kU][4];
+    unsigned fin;
+    if (blockIdx.x < chunks) load_chunk_keys(v, n, blockIdx.x, warp, lane, x, fin);
+    __syncthreads();
+    int par = 0;
+    for (long long c = blockIdx.x; c < chunks; c += gridDim.x, par ^= 1) {
+        unsigned mine = 0u;                    // bit 4u + k: element is a candidate
+        unsigned gt = 0u;
+#pragma unroll
+        for (int u = 0; u < kU; ++u)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const unsigned key = key_of(x[u][k]);
+                const unsigned top = key >> 20;
+                const bool in = (fin >> (4 * u + k)) & 1u;
+                gt += (in && top > P0) ? 1u : 0u;
+                if (in && top == P0) {
+                    mine |= 1u << (4 * u + k);
+                    atomicAdd(&s_hist[(key >> 9) & (kBins - 1)], 1u);
+                }
+            }
+        // sure keys of the chunk; list positions of the warp's candidates (one shared atomic per warp)
+        const unsigned packed = warp_inclusive_scan32(gt | ((unsigned)__popc(mine) << 16), lane);
+        const unsigned wtot = __shfl_sync(kFull, packed, 31);
+        unsigned wbase = 0u;
+        if (lane == 31) {
+            s_gt[par][warp] = wtot & 0xffffu;
+            if (compact && (wtot >> 16)) wbase = atomicAdd(&s_cnt[par], wtot >> 16);
+        }
+        wbase = __shfl_sync(kFull, wbase, 31);
+        if (compact && mine) {
+            unsigned pos = wbase + (packed >> 16) - (unsigned)__popc(mine);
+#pragma unroll
+            for (int u = 0; u < kU; ++u)
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if ((mine >> (4 * u + k)) & 1u) s_list[par][pos++] = key_of(x[u][k]);
+        }
+        __syncthreads();                       // list and counts of chunk c are complete
+        unsigned long long base = 0ull;
+        unsigned cnt = 0u;
+        if (threadIdx.x == 0) {
+            cnt = s_cnt[par];
+            if (cnt) base = atomicAdd(&st->cursor, (unsigned long long)cnt);     // in flight ...
+        }
+        const long long next = c + gridDim.x;
+        if (next < chunks) load_chunk_keys(v, n, next, warp, lane, x, fin);      // ... with the next chunk's loads
+        if (threadIdx.x == 0) {
+            unsigned a = 0;
+            for (int w = 0; w < kWarps; ++w) a += s_gt[par][w];
+            cgt[c] = a;
+            seg_cnt[c] = cnt;
+            seg_start[c] = base;
+            s_base = base;
+            s_cnt[par ^ 1] = 0u;               // its last readers passed the barrier above
+        }
+        __syncthreads();
+        cnt = s_cnt[par];
+        base = s_base;
+        for (unsigned i = threadIdx.x; i < cnt; i += kThreads) cand[base + i] = s_list[par][i];
+        // s_base and list `par` are next written after the next chunk's first barrier
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < kBins; b += kThreads)
+        if (s_hist[b]) atomicAdd(&hist[b], (unsigned long long)s_hist[b]);
+}
+
+// ---- 1b, third digit: histogram over the candidate list (ends at once in the fallback).
+__global__ void __launch_bounds__(kThreads) ef_topk_hist_list_kernel(const unsigned* __restrict__ cand,
+                                                                     const TopkState* __restrict__ st,
+                                                                     unsigned long long* __restrict__ hist) {
+    __shared__ unsigned s_hist[1 << pass_bits(2)];
+    if (!st->compact) return;
+    for (int b = threadIdx.x; b < (1 << pass_bits(2)); b += kThreads) s_hist[b] = 0u;
+    __syncthreads();
+    const unsigned long long ncand = st->ncand;
+    const unsigned prefix = st->prefix;            // 22 bits
+    for (unsigned long long i = (unsigned long long)blockIdx.x * kThreads + threadIdx.x; i < ncand;
+         i += (unsigned long long)gridDim.x * kThreads) {
+        const unsigned key = cand[i];
+        if ((key >> pass_bits(2)) == prefix) atomicAdd(&s_hist[key & ((1u << pass_bits(2)) - 1u)], 1u);
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < (1 << pass_bits(2)); b += kThreads)
+        if (s_hist[b]) atomicAdd(&hist[b], (unsigned long long)s_hist[b]);
+}
+
 // One CTA fixes the next digit: it finds, from the largest digit down, the bin in which the
 // count of keys seen so far reaches `remaining`.  Thread t adds up bins 8t .. 8t+7; thread 0
 // walks the 256 sums from the top and then the eight bins of the group it stops in.
 template <int PASS>
 __global__ void __launch_bounds__(kThreads) ef_topk_select_kernel(const unsigned long long* __restrict__ hist,
-                                                                  TopkState* st, unsigned long long k) {
+                                                                  TopkState* st, unsigned long long k,
+                                                                  unsigned long long cap) {
     constexpr int bits = pass_bits(PASS), nbins = 1 << bits, per = kBins / kThreads;
     __shared__ unsigned long long s_bin[kBins], s_grp[kThreads];
     unsigned long long g = 0;
@@ -145,49 +312,100 @@ __global__ void __launch_bounds__(kThreads) ef_topk_select_kernel(const unsigned
     remaining -= above;                       // still to keep among the keys of bin b
     st->prefix = (prefix << bits) | (unsigned)b;
     st->remaining = remaining;
+    if (PASS == 0) {
+        st->ncand = s_bin[b];
+        st->compact = s_bin[b] <= cap ? 1u : 0u;
+    }
     if (PASS == kPasses - 1) {
         st->threshold = st->prefix;
         st->need_eq = remaining;
     }
 }
 
-// ---- 2. per chunk: how many keys are > T and == T
-__global__ void __launch_bounds__(kThreads) ef_topk_count_kernel(const float* __restrict__ v, long long n,
-                                                                 const TopkState* __restrict__ st,
-                                                                 unsigned* __restrict__ cgt,
-                                                                 unsigned* __restrict__ ceq) {
-    __shared__ unsigned s_gt[kWarps], s_eq[kWarps];
+// ---- 2. per chunk: how many keys are > T and == T.  From the list: one warp per chunk adds
+// the chunk's candidates above T to its sure count.
+__global__ void __launch_bounds__(kThreads) ef_topk_count_list_kernel(const unsigned* __restrict__ cand,
+                                                                      const TopkState* __restrict__ st,
+                                                                      const unsigned long long* __restrict__ seg_start,
+                                                                      const unsigned* __restrict__ seg_cnt,
+                                                                      long long chunks,
+                                                                      unsigned* __restrict__ cgt,
+                                                                      unsigned* __restrict__ ceq,
+                                                                      unsigned* __restrict__ tgt,
+                                                                      unsigned* __restrict__ teq) {
+    if (!st->compact) return;
     const unsigned T = st->threshold;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    unsigned gt = 0, eq = 0;
-#pragma unroll
-    for (int u = 0; u < kU; ++u) {
-        const long long base = (long long)blockIdx.x * kChunkLen + warp * (128 * kU) + u * 128 + lane * 4;
-        if (base >= n) continue;
-        float x[4]; bool in[4];
-        load_keys(v, base, n, x, in);
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const unsigned key = key_of(x[k]);
-            gt += (in[k] && key > T) ? 1u : 0u;
-            eq += (in[k] && key == T) ? 1u : 0u;
-        }
+    const long long c = (long long)blockIdx.x * kWarps + warp;
+    if (c >= chunks) return;
+    const unsigned cnt = seg_cnt[c];
+    const unsigned* seg = cand + seg_start[c];
+    unsigned both = 0u;                       // at most 4096 each: two 16-bit fields
+    for (unsigned i = lane; i < cnt; i += 32) {
+        const unsigned key = seg[i];
+        both += (key > T ? 1u : 0u) + (key == T ? 1u << 16 : 0u);
     }
-    unsigned both = gt | (eq << 16);          // at most 512 elements per warp each: two 16-bit fields
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) both += __shfl_xor_sync(kFull, both, o);
-    if (lane == 0) { s_gt[warp] = both & 0xffffu; s_eq[warp] = both >> 16; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        unsigned a = 0, b = 0;
-        for (int w = 0; w < kWarps; ++w) { a += s_gt[w]; b += s_eq[w]; }
-        cgt[blockIdx.x] = a;
-        ceq[blockIdx.x] = b;
+    if (lane == 0) {
+        const unsigned gt = cgt[c] + (both & 0xffffu), eq = both >> 16;
+        cgt[c] = gt;
+        ceq[c] = eq;
+        if (gt) atomicAdd(&tgt[c / kTileOfChunks], gt);      // totals of the tile, for the scan
+        if (eq) atomicAdd(&teq[c / kTileOfChunks], eq);
     }
 }
 
-// ---- 3. exclusive prefix sums of the two count arrays over the chunks (one CTA)
+// Fallback: the same counts from v itself (ends at once when the list was used).
+__global__ void __launch_bounds__(kThreads) ef_topk_count_kernel(const float* __restrict__ v, long long n,
+                                                                 long long chunks,
+                                                                 const TopkState* __restrict__ st,
+                                                                 unsigned* __restrict__ cgt,
+                                                                 unsigned* __restrict__ ceq,
+                                                                 unsigned* __restrict__ tgt,
+                                                                 unsigned* __restrict__ teq) {
+    __shared__ unsigned s_gt[kWarps], s_eq[kWarps];
+    if (st->compact) return;
+    const unsigned T = st->threshold;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (long long c = blockIdx.x; c < chunks; c += gridDim.x) {
+        unsigned gt = 0, eq = 0;
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const long long base = c * kChunkLen + warp * (128 * kU) + u * 128 + lane * 4;
+            if (base >= n) continue;
+            float x[4]; bool in[4];
+            load_keys(v, base, n, x, in);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const unsigned key = key_of(x[k]);
+                gt += (in[k] && key > T) ? 1u : 0u;
+                eq += (in[k] && key == T) ? 1u : 0u;
+            }
+        }
+        unsigned both = gt | (eq << 16);      // at most 512 elements per warp each: two 16-bit fields
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) both += __shfl_xor_sync(kFull, both, o);
+        if (lane == 0) { s_gt[warp] = both & 0xffffu; s_eq[warp] = both >> 16; }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            unsigned a = 0, b = 0;
+            for (int w = 0; w < kWarps; ++w) { a += s_gt[w]; b += s_eq[w]; }
+            cgt[c] = a;
+            ceq[c] = b;
+            if (a) atomicAdd(&tgt[c / kTileOfChunks], a);
+            if (b) atomicAdd(&teq[c / kTileOfChunks], b);
+        }
+        __syncthreads();
+    }
+}
+
+// ---- 3. exclusive prefix sums of the two per-tile count arrays (a tile is kTileOfChunks chunks;
+// one CTA).  The CTA walks the arrays in pieces of kScanThreads * kScanPer entries: every thread takes kScanPer
+// consecutive entries, the threads' totals are scanned over the CTA (warps, then the warps'
+// totals), and the piece's total is carried to the next piece.
 constexpr int kScanThreads = 1024;
+constexpr int kScanPer = 8;
 __device__ __forceinline__ unsigned long long warp_inclusive_scan(unsigned long long v, int lane) {
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -202,111 +420,175 @@ __global__ void __launch_bounds__(kScanThreads) ef_topk_scan_kernel(const unsign
                                                                     unsigned long long* __restrict__ peq,
                                                                     long long chunks) {
     __shared__ unsigned long long s_a[32], s_b[32];
+    __shared__ unsigned long long s_carry[2];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const long long per = (chunks + kScanThreads - 1) / kScanThreads;
-    const long long lo = min(chunks, (long long)threadIdx.x * per), hi = min(chunks, lo + per);
-    unsigned long long a = 0, b = 0;
-    for (long long c = lo; c < hi; ++c) { a += cgt[c]; b += ceq[c]; }
-    // exclusive scan of the per-thread totals over the CTA: warps, then the warps' totals
-    const unsigned long long ia = warp_inclusive_scan(a, lane), ib = warp_inclusive_scan(b, lane);
-    if (lane == 31) { s_a[warp] = ia; s_b[warp] = ib; }
+    if (threadIdx.x == 0) { s_carry[0] = 0ull; s_carry[1] = 0ull; }
     __syncthreads();
-    if (warp == 0) {
-        const unsigned long long wa = warp_inclusive_scan(s_a[lane], lane), wb = warp_inclusive_scan(s_b[lane], lane);
-        s_a[lane] = wa - s_a[lane];            // exclusive
-        s_b[lane] = wb - s_b[lane];
-    }
-    __syncthreads();
-    a = s_a[warp] + ia - a;
-    b = s_b[warp] + ib - b;
-    for (long long c = lo; c < hi; ++c) {
-        pgt[c] = a; peq[c] = b;
-        a += cgt[c]; b += ceq[c];
+    for (long long piece = 0; piece < chunks; piece += (long long)kScanThreads * kScanPer) {
+        const long long lo = piece + (long long)threadIdx.x * kScanPer;
+        unsigned ga[kScanPer], gb[kScanPer];
+        unsigned long long a = 0, b = 0;
+#pragma unroll
+        for (int j = 0; j < kScanPer; ++j) {
+            ga[j] = lo + j < chunks ? cgt[lo + j] : 0u;
+            gb[j] = lo + j < chunks ? ceq[lo + j] : 0u;
+            a += ga[j]; b += gb[j];
+        }
+        const unsigned long long ia = warp_inclusive_scan(a, lane), ib = warp_inclusive_scan(b, lane);
+        if (lane == 31) { s_a[warp] = ia; s_b[warp] = ib; }
+        __syncthreads();
+        if (warp == 0) {
+            const unsigned long long ta = s_a[lane], tb = s_b[lane];
+            const unsigned long long wa = warp_inclusive_scan(ta, lane), wb = warp_inclusive_scan(tb, lane);
+            s_a[lane] = wa - ta;               // exclusive
+            s_b[lane] = wb - tb;
+        }
+        __syncthreads();
+        a = s_carry[0] + s_a[warp] + ia - a;   // entries before this thread's first one
+        b = s_carry[1] + s_b[warp] + ib - b;
+#pragma unroll
+        for (int j = 0; j < kScanPer; ++j) {
+            if (lo + j < chunks) { pgt[lo + j] = a; peq[lo + j] = b; }
+            a += ga[j]; b += gb[j];
+        }
+        __syncthreads();                       // everyone has read the carry and the warp offsets
+        if (threadIdx.x == kScanThreads - 1) { s_carry[0] = a; s_carry[1] = b; }
+        __syncthreads();
     }
 }
 
 // ---- 4. scatter: kept = key > T, or key == T and fewer than need_eq equal keys precede it
-__global__ void __launch_bounds__(kThreads) ef_topk_scatter_kernel(const float* v, long long n,
-                                                                   const TopkState* __restrict__ st,
-                                                                   const unsigned long long* __restrict__ pgt,
-                                                                   const unsigned long long* __restrict__ peq,
-                                                                   long long* __restrict__ idx_out,
-                                                                   float* __restrict__ val_out,
-                                                                   float* resid, unsigned long long kmax) {
-    // resid may alias v: every thread has read its own elements before it writes them.
-    // element order inside a chunk: warp, then row, then lane, then the lane's four elements
-    __shared__ unsigned s_eq[kWarps], s_gt[kWarps];
-    const unsigned T = st->threshold;
-    const unsigned long long need_eq = st->need_eq;
+// element order inside a chunk: warp, then row, then lane, then the lane's four elements.
+// Ranks come from per-lane counts (0..4 per row, the four rows packed into one word of four
+// 8-bit fields: a row of a warp has at most 128 kept elements) and one shuffle scan per warp.
+// A CTA handles kScatterChunks consecutive chunks, the next chunk's loads in flight while the
+// current one is ranked and written; its first rank is the tile's prefix plus the counts of the
+// tile's chunks before it.
+struct ScatterArgs {
+    const float* v;
+    long long n, chunks;
+    const TopkState* st;
+    const unsigned* cgt;
+    const unsigned* ceq;
+    const unsigned long long* pgt;     // per tile
+    const unsigned long long* peq;
+    long long* idx_out;
+    float* val_out;
+    float* resid;                      // may alias v: every thread has read its own elements before it writes them
+    unsigned long long kmax;
+};
+
+__device__ __forceinline__ unsigned row_counts(unsigned f) {
+    return (unsigned)__popc(f & 0xfu) | ((unsigned)__popc(f & 0xf0u) << 8) |
+           ((unsigned)__popc(f & 0xf00u) << 16) | ((unsigned)__popc(f & 0xf000u) << 24);
+}
+__device__ __forceinline__ unsigned field_sum(unsigned t) {
+    return (t & 0xffu) + ((t >> 8) & 0xffu) + ((t >> 16) & 0xffu) + (t >> 24);
+}
+
+// One chunk, its elements in x/fin.  gt_run / eq_run: kept-candidate counts before the chunk
+// (advanced by the chunk's totals).  s_gt / s_eq: this chunk's buffer of per-warp totals.
+__device__ __forceinline__ void scatter_chunk(const ScatterArgs& a, long long c, unsigned T,
+                                              unsigned long long need_eq, const float (&x)[kU][4],
+                                              unsigned fin, unsigned* s_gt, unsigned* s_eq,
+                                              unsigned long long& gt_run, unsigned long long& eq_run) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const unsigned lt_mask = (1u << lane) - 1u;
-    float x[kU][4]; bool in[kU][4];
-    unsigned feq[kU], fgt[kU];                 // nibbles of flags
-    unsigned eq_lanes_before[kU], gt_lanes_before[kU], eq_row[kU], gt_row[kU];
-    unsigned weq = 0, wgt = 0;                 // this warp's totals
+    const long long cbase = c * kChunkLen + warp * (128 * kU) + lane * 4;
+    unsigned fgt = 0u, feq = 0u;               // bit 4u + k: key > T, key == T
 #pragma unroll
-    for (int u = 0; u < kU; ++u) {
-        const long long base = (long long)blockIdx.x * kChunkLen + warp * (128 * kU) + u * 128 + lane * 4;
-        feq[u] = fgt[u] = 0u;
-        if (base < n) {
-            load_keys(v, base, n, x[u], in[u]);
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const unsigned key = key_of(x[u][k]);
-                if (in[u][k] && key == T) feq[u] |= 1u << k;
-                if (in[u][k] && key > T) fgt[u] |= 1u << k;
-            }
-        } else {
-#pragma unroll
-            for (int k = 0; k < 4; ++k) { in[u][k] = false; x[u][k] = 0.f; }
-        }
-        // keys of this row before this lane, and in the whole row: one ballot per element position
-        eq_lanes_before[u] = gt_lanes_before[u] = eq_row[u] = gt_row[u] = 0u;
-        if (__any_sync(kFull, (feq[u] | fgt[u]) != 0u)) {      // most rows keep nothing
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const unsigned be = __ballot_sync(kFull, (feq[u] >> k) & 1u);
-                const unsigned bg = __ballot_sync(kFull, (fgt[u] >> k) & 1u);
-                eq_lanes_before[u] += __popc(be & lt_mask); eq_row[u] += __popc(be);
-                gt_lanes_before[u] += __popc(bg & lt_mask); gt_row[u] += __popc(bg);
-            }
-        }
-        weq += eq_row[u];
-        wgt += gt_row[u];
-    }
-    if (lane == 0) { s_eq[warp] = weq; s_gt[warp] = wgt; }
-    __syncthreads();
-    unsigned long long eq_before = peq[blockIdx.x], gt_before = pgt[blockIdx.x];
-    for (int w = 0; w < warp; ++w) { eq_before += s_eq[w]; gt_before += s_gt[w]; }
-#pragma unroll
-    for (int u = 0; u < kU; ++u) {
-        const long long base = (long long)blockIdx.x * kChunkLen + warp * (128 * kU) + u * 128 + lane * 4;
-        unsigned long long eq_rank = eq_before + eq_lanes_before[u];     // equal keys before element 0 of this lane
-        unsigned long long gt_rank = gt_before + gt_lanes_before[u];
-        float r[4];
+    for (int u = 0; u < kU; ++u)
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            const bool is_eq = (feq[u] >> k) & 1u, is_gt = (fgt[u] >> k) & 1u;
-            const bool kept = is_gt || (is_eq && eq_rank < need_eq);
-            if (kept) {
-                // kept elements before this one = (keys > T before it) + min(equal keys before it, need_eq)
-                const unsigned long long pos = gt_rank + (eq_rank < need_eq ? eq_rank : need_eq);
-                if (pos < kmax) {              // always true when the counts are consistent
-                    idx_out[pos] = base + k;
-                    val_out[pos] = x[u][k];
+            const unsigned key = key_of(x[u][k]);
+            fgt |= key > T ? 1u << (4 * u + k) : 0u;
+            feq |= key == T ? 1u << (4 * u + k) : 0u;
+        }
+    fgt &= fin; feq &= fin;
+    const unsigned cg = row_counts(fgt);
+    unsigned ig = 0u, ie = 0u, ce = 0u;        // inclusive scans over the lanes; lane 31 holds the rows' totals
+    if (__any_sync(kFull, fgt != 0u)) ig = warp_inclusive_scan32(cg, lane);
+    if (__any_sync(kFull, feq != 0u)) { ce = row_counts(feq); ie = warp_inclusive_scan32(ce, lane); }
+    const unsigned tg = __shfl_sync(kFull, ig, 31), te = __shfl_sync(kFull, ie, 31);
+    if (lane == 0) { s_gt[warp] = field_sum(tg); s_eq[warp] = field_sum(te); }
+    __syncthreads();
+    unsigned long long gt_before = gt_run, eq_before = eq_run;
+    unsigned all_gt = 0u, all_eq = 0u;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+        if (w < warp) { gt_before += s_gt[w]; eq_before += s_eq[w]; }
+        all_gt += s_gt[w]; all_eq += s_eq[w];
+    }
+    gt_run += all_gt; eq_run += all_eq;
+    const unsigned xg = ig - cg, xe = ie - ce; // exclusive: kept keys of the row in lower lanes
+    const bool any_kept = (fgt | feq) != 0u;
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+        const long long base = cbase + u * 128;
+        float r[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) r[k] = x[u][k];
+        if (any_kept) {
+            unsigned long long eq_rank = eq_before + ((xe >> (8 * u)) & 0xffu);   // equal keys before element 0 of this lane
+            unsigned long long gt_rank = gt_before + ((xg >> (8 * u)) & 0xffu);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const bool is_eq = (feq >> (4 * u + k)) & 1u, is_gt = (fgt >> (4 * u + k)) & 1u;
+                const bool kept = is_gt || (is_eq && eq_rank < need_eq);
+                if (kept) {
+                    // kept elements before this one = (keys > T before it) + min(equal keys before it, need_eq)
+                    const unsigned long long pos = gt_rank + (eq_rank < need_eq ? eq_rank : need_eq);
+                    if (pos < a.kmax) {        // always true when the counts are consistent
+                        a.idx_out[pos] = base + k;
+                        a.val_out[pos] = x[u][k];
+                    }
+                    r[k] = __fsub_rn(x[u][k], x[u][k]);      // e = v - C(v)
                 }
+                eq_rank += is_eq ? 1u : 0u;
+                gt_rank += is_gt ? 1u : 0u;
             }
-            r[k] = kept ? __fsub_rn(x[u][k], x[u][k]) : x[u][k];      // e = v - C(v)
-            eq_rank += is_eq ? 1u : 0u;
-            gt_rank += is_gt ? 1u : 0u;
         }
-        if (resid != nullptr && base < n) {
-            if (base + 4 <= n) efk::st_stream(resid + base, make_float4(r[0], r[1], r[2], r[3]));
+        if (a.resid != nullptr && base < a.n) {
+            if (base + 4 <= a.n) efk::st_stream(a.resid + base, make_float4(r[0], r[1], r[2], r[3]));
             else
-                for (int k = 0; k < 4; ++k) if (in[u][k]) resid[base + k] = r[k];
+                for (int k = 0; k < 4; ++k) if ((fin >> (4 * u + k)) & 1u) a.resid[base + k] = r[k];
         }
-        eq_before += eq_row[u];
-        gt_before += gt_row[u];
+        eq_before += (te >> (8 * u)) & 0xffu;
+        gt_before += (tg >> (8 * u)) & 0xffu;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 3) ef_topk_scatter_kernel(const ScatterArgs a) {
+    __shared__ unsigned s_eq[2][kWarps], s_gt[2][kWarps];
+    __shared__ unsigned long long s_first[2];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long c0 = (long long)blockIdx.x * kScatterChunks;
+    const int nch = (int)min((long long)kScatterChunks, a.chunks - c0);
+    float xA[kU][4], xB[kU][4];
+    unsigned finA, finB = 0u;
+    load_chunk_keys(a.v, a.n, c0, warp, lane, xA, finA);
+    // rank of the CTA's first element: the tile's prefix plus the tile's chunks before c0
+    if (warp == 0) {
+        const long long tile = c0 / kTileOfChunks, first = tile * kTileOfChunks;
+        unsigned g = first + lane < c0 ? a.cgt[first + lane] : 0u;
+        unsigned e = first + lane < c0 ? a.ceq[first + lane] : 0u;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            g += __shfl_xor_sync(kFull, g, o);
+            e += __shfl_xor_sync(kFull, e, o);
+        }
+        if (lane == 0) { s_first[0] = a.pgt[tile] + g; s_first[1] = a.peq[tile] + e; }
+    }
+    const unsigned T = a.st->threshold;
+    const unsigned long long need_eq = a.st->need_eq;
+    __syncthreads();
+    unsigned long long gt_run = s_first[0], eq_run = s_first[1];
+    for (int j = 0; j < nch; j += 2) {
+        if (j + 1 < nch) load_chunk_keys(a.v, a.n, c0 + j + 1, warp, lane, xB, finB);
+        scatter_chunk(a, c0 + j, T, need_eq, xA, finA, s_gt[0], s_eq[0], gt_run, eq_run);
+        if (j + 1 < nch) {
+            if (j + 2 < nch) load_chunk_keys(a.v, a.n, c0 + j + 2, warp, lane, xA, finA);
+            scatter_chunk(a, c0 + j + 1, T, need_eq, xB, finB, s_gt[1], s_eq[1], gt_run, eq_run);
+        }
     }
 }
 
@@ -337,23 +619,36 @@ int ef_topk_compress(const float* v, int64_t n, int64_t k, int64_t* idx_out, flo
     char* ws = (char*)workspace;
     unsigned long long* hist = (unsigned long long*)(ws + L.off_hist);
     TopkState* state = (TopkState*)(ws + L.off_state);
+    unsigned* tgt = (unsigned*)(ws + L.off_tgt);
+    unsigned* teq = (unsigned*)(ws + L.off_teq);
     unsigned* cgt = (unsigned*)(ws + L.off_cgt);
     unsigned* ceq = (unsigned*)(ws + L.off_ceq);
     unsigned long long* pgt = (unsigned long long*)(ws + L.off_pgt);
     unsigned long long* peq = (unsigned long long*)(ws + L.off_peq);
-    if (cudaMemsetAsync(ws, 0, L.off_cgt, st) != cudaSuccess) return EF_ERR_CUDA;   // histograms + state
+    unsigned long long* seg_start = (unsigned long long*)(ws + L.off_seg_start);
+    unsigned* seg_cnt = (unsigned*)(ws + L.off_seg_cnt);
+    unsigned* cand = (unsigned*)(ws + L.off_cand);
+    if (cudaMemsetAsync(ws, 0, L.off_cgt, st) != cudaSuccess) return EF_ERR_CUDA;   // histograms, state, tile totals
     const unsigned hgrid = (unsigned)std::min<long long>(L.chunks, 148 * 8);
+    const unsigned cgrid = (unsigned)std::min<long long>(L.chunks, 148 * 5);       // five CTAs of 41 KB per SM
+    const unsigned lgrid = (unsigned)std::min<unsigned long long>((L.cap + kThreads - 1) / kThreads, 148 * 8);
     const unsigned long long kk = (unsigned long long)k;
     ef_topk_hist_kernel<0><<<hgrid, kThreads, 0, st>>>(v, n, L.chunks, state, hist);
-    ef_topk_select_kernel<0><<<1, kThreads, 0, st>>>(hist, state, kk);
-    ef_topk_hist_kernel<1><<<hgrid, kThreads, 0, st>>>(v, n, L.chunks, state, hist + kBins);
-    ef_topk_select_kernel<1><<<1, kThreads, 0, st>>>(hist + kBins, state, kk);
-    ef_topk_hist_kernel<2><<<hgrid, kThreads, 0, st>>>(v, n, L.chunks, state, hist + 2 * kBins);
-    ef_topk_select_kernel<2><<<1, kThreads, 0, st>>>(hist + 2 * kBins, state, kk);
-    ef_topk_count_kernel<<<(unsigned)L.chunks, kThreads, 0, st>>>(v, n, state, cgt, ceq);
-    ef_topk_scan_kernel<<<1, kScanThreads, 0, st>>>(cgt, ceq, pgt, peq, L.chunks);
-    ef_topk_scatter_kernel<<<(unsigned)L.chunks, kThreads, 0, st>>>(v, n, state, pgt, peq,
-                                                                    (long long*)idx_out, val_out, resid_out, kk);
+    ef_topk_select_kernel<0><<<1, kThreads, 0, st>>>(hist, state, kk, L.cap);
+    ef_topk_candidates_kernel<<<cgrid, kThreads, 0, st>>>(v, n, L.chunks, state, hist + kBins, cgt,
+                                                          seg_start, seg_cnt, cand);
+    ef_topk_select_kernel<1><<<1, kThreads, 0, st>>>(hist + kBins, state, kk, L.cap);
+    ef_topk_hist_list_kernel<<<lgrid, kThreads, 0, st>>>(cand, state, hist + 2 * kBins);     // list ...
+    ef_topk_hist_kernel<2><<<hgrid, kThreads, 0, st>>>(v, n, L.chunks, state, hist + 2 * kBins);   // ... or v
+    ef_topk_select_kernel<2><<<1, kThreads, 0, st>>>(hist + 2 * kBins, state, kk, L.cap);
+    ef_topk_count_list_kernel<<<(unsigned)((L.chunks + kWarps - 1) / kWarps), kThreads, 0, st>>>(
+        cand, state, seg_start, seg_cnt, L.chunks, cgt, ceq, tgt, teq);
+    ef_topk_count_kernel<<<hgrid, kThreads, 0, st>>>(v, n, L.chunks, state, cgt, ceq, tgt, teq);
+    ef_topk_scan_kernel<<<1, kScanThreads, 0, st>>>(tgt, teq, pgt, peq, L.tiles);
+    ScatterArgs sa;
+    sa.v = v; sa.n = n; sa.chunks = L.chunks; sa.st = state; sa.cgt = cgt; sa.ceq = ceq; sa.pgt = pgt; sa.peq = peq;
+    sa.idx_out = (long long*)idx_out; sa.val_out = val_out; sa.resid = resid_out; sa.kmax = kk;
+    ef_topk_scatter_kernel<<<(unsigned)((L.chunks + kScatterChunks - 1) / kScatterChunks), kThreads, 0, st>>>(sa);
     return cudaGetLastError() == cudaSuccess ? EF_OK : EF_ERR_CUDA;
 }
 

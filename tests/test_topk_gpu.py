@@ -76,6 +76,37 @@ def test_large_vectors(n, k):
     check(v.cpu(), k)
 
 
+@pytest.mark.parametrize("law", ["one-bin", "constant", "two-levels", "narrow-then-wide"])
+def test_vectors_whose_candidates_do_not_fit_the_list(law):
+    """The keys that share the threshold's leading digit are normally a few per cent of the
+    vector and are copied to a list; here they are (nearly) all of it, more than the list holds,
+    and the later digits and the counts must come from the vector itself."""
+    n = 300_000 + 77
+    gen = torch.Generator().manual_seed(11)
+    if law == "one-bin":
+        v = (1.0 + torch.rand(n, generator=gen) * 0.05) * torch.where(torch.rand(n, generator=gen) < 0.5, -1.0, 1.0)
+    elif law == "constant":
+        v = torch.where(torch.rand(n, generator=gen) < 0.5, -2.5, 2.5)
+    elif law == "two-levels":
+        v = torch.where(torch.rand(n, generator=gen) < 0.3, 4.0, 1.0)          # k decides which level ties
+    else:
+        v = torch.randn(n, generator=gen)
+        v[: n // 2] = 3.0 + torch.rand(n // 2, generator=gen) * 1e-3
+    for k in (1, n // 1000, n // 10, n // 2 + 5, n - 1):
+        check(v, k)
+
+
+@pytest.mark.parametrize("n", [65536, 65537, 8 * 65536, 8 * 65536 + 8, 1_000_003])
+def test_sizes_around_the_list_capacity(n):
+    """The list holds max(n/8, min(n, 65536)) keys; vectors on both sides of the two break points,
+    ordinary values (the list is used) and all-equal magnitudes (it is not, beyond 65536)."""
+    gen = torch.Generator().manual_seed(n % 97)
+    v = torch.randn(n, generator=gen)
+    for k in (n // 100, n // 7):
+        check(v, k)
+    check(torch.full((n,), -0.75), n // 3)
+
+
 def test_arguments_are_checked():
     v = torch.zeros(64, device="cuda")
     idx = torch.zeros(64, dtype=torch.int64, device="cuda")
