@@ -30,6 +30,7 @@
 #include "ef_internal.h"
 
 #include <algorithm>
+#include <type_traits>
 
 namespace {
 
@@ -149,6 +150,47 @@ __global__ void __launch_bounds__(kThreads) ef_topk_hist_kernel(const float* __r
         if (s_hist[b]) atomicAdd(&hist[b], (unsigned long long)s_hist[b]);
 }
 
+// ---- Both passes below are bound by instruction issue, not by memory, if every element is
+// classified by its own lane: only a few per cent of the elements matter (keys at or above the
+// threshold bin resp. the threshold), but nearly every warp instruction of a per-element test
+// has some lane that needs it.  So a lane first tests its four elements of a row together (the
+// largest of the four keys against the bound), and the lanes whose row holds such a key copy the
+// row to a staging area of their warp, packed densely in index order (ballot + population
+// count).  The warp then classifies the staged rows, one row per lane: a handful of dense
+// iterations instead of sixteen sparse ones.
+struct WarpStage {
+    uint4 row[128];                 // raw bits of the four elements of a staged lane-row
+    unsigned short tag[128];        // (in-range nibble << 8) | (row u << 5) | lane
+};
+
+// Stages the lane-rows of this warp's part of a chunk whose largest key is >= lo (and that lie
+// inside the vector).  Returns the number of staged rows (the same in every lane).
+// FULL: the chunk lies wholly inside the vector (every chunk but the last): no range tests.
+template <bool FULL>
+__device__ __forceinline__ int stage_rows(const float (&x)[kU][4], unsigned fin, unsigned lo,
+                                          WarpStage& st, int lane) {
+    const unsigned lt_mask = (1u << lane) - 1u;
+    int H = 0;
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+        const unsigned b0 = __float_as_uint(x[u][0]), b1 = __float_as_uint(x[u][1]),
+                       b2 = __float_as_uint(x[u][2]), b3 = __float_as_uint(x[u][3]);
+        const unsigned m = max(__vimax3_u32(b0 & 0x7fffffffu, b1 & 0x7fffffffu, b2 & 0x7fffffffu),
+                               b3 & 0x7fffffffu);
+        const unsigned nib = FULL ? 0xfu : (fin >> (4 * u)) & 0xfu;
+        const bool hit = m >= lo && nib != 0u;
+        const unsigned ballot = __ballot_sync(kFull, hit);
+        if (hit) {
+            const int e = H + __popc(ballot & lt_mask);
+            st.row[e] = make_uint4(b0, b1, b2, b3);
+            st.tag[e] = (unsigned short)((nib << 8) | (u << 5) | lane);
+        }
+        H += __popc(ballot);
+    }
+    __syncwarp();
+    return H;
+}
+
 // ---- 1b. second pass over v.  Per chunk: histogram of the second digit of the candidates (keys
 // whose first digit is P0), the number of sure keys (first digit > P0) into cgt, and -- if the
 // candidates fit the list -- the candidates' keys as one segment of the list.
@@ -157,6 +199,16 @@ __global__ void __launch_bounds__(kThreads) ef_topk_hist_kernel(const float* __r
 // shared-memory lists used in turn, so that a chunk costs two barriers.
 __device__ __forceinline__ void load_chunk_keys(const float* __restrict__ v, long long n, long long c,
                                                 int warp, int lane, float (&x)[kU][4], unsigned& fin) {
+    if ((c + 1) * kChunkLen <= n) {            // the whole chunk is inside the vector
+        const float* p = v + c * kChunkLen + warp * (128 * kU) + lane * 4;
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const float4 q = efk::ld_stream(p + u * 128);
+            x[u][0] = q.x; x[u][1] = q.y; x[u][2] = q.z; x[u][3] = q.w;
+        }
+        fin = 0xffffu;
+        return;
+    }
     fin = 0u;
 #pragma unroll
     for (int u = 0; u < kU; ++u) {
@@ -179,54 +231,73 @@ __global__ void __launch_bounds__(kThreads) ef_topk_candidates_kernel(const floa
                                                                       unsigned long long* __restrict__ seg_start,
                                                                       unsigned* __restrict__ seg_cnt,
                                                                       unsigned* __restrict__ cand) {
+    extern __shared__ __align__(16) unsigned char s_dyn[];
+    // dynamic: [two lists of kChunkLen keys][one staging area per warp]
+    unsigned (*s_list)[kChunkLen] = reinterpret_cast<unsigned (*)[kChunkLen]>(s_dyn);
+    WarpStage* s_stage = reinterpret_cast<WarpStage*>(s_dyn + 2 * kChunkLen * sizeof(unsigned));
     __shared__ unsigned s_hist[kBins];
-    __shared__ unsigned s_list[2][kChunkLen];
     __shared__ unsigned s_gt[2][kWarps];
     __shared__ unsigned s_cnt[2];
     __shared__ unsigned long long s_base;
     for (int b = threadIdx.x; b < kBins; b += kThreads) s_hist[b] = 0u;
     if (threadIdx.x == 0) { s_cnt[0] = 0u; s_cnt[1] = 0u; }
     const unsigned P0 = st->prefix;
+    const unsigned lo = P0 << 20, hi_top = P0 + 1u;       // candidates: lo <= key and (key >> 20) < hi_top
     const bool compact = st->compact != 0u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    WarpStage& stage = s_stage[warp];
     float x[kU][4];
     unsigned fin;
     if (blockIdx.x < chunks) load_chunk_keys(v, n, blockIdx.x, warp, lane, x, fin);
     __syncthreads();
     int par = 0;
-    for (long long c = blockIdx.x; c < chunks; c += gridDim.x, par ^= 1) {
-        unsigned mine = 0u;                    // bit 4u + k: element is a candidate
+    // the staged rows of one chunk: second-digit histogram, candidates to list `par`, sure keys counted
+    auto classify = [&](auto full_c) -> unsigned {
+        constexpr bool FULL = decltype(full_c)::value;
+        const int H = stage_rows<FULL>(x, fin, lo, stage, lane);
         unsigned gt = 0u;
+        for (int e0 = 0; e0 < H; e0 += 32) {
+            const int e = e0 + lane;
+            unsigned keys[4] = {0u, 0u, 0u, 0u};
+            unsigned mine = 0u;                // bit k: element k of the staged row is a candidate
+            if (e < H) {
+                const uint4 q = stage.row[e];
+                const unsigned nib = FULL ? 0xfu : stage.tag[e] >> 8;
+                keys[0] = q.x & 0x7fffffffu; keys[1] = q.y & 0x7fffffffu;
+                keys[2] = q.z & 0x7fffffffu; keys[3] = q.w & 0x7fffffffu;
 #pragma unroll
-        for (int u = 0; u < kU; ++u)
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const unsigned key = key_of(x[u][k]);
-                const unsigned top = key >> 20;
-                const bool in = (fin >> (4 * u + k)) & 1u;
-                gt += (in && top > P0) ? 1u : 0u;
-                if (in && top == P0) {
-                    mine |= 1u << (4 * u + k);
-                    atomicAdd(&s_hist[(key >> 9) & (kBins - 1)], 1u);
+                for (int k = 0; k < 4; ++k) {
+                    const bool in = (nib >> k) & 1u;
+                    const unsigned top = keys[k] >> 20;
+                    gt += (in && top >= hi_top) ? 1u : 0u;
+                    if (in && top == P0) {
+                        mine |= 1u << k;
+                        atomicAdd(&s_hist[(keys[k] >> 9) & (kBins - 1)], 1u);
+                    }
                 }
             }
-        // sure keys of the chunk; list positions of the warp's candidates (one shared atomic per warp)
-        const unsigned packed = warp_inclusive_scan32(gt | ((unsigned)__popc(mine) << 16), lane);
-        const unsigned wtot = __shfl_sync(kFull, packed, 31);
-        unsigned wbase = 0u;
-        if (lane == 31) {
-            s_gt[par][warp] = wtot & 0xffffu;
-            if (compact && (wtot >> 16)) wbase = atomicAdd(&s_cnt[par], wtot >> 16);
-        }
-        wbase = __shfl_sync(kFull, wbase, 31);
-        if (compact && mine) {
-            unsigned pos = wbase + (packed >> 16) - (unsigned)__popc(mine);
-#pragma unroll
-            for (int u = 0; u < kU; ++u)
+            if (compact && __any_sync(kFull, mine != 0u)) {
+                // list positions of the warp's candidates: one shared atomic per dense iteration
+                const unsigned cnt = (unsigned)__popc(mine);
+                const unsigned incl = warp_inclusive_scan32(cnt, lane);
+                unsigned wbase = 0u;
+                if (lane == 31) wbase = atomicAdd(&s_cnt[par], incl);
+                wbase = __shfl_sync(kFull, wbase, 31);
+                unsigned pos = wbase + incl - cnt;
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
-                    if ((mine >> (4 * u + k)) & 1u) s_list[par][pos++] = key_of(x[u][k]);
+                    if ((mine >> k) & 1u) s_list[par][pos++] = keys[k];
+            }
         }
+        return gt;
+    };
+    for (long long c = blockIdx.x; c < chunks; c += gridDim.x, par ^= 1) {
+        // the choice must be the same in every thread of the CTA (the paths hold warp-wide operations):
+        // it is made on the chunk, not on the thread's own range flags
+        unsigned gt = (c + 1) * kChunkLen <= n ? classify(std::true_type{}) : classify(std::false_type{});
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) gt += __shfl_xor_sync(kFull, gt, o);
+        if (lane == 0) s_gt[par][warp] = gt;
         __syncthreads();                       // list and counts of chunk c are complete
         unsigned long long base = 0ull;
         unsigned cnt = 0u;
@@ -255,6 +326,7 @@ __global__ void __launch_bounds__(kThreads) ef_topk_candidates_kernel(const floa
     for (int b = threadIdx.x; b < kBins; b += kThreads)
         if (s_hist[b]) atomicAdd(&hist[b], (unsigned long long)s_hist[b]);
 }
+constexpr size_t kCandidatesSmem = 2 * kChunkLen * sizeof(unsigned) + kWarps * sizeof(WarpStage);
 
 // ---- 1b, third digit: histogram over the candidate list (ends at once in the fallback).
 __global__ void __launch_bounds__(kThreads) ef_topk_hist_list_kernel(const unsigned* __restrict__ cand,
@@ -478,38 +550,50 @@ struct ScatterArgs {
     unsigned long long kmax;
 };
 
-__device__ __forceinline__ unsigned row_counts(unsigned f) {
-    return (unsigned)__popc(f & 0xfu) | ((unsigned)__popc(f & 0xf0u) << 8) |
-           ((unsigned)__popc(f & 0xf00u) << 16) | ((unsigned)__popc(f & 0xf000u) << 24);
-}
-__device__ __forceinline__ unsigned field_sum(unsigned t) {
-    return (t & 0xffu) + ((t >> 8) & 0xffu) + ((t >> 16) & 0xffu) + (t >> 24);
-}
-
 // One chunk, its elements in x/fin.  gt_run / eq_run: kept-candidate counts before the chunk
 // (advanced by the chunk's totals).  s_gt / s_eq: this chunk's buffer of per-warp totals.
+// Lane-rows without a key >= T keep nothing: their residual is the input, stored at once.  The
+// others are staged and handled densely: a first sweep counts, the CTA's warps exchange their
+// totals, a second sweep ranks, writes idx/val and stores the staged rows' residual.
+template <bool FULL>
 __device__ __forceinline__ void scatter_chunk(const ScatterArgs& a, long long c, unsigned T,
                                               unsigned long long need_eq, const float (&x)[kU][4],
-                                              unsigned fin, unsigned* s_gt, unsigned* s_eq,
+                                              unsigned fin, WarpStage& stage, unsigned* s_gt, unsigned* s_eq,
                                               unsigned long long& gt_run, unsigned long long& eq_run) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long cbase = c * kChunkLen + warp * (128 * kU) + lane * 4;
-    unsigned fgt = 0u, feq = 0u;               // bit 4u + k: key > T, key == T
+    const long long wbase = c * kChunkLen + warp * (128 * kU);
+    const int H = stage_rows<FULL>(x, fin, T, stage, lane);
+    // residual of the rows that keep nothing (a staged row is recognised by its largest key again)
+    if (a.resid != nullptr) {
 #pragma unroll
-    for (int u = 0; u < kU; ++u)
+        for (int u = 0; u < kU; ++u) {
+            const long long base = wbase + u * 128 + lane * 4;
+            const unsigned nib = FULL ? 0xfu : (fin >> (4 * u)) & 0xfu;
+            const unsigned m = max(__vimax3_u32(__float_as_uint(x[u][0]) & 0x7fffffffu,
+                                                __float_as_uint(x[u][1]) & 0x7fffffffu,
+                                                __float_as_uint(x[u][2]) & 0x7fffffffu),
+                                   __float_as_uint(x[u][3]) & 0x7fffffffu);
+            if (m >= T || nib == 0u) continue;
+            if (nib == 0xfu) efk::st_stream(a.resid + base, make_float4(x[u][0], x[u][1], x[u][2], x[u][3]));
+            else
+                for (int k = 0; k < 4; ++k) if ((nib >> k) & 1u) a.resid[base + k] = x[u][k];
+        }
+    }
+    // first sweep: this warp's numbers of keys > T and == T
+    unsigned both = 0u;                        // two 16-bit fields (at most 512 each)
+    for (int e = lane; e < H; e += 32) {
+        const uint4 q = stage.row[e];
+        const unsigned nib = FULL ? 0xfu : stage.tag[e] >> 8;
+        const unsigned key[4] = {q.x & 0x7fffffffu, q.y & 0x7fffffffu, q.z & 0x7fffffffu, q.w & 0x7fffffffu};
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            const unsigned key = key_of(x[u][k]);
-            fgt |= key > T ? 1u << (4 * u + k) : 0u;
-            feq |= key == T ? 1u << (4 * u + k) : 0u;
+            const bool in = (nib >> k) & 1u;
+            both += (in && key[k] > T ? 1u : 0u) + (in && key[k] == T ? 1u << 16 : 0u);
         }
-    fgt &= fin; feq &= fin;
-    const unsigned cg = row_counts(fgt);
-    unsigned ig = 0u, ie = 0u, ce = 0u;        // inclusive scans over the lanes; lane 31 holds the rows' totals
-    if (__any_sync(kFull, fgt != 0u)) ig = warp_inclusive_scan32(cg, lane);
-    if (__any_sync(kFull, feq != 0u)) { ce = row_counts(feq); ie = warp_inclusive_scan32(ce, lane); }
-    const unsigned tg = __shfl_sync(kFull, ig, 31), te = __shfl_sync(kFull, ie, 31);
-    if (lane == 0) { s_gt[warp] = field_sum(tg); s_eq[warp] = field_sum(te); }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) both += __shfl_xor_sync(kFull, both, o);
+    if (lane == 0) { s_gt[warp] = both & 0xffffu; s_eq[warp] = both >> 16; }
     __syncthreads();
     unsigned long long gt_before = gt_run, eq_before = eq_run;
     unsigned all_gt = 0u, all_eq = 0u;
@@ -519,47 +603,63 @@ __device__ __forceinline__ void scatter_chunk(const ScatterArgs& a, long long c,
         all_gt += s_gt[w]; all_eq += s_eq[w];
     }
     gt_run += all_gt; eq_run += all_eq;
-    const unsigned xg = ig - cg, xe = ie - ce; // exclusive: kept keys of the row in lower lanes
-    const bool any_kept = (fgt | feq) != 0u;
-#pragma unroll
-    for (int u = 0; u < kU; ++u) {
-        const long long base = cbase + u * 128;
-        float r[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) r[k] = x[u][k];
-        if (any_kept) {
-            unsigned long long eq_rank = eq_before + ((xe >> (8 * u)) & 0xffu);   // equal keys before element 0 of this lane
-            unsigned long long gt_rank = gt_before + ((xg >> (8 * u)) & 0xffu);
+    // second sweep: staged rows are in index order, so ranks are running counts
+    for (int e0 = 0; e0 < H; e0 += 32) {
+        const int e = e0 + lane;
+        uint4 q = make_uint4(0u, 0u, 0u, 0u);
+        unsigned tag = 0u, fgt = 0u, feq = 0u;
+        if (e < H) {
+            q = stage.row[e];
+            tag = stage.tag[e];
+            const unsigned key[4] = {q.x & 0x7fffffffu, q.y & 0x7fffffffu, q.z & 0x7fffffffu, q.w & 0x7fffffffu};
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const bool is_eq = (feq >> (4 * u + k)) & 1u, is_gt = (fgt >> (4 * u + k)) & 1u;
+                fgt |= key[k] > T ? 1u << k : 0u;
+                feq |= key[k] == T ? 1u << k : 0u;
+            }
+            if (!FULL) { fgt &= tag >> 8; feq &= tag >> 8; }
+        }
+        const unsigned cnt = (unsigned)__popc(fgt) | ((unsigned)__popc(feq) << 16);
+        const unsigned incl = warp_inclusive_scan32(cnt, lane);
+        const unsigned tot = __shfl_sync(kFull, incl, 31);
+        if (e < H) {
+            unsigned long long gt_rank = gt_before + ((incl - cnt) & 0xffffu);
+            unsigned long long eq_rank = eq_before + ((incl - cnt) >> 16);
+            const long long base = wbase + ((tag >> 5) & 3u) * 128 + (tag & 31u) * 4;
+            const float xv[4] = {__uint_as_float(q.x), __uint_as_float(q.y), __uint_as_float(q.z), __uint_as_float(q.w)};
+            float r[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const bool is_eq = (feq >> k) & 1u, is_gt = (fgt >> k) & 1u;
                 const bool kept = is_gt || (is_eq && eq_rank < need_eq);
                 if (kept) {
                     // kept elements before this one = (keys > T before it) + min(equal keys before it, need_eq)
                     const unsigned long long pos = gt_rank + (eq_rank < need_eq ? eq_rank : need_eq);
                     if (pos < a.kmax) {        // always true when the counts are consistent
                         a.idx_out[pos] = base + k;
-                        a.val_out[pos] = x[u][k];
+                        a.val_out[pos] = xv[k];
                     }
-                    r[k] = __fsub_rn(x[u][k], x[u][k]);      // e = v - C(v)
                 }
+                r[k] = kept ? __fsub_rn(xv[k], xv[k]) : xv[k];      // e = v - C(v)
                 eq_rank += is_eq ? 1u : 0u;
                 gt_rank += is_gt ? 1u : 0u;
             }
+            if (a.resid != nullptr) {
+                if (FULL || (tag >> 8) == 0xfu) efk::st_stream(a.resid + base, make_float4(r[0], r[1], r[2], r[3]));
+                else
+                    for (int k = 0; k < 4; ++k) if ((tag >> (8 + k)) & 1u) a.resid[base + k] = r[k];
+            }
         }
-        if (a.resid != nullptr && base < a.n) {
-            if (base + 4 <= a.n) efk::st_stream(a.resid + base, make_float4(r[0], r[1], r[2], r[3]));
-            else
-                for (int k = 0; k < 4; ++k) if ((fin >> (4 * u + k)) & 1u) a.resid[base + k] = r[k];
-        }
-        eq_before += (te >> (8 * u)) & 0xffu;
-        gt_before += (tg >> (8 * u)) & 0xffu;
+        gt_before += tot & 0xffffu;
+        eq_before += tot >> 16;
     }
+    __syncwarp();                              // the staging area is rewritten by the next chunk
 }
 
 __global__ void __launch_bounds__(kThreads, 3) ef_topk_scatter_kernel(const ScatterArgs a) {
     __shared__ unsigned s_eq[2][kWarps], s_gt[2][kWarps];
     __shared__ unsigned long long s_first[2];
+    __shared__ WarpStage s_stage[kWarps];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long c0 = (long long)blockIdx.x * kScatterChunks;
     const int nch = (int)min((long long)kScatterChunks, a.chunks - c0);
@@ -584,10 +684,13 @@ __global__ void __launch_bounds__(kThreads, 3) ef_topk_scatter_kernel(const Scat
     unsigned long long gt_run = s_first[0], eq_run = s_first[1];
     for (int j = 0; j < nch; j += 2) {
         if (j + 1 < nch) load_chunk_keys(a.v, a.n, c0 + j + 1, warp, lane, xB, finB);
-        scatter_chunk(a, c0 + j, T, need_eq, xA, finA, s_gt[0], s_eq[0], gt_run, eq_run);
+        // whole chunk or not: decided on the chunk, identically in every thread (the paths hold barriers)
+        if ((c0 + j + 1) * kChunkLen <= a.n) scatter_chunk<true>(a, c0 + j, T, need_eq, xA, finA, s_stage[warp], s_gt[0], s_eq[0], gt_run, eq_run);
+        else scatter_chunk<false>(a, c0 + j, T, need_eq, xA, finA, s_stage[warp], s_gt[0], s_eq[0], gt_run, eq_run);
         if (j + 1 < nch) {
             if (j + 2 < nch) load_chunk_keys(a.v, a.n, c0 + j + 2, warp, lane, xA, finA);
-            scatter_chunk(a, c0 + j + 1, T, need_eq, xB, finB, s_gt[1], s_eq[1], gt_run, eq_run);
+            if ((c0 + j + 2) * kChunkLen <= a.n) scatter_chunk<true>(a, c0 + j + 1, T, need_eq, xB, finB, s_stage[warp], s_gt[1], s_eq[1], gt_run, eq_run);
+            else scatter_chunk<false>(a, c0 + j + 1, T, need_eq, xB, finB, s_stage[warp], s_gt[1], s_eq[1], gt_run, eq_run);
         }
     }
 }
@@ -615,6 +718,17 @@ int ef_topk_compress(const float* v, int64_t n, int64_t k, int64_t* idx_out, flo
         cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
         return EF_ERR_CUDA;
     if (major != 10) return EF_ERR_UNSUPPORTED_DEVICE;
+    {
+        // the candidates kernel needs more dynamic shared memory than the default limit: once per device
+        static bool raised[64] = {};
+        if (dev < 0 || dev >= 64) return EF_ERR_UNSUPPORTED_DEVICE;
+        if (!raised[dev]) {
+            if (cudaFuncSetAttribute(ef_topk_candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)kCandidatesSmem) != cudaSuccess)
+                return EF_ERR_CUDA;
+            raised[dev] = true;
+        }
+    }
     cudaStream_t st = (cudaStream_t)cuda_stream;
     char* ws = (char*)workspace;
     unsigned long long* hist = (unsigned long long*)(ws + L.off_hist);
@@ -630,13 +744,13 @@ int ef_topk_compress(const float* v, int64_t n, int64_t k, int64_t* idx_out, flo
     unsigned* cand = (unsigned*)(ws + L.off_cand);
     if (cudaMemsetAsync(ws, 0, L.off_cgt, st) != cudaSuccess) return EF_ERR_CUDA;   // histograms, state, tile totals
     const unsigned hgrid = (unsigned)std::min<long long>(L.chunks, 148 * 8);
-    const unsigned cgrid = (unsigned)std::min<long long>(L.chunks, 148 * 5);       // five CTAs of 41 KB per SM
+    const unsigned cgrid = (unsigned)std::min<long long>(L.chunks, 148 * 3);       // three CTAs of 59 KB per SM
     const unsigned lgrid = (unsigned)std::min<unsigned long long>((L.cap + kThreads - 1) / kThreads, 148 * 8);
     const unsigned long long kk = (unsigned long long)k;
     ef_topk_hist_kernel<0><<<hgrid, kThreads, 0, st>>>(v, n, L.chunks, state, hist);
     ef_topk_select_kernel<0><<<1, kThreads, 0, st>>>(hist, state, kk, L.cap);
-    ef_topk_candidates_kernel<<<cgrid, kThreads, 0, st>>>(v, n, L.chunks, state, hist + kBins, cgt,
-                                                          seg_start, seg_cnt, cand);
+    ef_topk_candidates_kernel<<<cgrid, kThreads, kCandidatesSmem, st>>>(v, n, L.chunks, state, hist + kBins,
+                                                                        cgt, seg_start, seg_cnt, cand);
     ef_topk_select_kernel<1><<<1, kThreads, 0, st>>>(hist + kBins, state, kk, L.cap);
     ef_topk_hist_list_kernel<<<lgrid, kThreads, 0, st>>>(cand, state, hist + 2 * kBins);     // list ...
     ef_topk_hist_kernel<2><<<hgrid, kThreads, 0, st>>>(v, n, L.chunks, state, hist + 2 * kBins);   // ... or v
