@@ -353,8 +353,9 @@ int ef_vote_server_step(ef_ctx* ctx);
  *                 v elsewhere); may alias v
  * Among equal magnitudes the lower index is kept (the paper does not say), +0 and -0 have the
  * same magnitude, NaN is unspecified.  workspace: device, 256-byte aligned, at least
- * ef_topk_workspace_bytes(n) bytes (histograms and per-chunk counts), owned by the caller and
- * overwritten by every call; calls that share a workspace must not overlap on the GPU.
+ * ef_topk_workspace_bytes(n) bytes (histograms, per-chunk counts and a list of candidate keys:
+ * about n/2 bytes), owned by the caller and overwritten by every call; calls that share a
+ * workspace must not overlap on the GPU.
  * Work is enqueued on cuda_stream without synchronisation; the library allocates nothing.
  * Errors: INVALID_ARG (n < 1, k outside [1, n], null), WORKSPACE, ALIGNMENT,
  * UNSUPPORTED_DEVICE, CUDA. */
