@@ -231,6 +231,10 @@ uint32_t* ef_status_word(ef_ctx* ctx);   /* the word itself (device, inside the 
 int ef_debug_build(void);
 int ef_debug_shift_tile(ef_ctx* ctx, int64_t tile, int64_t delta);
 
+/* Tracing: every entry point that enqueues work runs inside an NVTX range named after itself
+ * ("ef_worker_step", "ef_server_step", ...), so that a profiler can group or filter the kernels
+ * by call; without an attached tool the ranges do nothing. */
+
 /* Number of kernels this context has launched so far (for launch accounting). */
 int64_t ef_launch_count(ef_ctx* ctx);
 

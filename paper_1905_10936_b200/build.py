@@ -19,6 +19,7 @@ NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
     "-fmad=false",                      # no implicit contraction: every fused op is explicit
     "-Xcompiler", "-fPIC", "-shared",
+    "-ldl",                             # NVTX (header-only) looks for an attached tool with dlopen
 ]
 
 

@@ -10,6 +10,8 @@
 #include <utility>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 namespace efh {
 
 using efk::Block;
@@ -106,6 +108,17 @@ struct ef_ctx {
 };
 
 namespace efh {
+
+// NVTX range around one call of the interface, named after the call: a profiler that is
+// attached can group or filter the kernels by call (e.g. ncu --nvtx --nvtx-include
+// "ef_server_step/"); without one the two calls cost a pointer test each.
+struct ApiRange {
+    explicit ApiRange(const char* name) { nvtxRangePushA(name); }
+    ~ApiRange() { nvtxRangePop(); }
+    ApiRange(const ApiRange&) = delete;
+    ApiRange& operator=(const ApiRange&) = delete;
+};
+#define EF_API_RANGE() efh::ApiRange ef_api_range_(__func__)
 
 // Which method the worker calls of the current iteration belong to: the two methods share the
 // context's momentum, parameter and packed-word buffers and must not be mixed inside one

@@ -315,6 +315,7 @@ int ef_workspace_bytes(int64_t d, int32_t B, const int64_t* offsets, int32_t M, 
 int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t M, float mu,
             float eta, uint32_t flags, void* workspace, size_t workspace_bytes,
             void* cuda_stream) {
+    EF_API_RANGE();
     if (!out) return EF_ERR_INVALID_ARG;
     *out = nullptr;
     Layout L;
@@ -422,6 +423,7 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
 }
 
 int ef_worker_step(ef_ctx* c, int32_t i, const float* grad) {
+    EF_API_RANGE();
     int rc = check_worker_call(c, i, grad, kModeEF);
     if (rc != EF_OK) return rc;
     if (!aligned16(grad)) return EF_ERR_ALIGNMENT;
@@ -434,6 +436,7 @@ int ef_worker_step(ef_ctx* c, int32_t i, const float* grad) {
 }
 
 int ef_worker_step_push(ef_ctx* c, int32_t i, const float* grad, uint32_t* const* block_dst) {
+    EF_API_RANGE();
     int rc = check_worker_call(c, i, grad, kModeEF);
     if (rc != EF_OK) return rc;
     if (!block_dst) return EF_ERR_INVALID_ARG;
@@ -446,6 +449,7 @@ int ef_worker_step_push(ef_ctx* c, int32_t i, const float* grad, uint32_t* const
 }
 
 int ef_worker_step_all(ef_ctx* c, const float* grads, int64_t stride) {
+    EF_API_RANGE();
     if (!c || !grads || stride < c->L.d) return EF_ERR_INVALID_ARG;
     if (!aligned16(grads) || (stride & 3) != 0) return EF_ERR_ALIGNMENT;
     if (c->pending != 0) return EF_ERR_BAD_STATE;
@@ -459,6 +463,7 @@ int ef_worker_step_all(ef_ctx* c, const float* grads, int64_t stride) {
 }
 
 int ef_worker_step_host(ef_ctx* c, int32_t i, const float* grad) {
+    EF_API_RANGE();
     int rc = check_worker_call(c, i, grad, kModeEF);
     if (rc != EF_OK) return rc;
     if (!(c->flags & EF_FLAG_HOST_STAGING) || c->scales_open[i]) return EF_ERR_BAD_STATE;
@@ -479,6 +484,7 @@ int ef_worker_step_host(ef_ctx* c, int32_t i, const float* grad) {
 }
 
 int ef_server_step(ef_ctx* c) {
+    EF_API_RANGE();
     if (!c) return EF_ERR_INVALID_ARG;
     if (c->pending != c->L.M || c->L.Ml != c->L.M || c->mode != kModeEF) return EF_ERR_BAD_STATE;
     if (c->n_served != 0 || c->n_applied != 0) return EF_ERR_BAD_STATE;   // finish the range calls instead
@@ -503,6 +509,7 @@ int ef_pack_message(ef_ctx* c, int32_t who, int32_t b0, int32_t b1, uint32_t* ds
 }
 
 int ef_push_message(ef_ctx* c, int32_t who, int32_t b0, int32_t b1, int32_t n_dst, uint32_t* const* dst) {
+    EF_API_RANGE();
     if (check_block_range(c, b0, b1) != EF_OK || !dst || who < -1 || who >= c->L.Ml ||
         n_dst < 1 || n_dst > efk::kMaxPackTargets)
         return EF_ERR_INVALID_ARG;
@@ -525,6 +532,7 @@ int ef_push_message(ef_ctx* c, int32_t who, int32_t b0, int32_t b1, int32_t n_ds
 }
 
 int ef_server_step_range(ef_ctx* c, int32_t b0, int32_t b1, const uint32_t* msgs, int64_t msg_stride) {
+    EF_API_RANGE();
     if (check_block_range(c, b0, b1) != EF_OK) return EF_ERR_INVALID_ARG;
     if (c->pending != c->L.Ml || c->mode != kModeEF) return EF_ERR_BAD_STATE;
     if (!msgs && c->L.Ml != c->L.M) return EF_ERR_BAD_STATE;     // the other workers' messages are needed
@@ -544,6 +552,7 @@ int ef_server_step_range(ef_ctx* c, int32_t b0, int32_t b1, const uint32_t* msgs
 }
 
 int ef_apply_update(ef_ctx* c, int32_t b0, int32_t b1, const uint32_t* update) {
+    EF_API_RANGE();
     if (check_block_range(c, b0, b1) != EF_OK) return EF_ERR_INVALID_ARG;
     if (c->pending != c->L.Ml || c->mode != kModeEF) return EF_ERR_BAD_STATE;
     for (int32_t b = b0; b < b1; ++b)
@@ -577,6 +586,7 @@ int ef_set_block_divisors(ef_ctx* c, const int64_t* full_len) {
 }
 
 int ef_block_sums(ef_ctx* c, int32_t who, double* dst) {
+    EF_API_RANGE();
     if (!c || !dst || who < -1 || who >= c->L.Ml) return EF_ERR_INVALID_ARG;
     const int k = who < 0 ? c->srv() : who;
     launch_kernel(c, efk::ef_block_sums_kernel, dim3((unsigned)((c->L.B + efk::kThreads - 1) / efk::kThreads)), 0,
@@ -587,6 +597,7 @@ int ef_block_sums(ef_ctx* c, int32_t who, double* dst) {
 }
 
 int ef_complete_scales(ef_ctx* c, int32_t who, const double* totals) {
+    EF_API_RANGE();
     if (!c || !totals || who < -1 || who >= c->L.Ml) return EF_ERR_INVALID_ARG;
     const int k = who < 0 ? c->srv() : who;
     if (!c->scales_open[k]) return EF_ERR_BAD_STATE;
@@ -622,6 +633,7 @@ float* ef_decay_momentum(ef_ctx* c) {
 }
 
 int ef_read_update_host(ef_ctx* c, uint32_t* words, float* scales) {
+    EF_API_RANGE();
     if (!c || !words || !scales) return EF_ERR_INVALID_ARG;
     const int M = c->srv();
     EF_CUDA(c, cudaMemcpyAsync(words, c->words(M), (size_t)c->L.W * 4, cudaMemcpyDeviceToHost,
@@ -643,6 +655,7 @@ float* ef_params(ef_ctx* c) { return c ? c->x() : nullptr; }
 int64_t ef_num_words(ef_ctx* c) { return c ? c->L.W : -1; }
 
 int ef_get_momentum(ef_ctx* c, int32_t i, float* dst) {
+    EF_API_RANGE();
     if (!c || !dst || i < 0 || i >= c->L.Ml) return EF_ERR_INVALID_ARG;
     if (!aligned16(dst)) return EF_ERR_ALIGNMENT;
     EF_CUDA(c, cudaMemcpyAsync(dst, c->m(i), (size_t)c->L.d * 4, cudaMemcpyDeviceToDevice,
@@ -651,6 +664,7 @@ int ef_get_momentum(ef_ctx* c, int32_t i, float* dst) {
 }
 
 int ef_get_residual(ef_ctx* c, int32_t i, float* dst) {
+    EF_API_RANGE();
     if (!c || !dst || i < -1 || i >= c->L.Ml) return EF_ERR_INVALID_ARG;
     if (!aligned16(dst)) return EF_ERR_ALIGNMENT;
     const int k = (i < 0) ? c->srv() : i;
@@ -664,6 +678,7 @@ int ef_get_residual(ef_ctx* c, int32_t i, float* dst) {
 }
 
 int ef_set_state(ef_ctx* c, int32_t i, const float* momentum, const float* residual) {
+    EF_API_RANGE();
     if (!c || !residual || i < -1 || i >= c->L.Ml) return EF_ERR_INVALID_ARG;
     if (i >= 0 && !momentum) return EF_ERR_INVALID_ARG;
     if (!aligned16(residual) || (momentum && !aligned16(momentum))) return EF_ERR_ALIGNMENT;

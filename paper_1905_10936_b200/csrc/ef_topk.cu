@@ -707,6 +707,7 @@ int ef_topk_workspace_bytes(int64_t n, size_t* bytes) {
 
 int ef_topk_compress(const float* v, int64_t n, int64_t k, int64_t* idx_out, float* val_out,
                      float* resid_out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    EF_API_RANGE();
     if (!v || n < 1 || k < 1 || k > n || !idx_out || !val_out) return EF_ERR_INVALID_ARG;
     const TopkLayout L = topk_layout(n);
     if (L.chunks > 0x7fffffffLL) return EF_ERR_INVALID_ARG;

@@ -309,6 +309,7 @@ int launch_vote_worker(ef_ctx* c, int i, const float* grad, int count, long long
 extern "C" {
 
 int ef_vote_worker_step(ef_ctx* c, int32_t i, const float* grad) {
+    EF_API_RANGE();
     int rc = check_worker_call(c, i, grad, kModeVote);
     if (rc != EF_OK) return rc;
     if (!aligned16(grad)) return EF_ERR_ALIGNMENT;
@@ -319,6 +320,7 @@ int ef_vote_worker_step(ef_ctx* c, int32_t i, const float* grad) {
 }
 
 int ef_vote_worker_step_all(ef_ctx* c, const float* grads, int64_t stride) {
+    EF_API_RANGE();
     if (!c || !grads || stride < c->L.d) return EF_ERR_INVALID_ARG;
     if (!aligned16(grads) || (stride & 3) != 0) return EF_ERR_ALIGNMENT;
     if (c->pending != 0) return EF_ERR_BAD_STATE;
@@ -329,6 +331,7 @@ int ef_vote_worker_step_all(ef_ctx* c, const float* grads, int64_t stride) {
 }
 
 int ef_vote_server_step(ef_ctx* c) {
+    EF_API_RANGE();
     if (!c) return EF_ERR_INVALID_ARG;
     if (c->pending != c->L.M || c->mode != kModeVote) return EF_ERR_BAD_STATE;   // needs all M workers local
     const int M = c->L.M;
