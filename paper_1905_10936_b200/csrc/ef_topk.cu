@@ -25,7 +25,7 @@
 // element (the definition needs 8).  The list has room for n/8 candidates; when the bin holds
 // more (e.g. a vector whose magnitudes are all equal) steps 1b's list is skipped and the third
 // digit and the counts are taken from v itself (two more reads of v).  Which way a call goes is
-// decided on the device; the kernels of the other way end at once.
+// decided on the device, inside the kernels of the third digit and of the counts.
 // Nothing waits on another CTA; kernel boundaries order the passes.
 #include "ef_internal.h"
 
@@ -116,19 +116,13 @@ __device__ __forceinline__ unsigned warp_inclusive_scan32(unsigned v, int lane) 
     return v;
 }
 
-// ---- 1a / fallback of 1b: histogram of digit PASS over the keys of v that match the prefix so far.
-// PASS 2 is the fallback (the candidates did not fit the list) and ends at once otherwise.
+// ---- 1a: histogram of digit PASS over the keys of v that match the prefix so far (a device
+// function: the first pass is a kernel of its own, the third digit's fallback shares a kernel
+// with the pass over the list).
 template <int PASS>
-__global__ void __launch_bounds__(kThreads) ef_topk_hist_kernel(const float* __restrict__ v, long long n,
-                                                                long long chunks,
-                                                                const TopkState* __restrict__ st,
-                                                                unsigned long long* __restrict__ hist) {
-    __shared__ unsigned s_hist[kBins];
-    if (PASS == 2 && st->compact) return;
-    for (int b = threadIdx.x; b < kBins; b += kThreads) s_hist[b] = 0u;
-    __syncthreads();
+__device__ __forceinline__ void hist_over_vector(const float* __restrict__ v, long long n, long long chunks,
+                                                 unsigned prefix, unsigned* s_hist) {
     constexpr int shift = pass_shift(PASS), bits = pass_bits(PASS);
-    const unsigned prefix = PASS == 0 ? 0u : st->prefix;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (long long c = blockIdx.x; c < chunks; c += gridDim.x) {
 #pragma unroll
@@ -145,6 +139,18 @@ __global__ void __launch_bounds__(kThreads) ef_topk_hist_kernel(const float* __r
             }
         }
     }
+}
+
+template <int PASS>
+__global__ void __launch_bounds__(kThreads) ef_topk_hist_kernel(const float* __restrict__ v, long long n,
+                                                                long long chunks,
+                                                                const TopkState* __restrict__ st,
+                                                                unsigned long long* __restrict__ hist) {
+    __shared__ unsigned s_hist[kBins];
+    for (int b = threadIdx.x; b < kBins; b += kThreads) s_hist[b] = 0u;
+    __syncthreads();
+    constexpr int bits = pass_bits(PASS);
+    hist_over_vector<PASS>(v, n, chunks, PASS == 0 ? 0u : st->prefix, s_hist);
     __syncthreads();
     for (int b = threadIdx.x; b < (1 << bits); b += kThreads)
         if (s_hist[b]) atomicAdd(&hist[b], (unsigned long long)s_hist[b]);
@@ -328,119 +334,127 @@ __global__ void __launch_bounds__(kThreads) ef_topk_candidates_kernel(const floa
 }
 constexpr size_t kCandidatesSmem = 2 * kChunkLen * sizeof(unsigned) + kWarps * sizeof(WarpStage);
 
-// ---- 1b, third digit: histogram over the candidate list (ends at once in the fallback).
-__global__ void __launch_bounds__(kThreads) ef_topk_hist_list_kernel(const unsigned* __restrict__ cand,
-                                                                     const TopkState* __restrict__ st,
-                                                                     unsigned long long* __restrict__ hist) {
-    __shared__ unsigned s_hist[1 << pass_bits(2)];
-    if (!st->compact) return;
-    for (int b = threadIdx.x; b < (1 << pass_bits(2)); b += kThreads) s_hist[b] = 0u;
+// ---- 1b, third digit: histogram over the candidate list, or over v when the list was not used.
+__global__ void __launch_bounds__(kThreads) ef_topk_third_digit_kernel(const float* __restrict__ v, long long n,
+                                                                       long long chunks,
+                                                                       const unsigned* __restrict__ cand,
+                                                                       const TopkState* __restrict__ st,
+                                                                       unsigned long long* __restrict__ hist) {
+    constexpr int nbins = 1 << pass_bits(2);
+    __shared__ unsigned s_hist[nbins];
+    for (int b = threadIdx.x; b < nbins; b += kThreads) s_hist[b] = 0u;
     __syncthreads();
-    const unsigned long long ncand = st->ncand;
     const unsigned prefix = st->prefix;            // 22 bits
-    for (unsigned long long i = (unsigned long long)blockIdx.x * kThreads + threadIdx.x; i < ncand;
-         i += (unsigned long long)gridDim.x * kThreads) {
-        const unsigned key = cand[i];
-        if ((key >> pass_bits(2)) == prefix) atomicAdd(&s_hist[key & ((1u << pass_bits(2)) - 1u)], 1u);
+    if (st->compact) {
+        const unsigned long long ncand = st->ncand;
+        for (unsigned long long i = (unsigned long long)blockIdx.x * kThreads + threadIdx.x; i < ncand;
+             i += (unsigned long long)gridDim.x * kThreads) {
+            const unsigned key = cand[i];
+            if ((key >> pass_bits(2)) == prefix) atomicAdd(&s_hist[key & (nbins - 1u)], 1u);
+        }
+    } else {
+        hist_over_vector<2>(v, n, chunks, prefix, s_hist);
     }
     __syncthreads();
-    for (int b = threadIdx.x; b < (1 << pass_bits(2)); b += kThreads)
+    for (int b = threadIdx.x; b < nbins; b += kThreads)
         if (s_hist[b]) atomicAdd(&hist[b], (unsigned long long)s_hist[b]);
 }
 
 // One CTA fixes the next digit: it finds, from the largest digit down, the bin in which the
-// count of keys seen so far reaches `remaining`.  Thread t adds up bins 8t .. 8t+7; thread 0
-// walks the 256 sums from the top and then the eight bins of the group it stops in.
+// count of keys seen so far reaches `remaining`.  Thread t adds up the eight bins of group
+// 255 - t (so thread order is from the top down); a scan over the threads gives every group the
+// count above it, the one thread whose group holds the crossing walks its eight bins.
 template <int PASS>
 __global__ void __launch_bounds__(kThreads) ef_topk_select_kernel(const unsigned long long* __restrict__ hist,
                                                                   TopkState* st, unsigned long long k,
                                                                   unsigned long long cap) {
     constexpr int bits = pass_bits(PASS), nbins = 1 << bits, per = kBins / kThreads;
-    __shared__ unsigned long long s_bin[kBins], s_grp[kThreads];
+    __shared__ unsigned long long s_warp[kWarps];
+    __shared__ int s_found;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int grp = kThreads - 1 - threadIdx.x;
+    unsigned long long bin[per];
     unsigned long long g = 0;
 #pragma unroll
     for (int j = 0; j < per; ++j) {
-        const int b = threadIdx.x * per + j;
-        const unsigned long long v = b < nbins ? hist[b] : 0ull;
-        s_bin[b] = v;
-        g += v;
+        const int b = grp * per + j;
+        bin[j] = b < nbins ? hist[b] : 0ull;
+        g += bin[j];
     }
-    s_grp[threadIdx.x] = g;
+    if (threadIdx.x == 0) s_found = 0;
+    unsigned long long incl = g;               // keys in this group and all groups above it
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long u = __shfl_up_sync(kFull, incl, o);
+        if (lane >= o) incl += u;
+    }
+    if (lane == 31) s_warp[warp] = incl;
     __syncthreads();
-    if (threadIdx.x != 0) return;
-    unsigned long long remaining = PASS == 0 ? k : st->remaining;
+    for (int w = 0; w < warp; ++w) incl += s_warp[w];
+    const unsigned long long remaining = PASS == 0 ? k : st->remaining;
+    unsigned long long above = incl - g;
+    // the crossing group; if the counts never reach `remaining` (they always do for k <= n) the lowest group
+    const bool mine = above < remaining && (incl >= remaining || grp == 0);
+    if (!mine) return;
+    if (atomicExch(&s_found, 1) != 0) return;  // defensive: exactly one thread writes
+    int j = per - 1;
+    for (; j > 0; --j) {
+        if (above + bin[j] >= remaining) break;
+        above += bin[j];
+    }
     const unsigned prefix = PASS == 0 ? 0u : st->prefix;
-    unsigned long long above = 0;
-    int grp = kThreads - 1;
-    for (; grp > 0; --grp) {
-        if (above + s_grp[grp] >= remaining) break;
-        above += s_grp[grp];
-    }
-    int b = grp * per + per - 1;
-    for (; b > grp * per; --b) {
-        if (above + s_bin[b] >= remaining) break;
-        above += s_bin[b];
-    }
-    remaining -= above;                       // still to keep among the keys of bin b
-    st->prefix = (prefix << bits) | (unsigned)b;
-    st->remaining = remaining;
+    st->prefix = (prefix << bits) | (unsigned)(grp * per + j);
+    st->remaining = remaining - above;         // still to keep among the keys of the bin
     if (PASS == 0) {
-        st->ncand = s_bin[b];
-        st->compact = s_bin[b] <= cap ? 1u : 0u;
+        st->ncand = bin[j];
+        st->compact = bin[j] <= cap ? 1u : 0u;
     }
     if (PASS == kPasses - 1) {
         st->threshold = st->prefix;
-        st->need_eq = remaining;
+        st->need_eq = remaining - above;
     }
 }
 
-// ---- 2. per chunk: how many keys are > T and == T.  From the list: one warp per chunk adds
-// the chunk's candidates above T to its sure count.
-__global__ void __launch_bounds__(kThreads) ef_topk_count_list_kernel(const unsigned* __restrict__ cand,
-                                                                      const TopkState* __restrict__ st,
-                                                                      const unsigned long long* __restrict__ seg_start,
-                                                                      const unsigned* __restrict__ seg_cnt,
-                                                                      long long chunks,
-                                                                      unsigned* __restrict__ cgt,
-                                                                      unsigned* __restrict__ ceq,
-                                                                      unsigned* __restrict__ tgt,
-                                                                      unsigned* __restrict__ teq) {
-    if (!st->compact) return;
-    const unsigned T = st->threshold;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long c = (long long)blockIdx.x * kWarps + warp;
-    if (c >= chunks) return;
-    const unsigned cnt = seg_cnt[c];
-    const unsigned* seg = cand + seg_start[c];
-    unsigned both = 0u;                       // at most 4096 each: two 16-bit fields
-    for (unsigned i = lane; i < cnt; i += 32) {
-        const unsigned key = seg[i];
-        both += (key > T ? 1u : 0u) + (key == T ? 1u << 16 : 0u);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) both += __shfl_xor_sync(kFull, both, o);
-    if (lane == 0) {
-        const unsigned gt = cgt[c] + (both & 0xffffu), eq = both >> 16;
-        cgt[c] = gt;
-        ceq[c] = eq;
-        if (gt) atomicAdd(&tgt[c / kTileOfChunks], gt);      // totals of the tile, for the scan
-        if (eq) atomicAdd(&teq[c / kTileOfChunks], eq);
-    }
-}
-
-// Fallback: the same counts from v itself (ends at once when the list was used).
+// ---- 2. per chunk: how many keys are > T and == T, and the totals per tile for the scan.
+// A CTA takes kWarps consecutive chunks.  With the list: one warp per chunk adds the chunk's
+// candidates above T to its sure count.  Without: the CTA counts its chunks in v one by one.
 __global__ void __launch_bounds__(kThreads) ef_topk_count_kernel(const float* __restrict__ v, long long n,
                                                                  long long chunks,
+                                                                 const unsigned* __restrict__ cand,
                                                                  const TopkState* __restrict__ st,
+                                                                 const unsigned long long* __restrict__ seg_start,
+                                                                 const unsigned* __restrict__ seg_cnt,
                                                                  unsigned* __restrict__ cgt,
                                                                  unsigned* __restrict__ ceq,
                                                                  unsigned* __restrict__ tgt,
                                                                  unsigned* __restrict__ teq) {
     __shared__ unsigned s_gt[kWarps], s_eq[kWarps];
-    if (st->compact) return;
     const unsigned T = st->threshold;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (long long c = blockIdx.x; c < chunks; c += gridDim.x) {
+    if (st->compact) {
+        const long long c = (long long)blockIdx.x * kWarps + warp;
+        if (c >= chunks) return;
+        const unsigned cnt = seg_cnt[c];
+        const unsigned* seg = cand + seg_start[c];
+        unsigned both = 0u;                   // at most 4096 each: two 16-bit fields
+        for (unsigned i = lane; i < cnt; i += 32) {
+            const unsigned key = seg[i];
+            both += (key > T ? 1u : 0u) + (key == T ? 1u << 16 : 0u);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) both += __shfl_xor_sync(kFull, both, o);
+        if (lane == 0) {
+            const unsigned gt = cgt[c] + (both & 0xffffu), eq = both >> 16;
+            cgt[c] = gt;
+            ceq[c] = eq;
+            if (gt) atomicAdd(&tgt[c / kTileOfChunks], gt);
+            if (eq) atomicAdd(&teq[c / kTileOfChunks], eq);
+        }
+        return;
+    }
+    for (int j = 0; j < kWarps; ++j) {
+        const long long c = (long long)blockIdx.x * kWarps + j;
+        if (c >= chunks) return;              // the same in every thread
         unsigned gt = 0, eq = 0;
 #pragma unroll
         for (int u = 0; u < kU; ++u) {
@@ -746,19 +760,16 @@ int ef_topk_compress(const float* v, int64_t n, int64_t k, int64_t* idx_out, flo
     if (cudaMemsetAsync(ws, 0, L.off_cgt, st) != cudaSuccess) return EF_ERR_CUDA;   // histograms, state, tile totals
     const unsigned hgrid = (unsigned)std::min<long long>(L.chunks, 148 * 8);
     const unsigned cgrid = (unsigned)std::min<long long>(L.chunks, 148 * 3);       // three CTAs of 59 KB per SM
-    const unsigned lgrid = (unsigned)std::min<unsigned long long>((L.cap + kThreads - 1) / kThreads, 148 * 8);
     const unsigned long long kk = (unsigned long long)k;
     ef_topk_hist_kernel<0><<<hgrid, kThreads, 0, st>>>(v, n, L.chunks, state, hist);
     ef_topk_select_kernel<0><<<1, kThreads, 0, st>>>(hist, state, kk, L.cap);
     ef_topk_candidates_kernel<<<cgrid, kThreads, kCandidatesSmem, st>>>(v, n, L.chunks, state, hist + kBins,
                                                                         cgt, seg_start, seg_cnt, cand);
     ef_topk_select_kernel<1><<<1, kThreads, 0, st>>>(hist + kBins, state, kk, L.cap);
-    ef_topk_hist_list_kernel<<<lgrid, kThreads, 0, st>>>(cand, state, hist + 2 * kBins);     // list ...
-    ef_topk_hist_kernel<2><<<hgrid, kThreads, 0, st>>>(v, n, L.chunks, state, hist + 2 * kBins);   // ... or v
+    ef_topk_third_digit_kernel<<<hgrid, kThreads, 0, st>>>(v, n, L.chunks, cand, state, hist + 2 * kBins);
     ef_topk_select_kernel<2><<<1, kThreads, 0, st>>>(hist + 2 * kBins, state, kk, L.cap);
-    ef_topk_count_list_kernel<<<(unsigned)((L.chunks + kWarps - 1) / kWarps), kThreads, 0, st>>>(
-        cand, state, seg_start, seg_cnt, L.chunks, cgt, ceq, tgt, teq);
-    ef_topk_count_kernel<<<hgrid, kThreads, 0, st>>>(v, n, L.chunks, state, cgt, ceq, tgt, teq);
+    ef_topk_count_kernel<<<(unsigned)((L.chunks + kWarps - 1) / kWarps), kThreads, 0, st>>>(
+        v, n, L.chunks, cand, state, seg_start, seg_cnt, cgt, ceq, tgt, teq);
     ef_topk_scan_kernel<<<1, kScanThreads, 0, st>>>(tgt, teq, pgt, peq, L.tiles);
     ScatterArgs sa;
     sa.v = v; sa.n = n; sa.chunks = L.chunks; sa.st = state; sa.cgt = cgt; sa.ceq = ceq; sa.pgt = pgt; sa.peq = peq;
