@@ -13,8 +13,8 @@
 //         keys IN the bin (the candidates, typically a few per cent of n) still matter.
 //      b. second pass over v: histogram of the second digit of the candidates, the number of
 //         sure keys per 4096-element chunk, and the candidates' keys copied to a compact list
-//         (one segment per chunk; the order inside a segment is arbitrary and nothing depends
-//         on it).  The third digit is then histogrammed over the list, not over v.
+//         (one segment per warp and chunk; the order inside a segment is arbitrary and nothing
+//         depends on it).  The third digit is then histogrammed over the list, not over v.
 //      Result: T and how many keys equal to T have to be kept (need_eq).
 //   2. per chunk the number of keys > T and == T, from the chunk's sure count and its segment
 //      of the list (no pass over v);
@@ -72,18 +72,18 @@ TopkLayout topk_layout(int64_t n) {
     // room for an eighth of the vector; short vectors always fit
     L.cap = (unsigned long long)std::max<int64_t>(n / 8, std::min<int64_t>(n, 65536));
     size_t o = 0;
-    // zeroed at the start of every call: histograms, state, per-tile totals
+    // zeroed at the start of every call: histograms, state, per-tile totals, per-chunk sure counts
     L.off_hist = o;  o += align_up(sizeof(unsigned long long) * kBins * kPasses);
     L.off_state = o; o += align_up(sizeof(TopkState));
     L.off_tgt = o;   o += align_up(sizeof(unsigned) * (size_t)L.tiles);
     L.off_teq = o;   o += align_up(sizeof(unsigned) * (size_t)L.tiles);
-    // written before they are read
     L.off_cgt = o;   o += align_up(sizeof(unsigned) * (size_t)L.chunks);
+    // written before they are read
     L.off_ceq = o;   o += align_up(sizeof(unsigned) * (size_t)L.chunks);
     L.off_pgt = o;   o += align_up(sizeof(unsigned long long) * (size_t)L.tiles);
     L.off_peq = o;   o += align_up(sizeof(unsigned long long) * (size_t)L.tiles);
-    L.off_seg_start = o; o += align_up(sizeof(unsigned long long) * (size_t)L.chunks);
-    L.off_seg_cnt = o;   o += align_up(sizeof(unsigned) * (size_t)L.chunks);
+    L.off_seg_start = o; o += align_up(sizeof(unsigned long long) * (size_t)L.chunks * kWarps);   // one segment
+    L.off_seg_cnt = o;   o += align_up(sizeof(unsigned) * (size_t)L.chunks * kWarps);             // per warp and chunk
     L.off_cand = o;  o += align_up(sizeof(unsigned) * (size_t)L.cap);
     L.total = o;
     return L;
@@ -199,10 +199,9 @@ __device__ __forceinline__ int stage_rows(const float (&x)[kU][4], unsigned fin,
 
 // ---- 1b. second pass over v.  Per chunk: histogram of the second digit of the candidates (keys
 // whose first digit is P0), the number of sure keys (first digit > P0) into cgt, and -- if the
-// candidates fit the list -- the candidates' keys as one segment of the list.
-// A CTA walks its chunks with the next chunk's loads issued before it waits for the list
-// position of the current one (one atomic on the global cursor per chunk), and with two
-// shared-memory lists used in turn, so that a chunk costs two barriers.
+// candidates fit the list -- the candidates' keys on the list.
+
+// This warp's 512 elements of chunk c, four rows of four per lane; fin: bit 4u + k = element exists.
 __device__ __forceinline__ void load_chunk_keys(const float* __restrict__ v, long long n, long long c,
                                                 int warp, int lane, float (&x)[kU][4], unsigned& fin) {
     if ((c + 1) * kChunkLen <= n) {            // the whole chunk is inside the vector
@@ -230,6 +229,40 @@ __device__ __forceinline__ void load_chunk_keys(const float* __restrict__ v, lon
     }
 }
 
+// Every warp works for itself: it keeps its candidates of up to 32 chunks in a list of its own in
+// shared memory, and when that is half full (or 32 chunks are logged) it reserves room on the
+// global list with ONE atomic, copies the keys out and records where each logged chunk's keys
+// went.  So a chunk has kWarps segments on the global list (one per warp), no CTA barrier lies on
+// the path, and the global cursor sees one atomic per ~500 candidates.
+constexpr int kWarpListKeys = 1024;     // a warp's slice of a chunk holds at most 512 keys: flushed above 512, it always fits
+constexpr int kWarpListLog = 32;
+struct WarpList {
+    unsigned key[kWarpListKeys];
+    long long seg[kWarpListLog];        // which segment (chunk * kWarps + warp) ...
+    unsigned short off[kWarpListLog];   // ... starts where in key[] ...
+    unsigned short cnt[kWarpListLog];   // ... and holds how many keys
+};
+
+__device__ __forceinline__ void flush_warp_list(WarpList& wl, int& fill, int& nlog, TopkState* st,
+                                                unsigned long long* __restrict__ seg_start,
+                                                unsigned* __restrict__ seg_cnt,
+                                                unsigned* __restrict__ cand, int lane) {
+    __syncwarp();
+    if (fill > 0) {
+        unsigned long long base = 0ull;
+        if (lane == 0) base = atomicAdd(&st->cursor, (unsigned long long)fill);
+        base = __shfl_sync(kFull, base, 0);
+        for (int i = lane; i < fill; i += 32) cand[base + i] = wl.key[i];
+        if (lane < nlog) {
+            seg_start[wl.seg[lane]] = base + wl.off[lane];
+            seg_cnt[wl.seg[lane]] = wl.cnt[lane];
+        }
+    }
+    __syncwarp();
+    fill = 0;
+    nlog = 0;
+}
+
 __global__ void __launch_bounds__(kThreads) ef_topk_candidates_kernel(const float* __restrict__ v, long long n,
                                                                       long long chunks, TopkState* st,
                                                                       unsigned long long* __restrict__ hist,
@@ -238,30 +271,33 @@ __global__ void __launch_bounds__(kThreads) ef_topk_candidates_kernel(const floa
                                                                       unsigned* __restrict__ seg_cnt,
                                                                       unsigned* __restrict__ cand) {
     extern __shared__ __align__(16) unsigned char s_dyn[];
-    // dynamic: [two lists of kChunkLen keys][one staging area per warp]
-    unsigned (*s_list)[kChunkLen] = reinterpret_cast<unsigned (*)[kChunkLen]>(s_dyn);
-    WarpStage* s_stage = reinterpret_cast<WarpStage*>(s_dyn + 2 * kChunkLen * sizeof(unsigned));
+    // dynamic: [one list per warp][one staging area per warp]
+    WarpList* s_lists = reinterpret_cast<WarpList*>(s_dyn);
+    WarpStage* s_stage = reinterpret_cast<WarpStage*>(s_dyn + kWarps * sizeof(WarpList));
     __shared__ unsigned s_hist[kBins];
-    __shared__ unsigned s_gt[2][kWarps];
-    __shared__ unsigned s_cnt[2];
-    __shared__ unsigned long long s_base;
     for (int b = threadIdx.x; b < kBins; b += kThreads) s_hist[b] = 0u;
-    if (threadIdx.x == 0) { s_cnt[0] = 0u; s_cnt[1] = 0u; }
     const unsigned P0 = st->prefix;
     const unsigned lo = P0 << 20, hi_top = P0 + 1u;       // candidates: lo <= key and (key >> 20) < hi_top
     const bool compact = st->compact != 0u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     WarpStage& stage = s_stage[warp];
+    WarpList& wl = s_lists[warp];
     float x[kU][4];
-    unsigned fin;
+    unsigned fin = 0u;
+    int fill = 0, nlog = 0;                    // the same in every lane of the warp
     if (blockIdx.x < chunks) load_chunk_keys(v, n, blockIdx.x, warp, lane, x, fin);
-    __syncthreads();
-    int par = 0;
-    // the staged rows of one chunk: second-digit histogram, candidates to list `par`, sure keys counted
-    auto classify = [&](auto full_c) -> unsigned {
+    __syncthreads();                           // the histogram is zero
+    // the staged rows of this warp's slice of chunk c: second-digit histogram, candidates to the
+    // warp's list, sure keys counted.  The next chunk's loads are issued once the rows are staged.
+    auto classify = [&](auto full_c, long long c) {
         constexpr bool FULL = decltype(full_c)::value;
+        if (compact && (fill > kWarpListKeys / 2 || nlog == kWarpListLog))
+            flush_warp_list(wl, fill, nlog, st, seg_start, seg_cnt, cand, lane);
         const int H = stage_rows<FULL>(x, fin, lo, stage, lane);
+        const long long next = c + gridDim.x;
+        if (next < chunks) load_chunk_keys(v, n, next, warp, lane, x, fin);
         unsigned gt = 0u;
+        const int fill0 = fill;
         for (int e0 = 0; e0 < H; e0 += 32) {
             const int e = e0 + lane;
             unsigned keys[4] = {0u, 0u, 0u, 0u};
@@ -283,56 +319,42 @@ __global__ void __launch_bounds__(kThreads) ef_topk_candidates_kernel(const floa
                 }
             }
             if (compact && __any_sync(kFull, mine != 0u)) {
-                // list positions of the warp's candidates: one shared atomic per dense iteration
                 const unsigned cnt = (unsigned)__popc(mine);
                 const unsigned incl = warp_inclusive_scan32(cnt, lane);
-                unsigned wbase = 0u;
-                if (lane == 31) wbase = atomicAdd(&s_cnt[par], incl);
-                wbase = __shfl_sync(kFull, wbase, 31);
-                unsigned pos = wbase + incl - cnt;
+                int pos = fill + (int)(incl - cnt);
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
-                    if ((mine >> k) & 1u) s_list[par][pos++] = keys[k];
+                    if ((mine >> k) & 1u) wl.key[pos++] = keys[k];
+                fill += (int)__shfl_sync(kFull, incl, 31);
             }
         }
-        return gt;
-    };
-    for (long long c = blockIdx.x; c < chunks; c += gridDim.x, par ^= 1) {
-        // the choice must be the same in every thread of the CTA (the paths hold warp-wide operations):
-        // it is made on the chunk, not on the thread's own range flags
-        unsigned gt = (c + 1) * kChunkLen <= n ? classify(std::true_type{}) : classify(std::false_type{});
+        __syncwarp();                          // the staging area is rewritten by the next chunk
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) gt += __shfl_xor_sync(kFull, gt, o);
-        if (lane == 0) s_gt[par][warp] = gt;
-        __syncthreads();                       // list and counts of chunk c are complete
-        unsigned long long base = 0ull;
-        unsigned cnt = 0u;
-        if (threadIdx.x == 0) {
-            cnt = s_cnt[par];
-            if (cnt) base = atomicAdd(&st->cursor, (unsigned long long)cnt);     // in flight ...
+        if (lane == 0) {
+            if (gt) atomicAdd(&cgt[c], gt);    // cgt is zeroed at the start of the call
+            const long long seg = c * kWarps + warp;
+            if (!compact || fill == fill0) seg_cnt[seg] = 0u;
+            else {
+                wl.seg[nlog] = seg;
+                wl.off[nlog] = (unsigned short)fill0;
+                wl.cnt[nlog] = (unsigned short)(fill - fill0);
+            }
         }
-        const long long next = c + gridDim.x;
-        if (next < chunks) load_chunk_keys(v, n, next, warp, lane, x, fin);      // ... with the next chunk's loads
-        if (threadIdx.x == 0) {
-            unsigned a = 0;
-            for (int w = 0; w < kWarps; ++w) a += s_gt[par][w];
-            cgt[c] = a;
-            seg_cnt[c] = cnt;
-            seg_start[c] = base;
-            s_base = base;
-            s_cnt[par ^ 1] = 0u;               // its last readers passed the barrier above
-        }
-        __syncthreads();
-        cnt = s_cnt[par];
-        base = s_base;
-        for (unsigned i = threadIdx.x; i < cnt; i += kThreads) cand[base + i] = s_list[par][i];
-        // s_base and list `par` are next written after the next chunk's first barrier
+        if (compact && fill != fill0) nlog += 1;
+    };
+    for (long long c = blockIdx.x; c < chunks; c += gridDim.x) {
+        // the choice must be the same in every thread of a warp (the paths hold warp-wide
+        // operations): it is made on the chunk, not on the thread's own range flags
+        if ((c + 1) * kChunkLen <= n) classify(std::true_type{}, c);
+        else classify(std::false_type{}, c);
     }
+    if (compact) flush_warp_list(wl, fill, nlog, st, seg_start, seg_cnt, cand, lane);
     __syncthreads();
     for (int b = threadIdx.x; b < kBins; b += kThreads)
         if (s_hist[b]) atomicAdd(&hist[b], (unsigned long long)s_hist[b]);
 }
-constexpr size_t kCandidatesSmem = 2 * kChunkLen * sizeof(unsigned) + kWarps * sizeof(WarpStage);
+constexpr size_t kCandidatesSmem = kWarps * (sizeof(WarpList) + sizeof(WarpStage));
 
 // ---- 1b, third digit: histogram over the candidate list, or over v when the list was not used.
 __global__ void __launch_bounds__(kThreads) ef_topk_third_digit_kernel(const float* __restrict__ v, long long n,
@@ -434,12 +456,16 @@ __global__ void __launch_bounds__(kThreads) ef_topk_count_kernel(const float* __
     if (st->compact) {
         const long long c = (long long)blockIdx.x * kWarps + warp;
         if (c >= chunks) return;
-        const unsigned cnt = seg_cnt[c];
-        const unsigned* seg = cand + seg_start[c];
         unsigned both = 0u;                   // at most 4096 each: two 16-bit fields
-        for (unsigned i = lane; i < cnt; i += 32) {
-            const unsigned key = seg[i];
-            both += (key > T ? 1u : 0u) + (key == T ? 1u << 16 : 0u);
+        {   // the chunk's kWarps segments (one per warp of the pass that listed them), four lanes each
+            static_assert(kWarps == 8, "four lanes per segment");
+            const long long sg = c * kWarps + (lane >> 2);
+            const unsigned cnt = seg_cnt[sg];
+            const unsigned* seg = cand + (cnt ? seg_start[sg] : 0ull);
+            for (unsigned i = lane & 3; i < cnt; i += 4) {
+                const unsigned key = seg[i];
+                both += (key > T ? 1u : 0u) + (key == T ? 1u << 16 : 0u);
+            }
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) both += __shfl_xor_sync(kFull, both, o);
@@ -757,7 +783,7 @@ int ef_topk_compress(const float* v, int64_t n, int64_t k, int64_t* idx_out, flo
     unsigned long long* seg_start = (unsigned long long*)(ws + L.off_seg_start);
     unsigned* seg_cnt = (unsigned*)(ws + L.off_seg_cnt);
     unsigned* cand = (unsigned*)(ws + L.off_cand);
-    if (cudaMemsetAsync(ws, 0, L.off_cgt, st) != cudaSuccess) return EF_ERR_CUDA;   // histograms, state, tile totals
+    if (cudaMemsetAsync(ws, 0, L.off_ceq, st) != cudaSuccess) return EF_ERR_CUDA;   // histograms, state, totals, sure counts
     const unsigned hgrid = (unsigned)std::min<long long>(L.chunks, 148 * 8);
     const unsigned cgrid = (unsigned)std::min<long long>(L.chunks, 148 * 3);       // three CTAs of 59 KB per SM
     const unsigned long long kk = (unsigned long long)k;
