@@ -72,14 +72,15 @@ TopkLayout topk_layout(int64_t n) {
     // room for an eighth of the vector; short vectors always fit
     L.cap = (unsigned long long)std::max<int64_t>(n / 8, std::min<int64_t>(n, 65536));
     size_t o = 0;
-    // zeroed at the start of every call: histograms, state, per-tile totals, per-chunk sure counts
+    // zeroed at the start of every call: histograms, state, per-tile totals
     L.off_hist = o;  o += align_up(sizeof(unsigned long long) * kBins * kPasses);
     L.off_state = o; o += align_up(sizeof(TopkState));
     L.off_tgt = o;   o += align_up(sizeof(unsigned) * (size_t)L.tiles);
     L.off_teq = o;   o += align_up(sizeof(unsigned) * (size_t)L.tiles);
-    L.off_cgt = o;   o += align_up(sizeof(unsigned) * (size_t)L.chunks);
-    // written before they are read
-    L.off_ceq = o;   o += align_up(sizeof(unsigned) * (size_t)L.chunks);
+    // written before they are read; counts and list segments are kept per SLICE: the 512 elements
+    // of a chunk that one warp handles (slice = chunk * kWarps + warp)
+    L.off_cgt = o;   o += align_up(sizeof(unsigned) * (size_t)L.chunks * kWarps);
+    L.off_ceq = o;   o += align_up(sizeof(unsigned) * (size_t)L.chunks * kWarps);
     L.off_pgt = o;   o += align_up(sizeof(unsigned long long) * (size_t)L.tiles);
     L.off_peq = o;   o += align_up(sizeof(unsigned long long) * (size_t)L.tiles);
     L.off_seg_start = o; o += align_up(sizeof(unsigned long long) * (size_t)L.chunks * kWarps);   // one segment
@@ -332,8 +333,8 @@ __global__ void __launch_bounds__(kThreads) ef_topk_candidates_kernel(const floa
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) gt += __shfl_xor_sync(kFull, gt, o);
         if (lane == 0) {
-            if (gt) atomicAdd(&cgt[c], gt);    // cgt is zeroed at the start of the call
             const long long seg = c * kWarps + warp;
+            cgt[seg] = gt;
             if (!compact || fill == fill0) seg_cnt[seg] = 0u;
             else {
                 wl.seg[nlog] = seg;
@@ -437,9 +438,10 @@ __global__ void __launch_bounds__(kThreads) ef_topk_select_kernel(const unsigned
     }
 }
 
-// ---- 2. per chunk: how many keys are > T and == T, and the totals per tile for the scan.
-// A CTA takes kWarps consecutive chunks.  With the list: one warp per chunk adds the chunk's
-// candidates above T to its sure count.  Without: the CTA counts its chunks in v one by one.
+// ---- 2. per slice (the 512 elements of a chunk that one warp handles): how many keys are > T and
+// == T, and the totals per tile for the scan.  A CTA takes kWarps consecutive chunks.  With the
+// list: one warp per chunk, four lanes per slice, adds the slice's candidates above T to its sure
+// count.  Without: the CTA counts its chunks in v one by one, every warp its own slice.
 __global__ void __launch_bounds__(kThreads) ef_topk_count_kernel(const float* __restrict__ v, long long n,
                                                                  long long chunks,
                                                                  const unsigned* __restrict__ cand,
@@ -450,37 +452,41 @@ __global__ void __launch_bounds__(kThreads) ef_topk_count_kernel(const float* __
                                                                  unsigned* __restrict__ ceq,
                                                                  unsigned* __restrict__ tgt,
                                                                  unsigned* __restrict__ teq) {
-    __shared__ unsigned s_gt[kWarps], s_eq[kWarps];
     const unsigned T = st->threshold;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (st->compact) {
         const long long c = (long long)blockIdx.x * kWarps + warp;
         if (c >= chunks) return;
-        unsigned both = 0u;                   // at most 4096 each: two 16-bit fields
-        {   // the chunk's kWarps segments (one per warp of the pass that listed them), four lanes each
-            static_assert(kWarps == 8, "four lanes per segment");
-            const long long sg = c * kWarps + (lane >> 2);
-            const unsigned cnt = seg_cnt[sg];
-            const unsigned* seg = cand + (cnt ? seg_start[sg] : 0ull);
-            for (unsigned i = lane & 3; i < cnt; i += 4) {
-                const unsigned key = seg[i];
-                both += (key > T ? 1u : 0u) + (key == T ? 1u << 16 : 0u);
-            }
+        // the chunk's kWarps slices, four lanes each
+        static_assert(kWarps == 8, "four lanes per slice");
+        const long long sl = c * kWarps + (lane >> 2);
+        const unsigned cnt = seg_cnt[sl];
+        const unsigned* seg = cand + (cnt ? seg_start[sl] : 0ull);
+        unsigned both = 0u;                   // at most 512 each: two 16-bit fields
+        for (unsigned i = lane & 3; i < cnt; i += 4) {
+            const unsigned key = seg[i];
+            both += (key > T ? 1u : 0u) + (key == T ? 1u << 16 : 0u);
+        }
+        both += __shfl_xor_sync(kFull, both, 1);
+        both += __shfl_xor_sync(kFull, both, 2);
+        if ((lane & 3) == 0) {
+            both += cgt[sl];                  // the slice's sure keys
+            cgt[sl] = both & 0xffffu;
+            ceq[sl] = both >> 16;
+        } else {
+            both = 0u;
         }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) both += __shfl_xor_sync(kFull, both, o);
-        if (lane == 0) {
-            const unsigned gt = cgt[c] + (both & 0xffffu), eq = both >> 16;
-            cgt[c] = gt;
-            ceq[c] = eq;
-            if (gt) atomicAdd(&tgt[c / kTileOfChunks], gt);
-            if (eq) atomicAdd(&teq[c / kTileOfChunks], eq);
+        for (int o = 16; o > 2; o >>= 1) both += __shfl_xor_sync(kFull, both, o);
+        if (lane == 0) {                      // at most 4096 each
+            if (both & 0xffffu) atomicAdd(&tgt[c / kTileOfChunks], both & 0xffffu);
+            if (both >> 16) atomicAdd(&teq[c / kTileOfChunks], both >> 16);
         }
         return;
     }
     for (int j = 0; j < kWarps; ++j) {
         const long long c = (long long)blockIdx.x * kWarps + j;
-        if (c >= chunks) return;              // the same in every thread
+        if (c >= chunks) return;
         unsigned gt = 0, eq = 0;
 #pragma unroll
         for (int u = 0; u < kU; ++u) {
@@ -498,17 +504,12 @@ __global__ void __launch_bounds__(kThreads) ef_topk_count_kernel(const float* __
         unsigned both = gt | (eq << 16);      // at most 512 elements per warp each: two 16-bit fields
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) both += __shfl_xor_sync(kFull, both, o);
-        if (lane == 0) { s_gt[warp] = both & 0xffffu; s_eq[warp] = both >> 16; }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            unsigned a = 0, b = 0;
-            for (int w = 0; w < kWarps; ++w) { a += s_gt[w]; b += s_eq[w]; }
-            cgt[c] = a;
-            ceq[c] = b;
-            if (a) atomicAdd(&tgt[c / kTileOfChunks], a);
-            if (b) atomicAdd(&teq[c / kTileOfChunks], b);
+        if (lane == 0) {
+            cgt[c * kWarps + warp] = both & 0xffffu;
+            ceq[c * kWarps + warp] = both >> 16;
+            if (both & 0xffffu) atomicAdd(&tgt[c / kTileOfChunks], both & 0xffffu);
+            if (both >> 16) atomicAdd(&teq[c / kTileOfChunks], both >> 16);
         }
-        __syncthreads();
     }
 }
 
@@ -569,18 +570,17 @@ __global__ void __launch_bounds__(kScanThreads) ef_topk_scan_kernel(const unsign
     }
 }
 
-// ---- 4. scatter: kept = key > T, or key == T and fewer than need_eq equal keys precede it
-// element order inside a chunk: warp, then row, then lane, then the lane's four elements.
-// Ranks come from per-lane counts (0..4 per row, the four rows packed into one word of four
-// 8-bit fields: a row of a warp has at most 128 kept elements) and one shuffle scan per warp.
-// A CTA handles kScatterChunks consecutive chunks, the next chunk's loads in flight while the
-// current one is ranked and written; its first rank is the tile's prefix plus the counts of the
-// tile's chunks before it.
+// ---- 4. scatter: kept = key > T, or key == T and fewer than need_eq equal keys precede it.
+// Element order inside a chunk: warp, then row, then lane, then the lane's four elements, i.e.
+// slice after slice.  A CTA handles kScatterChunks consecutive chunks; every warp walks its own
+// slices of them with the next slice's loads in flight, without any CTA barrier: the number of
+// kept keys before each slice is known up front from the per-slice counts (the tile's prefix,
+// the tile's slices before the CTA's, and a scan over the CTA's own 64 slices by its first warp).
 struct ScatterArgs {
     const float* v;
     long long n, chunks;
     const TopkState* st;
-    const unsigned* cgt;
+    const unsigned* cgt;               // per slice
     const unsigned* ceq;
     const unsigned long long* pgt;     // per tile
     const unsigned long long* peq;
@@ -590,16 +590,15 @@ struct ScatterArgs {
     unsigned long long kmax;
 };
 
-// One chunk, its elements in x/fin.  gt_run / eq_run: kept-candidate counts before the chunk
-// (advanced by the chunk's totals).  s_gt / s_eq: this chunk's buffer of per-warp totals.
-// Lane-rows without a key >= T keep nothing: their residual is the input, stored at once.  The
-// others are staged and handled densely: a first sweep counts, the CTA's warps exchange their
-// totals, a second sweep ranks, writes idx/val and stores the staged rows' residual.
+// One slice (this warp's 512 elements of chunk c), its elements in x/fin.  gt_base / eq_base: keys
+// > T and == T before the slice.  Lane-rows without a key >= T keep nothing: their residual is the
+// input, stored at once.  The others are staged in index order and handled one row per lane:
+// ranks are running counts from one shuffle scan per 32 staged rows.
 template <bool FULL>
-__device__ __forceinline__ void scatter_chunk(const ScatterArgs& a, long long c, unsigned T,
+__device__ __forceinline__ void scatter_slice(const ScatterArgs& a, long long c, unsigned T,
                                               unsigned long long need_eq, const float (&x)[kU][4],
-                                              unsigned fin, WarpStage& stage, unsigned* s_gt, unsigned* s_eq,
-                                              unsigned long long& gt_run, unsigned long long& eq_run) {
+                                              unsigned fin, WarpStage& stage,
+                                              unsigned long long gt_base, unsigned long long eq_base) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long wbase = c * kChunkLen + warp * (128 * kU);
     const int H = stage_rows<FULL>(x, fin, T, stage, lane);
@@ -619,31 +618,12 @@ __device__ __forceinline__ void scatter_chunk(const ScatterArgs& a, long long c,
                 for (int k = 0; k < 4; ++k) if ((nib >> k) & 1u) a.resid[base + k] = x[u][k];
         }
     }
-    // first sweep: this warp's numbers of keys > T and == T
-    unsigned both = 0u;                        // two 16-bit fields (at most 512 each)
-    for (int e = lane; e < H; e += 32) {
-        const uint4 q = stage.row[e];
-        const unsigned nib = FULL ? 0xfu : stage.tag[e] >> 8;
-        const unsigned key[4] = {q.x & 0x7fffffffu, q.y & 0x7fffffffu, q.z & 0x7fffffffu, q.w & 0x7fffffffu};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const bool in = (nib >> k) & 1u;
-            both += (in && key[k] > T ? 1u : 0u) + (in && key[k] == T ? 1u << 16 : 0u);
-        }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) both += __shfl_xor_sync(kFull, both, o);
-    if (lane == 0) { s_gt[warp] = both & 0xffffu; s_eq[warp] = both >> 16; }
-    __syncthreads();
-    unsigned long long gt_before = gt_run, eq_before = eq_run;
-    unsigned all_gt = 0u, all_eq = 0u;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-        if (w < warp) { gt_before += s_gt[w]; eq_before += s_eq[w]; }
-        all_gt += s_gt[w]; all_eq += s_eq[w];
-    }
-    gt_run += all_gt; eq_run += all_eq;
-    // second sweep: staged rows are in index order, so ranks are running counts
+    // position of a kept element = gt_rank + min(eq_rank, need_eq), split into a 64-bit part that
+    // is fixed for the slice and small local counts:
+    //   gt_base + min(eq_base, need_eq)  +  gt_local + min(eq_local, eq_room)
+    const unsigned long long pos_base = gt_base + (eq_base < need_eq ? eq_base : need_eq);
+    const unsigned eq_room = eq_base < need_eq ? (unsigned)min(need_eq - eq_base, 1024ull) : 0u;
+    unsigned gt_local = 0u, eq_local = 0u;     // staged keys > T / == T in the rows before this iteration
     for (int e0 = 0; e0 < H; e0 += 32) {
         const int e = e0 + lane;
         uint4 q = make_uint4(0u, 0u, 0u, 0u);
@@ -663,18 +643,17 @@ __device__ __forceinline__ void scatter_chunk(const ScatterArgs& a, long long c,
         const unsigned incl = warp_inclusive_scan32(cnt, lane);
         const unsigned tot = __shfl_sync(kFull, incl, 31);
         if (e < H) {
-            unsigned long long gt_rank = gt_before + ((incl - cnt) & 0xffffu);
-            unsigned long long eq_rank = eq_before + ((incl - cnt) >> 16);
+            unsigned gt_rank = gt_local + ((incl - cnt) & 0xffffu);
+            unsigned eq_rank = eq_local + ((incl - cnt) >> 16);
             const long long base = wbase + ((tag >> 5) & 3u) * 128 + (tag & 31u) * 4;
             const float xv[4] = {__uint_as_float(q.x), __uint_as_float(q.y), __uint_as_float(q.z), __uint_as_float(q.w)};
             float r[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 const bool is_eq = (feq >> k) & 1u, is_gt = (fgt >> k) & 1u;
-                const bool kept = is_gt || (is_eq && eq_rank < need_eq);
+                const bool kept = is_gt || (is_eq && eq_rank < eq_room);
                 if (kept) {
-                    // kept elements before this one = (keys > T before it) + min(equal keys before it, need_eq)
-                    const unsigned long long pos = gt_rank + (eq_rank < need_eq ? eq_rank : need_eq);
+                    const unsigned long long pos = pos_base + gt_rank + (eq_rank < eq_room ? eq_rank : eq_room);
                     if (pos < a.kmax) {        // always true when the counts are consistent
                         a.idx_out[pos] = base + k;
                         a.val_out[pos] = xv[k];
@@ -690,15 +669,16 @@ __device__ __forceinline__ void scatter_chunk(const ScatterArgs& a, long long c,
                     for (int k = 0; k < 4; ++k) if ((tag >> (8 + k)) & 1u) a.resid[base + k] = r[k];
             }
         }
-        gt_before += tot & 0xffffu;
-        eq_before += tot >> 16;
+        gt_local += tot & 0xffffu;
+        eq_local += tot >> 16;
     }
-    __syncwarp();                              // the staging area is rewritten by the next chunk
+    __syncwarp();                              // the staging area is rewritten by the next slice
 }
 
 __global__ void __launch_bounds__(kThreads, 3) ef_topk_scatter_kernel(const ScatterArgs a) {
-    __shared__ unsigned s_eq[2][kWarps], s_gt[2][kWarps];
-    __shared__ unsigned long long s_first[2];
+    constexpr int kSlices = kScatterChunks * kWarps;            // 64: two per lane of the first warp
+    static_assert(kSlices == 64, "the first warp scans two slices per lane");
+    __shared__ unsigned long long s_gt[kSlices], s_eq[kSlices]; // keys > T / == T before each slice of the CTA
     __shared__ WarpStage s_stage[kWarps];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long c0 = (long long)blockIdx.x * kScatterChunks;
@@ -706,31 +686,46 @@ __global__ void __launch_bounds__(kThreads, 3) ef_topk_scatter_kernel(const Scat
     float xA[kU][4], xB[kU][4];
     unsigned finA, finB = 0u;
     load_chunk_keys(a.v, a.n, c0, warp, lane, xA, finA);
-    // rank of the CTA's first element: the tile's prefix plus the tile's chunks before c0
     if (warp == 0) {
-        const long long tile = c0 / kTileOfChunks, first = tile * kTileOfChunks;
-        unsigned g = first + lane < c0 ? a.cgt[first + lane] : 0u;
-        unsigned e = first + lane < c0 ? a.ceq[first + lane] : 0u;
+        // before the CTA's first slice: the tile's prefix plus the tile's slices before it
+        const long long tile = c0 / kTileOfChunks, first = tile * kTileOfChunks * kWarps, mine = c0 * kWarps;
+        unsigned long long g = 0ull, e = 0ull;
+        for (long long i = first + lane; i < mine; i += 32) { g += a.cgt[i]; e += a.ceq[i]; }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             g += __shfl_xor_sync(kFull, g, o);
             e += __shfl_xor_sync(kFull, e, o);
         }
-        if (lane == 0) { s_first[0] = a.pgt[tile] + g; s_first[1] = a.peq[tile] + e; }
+        g += a.pgt[tile];
+        e += a.peq[tile];
+        // exclusive scan over the CTA's own slices, lane l holding slices 2l and 2l + 1
+        const long long last = a.chunks * kWarps;
+        const unsigned g0 = mine + 2 * lane < last ? a.cgt[mine + 2 * lane] : 0u;
+        const unsigned g1 = mine + 2 * lane + 1 < last ? a.cgt[mine + 2 * lane + 1] : 0u;
+        const unsigned e0 = mine + 2 * lane < last ? a.ceq[mine + 2 * lane] : 0u;
+        const unsigned e1 = mine + 2 * lane + 1 < last ? a.ceq[mine + 2 * lane + 1] : 0u;
+        const unsigned ig = warp_inclusive_scan32(g0 + g1, lane), ie = warp_inclusive_scan32(e0 + e1, lane);
+        s_gt[2 * lane] = g + (ig - g0 - g1);
+        s_gt[2 * lane + 1] = g + (ig - g1);
+        s_eq[2 * lane] = e + (ie - e0 - e1);
+        s_eq[2 * lane + 1] = e + (ie - e1);
     }
     const unsigned T = a.st->threshold;
     const unsigned long long need_eq = a.st->need_eq;
-    __syncthreads();
-    unsigned long long gt_run = s_first[0], eq_run = s_first[1];
+    __syncthreads();                           // the only barrier: from here on every warp runs for itself
     for (int j = 0; j < nch; j += 2) {
         if (j + 1 < nch) load_chunk_keys(a.v, a.n, c0 + j + 1, warp, lane, xB, finB);
-        // whole chunk or not: decided on the chunk, identically in every thread (the paths hold barriers)
-        if ((c0 + j + 1) * kChunkLen <= a.n) scatter_chunk<true>(a, c0 + j, T, need_eq, xA, finA, s_stage[warp], s_gt[0], s_eq[0], gt_run, eq_run);
-        else scatter_chunk<false>(a, c0 + j, T, need_eq, xA, finA, s_stage[warp], s_gt[0], s_eq[0], gt_run, eq_run);
+        // whole chunk or not: decided on the chunk, identically in every lane (the paths hold warp-wide operations)
+        if ((c0 + j + 1) * kChunkLen <= a.n)
+            scatter_slice<true>(a, c0 + j, T, need_eq, xA, finA, s_stage[warp], s_gt[j * kWarps + warp], s_eq[j * kWarps + warp]);
+        else
+            scatter_slice<false>(a, c0 + j, T, need_eq, xA, finA, s_stage[warp], s_gt[j * kWarps + warp], s_eq[j * kWarps + warp]);
         if (j + 1 < nch) {
             if (j + 2 < nch) load_chunk_keys(a.v, a.n, c0 + j + 2, warp, lane, xA, finA);
-            if ((c0 + j + 2) * kChunkLen <= a.n) scatter_chunk<true>(a, c0 + j + 1, T, need_eq, xB, finB, s_stage[warp], s_gt[1], s_eq[1], gt_run, eq_run);
-            else scatter_chunk<false>(a, c0 + j + 1, T, need_eq, xB, finB, s_stage[warp], s_gt[1], s_eq[1], gt_run, eq_run);
+            if ((c0 + j + 2) * kChunkLen <= a.n)
+                scatter_slice<true>(a, c0 + j + 1, T, need_eq, xB, finB, s_stage[warp], s_gt[(j + 1) * kWarps + warp], s_eq[(j + 1) * kWarps + warp]);
+            else
+                scatter_slice<false>(a, c0 + j + 1, T, need_eq, xB, finB, s_stage[warp], s_gt[(j + 1) * kWarps + warp], s_eq[(j + 1) * kWarps + warp]);
         }
     }
 }
@@ -783,7 +778,7 @@ int ef_topk_compress(const float* v, int64_t n, int64_t k, int64_t* idx_out, flo
     unsigned long long* seg_start = (unsigned long long*)(ws + L.off_seg_start);
     unsigned* seg_cnt = (unsigned*)(ws + L.off_seg_cnt);
     unsigned* cand = (unsigned*)(ws + L.off_cand);
-    if (cudaMemsetAsync(ws, 0, L.off_ceq, st) != cudaSuccess) return EF_ERR_CUDA;   // histograms, state, totals, sure counts
+    if (cudaMemsetAsync(ws, 0, L.off_cgt, st) != cudaSuccess) return EF_ERR_CUDA;   // histograms, state, tile totals
     const unsigned hgrid = (unsigned)std::min<long long>(L.chunks, 148 * 8);
     const unsigned cgrid = (unsigned)std::min<long long>(L.chunks, 148 * 3);       // three CTAs of 59 KB per SM
     const unsigned long long kk = (unsigned long long)k;
