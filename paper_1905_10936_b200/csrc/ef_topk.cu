@@ -12,15 +12,17 @@
 //         the count reaches k.  Keys above that bin are kept for sure, keys below never; only the
 //         keys IN the bin (the candidates, typically a few per cent of n) still matter.
 //      b. second pass over v: histogram of the second digit of the candidates, the number of
-//         sure keys per 4096-element chunk, and the candidates' keys copied to a compact list
-//         (one segment per warp and chunk; the order inside a segment is arbitrary and nothing
-//         depends on it).  The third digit is then histogrammed over the list, not over v.
+//         sure keys per slice (the 512 elements of a 4096-element chunk that one warp handles),
+//         and the candidates' keys copied to a compact list (one segment per slice; the order
+//         inside a segment is arbitrary and nothing depends on it).  The third digit is then
+//         histogrammed over the list, not over v.
 //      Result: T and how many keys equal to T have to be kept (need_eq).
-//   2. per chunk the number of keys > T and == T, from the chunk's sure count and its segment
-//      of the list (no pass over v);
-//   3. a scan of those counts over the chunks (one CTA);
-//   4. a scatter pass: every chunk recomputes its flags, ranks its kept elements in index order
-//      (a shuffle scan of per-lane counts, no sorting) and writes idx, val and the residual.
+//   2. per slice the number of keys > T and == T, from the slice's sure count and its segment
+//      of the list (no pass over v), and their totals per tile of 32 chunks;
+//   3. a scan of the tile totals (one CTA);
+//   4. a scatter pass: every warp recomputes the flags of its slices, ranks the kept elements in
+//      index order (a shuffle scan of per-lane counts, no sorting) and writes idx, val and the
+//      residual.
 // Traffic: three reads of v, one write of the residual, k index/value pairs: about 16 bytes per
 // element (the definition needs 8).  The list has room for n/8 candidates; when the bin holds
 // more (e.g. a vector whose magnitudes are all equal) steps 1b's list is skipped and the third
