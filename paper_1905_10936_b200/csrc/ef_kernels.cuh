@@ -759,8 +759,8 @@ constexpr int kServerStages = 2;
 
 // ---- bulk staging (TMA, 1-D): one elected thread copies a whole chunk of ptilde (16 KB) and
 // each worker's 128 packed words (512 B) into a shared-memory stage with cp.async.bulk and an
-// mbarrier that counts the bytes; the other threads only wait.  Never multicast, and only this
-// GPU's own memory is read.  Every wait is bounded: when the limit runs out the kernel records
+// mbarrier that counts the bytes; the other threads only wait.  Each copy has this CTA as its
+// only destination, and only this GPU's own memory is read.  Every wait is bounded: when the limit runs out the kernel records
 // kStatusWaitTimeout in the context's status word, waits (bounded again) for the copies it
 // still has in flight, and ends.
 constexpr unsigned kStatusWaitTimeout = 1u;
