@@ -93,6 +93,13 @@ enum ef_status {
                                       it did not shorten the launch-bound small layouts (results are
                                       identical either way). */
 
+#define EF_FLAG_SEPARATE_UPDATE 2048u /* On layouts of few chunks in which no block spans more than 16 chunks,
+                                      ef_server_step runs the server lines and the parameter update as ONE
+                                      kernel launched in thread-block clusters (a cluster per block; the
+                                      block's scale is agreed at the cluster barrier and every CTA updates
+                                      its own chunk of x); this flag keeps the two kernels every other
+                                      layout uses (for comparisons; results are identical). */
+
 /* Maximum number of simulated workers. */
 #define EF_MAX_WORKERS 4096
 

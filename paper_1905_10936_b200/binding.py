@@ -36,6 +36,7 @@ EF_FLAG_DIAGNOSTICS = 16
 EF_FLAG_ONE_LOCAL_WORKER = 32
 EF_FLAG_SERVER_NO_BULK = 512
 EF_FLAG_PROGRAMMATIC_LAUNCH = 1024
+EF_FLAG_SEPARATE_UPDATE = 2048
 EF_MAX_WORKERS = 4096
 EF_PROBE_3R2W, EF_PROBE_1R1W, EF_PROBE_COPY = 0, 1, 2
 

@@ -41,10 +41,11 @@ struct Layout {
     size_t dpad = 0, wpad = 0, bpad = 0, tpad = 0;    // padded element counts per sub-buffer
     size_t off_x = 0, off_m = 0, off_pb = 0, off_spb = 0, off_words = 0, off_scales = 0,
            off_rscale = 0, off_partials = 0, off_tickets = 0, off_tiles = 0, off_blocks = 0,
-           off_multi = 0, off_multi_big = 0, off_stage = 0, off_mt = 0, off_dpartials = 0,
+           off_multi = 0, off_multi_big = 0, off_ctiles = 0, off_stage = 0, off_mt = 0, off_dpartials = 0,
            off_diag = 0, off_status = 0, total = 0;
     int32_t num_multi = 0;                            // blocks that span more than one chunk
     int32_t num_multi_big = 0;                        // ... and more than kSelfScaleTiles tiles
+    int32_t num_ctiles = 0;                           // work items of the one-launch server call (0: not used)
 };
 
 }  // namespace efh
@@ -69,6 +70,7 @@ struct ef_ctx {
     std::vector<efk::Tile> h_tiles;             // kept alive: source of an asynchronous upload
     std::vector<efk::Block> h_blocks;
     std::vector<int32_t> h_multi, h_multi_big;
+    std::vector<efk::Tile> h_ctiles;            // cluster work items of the one-launch server call
     int fused = 0;                         // block scales finalised inside the main kernels
     // blocks cut across devices (ef_set_block_divisors): slot k's scales of the pieces are still
     // to be completed from the sum over all pieces (ef_complete_scales)
@@ -99,6 +101,7 @@ struct ef_ctx {
     const efk::Block* blocks() const { return (const efk::Block*)(ws + L.off_blocks); }
     const int* multi() const { return (const int*)(ws + L.off_multi); }
     const int* multi_big() const { return (const int*)(ws + L.off_multi_big); }
+    const efk::Tile* ctiles() const { return (const efk::Tile*)(ws + L.off_ctiles); }
     float* mt() const { return (float*)(ws + L.off_mt); }
     double* dpartials(int i) const { return (double*)(ws + L.off_dpartials) + (size_t)i * 3 * L.tpad; }
     double* diag(int i) const { return (double*)(ws + L.off_diag) + (size_t)i * 4 * L.bpad; }

@@ -822,7 +822,7 @@ template <int U, int MT, bool BULK>
 __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Tile& t, float sp,
                                                   unsigned char* ring, float* s_c, float* s_base,
                                                   float* s_lut, unsigned long long* full,
-                                                  unsigned& phase, bool* failed) {
+                                                  unsigned& phase, bool* failed, unsigned* signs = nullptr) {
     constexpr int kChunk = 1024 * U;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q = lane & 7;
@@ -928,6 +928,7 @@ __device__ __forceinline__ double server_tile_lut(const ServerArgs& a, const Til
                 p[u][k] = pv;
             }
             const unsigned nib = sign_nibble(p[u]);
+            if (signs) *signs |= nib << (4 * u);         // one-chunk tiles only: the caller keeps the signs
             acc += abs_sum4(p[u]);
             const unsigned word = pack_nibbles(nib, lane);
             store4(pp + u * 128, o, clen, full, p[u]);
@@ -1030,9 +1031,10 @@ __device__ __forceinline__ void average4(const ServerArgs& a, const float* s_c, 
     }
 }
 
+// signs (optional): bit 4u + k = sign bit of this thread's element k of row u.
 template <int U>
 __device__ __forceinline__ double server_rows(const ServerArgs& a, const Tile& t, float sp,
-                                              const float* s_c) {
+                                              const float* s_c, unsigned* signs = nullptr) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int o0 = warp * (128 * U) + lane * 4;
     const int sh = (lane & 7) * 4;
@@ -1054,6 +1056,7 @@ __device__ __forceinline__ double server_rows(const ServerArgs& a, const Tile& t
             p[u][k] = pv;
         }
         const unsigned nib = sign_nibble(p[u]);
+        if (signs) *signs |= nib << (4 * u);
         acc += abs_sum4(p[u]);
         const unsigned w = pack_nibbles(nib, lane);
         store4(pp + u * 128, o, t.len, full, p[u]);
@@ -1062,9 +1065,10 @@ __device__ __forceinline__ double server_rows(const ServerArgs& a, const Tile& t
     return acc;
 }
 
-// Any alignment, any M, any tile length.
+// Any alignment, any M, any tile length.  signs (optional): bit n = sign bit of the element this
+// thread handled in its n-th row (row warp + n * kWarps).
 __device__ __forceinline__ double server_rows_scalar(const ServerArgs& a, const Tile& t, float sp,
-                                                     const float* s_c) {
+                                                     const float* s_c, unsigned* signs = nullptr) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rows = (t.len + 31) >> 5;
     double acc = 0.0;
@@ -1085,6 +1089,7 @@ __device__ __forceinline__ double server_rows_scalar(const ServerArgs& a, const 
         }
         acc += (double)fabsf(pv);
         const unsigned w = __ballot_sync(kFull, valid && pv < 0.f);
+        if (signs) *signs |= ((w >> lane) & 1u) << ((r - warp) / kWarps);
         if (lane == 0) a.words[t.word + r] = w;
     }
     return acc;
@@ -1133,6 +1138,108 @@ __global__ void __launch_bounds__(kThreads) ef_server_kernel(const ServerArgs a)
     finish_block(acc, (long long)(blockIdx.x + a.tile0) * a.lim.tc, a.lim.tc - 1, b.len <= 1024 * U,
                  (unsigned)b.tile_count, t.block, a.blocks, a.partials, a.tickets, a.scale_out,
                  a.rscale, a.fused, a.lim.tc);
+}
+
+// ------------------------------------------------------------------ server lines + update, one launch
+// Layouts of few chunks are bound by the latency of their short kernels, not by memory.  When no
+// block spans more than kClusterCtas chunks, ef_server_step runs as ONE kernel launched in
+// thread-block clusters: a cluster owns one block (CTA r takes chunk r; the rest of the cluster
+// idles) or up to kClusterCtas single-chunk blocks.  A CTA keeps its chunk's sign bits and x values
+// in registers; the CTAs of a block publish their partial L1 sums, meet at the cluster barrier
+// (hardware, all CTAs of a cluster are co-scheduled: nothing polls memory), add the partial sums
+// in the usual fixed order -- every CTA for itself, so the scale has the same bits everywhere and
+// the same bits as in the two-kernel path -- and apply  x <- x - eta * stilde_b * sign(ptilde).
+constexpr int kClusterCtas = 16;
+constexpr int kClusterTileSync = 1;     // Tile::pad0 of a cluster work item: the cluster meets at its barrier
+
+struct ServerUpdateArgs {
+    ServerArgs s;          // plain inputs (the context's own worker words and scales), whole layout
+    const Tile* ctiles;    // one work item per CTA in cluster order: len 0 = idle, pad0 = flags,
+                           // pad1 = index of the tile in the ordinary tile table (its partial-sum slot)
+    float* x;
+    float eta;
+};
+
+__device__ __forceinline__ void cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+template <int U, int MT>
+__global__ void __launch_bounds__(kThreads) ef_server_update_kernel(const ServerUpdateArgs aa) {
+    extern __shared__ __align__(128) unsigned char s_dyn[];
+    float* s_c = reinterpret_cast<float*>(s_dyn + (MT > 0 ? server_ring_bytes<U>(MT, false) : 0));
+    __shared__ float s_base[(MT > 0 && !kUseWideLut(MT)) ? kLutEntries(MT) : 1];
+    __shared__ float s_lut[MT > 0 ? kLutFloats(MT, false) : 1];
+    __shared__ unsigned long long s_full[kServerStages];      // unused: the stages are filled per thread
+    __shared__ double s_sum[kWarps];
+    __shared__ float s_scale;
+    const ServerArgs& a = aa.s;
+    pdl_enter();
+    const Tile t = aa.ctiles[blockIdx.x];
+    const bool meet = (t.pad0 & kClusterTileSync) != 0;
+    // An idle CTA, or (checked build) one whose work item is refused, only keeps its appointment.
+    if (t.len <= 0 || !work_item_ok(t, a.lim, 1024 * U)) {
+        if (meet) cluster_barrier();
+        return;
+    }
+    const float sp = a.rscale[t.block];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool vec = (t.start & 3) == 0;
+    const bool full = t.len == 1024 * U;
+    const int o0 = warp * (128 * U) + lane * 4;
+    float x[U][4];
+    if (vec) {                                 // needed at the very end only: the loads overlap everything
+#pragma unroll
+        for (int u = 0; u < U; ++u) load4(aa.x + t.start + o0 + u * 128, o0 + u * 128, t.len, full, x[u]);
+    }
+    unsigned signs = 0u;
+    double acc;
+    if (MT > 0 && vec) {
+        unsigned phase = 0u;
+        bool failed = false;
+        acc = server_tile_lut<U, (MT > 0 ? MT : 1), false>(a, t, sp, s_dyn, s_c, s_base, s_lut, s_full, phase,
+                                                            &failed, &signs);
+    } else {
+        build_scaled(a, t, a.M, s_c);
+        __syncthreads();
+        acc = vec ? server_rows<U>(a, t, sp, s_c, &signs) : server_rows_scalar(a, t, sp, s_c, &signs);
+    }
+    const Block b = a.blocks[t.block];
+    double S = cta_sum(acc, s_sum);            // valid in thread 0
+    if (meet) {
+        if (threadIdx.x == 0) a.partials[t.pad1] = S;
+        cluster_barrier();                     // every CTA of the block has published its sum
+        S = sum_slots(b, a.partials, s_sum, 1);
+    }
+    if (threadIdx.x == 0) {
+        const float s = (float)(S / (double)b.div);
+        s_scale = s;
+        if (t.start == b.start) {              // the block's first chunk records the scale
+            a.scale_out[t.block] = s;
+            a.rscale[t.block] = s;             // every CTA of the block read the old one before the barrier
+        }
+    }
+    __syncthreads();
+    const float step = __fmul_rn(aa.eta, s_scale);
+    if (vec) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                x[u][k] = __fsub_rn(x[u][k], __uint_as_float(__float_as_uint(step) ^
+                                                             ((signs << (31 - 4 * u - k)) & 0x80000000u)));
+            store4(aa.x + t.start + o0 + u * 128, o0 + u * 128, t.len, full, x[u]);
+        }
+    } else {
+        const int rows = (t.len + 31) >> 5;
+        for (int r = warp, n = 0; r < rows; r += kWarps, ++n) {
+            const int o = r * 32 + lane;
+            if (o < t.len) {
+                const long long j = t.start + o;
+                aa.x[j] = __fsub_rn(aa.x[j], ((signs >> n) & 1u) ? -step : step);
+            }
+        }
+    }
 }
 
 // ------------------------------------------------------------------ parameter update

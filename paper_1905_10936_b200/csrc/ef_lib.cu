@@ -31,7 +31,7 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
     if (rc != EF_OK) return rc;
     if (flags & ~(EF_FLAG_HOST_STAGING | EF_FLAG_FUSED_SCALE | EF_FLAG_SPLIT_SCALE |
                   EF_FLAG_WEIGHT_DECAY | EF_FLAG_DIAGNOSTICS | EF_FLAG_ONE_LOCAL_WORKER |
-                  EF_FLAG_SERVER_NO_BULK | EF_FLAG_PROGRAMMATIC_LAUNCH))
+                  EF_FLAG_SERVER_NO_BULK | EF_FLAG_PROGRAMMATIC_LAUNCH | EF_FLAG_SEPARATE_UPDATE))
         return EF_ERR_INVALID_ARG;
     if ((flags & EF_FLAG_FUSED_SCALE) && (flags & (EF_FLAG_SPLIT_SCALE | EF_FLAG_DIAGNOSTICS)))
         return EF_ERR_INVALID_ARG;
@@ -49,12 +49,20 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
     // kTileChunks chunks.
     L->tile_chunks = (chunks <= kFusedMaxChunks) ? 1 : efk::kTileChunks;
     const int64_t tile_len = (int64_t)kChunkLen * L->tile_chunks;
-    int64_t T = 0;
+    int64_t T = 0, most = 0, single = 0;
     for (int32_t b = 0; b < B; ++b) {
         const int64_t tiles_b = (offsets[b + 1] - offsets[b] + tile_len - 1) / tile_len;
         T += tiles_b;
+        most = std::max(most, tiles_b);
+        single += tiles_b == 1;
         if (tiles_b > kSelfScaleTiles) L->num_multi_big += 1;
     }
+    // One-launch server call (clusters): few chunks, all workers local, no block beyond one cluster.
+    // A cluster per multi-chunk block, single-chunk blocks share clusters.
+    if (L->tile_chunks == 1 && L->Ml == M && most <= efk::kClusterCtas &&
+        !(flags & (EF_FLAG_SEPARATE_UPDATE | EF_FLAG_SPLIT_SCALE | EF_FLAG_DIAGNOSTICS)))
+        L->num_ctiles = (int32_t)(efk::kClusterCtas *
+                                  ((B - single) + (single + efk::kClusterCtas - 1) / efk::kClusterCtas));
     if (T * L->tile_chunks > 0x7fffffffLL) return EF_ERR_INVALID_ARG;
     L->W = W; L->num_tiles = T;
     L->dpad = align_up((size_t)d * 4) / 4;
@@ -79,6 +87,7 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
     L->off_blocks = o;   o += align_up((size_t)B * sizeof(Block));
     L->off_multi = o;    o += align_up((size_t)L->num_multi * sizeof(int32_t) + 4);
     L->off_multi_big = o; o += align_up((size_t)L->num_multi_big * sizeof(int32_t) + 4);
+    L->off_ctiles = o;   o += align_up((size_t)L->num_ctiles * sizeof(Tile));
     L->off_status = o;   o += kAlign;
     L->off_stage = o;
     if (flags & EF_FLAG_HOST_STAGING) o += 2 * L->dpad * 4;
@@ -179,6 +188,53 @@ cudaError_t prepare_server(int M) {
     }
 }
 
+// The one-launch server call: clusters of kClusterCtas CTAs need the kernel's opt-in (above 8),
+// and its staging ring may need a raised dynamic shared-memory limit.
+template <int MT>
+cudaError_t prepare_server_update_t(int M) {
+    auto kernel = efk::ef_server_update_kernel<kU, MT>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (e != cudaSuccess) return e;
+    const size_t smem = server_smem_bytes<MT>(M, false);
+    if (smem <= 16 * 1024) return cudaSuccess;
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+}
+
+template <int MT>
+cudaError_t launch_server_update_t(ef_ctx* c, const efk::ServerUpdateArgs& aa) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)c->L.num_ctiles);
+    cfg.blockDim = dim3(efk::kThreads);
+    cfg.dynamicSmemBytes = server_smem_bytes<MT>(c->L.M, false);
+    cfg.stream = c->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = efk::kClusterCtas;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, efk::ef_server_update_kernel<kU, MT>, aa);
+}
+
+#define EF_FOR_WORKER_COUNT(M, CALL)                                                           \
+    switch (M) {                                                                               \
+        case 1: CALL(1); break;   case 2: CALL(2); break;   case 3: CALL(3); break;            \
+        case 4: CALL(4); break;   case 5: CALL(5); break;   case 6: CALL(6); break;            \
+        case 7: CALL(7); break;   case 8: CALL(8); break;   case 9: CALL(9); break;            \
+        case 10: CALL(10); break; case 11: CALL(11); break; case 12: CALL(12); break;          \
+        case 13: CALL(13); break; case 14: CALL(14); break; case 15: CALL(15); break;          \
+        case 16: CALL(16); break; default: CALL(0); break;                                     \
+    }
+
+cudaError_t prepare_server_update(int M) {
+    cudaError_t e = cudaSuccess;
+#define EF_CALL(MT) e = prepare_server_update_t<MT>(M)
+    EF_FOR_WORKER_COUNT(M, EF_CALL)
+#undef EF_CALL
+    return e;
+}
+
 // Range of tiles that covers the blocks [b0, b1).
 struct TileRange { int tile0; unsigned count; };
 TileRange tiles_of(const ef_ctx* c, int b0, int b1) {
@@ -202,10 +258,8 @@ cudaError_t launch_server_t(ef_ctx* c, const efk::ServerArgs& a, unsigned grid, 
 // starts at msgs + i * msg_stride.
 // defer_scales: the caller applies the update right away with launch_apply_range(.., self_scale):
 // only the blocks too large for that get their scale from ef_scale_kernel here.
-int launch_server_range(ef_ctx* c, int b0, int b1, const uint32_t* msgs, long long msg_stride,
-                        bool defer_scales = false) {
+efk::ServerArgs server_args(ef_ctx* c, int b0, int tile0, const uint32_t* msgs, long long msg_stride) {
     const int M = c->L.M, S = c->srv();
-    const TileRange tr = tiles_of(c, b0, b1);
     efk::ServerArgs a;
     a.wwords = msgs ? msgs : c->words(0);
     a.wstride = msgs ? msg_stride : (long long)c->L.wpad;
@@ -214,11 +268,19 @@ int launch_server_range(ef_ctx* c, int b0, int b1, const uint32_t* msgs, long lo
     a.partials = c->partials(S); a.tickets = c->tickets(S);
     a.tiles = c->tiles(); a.blocks = c->blocks(); a.fused = c->fused;
     a.ratio = c->eta_prev / c->eta;
-    a.tile0 = tr.tile0;
+    a.tile0 = tile0;
     a.fused_in = msgs ? 1 : 0;
     a.msg_base = efk::message_unit(c->h_blocks[b0].word, b0);
     a.status = c->status();
     a.lim = c->limits();
+    return a;
+}
+
+int launch_server_range(ef_ctx* c, int b0, int b1, const uint32_t* msgs, long long msg_stride,
+                        bool defer_scales = false) {
+    const int M = c->L.M, S = c->srv();
+    const TileRange tr = tiles_of(c, b0, b1);
+    const efk::ServerArgs a = server_args(c, b0, tr.tile0, msgs, msg_stride);
     // bulk staging needs every chunk's packed words on a 16-byte boundary: plain layout only
     const bool bulk = c->use_bulk && !msgs;
     cudaError_t le;
@@ -286,7 +348,24 @@ int launch_apply_range(ef_ctx* c, int b0, int b1, const uint32_t* update, bool s
     return EF_OK;
 }
 
+// Few chunks, no block beyond one cluster: server lines and update in one launch.
+int launch_server_update(ef_ctx* c) {
+    efk::ServerUpdateArgs aa;
+    aa.s = server_args(c, 0, 0, nullptr, 0);
+    aa.ctiles = c->ctiles();
+    aa.x = c->x();
+    aa.eta = c->eta;
+    cudaError_t e = cudaSuccess;
+#define EF_CALL(MT) e = launch_server_update_t<MT>(c, aa)
+    EF_FOR_WORKER_COUNT(c->L.M, EF_CALL)
+#undef EF_CALL
+    EF_CUDA(c, e);
+    c->launches += 1;
+    return EF_OK;
+}
+
 int launch_server(ef_ctx* c) {
+    if (c->L.num_ctiles > 0 && c->lambda == 0.f) return launch_server_update(c);
     // Large layouts: the update kernel completes the scales of all but the largest blocks itself.
     const bool self_scale = !c->fused;
     const int rc = launch_server_range(c, 0, c->L.B, nullptr, 0, self_scale);
@@ -370,6 +449,31 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
         if (blk.tile_count > kSelfScaleTiles) c->h_multi_big.push_back(b);
         word += (len + 31) / 32;
     }
+    if (L.num_ctiles > 0) {
+        // cluster work items: a cluster per multi-chunk block (CTA r takes its r-th chunk and the
+        // cluster meets at its barrier), then the single-chunk blocks, kClusterCtas to a cluster
+        const Tile idle = {0, 0, 0, 0, 0, 0};
+        for (int32_t b = 0; b < B; ++b) {
+            const Block& blk = c->h_blocks[b];
+            if (blk.tile_count == 1) continue;
+            for (int r = 0; r < efk::kClusterCtas; ++r) {
+                Tile t = idle;
+                if (r < blk.tile_count) { t = c->h_tiles[blk.tile_begin + r]; t.pad1 = blk.tile_begin + r; }
+                t.block = b;
+                t.pad0 = efk::kClusterTileSync;
+                c->h_ctiles.push_back(t);
+            }
+        }
+        for (int32_t b = 0; b < B; ++b) {
+            const Block& blk = c->h_blocks[b];
+            if (blk.tile_count != 1) continue;
+            Tile t = c->h_tiles[blk.tile_begin];
+            t.pad1 = blk.tile_begin;
+            c->h_ctiles.push_back(t);
+        }
+        while (c->h_ctiles.size() % efk::kClusterCtas != 0) c->h_ctiles.push_back(idle);
+        if ((int64_t)c->h_ctiles.size() != L.num_ctiles) { delete c; return EF_ERR_INVALID_ARG; }
+    }
     } catch (const std::bad_alloc&) {
         delete c;
         return EF_ERR_NO_MEMORY;
@@ -398,7 +502,11 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
         (ce = cudaMemcpyAsync(c->ws + L.off_multi_big, c->h_multi_big.data(),
                               c->h_multi_big.size() * sizeof(int32_t), cudaMemcpyHostToDevice,
                               c->stream)) != cudaSuccess) return fail(ce);
+    if (!c->h_ctiles.empty() &&
+        (ce = cudaMemcpyAsync(c->ws + L.off_ctiles, c->h_ctiles.data(), c->h_ctiles.size() * sizeof(Tile),
+                              cudaMemcpyHostToDevice, c->stream)) != cudaSuccess) return fail(ce);
     if ((ce = prepare_server(M)) != cudaSuccess) return fail(ce);
+    if (L.num_ctiles > 0 && (ce = prepare_server_update(M)) != cudaSuccess) return fail(ce);
     {
         // bulk staging: every block but the last must hold a multiple of 128 elements (so that
         // every chunk's 128 packed words start on a 16-byte boundary) and start 16-byte aligned

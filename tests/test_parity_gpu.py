@@ -599,7 +599,7 @@ def test_error_paths_on_device():
     assert ei.value.status == ef.EF_ERR_BAD_STATE          # in the middle of an iteration
     ef.ef_worker_step(e.ctx, 0, g.data_ptr())
     ef.ef_server_step(e.ctx)
-    assert e.step_count == 1 and e.launch_count == 4      # 2 worker + server + apply kernels
+    assert e.step_count == 1 and e.launch_count == 3      # 2 worker kernels + the one-launch server call
     ws = torch.empty(1024, dtype=torch.uint8, device="cuda")
     with pytest.raises(ef.EFError) as ei:
         ef.ef_init(w.d, w.B, w.offsets, w.M, 0.9, 0.1, 0, ws.data_ptr(), 1024, 0)
