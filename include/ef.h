@@ -89,10 +89,14 @@ enum ef_status {
                                       results are identical). */
 #define EF_FLAG_PROGRAMMATIC_LAUNCH 1024u /* Launch the kernels with programmatic stream serialization: each
                                       may be scheduled while its predecessor on the stream drains and waits
-                                      on the device for the predecessor's results.  Off by default: on B200
-                                      it did not shorten the launch-bound small layouts (results are
-                                      identical either way). */
-
+                                      on the device for the predecessor's results; the worker kernel loads
+                                      the worker's own state, and the one-launch server kernel its x values,
+                                      before that wait.  On B200 this shortens the launch-bound layouts whose
+                                      worker launch is a single wave of CTAs (flat 2^20, M = 2: 16.4 -> 14.5 us
+                                      per step from a CUDA graph) and does nothing for the others, so it is
+                                      off by default.  Results are identical.  While it is on, kernels of the
+                                      caller that write x or a worker's state through the raw pointers
+                                      directly before a call must not signal programmatic completion early. */
 #define EF_FLAG_SEPARATE_UPDATE 2048u /* On layouts of few chunks in which no block spans more than 16 chunks,
                                       ef_server_step runs the server lines and the parameter update as ONE
                                       kernel launched in thread-block clusters (a cluster per block; the

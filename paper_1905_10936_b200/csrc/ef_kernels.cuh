@@ -221,15 +221,29 @@ struct ResidualArgs {
 };
 
 // ------------------------------------------------------------------ programmatic dependent launch
-// Every kernel of the library starts with pdl_enter(): it waits until the kernel launched before
-// it on the stream has completed and its writes are visible (a no-op for an ordinary launch),
-// then lets the kernel launched after it be scheduled as soon as SM resources free up.  With the
-// launch attribute set on the host side this overlaps each kernel's launch latency and ramp-up
-// with its predecessor's tail; the data dependence is still enforced by the wait, so nothing
-// may touch global memory before pdl_enter().
+// pdl_wait(): until the kernel launched before this one on the stream has completed and its
+// writes are visible (a no-op for an ordinary launch).  pdl_trigger(): the kernel launched after
+// this one may be scheduled as soon as SM resources free up.  With the launch attribute set on
+// the host side (EF_FLAG_PROGRAMMATIC_LAUNCH) this overlaps a kernel's launch latency, its
+// descriptor loads and whatever else it may do before its wait with the predecessor's tail.
+//
+// Most kernels start with pdl_enter() = wait, then trigger: nothing of theirs touches global
+// memory before the predecessor is complete.  Two kernels do part of their work BEFORE the wait:
+//  * the worker kernel loads its descriptors and the worker's own state (m_i, the deferred
+//    residual and its scales) first; the gradient and every store come after the wait;
+//  * the one-launch server kernel loads its work item and its x values first.
+// That is safe as long as the kernel directly before them does not write what they read early
+// while having triggered early itself.  Inside the library the only writers of a worker's state
+// that can directly precede that worker's step are the state import and the completion of cut
+// blocks' scales: those two wait and never trigger (their dependents start when they are done).
+// x is written by the update kernels, and a server call is always preceded by worker kernels.
+// Kernels of the caller that write x or worker state through the raw pointers must not signal
+// early either when this mode is on.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_enter() {
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    pdl_wait();
+    pdl_trigger();
 }
 
 // ------------------------------------------------------------------ small helpers
@@ -482,10 +496,13 @@ __device__ __forceinline__ double worker_rows(const WorkerArgs& a, const Tile& t
     float g[U][4], m[U][4], p[U][4];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-        load4(gp + u * 128, o0 + u * 128, t.len, FULL, g[u]);
         load4(mp + u * 128, o0 + u * 128, t.len, FULL, m[u]);
         load4(pp + u * 128, o0 + u * 128, t.len, FULL, p[u]);
     }
+    // the worker's own state is in flight; the gradient (the caller's) and all stores follow the wait
+    pdl_wait();
+#pragma unroll
+    for (int u = 0; u < U; ++u) load4(gp + u * 128, o0 + u * 128, t.len, FULL, g[u]);
     double acc = 0.0;
     const bool rescale = a.ratio != 1.0f;
 #pragma unroll
@@ -534,6 +551,7 @@ __device__ __forceinline__ double worker_rows_scalar(const WorkerArgs& a, const 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rows = (t.len + 31) >> 5;
     double acc = 0.0;
+    pdl_wait();
     for (int r = warp; r < rows; r += kWarps) {
         const int o = r * 32 + lane;
         const bool valid = o < t.len;
@@ -563,7 +581,7 @@ __device__ __forceinline__ double worker_rows_scalar(const WorkerArgs& a, const 
 // grid.x = chunks, grid.y = workers stepped by this launch (1 for ef_worker_step).
 template <int U, bool DIAG>
 __global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a0) {
-    pdl_enter();
+    pdl_trigger();
     WorkerArgs a = a0;
     {
         const long long wi = blockIdx.y;
@@ -589,6 +607,7 @@ __global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a0
     if (a.push) a.words = a.push[t.block] + 1 - b.word;
     double acc = 0.0;
     DiagAcc dacc;
+    if (t.len <= 0) pdl_wait();
     if (t.len > 0) {
         const float sp = a.rscale[t.block];
         if ((t.start & 3) != 0)
@@ -1174,11 +1193,12 @@ __global__ void __launch_bounds__(kThreads) ef_server_update_kernel(const Server
     __shared__ double s_sum[kWarps];
     __shared__ float s_scale;
     const ServerArgs& a = aa.s;
-    pdl_enter();
+    pdl_trigger();
     const Tile t = aa.ctiles[blockIdx.x];
     const bool meet = (t.pad0 & kClusterTileSync) != 0;
     // An idle CTA, or (checked build) one whose work item is refused, only keeps its appointment.
     if (t.len <= 0 || !work_item_ok(t, a.lim, 1024 * U)) {
+        pdl_wait();
         if (meet) cluster_barrier();
         return;
     }
@@ -1192,6 +1212,7 @@ __global__ void __launch_bounds__(kThreads) ef_server_update_kernel(const Server
 #pragma unroll
         for (int u = 0; u < U; ++u) load4(aa.x + t.start + o0 + u * 128, o0 + u * 128, t.len, full, x[u]);
     }
+    pdl_wait();
     unsigned signs = 0u;
     double acc;
     if (MT > 0 && vec) {
@@ -1420,7 +1441,7 @@ static __global__ void __launch_bounds__(kThreads) ef_complete_scales_kernel(con
                                                                              const double* __restrict__ totals,
                                                                              int B, float* __restrict__ scale_out,
                                                                              float* __restrict__ rscale) {
-    pdl_enter();
+    pdl_wait();                        // writes a worker's scales: no early trigger (see pdl_wait above)
     const int b = blockIdx.x * kThreads + threadIdx.x;
     if (b < B && blocks[b].partial) {
         const float s = (float)(totals[b] / (double)blocks[b].div);
@@ -1433,7 +1454,7 @@ static __global__ void __launch_bounds__(kThreads) ef_complete_scales_kernel(con
 // keeps the "no -0 in a residual buffer" invariant of the sign-bit tests above.
 static __global__ void __launch_bounds__(kThreads) ef_import_kernel(const float* __restrict__ src,
                                                              float* __restrict__ dst, long long n) {
-    pdl_enter();
+    pdl_wait();                        // writes a worker's state: no early trigger (see pdl_wait above)
     for (long long j = blockIdx.x * (long long)kThreads + threadIdx.x; j < n;
          j += (long long)gridDim.x * kThreads)
         dst[j] = __fadd_rn(src[j], 0.0f);

@@ -212,8 +212,12 @@ cudaError_t launch_server_update_t(ef_ctx* c, const efk::ServerUpdateArgs& aa) {
     attr[0].val.clusterDim.x = efk::kClusterCtas;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cudaLaunchAttribute attr2[2];
+    attr2[0] = attr[0];
+    attr2[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr2[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr2;
+    cfg.numAttrs = c->pdl ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, efk::ef_server_update_kernel<kU, MT>, aa);
 }
 
@@ -839,6 +843,14 @@ int ef_debug_shift_tile(ef_ctx* c, int64_t tile, int64_t delta) {
     c->h_tiles[(size_t)tile].start += delta;
     EF_CUDA(c, cudaMemcpyAsync(c->ws + c->L.off_tiles + (size_t)tile * sizeof(Tile), &c->h_tiles[(size_t)tile],
                                sizeof(Tile), cudaMemcpyHostToDevice, c->stream));
+    // the same tile among the work items of the one-launch server call
+    for (size_t k = 0; k < c->h_ctiles.size(); ++k) {
+        Tile& ct = c->h_ctiles[k];
+        if (ct.len <= 0 || ct.pad1 != (int)tile) continue;
+        ct.start += delta;
+        EF_CUDA(c, cudaMemcpyAsync(c->ws + c->L.off_ctiles + k * sizeof(Tile), &ct, sizeof(Tile),
+                                   cudaMemcpyHostToDevice, c->stream));
+    }
     return EF_OK;
 #else
     (void)c; (void)tile; (void)delta;

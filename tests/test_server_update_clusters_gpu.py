@@ -100,3 +100,42 @@ def test_one_launch_replays_from_a_cuda_graph():
     # one eager step and three replays (the capture itself runs nothing) leave what four eager steps leave
     assert torch.equal(ga.params(), b.params())
     assert torch.equal(ga.residual(-1), b.residual(-1))
+
+
+@pytest.mark.parametrize("sizes,M", [([65536] * 16, 2), ([3 * CH + 5, 640, 10, 16 * CH, 333, 9 * CH + 1], 7)])
+def test_programmatic_launches_change_nothing(sizes, M):
+    """With EF_FLAG_PROGRAMMATIC_LAUNCH the worker kernel loads the worker's state, and the
+    one-launch server kernel its x values, before they wait for the kernel ahead of them.  State
+    imports (ef_set_state) directly before a step, steps back to back and a parameter overwrite by
+    a torch kernel in between must give what ordinary launches give."""
+    w = _wl(sizes, M, steps=6, cid=421)
+    pdl = EFEngine(w.offsets, M, w.mu, w.eta, extra_flags=ef.EF_FLAG_PROGRAMMATIC_LAUNCH)
+    ref = EFEngine(w.offsets, M, w.mu, w.eta, extra_flags=ef.EF_FLAG_SEPARATE_UPDATE)
+    es = w.element_scales("cuda")
+    gen = torch.Generator("cuda").manual_seed(5)
+    for t in range(w.steps):
+        stride = (w.d + 3) // 4 * 4                        # rows start on 16-byte boundaries
+        grads = torch.zeros(M, stride, device="cuda")
+        for i in range(M):
+            w.draw_grad(t, i, "cuda", es, out=grads[i, :w.d])
+        if t == 2:                                         # imported state, used by the very next kernel
+            m = torch.randn(w.d, device="cuda", generator=gen)
+            e = torch.randn(w.d, device="cuda", generator=gen) * 1e-2
+            for eng in (pdl, ref):
+                for i in range(M):
+                    eng.set_state(i, m, e)
+        if t == 4:
+            for eng in (pdl, ref):
+                eng.params().mul_(0.5)
+        for eng in (pdl, ref):
+            if t % 2:
+                eng.worker_step_all(grads)
+            else:
+                for i in range(M):
+                    eng.worker_step(i, grads[i, :w.d])
+            eng.server_step()
+        assert torch.equal(pdl.params(), ref.params()), f"x after step {t}"
+        assert torch.equal(pdl.server_words(), ref.server_words())
+        for i in range(M):
+            assert torch.equal(pdl.momentum(i), ref.momentum(i))
+            assert torch.equal(pdl.residual(i), ref.residual(i))
