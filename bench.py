@@ -383,7 +383,7 @@ def run_ours(args) -> None:
 
     # ---- end to end: host gradients in, packed update out, copies inside the timed region
     e2e = None
-    if not args.no_e2e and not signum:
+    if not args.no_e2e:
         hsrc = galls[0]
         del eng
         torch.cuda.empty_cache()
@@ -399,8 +399,8 @@ def run_ours(args) -> None:
 
         def e2e_step():
             for i in range(w.M):
-                eng2.worker_step_host(i, hgrads[i])
-            eng2.server_step()
+                (eng2.vote_worker_step_host if signum else eng2.worker_step_host)(i, hgrads[i])
+            (eng2.vote_server_step if signum else eng2.server_step)()
             eng2.read_update_host(hwords, hscales)
 
         for _ in range(2):
@@ -419,8 +419,10 @@ def run_ours(args) -> None:
                "h2d_bytes_per_step": int(w.M * w.d * 4),
                "d2h_bytes_per_step": int(eng2.W * 4 + eng2.B * 4),
                "steps": Ke, "ms_per_step": e2e_ms / Ke, "wall_ms_per_step": wall_ms / Ke,
-               "note": "pinned host gradients -> ef_worker_step_host (double-buffered H2D on a "
-                       "copy stream) -> ef_server_step -> ef_read_update_host; PCIe-bound"}
+               "note": ("pinned host gradients -> ef_vote_worker_step_host (double-buffered H2D on a copy "
+                        "stream) -> ef_vote_server_step -> ef_read_update_host; PCIe-bound" if signum else
+                        "pinned host gradients -> ef_worker_step_host (double-buffered H2D on a "
+                        "copy stream) -> ef_server_step -> ef_read_update_host; PCIe-bound")}
         del eng2, hgrads
 
     if rank != 0:

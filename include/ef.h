@@ -355,6 +355,10 @@ int ef_complete_scales(ef_ctx* ctx, int32_t who, const double* totals /* device,
  * ef_init / ef_set_eta; weight decay does not apply to this method. */
 int ef_vote_worker_step(ef_ctx* ctx, int32_t i, const float* grad /* device */);
 int ef_vote_worker_step_all(ef_ctx* ctx, const float* grads /* device, M gradients */, int64_t stride);
+/* As ef_worker_step_host: grad is a HOST buffer (pinned for an asynchronous copy), staged through
+ * the context's two staging buffers (EF_FLAG_HOST_STAGING, else BAD_STATE).  The voted signs are
+ * read back with ef_read_update_host (its scales output is not meaningful for this method). */
+int ef_vote_worker_step_host(ef_ctx* ctx, int32_t i, const float* grad /* host */);
 int ef_vote_server_step(ef_ctx* ctx);
 
 /* ---- top-k: the second example of a delta-approximate compressor after Definition 1

@@ -84,6 +84,7 @@ SIGNATURES = {
     "ef_complete_scales": (ctypes.c_int, [_vp, _i32, _vp]),
     "ef_vote_worker_step": (ctypes.c_int, [_vp, _i32, _vp]),
     "ef_vote_worker_step_all": (ctypes.c_int, [_vp, _vp, _i64]),
+    "ef_vote_worker_step_host": (ctypes.c_int, [_vp, _i32, _vp]),
     "ef_vote_server_step": (ctypes.c_int, [_vp]),
     "ef_topk_workspace_bytes": (ctypes.c_int, [_i64, ctypes.POINTER(ctypes.c_size_t)]),
     "ef_topk_compress": (ctypes.c_int, [_vp, _i64, _i64, _vp, _vp, _vp, _vp, ctypes.c_size_t, _vp]),
@@ -310,6 +311,10 @@ def ef_vote_worker_step(ctx: int, i: int, grad_ptr: int) -> None:
 
 def ef_vote_worker_step_all(ctx: int, grads_ptr: int, stride: int) -> None:
     _check(load_library().ef_vote_worker_step_all(ctx, grads_ptr, stride), "ef_vote_worker_step_all")
+
+
+def ef_vote_worker_step_host(ctx: int, i: int, grad_host_ptr: int) -> None:
+    _check(load_library().ef_vote_worker_step_host(ctx, i, grad_host_ptr), "ef_vote_worker_step_host")
 
 
 def ef_vote_server_step(ctx: int) -> None:

@@ -173,6 +173,27 @@ inline void mark_all_stepped(ef_ctx* c, int mode) {
     for (auto& v : c->stepped) v = 1;
     c->pending = c->L.Ml; c->mode = mode;
 }
+// Host gradients (EF_FLAG_HOST_STAGING): the copy into one of the two staging buffers runs on
+// the copy stream, the step kernel on the context's stream waits for it, and a buffer is reused
+// only after the kernel that last read it.  stage_host_gradient enqueues copy and wait and
+// returns the buffer; host_gradient_consumed is called after the kernel has been enqueued.
+inline int stage_host_gradient(ef_ctx* c, const float* grad, float** staged) {
+    const int s = (int)(c->host_calls & 1);
+    if (c->host_calls >= 2) EF_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->ev_free[s], 0));
+    EF_CUDA(c, cudaMemcpyAsync(c->stage(s), grad, (size_t)c->L.d * 4, cudaMemcpyHostToDevice,
+                               c->copy_stream));
+    EF_CUDA(c, cudaEventRecord(c->ev_copied[s], c->copy_stream));
+    EF_CUDA(c, cudaStreamWaitEvent(c->stream, c->ev_copied[s], 0));
+    *staged = c->stage(s);
+    return EF_OK;
+}
+inline int host_gradient_consumed(ef_ctx* c) {
+    const int s = (int)(c->host_calls & 1);
+    EF_CUDA(c, cudaEventRecord(c->ev_free[s], c->stream));
+    c->host_calls += 1;
+    return EF_OK;
+}
+
 inline void end_iteration(ef_ctx* c) {
     for (auto& v : c->stepped) v = 0;
     for (auto& v : c->served) v = 0;

@@ -579,17 +579,13 @@ int ef_worker_step_host(ef_ctx* c, int32_t i, const float* grad) {
     int rc = check_worker_call(c, i, grad, kModeEF);
     if (rc != EF_OK) return rc;
     if (!(c->flags & EF_FLAG_HOST_STAGING) || c->scales_open[i]) return EF_ERR_BAD_STATE;
-    const int s = (int)(c->host_calls & 1);
-    // the staging slot is free once the kernel that last read it has finished
-    if (c->host_calls >= 2) EF_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->ev_free[s], 0));
-    EF_CUDA(c, cudaMemcpyAsync(c->stage(s), grad, (size_t)c->L.d * 4, cudaMemcpyHostToDevice,
-                               c->copy_stream));
-    EF_CUDA(c, cudaEventRecord(c->ev_copied[s], c->copy_stream));
-    EF_CUDA(c, cudaStreamWaitEvent(c->stream, c->ev_copied[s], 0));
-    rc = launch_worker(c, i, c->stage(s));
+    float* staged = nullptr;
+    rc = stage_host_gradient(c, grad, &staged);
     if (rc != EF_OK) return rc;
-    EF_CUDA(c, cudaEventRecord(c->ev_free[s], c->stream));
-    c->host_calls += 1;
+    rc = launch_worker(c, i, staged);
+    if (rc != EF_OK) return rc;
+    rc = host_gradient_consumed(c);
+    if (rc != EF_OK) return rc;
     mark_stepped(c, i, kModeEF);
     if (c->has_partial) c->scales_open[i] = 1;
     return EF_OK;

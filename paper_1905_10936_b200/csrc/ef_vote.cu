@@ -319,6 +319,22 @@ int ef_vote_worker_step(ef_ctx* c, int32_t i, const float* grad) {
     return EF_OK;
 }
 
+int ef_vote_worker_step_host(ef_ctx* c, int32_t i, const float* grad) {
+    EF_API_RANGE();
+    int rc = check_worker_call(c, i, grad, kModeVote);
+    if (rc != EF_OK) return rc;
+    if (!(c->flags & EF_FLAG_HOST_STAGING)) return EF_ERR_BAD_STATE;
+    float* staged = nullptr;
+    rc = stage_host_gradient(c, grad, &staged);
+    if (rc != EF_OK) return rc;
+    rc = launch_vote_worker(c, i, staged, 1, 0);
+    if (rc != EF_OK) return rc;
+    rc = host_gradient_consumed(c);
+    if (rc != EF_OK) return rc;
+    mark_stepped(c, i, kModeVote);
+    return EF_OK;
+}
+
 int ef_vote_worker_step_all(ef_ctx* c, const float* grads, int64_t stride) {
     EF_API_RANGE();
     if (!c || !grads || stride < c->L.d) return EF_ERR_INVALID_ARG;

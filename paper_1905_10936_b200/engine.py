@@ -151,6 +151,11 @@ class EFEngine:
         assert grads.shape[0] == self.M and grads.shape[1] >= self.d and grads.stride(1) == 1
         ef.ef_vote_worker_step_all(self.ctx, grads.data_ptr(), grads.stride(0))
 
+    def vote_worker_step_host(self, i: int, grad: torch.Tensor) -> None:
+        assert (not grad.is_cuda) and grad.dtype == torch.float32 and grad.numel() == self.d
+        assert grad.is_contiguous()
+        ef.ef_vote_worker_step_host(self.ctx, i, grad.data_ptr())
+
     def vote_server_step(self) -> None:
         ef.ef_vote_server_step(self.ctx)
 

@@ -144,3 +144,30 @@ def test_methods_cannot_be_mixed_inside_one_iteration():
     e.vote_server_step()
     assert e.step_count == 2
     torch.cuda.synchronize()
+
+
+def test_host_gradients_match_device_gradients():
+    """ef_vote_worker_step_host (pinned host gradients through the two staging buffers) and the
+    voted signs read back with ef_read_update_host equal the device path bit for bit."""
+    w = wl.custom_workload("vote-host", [TILE * 3 + 11, 100, TILE], 3, 0.9, 0.1, 4, "normal", (1e-3, 1.0),
+                           config_id=330)
+    a = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    b = EFEngine(w.offsets, w.M, w.mu, w.eta, host_staging=True)
+    words = torch.empty(b.W, dtype=torch.int32).pin_memory()
+    scales = torch.empty(b.B, dtype=torch.float32).pin_memory()
+    for t in range(4):
+        hs = [w.draw_grad(t, i, "cpu").pin_memory() for i in range(w.M)]
+        for i in range(w.M):
+            a.vote_worker_step(i, hs[i].cuda())
+            b.vote_worker_step_host(i, hs[i])
+        a.vote_server_step(); b.vote_server_step()
+        b.read_update_host(words, scales)
+        torch.cuda.synchronize()
+        assert torch.equal(words, a.server_words().cpu())
+    assert torch.equal(a.params(), b.params())
+    for i in range(w.M):
+        assert torch.equal(a.momentum(i), b.momentum(i))
+    plain = EFEngine(w.offsets, w.M, w.mu, w.eta)
+    with pytest.raises(ef.EFError) as ei:
+        plain.vote_worker_step_host(0, hs[0])
+    assert ei.value.status == ef.EF_ERR_BAD_STATE            # no staging buffers requested
