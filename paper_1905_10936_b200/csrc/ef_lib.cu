@@ -166,26 +166,23 @@ cudaError_t prepare_server_t(int M) {
                                 (int)server_smem_bytes<MT>(M, true));
 }
 
-cudaError_t prepare_server(int M) {
-    switch (M) {
-        case 1: return prepare_server_t<1>(M);
-        case 2: return prepare_server_t<2>(M);
-        case 3: return prepare_server_t<3>(M);
-        case 4: return prepare_server_t<4>(M);
-        case 5: return prepare_server_t<5>(M);
-        case 6: return prepare_server_t<6>(M);
-        case 7: return prepare_server_t<7>(M);
-        case 8: return prepare_server_t<8>(M);
-        case 9: return prepare_server_t<9>(M);
-        case 10: return prepare_server_t<10>(M);
-        case 11: return prepare_server_t<11>(M);
-        case 12: return prepare_server_t<12>(M);
-        case 13: return prepare_server_t<13>(M);
-        case 14: return prepare_server_t<14>(M);
-        case 15: return prepare_server_t<15>(M);
-        case 16: return prepare_server_t<16>(M);
-        default: return prepare_server_t<0>(M);
+// Runs CALL(MT) with the template argument that serves M workers: M itself up to 16 (table path), else 0.
+#define EF_FOR_WORKER_COUNT(M, CALL)                                                           \
+    switch (M) {                                                                               \
+        case 1: CALL(1); break;   case 2: CALL(2); break;   case 3: CALL(3); break;            \
+        case 4: CALL(4); break;   case 5: CALL(5); break;   case 6: CALL(6); break;            \
+        case 7: CALL(7); break;   case 8: CALL(8); break;   case 9: CALL(9); break;            \
+        case 10: CALL(10); break; case 11: CALL(11); break; case 12: CALL(12); break;          \
+        case 13: CALL(13); break; case 14: CALL(14); break; case 15: CALL(15); break;          \
+        case 16: CALL(16); break; default: CALL(0); break;                                     \
     }
+
+cudaError_t prepare_server(int M) {
+    cudaError_t e = cudaSuccess;
+#define EF_CALL(MT) e = prepare_server_t<MT>(M)
+    EF_FOR_WORKER_COUNT(M, EF_CALL)
+#undef EF_CALL
+    return e;
 }
 
 // The one-launch server call: clusters of kClusterCtas CTAs need the kernel's opt-in (above 8),
@@ -220,16 +217,6 @@ cudaError_t launch_server_update_t(ef_ctx* c, const efk::ServerUpdateArgs& aa) {
     cfg.numAttrs = c->pdl ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, efk::ef_server_update_kernel<kU, MT>, aa);
 }
-
-#define EF_FOR_WORKER_COUNT(M, CALL)                                                           \
-    switch (M) {                                                                               \
-        case 1: CALL(1); break;   case 2: CALL(2); break;   case 3: CALL(3); break;            \
-        case 4: CALL(4); break;   case 5: CALL(5); break;   case 6: CALL(6); break;            \
-        case 7: CALL(7); break;   case 8: CALL(8); break;   case 9: CALL(9); break;            \
-        case 10: CALL(10); break; case 11: CALL(11); break; case 12: CALL(12); break;          \
-        case 13: CALL(13); break; case 14: CALL(14); break; case 15: CALL(15); break;          \
-        case 16: CALL(16); break; default: CALL(0); break;                                     \
-    }
 
 cudaError_t prepare_server_update(int M) {
     cudaError_t e = cudaSuccess;
@@ -287,26 +274,10 @@ int launch_server_range(ef_ctx* c, int b0, int b1, const uint32_t* msgs, long lo
     const efk::ServerArgs a = server_args(c, b0, tr.tile0, msgs, msg_stride);
     // bulk staging needs every chunk's packed words on a 16-byte boundary: plain layout only
     const bool bulk = c->use_bulk && !msgs;
-    cudaError_t le;
-    switch (M) {
-        case 1: le = launch_server_t<1>(c, a, tr.count, bulk); break;
-        case 2: le = launch_server_t<2>(c, a, tr.count, bulk); break;
-        case 3: le = launch_server_t<3>(c, a, tr.count, bulk); break;
-        case 4: le = launch_server_t<4>(c, a, tr.count, bulk); break;
-        case 5: le = launch_server_t<5>(c, a, tr.count, bulk); break;
-        case 6: le = launch_server_t<6>(c, a, tr.count, bulk); break;
-        case 7: le = launch_server_t<7>(c, a, tr.count, bulk); break;
-        case 8: le = launch_server_t<8>(c, a, tr.count, bulk); break;
-        case 9: le = launch_server_t<9>(c, a, tr.count, bulk); break;
-        case 10: le = launch_server_t<10>(c, a, tr.count, bulk); break;
-        case 11: le = launch_server_t<11>(c, a, tr.count, bulk); break;
-        case 12: le = launch_server_t<12>(c, a, tr.count, bulk); break;
-        case 13: le = launch_server_t<13>(c, a, tr.count, bulk); break;
-        case 14: le = launch_server_t<14>(c, a, tr.count, bulk); break;
-        case 15: le = launch_server_t<15>(c, a, tr.count, bulk); break;
-        case 16: le = launch_server_t<16>(c, a, tr.count, bulk); break;
-        default: le = launch_server_t<0>(c, a, tr.count, bulk); break;
-    }
+    cudaError_t le = cudaSuccess;
+#define EF_CALL(MT) le = launch_server_t<MT>(c, a, tr.count, bulk)
+    EF_FOR_WORKER_COUNT(M, EF_CALL)
+#undef EF_CALL
     EF_CUDA(c, le);
     c->launches += 1;
     const std::vector<int32_t>& list = defer_scales ? c->h_multi_big : c->h_multi;
