@@ -80,6 +80,7 @@ struct ef_ctx {
     std::vector<uint8_t> pushed;
     bool use_bulk = false;                 // the server kernel stages its inputs with cp.async.bulk
     bool pdl = false;                      // kernels are launched with programmatic stream serialization
+    bool one_launch_server = false;        // ef_server_step is the cluster-launched server + update kernel
     // host-staging path
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t ev_copied[2] = {nullptr, nullptr};

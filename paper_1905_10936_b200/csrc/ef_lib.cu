@@ -197,24 +197,43 @@ cudaError_t prepare_server_update_t(int M) {
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
 }
 
+// Launch configuration of the one-launch server call; attr must have room for two entries.
 template <int MT>
-cudaError_t launch_server_update_t(ef_ctx* c, const efk::ServerUpdateArgs& aa) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)c->L.num_ctiles);
-    cfg.blockDim = dim3(efk::kThreads);
-    cfg.dynamicSmemBytes = server_smem_bytes<MT>(c->L.M, false);
-    cfg.stream = c->stream;
-    cudaLaunchAttribute attr[1];
+void server_update_config(const ef_ctx* c, cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr) {
+    *cfg = cudaLaunchConfig_t{};
+    cfg->gridDim = dim3((unsigned)c->L.num_ctiles);
+    cfg->blockDim = dim3(efk::kThreads);
+    cfg->dynamicSmemBytes = server_smem_bytes<MT>(c->L.M, false);
+    cfg->stream = c->stream;
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = efk::kClusterCtas;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
-    cudaLaunchAttribute attr2[2];
-    attr2[0] = attr[0];
-    attr2[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr2[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr2;
-    cfg.numAttrs = c->pdl ? 2 : 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg->attrs = attr;
+    cfg->numAttrs = c->pdl ? 2 : 1;
+}
+
+// Can the device hold at least one cluster of this kernel at a time?  (If not, the call keeps
+// its two kernels.)
+template <int MT>
+cudaError_t server_update_fits_t(const ef_ctx* c, bool* fits) {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[2];
+    server_update_config<MT>(c, &cfg, attr);
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    const cudaError_t e = cudaOccupancyMaxActiveClusters(&clusters, efk::ef_server_update_kernel<kU, MT>, &cfg);
+    *fits = e == cudaSuccess && clusters >= 1;
+    return e;
+}
+
+template <int MT>
+cudaError_t launch_server_update_t(ef_ctx* c, const efk::ServerUpdateArgs& aa) {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[2];
+    server_update_config<MT>(c, &cfg, attr);
     return cudaLaunchKernelEx(&cfg, efk::ef_server_update_kernel<kU, MT>, aa);
 }
 
@@ -340,7 +359,7 @@ int launch_server_update(ef_ctx* c) {
 }
 
 int launch_server(ef_ctx* c) {
-    if (c->L.num_ctiles > 0 && c->lambda == 0.f) return launch_server_update(c);
+    if (c->one_launch_server && c->lambda == 0.f) return launch_server_update(c);
     // Large layouts: the update kernel completes the scales of all but the largest blocks itself.
     const bool self_scale = !c->fused;
     const int rc = launch_server_range(c, 0, c->L.B, nullptr, 0, self_scale);
@@ -481,7 +500,15 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
         (ce = cudaMemcpyAsync(c->ws + L.off_ctiles, c->h_ctiles.data(), c->h_ctiles.size() * sizeof(Tile),
                               cudaMemcpyHostToDevice, c->stream)) != cudaSuccess) return fail(ce);
     if ((ce = prepare_server(M)) != cudaSuccess) return fail(ce);
-    if (L.num_ctiles > 0 && (ce = prepare_server_update(M)) != cudaSuccess) return fail(ce);
+    if (L.num_ctiles > 0) {
+        if ((ce = prepare_server_update(M)) != cudaSuccess) return fail(ce);
+        bool fits = false;
+#define EF_CALL(MT) ce = server_update_fits_t<MT>(c, &fits)
+        EF_FOR_WORKER_COUNT(M, EF_CALL)
+#undef EF_CALL
+        (void)cudaGetLastError();          // a device without room for such a cluster keeps the two kernels
+        c->one_launch_server = fits;
+    }
     {
         // bulk staging: every block but the last must hold a multiple of 128 elements (so that
         // every chunk's 128 packed words start on a 16-byte boundary) and start 16-byte aligned
