@@ -593,6 +593,70 @@ def run_topk(args) -> None:
     print(json.dumps(line), flush=True)
 
 
+def run_ps_group(args) -> None:
+    """The paper's setting over a process group: one rank per GPU (torchrun), rank r = worker r
+    and the server of one block range, M = world size.  --push: buffers in symmetric memory, the
+    kernels store the messages into the peers' buffers, two one-element all-reduces per iteration;
+    otherwise all-to-all and all-gather.  Timed as the whole iteration, max over ranks."""
+    import torch.distributed as dist
+    from paper_1905_10936_b200 import ps
+    from paper_1905_10936_b200.engine import EFEngine
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29541")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    w0 = load_workload(args)
+    w = wl.custom_workload(f"{w0.name}-M{world}", w0.sizes, world, w0.mu, w0.eta, w0.steps, w0.law,
+                           w0.scale_range, config_id=w0.config_id)
+    K, W = args.steps, args.warmup
+    eng = EFEngine(w.offsets, world, w.mu, w.eta, one_local_worker=True)
+    if args.push:
+        recv, update, recv_ptrs, update_ptrs = ps.symmetric_buffers(w.sizes, rank, world, dev)
+        rk = ps.Rank(eng, w.sizes, rank, world, recv=recv, update=update)
+        rk.connect(recv_ptrs, update_ptrs)
+    else:
+        rk = ps.Rank(eng, w.sizes, rank, world)
+    flag = torch.zeros(1, device=dev)
+    grad = w.draw_grad(0, rank, "cuda", w.element_scales("cuda"))
+
+    def one():
+        if args.push:
+            ps.step_push(rk, grad, flag)
+        else:
+            ps.step(rk, grad)
+
+    for _ in range(W):
+        one()
+    dist.barrier(); torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(K):
+        one()
+    e1.record()
+    dist.barrier(); torch.cuda.synchronize()
+    tt = torch.tensor([e0.elapsed_time(e1)], device=dev, dtype=torch.float64)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    ms = float(tt.item()) / K
+    if rank == 0:
+        units = rk.total_units
+        line = {"metric": "parameters/sec through one iteration of the sharded parameter-server protocol "
+                          "(one worker and one server shard per GPU)",
+                "value": w.d / (ms * 1e-3), "unit": "params/s", "n_gpus": world, "steps": K, "warmup": W,
+                "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+                "dtype": "f32", "data": "synthetic", "config": config_dict(w),
+                "run": {"workload": "ps", "variant": "push" if args.push else "collective", "ranks": world,
+                        "process_group": "nccl",
+                        "exchange_bytes_per_rank": {"out": 4 * units * (world - 1) // world,
+                                                    "in": 4 * units * (world - 1) // world}},
+                "e2e": None, "gpu_launches": int(eng.launch_count)}
+        print(json.dumps(line), flush=True)
+    dist.destroy_process_group()
+
+
 def run_ps(args) -> None:
     """The paper's setting in pieces on ONE GPU: G ranks (rank r = worker r + the server of one
     block range) stepped one after the other, the exchange replaced by device copies.  Times the
@@ -720,6 +784,9 @@ def main():
                          "topk: the top-k compressor on one vector of the layout's size; "
                          "ps: the one-worker-per-rank protocol with a block-sharded server, its "
                          "compute pieces timed with the M ranks emulated on one GPU")
+    ap.add_argument("--process-group", action="store_true",
+                    help="--workload ps: run over the torch.distributed process group (one rank per GPU; "
+                         "implied under torchrun with more than one rank) instead of emulating the ranks")
     ap.add_argument("--push", action="store_true",
                     help="--workload ps: the push variant (messages stored where their readers are)")
     ap.add_argument("--topk-fraction", type=float, default=0.01, help="k / n for --workload topk")
@@ -753,7 +820,10 @@ def main():
     if args.workload == "topk":
         run_topk(args)
     elif args.workload == "ps":
-        run_ps(args)
+        if args.process_group or int(os.environ.get("WORLD_SIZE", "1")) > 1:
+            run_ps_group(args)
+        else:
+            run_ps(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

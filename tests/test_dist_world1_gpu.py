@@ -107,3 +107,23 @@ def test_push_variant_over_symmetric_memory(nccl_world1):
     sc, wd = ps.unpack_message(rk.update.cpu().numpy(), w.sizes, 0, w.B)
     assert np.array_equal(sc, ref.server_scales().cpu().numpy())
     assert np.array_equal(wd, ref.server_words().cpu().numpy().view(np.uint32))
+
+
+@pytest.mark.parametrize("push", [False, True])
+def test_bench_process_group_mode_runs_with_one_rank(push):
+    """bench.py --workload ps --process-group: the mode torchrun uses with one rank per GPU."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK="0", WORLD_SIZE="1", LOCAL_RANK="0")
+    cmd = [sys.executable, os.path.join(root, "bench.py"), "--workload", "ps", "--process-group", "--config", "1",
+           "--steps", "3", "--warmup", "3"] + (["--push"] if push else [])
+    out = subprocess.run(cmd, capture_output=True, text=True, env=env, cwd=root, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads([ln for ln in out.stdout.splitlines() if ln.startswith("{")][-1])
+    assert line["run"]["variant"] == ("push" if push else "collective") and line["run"]["process_group"] == "nccl"
+    assert line["value"] > 0 and line["gpu_launches"] > 0
