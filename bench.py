@@ -7,7 +7,8 @@ synthetic gradients (up to three batches are kept in HBM and rotated).  The defa
 the flat 2^28-parameter layout (256 blocks of 2^20, M = 7).  Prints ONE JSON line on rank 0.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
-                  [--workload ef|signum|topk] [--scaling weak|strong] [--graph] [--ceiling]
+                  [--workload ef|signum|topk|ps [--push] [--process-group]] [--scaling weak|strong]
+                  [--graph] [--ceiling] [--library-flags F]
                   [--per-worker-calls] [--weight-decay L] [--diagnostics] [--blocks N] [--workers M]
 
 Keys beyond the common ones: `roofline` (worker launch), `roofline_server` (server call),
@@ -19,6 +20,11 @@ With N > 1 (launched by torch.distributed.run): --scaling weak (default) gives e
 whole layout (a block-range shard of an N-times larger problem; no data-path collective);
 --scaling strong cuts ONE layout into N equal element ranges, blocks included, and all-reduces
 one fp64 sum per cut block and call.
+
+--workload ps: the sharded parameter server (one worker and one server shard per rank), with
+the ranks emulated on one GPU (the pieces timed one by one) or, with --process-group or under
+torchrun with N > 1, over the real process group; --push stores the messages directly into the
+peers' buffers instead of packing them and calling collectives.
 
 --impl reference times the CPU oracle (plain single-threaded C++) on a bounded sample of the
 same workload; it is a deliberately slow program, reported for context.
