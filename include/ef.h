@@ -93,8 +93,11 @@ enum ef_status {
                                       the worker's own state, and the one-launch server kernel its x values,
                                       before that wait.  On B200 this shortens the launch-bound layouts whose
                                       worker launch is a single wave of CTAs (flat 2^20, M = 2: 16.4 -> 14.5 us
-                                      per step from a CUDA graph) and does nothing for the others, so it is
-                                      off by default.  Results are identical.  While it is on, kernels of the
+                                      per step from a CUDA graph) and does nothing for the others, so by
+                                      default it is on only there (one-launch server call and all CTAs of
+                                      the M workers resident at once) and this flag forces it everywhere;
+                                      EF_FLAG_SEPARATE_UPDATE keeps ordinary launches.  Results are
+                                      identical.  While it is on, kernels of the
                                       caller that write x or a worker's state through the raw pointers
                                       directly before a call must not signal programmatic completion early. */
 #define EF_FLAG_SEPARATE_UPDATE 2048u /* On layouts of few chunks in which no block spans more than 16 chunks,

@@ -508,6 +508,14 @@ int ef_init(ef_ctx** out, int64_t d, int32_t B, const int64_t* offsets, int32_t 
 #undef EF_CALL
         (void)cudaGetLastError();          // a device without room for such a cluster keeps the two kernels
         c->one_launch_server = fits;
+        // Programmatic launches pay off exactly where the whole step is two single-wave kernels (the
+        // next kernel finds free SMs while its predecessor drains): switched on by default there.
+        int per_sm = 0, sms = 0;
+        if (fits && cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, efk::ef_worker_kernel<kU, false>,
+                                                                  efk::kThreads, 0) == cudaSuccess &&
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
+            L.num_tiles * L.tile_chunks * (int64_t)L.Ml <= (int64_t)per_sm * sms)
+            c->pdl = true;
     }
     {
         // bulk staging: every block but the last must hold a multiple of 128 elements (so that
