@@ -60,9 +60,11 @@ int make_layout(int64_t d, int32_t B, const int64_t* offsets, int32_t M, uint32_
     // One-launch server call (clusters): few chunks, all workers local, no block beyond one cluster.
     // A cluster per multi-chunk block, single-chunk blocks share clusters.
     if (L->tile_chunks == 1 && L->Ml == M && most <= efk::kClusterCtas &&
-        !(flags & (EF_FLAG_SEPARATE_UPDATE | EF_FLAG_SPLIT_SCALE | EF_FLAG_DIAGNOSTICS)))
-        L->num_ctiles = (int32_t)(efk::kClusterCtas *
-                                  ((B - single) + (single + efk::kClusterCtas - 1) / efk::kClusterCtas));
+        !(flags & (EF_FLAG_SEPARATE_UPDATE | EF_FLAG_SPLIT_SCALE | EF_FLAG_DIAGNOSTICS))) {
+        const int64_t ctas = efk::kClusterCtas *
+                             ((B - single) + (single + efk::kClusterCtas - 1) / efk::kClusterCtas);
+        if (ctas <= std::max<int64_t>(4 * T, 512)) L->num_ctiles = (int32_t)ctas;   // not where thousands of CTAs would idle
+    }
     if (T * L->tile_chunks > 0x7fffffffLL) return EF_ERR_INVALID_ARG;
     L->W = W; L->num_tiles = T;
     L->dpad = align_up((size_t)d * 4) / 4;
