@@ -579,8 +579,10 @@ __device__ __forceinline__ double worker_rows_scalar(const WorkerArgs& a, const 
 }
 
 // grid.x = chunks, grid.y = workers stepped by this launch (1 for ef_worker_step).
+// Four CTAs per SM (64 registers) for the plain form: the launch-bound layouts need all CTAs of
+// the M workers resident at once (flat 2^20, M = 2: 512 CTAs on 148 SMs).
 template <int U, bool DIAG>
-__global__ void __launch_bounds__(kThreads) ef_worker_kernel(const WorkerArgs a0) {
+__global__ void __launch_bounds__(kThreads, DIAG ? 3 : 4) ef_worker_kernel(const WorkerArgs a0) {
     pdl_trigger();
     WorkerArgs a = a0;
     {
