@@ -92,7 +92,7 @@ enum ef_status {
                                       on the device for the predecessor's results; the worker kernel loads
                                       the worker's own state, and the one-launch server kernel its x values,
                                       before that wait.  On B200 this shortens the launch-bound layouts whose
-                                      worker launch is a single wave of CTAs (flat 2^20, M = 2: 16.4 -> 14.5 us
+                                      worker launch is a single wave of CTAs (flat 2^20, M = 2: 16.4 -> 14.5-15.4 us
                                       per step from a CUDA graph) and does nothing for the others, so by
                                       default it is on only there (one-launch server call and all CTAs of
                                       the M workers resident at once) and this flag forces it everywhere;
