@@ -732,6 +732,125 @@ __global__ void __launch_bounds__(kThreads, 3) ef_topk_scatter_kernel(const Scat
     }
 }
 
+// ---- short vectors: everything in ONE CTA.  Up to kSmallN elements the nine launches above
+// cost more than the work; here one CTA of 1024 threads runs the three digit passes over v
+// (shared-memory histogram, selection by a scan over the CTA; v is re-read from L2), then goes
+// through v once more in index order, 4096 elements per round, ranks the kept elements (a scan
+// within each warp, then over the warps' totals, running totals over the rounds) and writes idx,
+// val and the residual.  Same keys, same tie rule, hence the same result as the general path.
+// (All keys of a vector fall into a few dozen bins of the first digit, so the histogram's
+// shared-memory atomics serialise: the cost grows with n and the general path wins from about
+// 2^15 elements on.  Keeping the vector in registers across the passes did not change that.)
+constexpr int kSmallThreads = 1024;
+constexpr long long kSmallN = 16384;
+
+__global__ void __launch_bounds__(kSmallThreads) ef_topk_small_kernel(const float* v, long long n,
+                                                                      unsigned long long k,
+                                                                      long long* __restrict__ idx_out,
+                                                                      float* __restrict__ val_out, float* resid) {
+    __shared__ unsigned s_hist[kBins];
+    __shared__ unsigned s_warp[32];            // per-warp totals (histogram scan, then packed gt | eq << 16)
+    __shared__ unsigned s_prefix, s_remaining;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    unsigned prefix = 0u, remaining = (unsigned)k;          // k <= n <= kSmallN
+#pragma unroll 1
+    for (int pass = 0; pass < kPasses; ++pass) {
+        const int shift = pass_shift(pass), bits = pass_bits(pass);
+        for (int b = tid; b < kBins; b += kSmallThreads) s_hist[b] = 0u;
+        __syncthreads();
+        for (long long i = 4LL * tid; i < n; i += 4 * kSmallThreads) {
+            float x[4]; bool in[4];
+            load_keys(v, i, n, x, in);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const unsigned key = key_of(x[j]);
+                if (in[j] && (pass == 0 || (key >> (shift + bits)) == prefix))
+                    atomicAdd(&s_hist[(key >> shift) & ((1u << bits) - 1u)], 1u);
+            }
+        }
+        __syncthreads();
+        // thread t owns bins 2047 - 2t and 2046 - 2t: from the top down; scan over the CTA
+        const unsigned h0 = s_hist[kBins - 1 - 2 * tid], h1 = s_hist[kBins - 2 - 2 * tid];
+        unsigned incl = warp_inclusive_scan32(h0 + h1, lane);
+        if (lane == 31) s_warp[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            const unsigned t = s_warp[lane];
+            const unsigned w = warp_inclusive_scan32(t, lane);
+            s_warp[lane] = w - t;              // exclusive
+        }
+        __syncthreads();
+        incl += s_warp[warp];
+        const unsigned above = incl - h0 - h1; // keys in the bins above this thread's pair
+        // the bin in which the count from the top reaches `remaining`
+        if (above < remaining && incl >= remaining) {
+            const bool first = above + h0 >= remaining;
+            const unsigned bin = kBins - 1 - 2 * tid - (first ? 0 : 1);
+            s_prefix = (prefix << bits) | bin;
+            s_remaining = remaining - above - (first ? 0u : h0);
+        }
+        __syncthreads();
+        prefix = s_prefix;
+        remaining = s_remaining;
+        __syncthreads();
+    }
+    const unsigned T = prefix;
+    const unsigned need_eq = remaining;
+    unsigned gt_run = 0u, eq_run = 0u;         // keys > T / == T before this round
+    for (long long base0 = 0; base0 < n; base0 += 4 * kSmallThreads) {
+        const long long base = base0 + 4 * tid;
+        float x[4] = {0.f, 0.f, 0.f, 0.f};
+        bool in[4] = {false, false, false, false};
+        if (base < n) load_keys(v, base, n, x, in);
+        unsigned fgt = 0u, feq = 0u, nib = 0u;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const unsigned key = key_of(x[j]);
+            nib |= in[j] ? 1u << j : 0u;
+            fgt |= key > T ? 1u << j : 0u;
+            feq |= key == T ? 1u << j : 0u;
+        }
+        fgt &= nib; feq &= nib;
+        const unsigned cnt = (unsigned)__popc(fgt) | ((unsigned)__popc(feq) << 16);
+        const unsigned incl = warp_inclusive_scan32(cnt, lane);
+        __syncthreads();                       // the previous round's totals have been read
+        if (lane == 31) s_warp[warp] = incl;
+        __syncthreads();
+        unsigned before = 0u, total = 0u;
+#pragma unroll 8
+        for (int w = 0; w < 32; ++w) {
+            const unsigned t = s_warp[w];
+            before += w < warp ? t : 0u;
+            total += t;
+        }
+        unsigned gt_rank = gt_run + ((before + incl - cnt) & 0xffffu);
+        unsigned eq_rank = eq_run + ((before + incl - cnt) >> 16);
+        float y[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const bool is_gt = (fgt >> j) & 1u, is_eq = (feq >> j) & 1u;
+            const bool kept = is_gt || (is_eq && eq_rank < need_eq);
+            if (kept) {
+                const unsigned long long pos = (unsigned long long)gt_rank + (eq_rank < need_eq ? eq_rank : need_eq);
+                if (pos < k) {                 // always true when the counts are consistent
+                    idx_out[pos] = base + j;
+                    val_out[pos] = x[j];
+                }
+            }
+            y[j] = kept ? __fsub_rn(x[j], x[j]) : x[j];        // e = v - C(v)
+            gt_rank += is_gt ? 1u : 0u;
+            eq_rank += is_eq ? 1u : 0u;
+        }
+        if (resid != nullptr && nib != 0u) {
+            if (nib == 0xfu) *reinterpret_cast<float4*>(resid + base) = make_float4(y[0], y[1], y[2], y[3]);
+            else
+                for (int j = 0; j < 4; ++j) if ((nib >> j) & 1u) resid[base + j] = y[j];
+        }
+        gt_run += total & 0xffffu;
+        eq_run += total >> 16;
+    }
+}
+
 }  // namespace
 
 extern "C" {
@@ -768,6 +887,11 @@ int ef_topk_compress(const float* v, int64_t n, int64_t k, int64_t* idx_out, flo
         }
     }
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (n <= kSmallN) {                        // short vectors: one CTA does it all (the workspace stays unused)
+        ef_topk_small_kernel<<<1, kSmallThreads, 0, st>>>(v, n, (unsigned long long)k, (long long*)idx_out,
+                                                          val_out, resid_out);
+        return cudaGetLastError() == cudaSuccess ? EF_OK : EF_ERR_CUDA;
+    }
     char* ws = (char*)workspace;
     unsigned long long* hist = (unsigned long long*)(ws + L.off_hist);
     TopkState* state = (TopkState*)(ws + L.off_state);

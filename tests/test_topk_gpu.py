@@ -40,9 +40,9 @@ def test_sizes_around_the_chunk_boundaries(n):
         check(v, k)
 
 
+@pytest.mark.parametrize("n", [10_000, 50_000])          # one-CTA path for short vectors, general path
 @pytest.mark.parametrize("law", ["normal", "laplace", "cauchy", "quantised", "constant", "zeros", "denormal"])
-def test_value_distributions_and_ties(law):
-    n = 50_000
+def test_value_distributions_and_ties(law, n):
     gen = torch.Generator().manual_seed(7)
     if law == "normal":
         v = torch.randn(n, generator=gen)
@@ -96,9 +96,10 @@ def test_vectors_whose_candidates_do_not_fit_the_list(law):
         check(v, k)
 
 
-@pytest.mark.parametrize("n", [65536, 65537, 8 * 65536, 8 * 65536 + 8, 1_000_003])
+@pytest.mark.parametrize("n", [16383, 16384, 16385, 65536, 65537, 8 * 65536, 8 * 65536 + 8, 1_000_003])
 def test_sizes_around_the_list_capacity(n):
-    """The list holds max(n/8, min(n, 65536)) keys; vectors on both sides of the two break points,
+    """Vectors of up to 16384 elements are handled by one CTA; beyond that the candidate list holds
+    max(n/8, min(n, 65536)) keys.  Vectors on both sides of the break points,
     ordinary values (the list is used) and all-equal magnitudes (it is not, beyond 65536)."""
     gen = torch.Generator().manual_seed(n % 97)
     v = torch.randn(n, generator=gen)
