@@ -32,6 +32,7 @@
 #include "ef_internal.h"
 
 #include <algorithm>
+#include <utility>
 #include <type_traits>
 
 namespace {
@@ -152,6 +153,7 @@ __global__ void __launch_bounds__(kThreads) ef_topk_hist_kernel(const float* __r
     __shared__ unsigned s_hist[kBins];
     for (int b = threadIdx.x; b < kBins; b += kThreads) s_hist[b] = 0u;
     __syncthreads();
+    efk::pdl_enter();
     constexpr int bits = pass_bits(PASS);
     hist_over_vector<PASS>(v, n, chunks, PASS == 0 ? 0u : st->prefix, s_hist);
     __syncthreads();
@@ -279,6 +281,7 @@ __global__ void __launch_bounds__(kThreads) ef_topk_candidates_kernel(const floa
     WarpStage* s_stage = reinterpret_cast<WarpStage*>(s_dyn + kWarps * sizeof(WarpList));
     __shared__ unsigned s_hist[kBins];
     for (int b = threadIdx.x; b < kBins; b += kThreads) s_hist[b] = 0u;
+    efk::pdl_enter();
     const unsigned P0 = st->prefix;
     const unsigned lo = P0 << 20, hi_top = P0 + 1u;       // candidates: lo <= key and (key >> 20) < hi_top
     const bool compact = st->compact != 0u;
@@ -369,6 +372,7 @@ __global__ void __launch_bounds__(kThreads) ef_topk_third_digit_kernel(const flo
     __shared__ unsigned s_hist[nbins];
     for (int b = threadIdx.x; b < nbins; b += kThreads) s_hist[b] = 0u;
     __syncthreads();
+    efk::pdl_enter();
     const unsigned prefix = st->prefix;            // 22 bits
     if (st->compact) {
         const unsigned long long ncand = st->ncand;
@@ -398,6 +402,7 @@ __global__ void __launch_bounds__(kThreads) ef_topk_select_kernel(const unsigned
     __shared__ int s_found;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int grp = kThreads - 1 - threadIdx.x;
+    efk::pdl_enter();
     unsigned long long bin[per];
     unsigned long long g = 0;
 #pragma unroll
@@ -454,6 +459,7 @@ __global__ void __launch_bounds__(kThreads) ef_topk_count_kernel(const float* __
                                                                  unsigned* __restrict__ ceq,
                                                                  unsigned* __restrict__ tgt,
                                                                  unsigned* __restrict__ teq) {
+    efk::pdl_enter();
     const unsigned T = st->threshold;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (st->compact) {
@@ -539,6 +545,7 @@ __global__ void __launch_bounds__(kScanThreads) ef_topk_scan_kernel(const unsign
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) { s_carry[0] = 0ull; s_carry[1] = 0ull; }
     __syncthreads();
+    efk::pdl_enter();
     for (long long piece = 0; piece < chunks; piece += (long long)kScanThreads * kScanPer) {
         const long long lo = piece + (long long)threadIdx.x * kScanPer;
         unsigned ga[kScanPer], gb[kScanPer];
@@ -687,6 +694,7 @@ __global__ void __launch_bounds__(kThreads, 3) ef_topk_scatter_kernel(const Scat
     const int nch = (int)min((long long)kScatterChunks, a.chunks - c0);
     float xA[kU][4], xB[kU][4];
     unsigned finA, finB = 0u;
+    efk::pdl_enter();
     load_chunk_keys(a.v, a.n, c0, warp, lane, xA, finA);
     if (warp == 0) {
         // before the CTA's first slice: the tile's prefix plus the tile's slices before it
@@ -851,6 +859,25 @@ __global__ void __launch_bounds__(kSmallThreads) ef_topk_small_kernel(const floa
     }
 }
 
+// Launch with programmatic stream serialization: every kernel of the call starts with
+// efk::pdl_enter() (or sets up its shared memory first), so a kernel's launch latency and set-up
+// overlap the tail of the one before it and its reads still follow that kernel's completion.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_after(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t st,
+                         Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 }  // namespace
 
 extern "C" {
@@ -908,20 +935,25 @@ int ef_topk_compress(const float* v, int64_t n, int64_t k, int64_t* idx_out, flo
     const unsigned hgrid = (unsigned)std::min<long long>(L.chunks, 148 * 8);
     const unsigned cgrid = (unsigned)std::min<long long>(L.chunks, 148 * 3);       // three CTAs of 59 KB per SM
     const unsigned long long kk = (unsigned long long)k;
-    ef_topk_hist_kernel<0><<<hgrid, kThreads, 0, st>>>(v, n, L.chunks, state, hist);
-    ef_topk_select_kernel<0><<<1, kThreads, 0, st>>>(hist, state, kk, L.cap);
-    ef_topk_candidates_kernel<<<cgrid, kThreads, kCandidatesSmem, st>>>(v, n, L.chunks, state, hist + kBins,
-                                                                        cgt, seg_start, seg_cnt, cand);
-    ef_topk_select_kernel<1><<<1, kThreads, 0, st>>>(hist + kBins, state, kk, L.cap);
-    ef_topk_third_digit_kernel<<<hgrid, kThreads, 0, st>>>(v, n, L.chunks, cand, state, hist + 2 * kBins);
-    ef_topk_select_kernel<2><<<1, kThreads, 0, st>>>(hist + 2 * kBins, state, kk, L.cap);
-    ef_topk_count_kernel<<<(unsigned)((L.chunks + kWarps - 1) / kWarps), kThreads, 0, st>>>(
-        v, n, L.chunks, cand, state, seg_start, seg_cnt, cgt, ceq, tgt, teq);
-    ef_topk_scan_kernel<<<1, kScanThreads, 0, st>>>(tgt, teq, pgt, peq, L.tiles);
+    launch_after(ef_topk_hist_kernel<0>, hgrid, kThreads, 0, st, v, (long long)n, L.chunks, (const TopkState*)state, hist);
+    launch_after(ef_topk_select_kernel<0>, 1, kThreads, 0, st, (const unsigned long long*)hist, state, kk, L.cap);
+    launch_after(ef_topk_candidates_kernel, cgrid, kThreads, kCandidatesSmem, st, v, (long long)n, L.chunks, state,
+                 hist + kBins, cgt, seg_start, seg_cnt, cand);
+    launch_after(ef_topk_select_kernel<1>, 1, kThreads, 0, st, (const unsigned long long*)(hist + kBins), state, kk, L.cap);
+    launch_after(ef_topk_third_digit_kernel, hgrid, kThreads, 0, st, v, (long long)n, L.chunks, (const unsigned*)cand,
+                 (const TopkState*)state, hist + 2 * kBins);
+    launch_after(ef_topk_select_kernel<2>, 1, kThreads, 0, st, (const unsigned long long*)(hist + 2 * kBins), state, kk,
+                 L.cap);
+    launch_after(ef_topk_count_kernel, (unsigned)((L.chunks + kWarps - 1) / kWarps), kThreads, 0, st, v, (long long)n,
+                 L.chunks, (const unsigned*)cand, (const TopkState*)state, (const unsigned long long*)seg_start,
+                 (const unsigned*)seg_cnt, cgt, ceq, tgt, teq);
+    launch_after(ef_topk_scan_kernel, 1, kScanThreads, 0, st, (const unsigned*)tgt, (const unsigned*)teq, pgt, peq,
+                 L.tiles);
     ScatterArgs sa;
     sa.v = v; sa.n = n; sa.chunks = L.chunks; sa.st = state; sa.cgt = cgt; sa.ceq = ceq; sa.pgt = pgt; sa.peq = peq;
     sa.idx_out = (long long*)idx_out; sa.val_out = val_out; sa.resid = resid_out; sa.kmax = kk;
-    ef_topk_scatter_kernel<<<(unsigned)((L.chunks + kScatterChunks - 1) / kScatterChunks), kThreads, 0, st>>>(sa);
+    launch_after(ef_topk_scatter_kernel, (unsigned)((L.chunks + kScatterChunks - 1) / kScatterChunks), kThreads, 0, st,
+                 sa);
     return cudaGetLastError() == cudaSuccess ? EF_OK : EF_ERR_CUDA;
 }
 
